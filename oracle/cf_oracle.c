@@ -1,0 +1,192 @@
+/*
+ * CPU oracle for mixed decode + chunked-prefill paged grouped-query attention.
+ *
+ * TEST INFRASTRUCTURE ONLY.  This file is the slow, plain definition the CUDA
+ * library is checked against.  It shares no code, header, table or helper with
+ * the CUDA path, and nothing in the product may call it: only the tests, the
+ * smoke check and the benchmark's CPU-baseline leg load it.
+ *
+ * What it computes.  The paper's decode node builds a mixed prefill/decode batch
+ * out of resident decode sequences plus locally queued prefill that reuses a
+ * resident prefix (Section 5), issued in bounded units (Section 4.4); prefill
+ * materialises KV and decode generates autoregressively (Section 2.1), hence the
+ * causal rule.  The paper gives no attention formula (it adds no model kernels,
+ * Section 5), so the arithmetic is the textbook definition of softmax attention
+ * over a paged cache:
+ *
+ *   for sequence s, new-token row i in [0, Lq[s]), query head h:
+ *     p = (Lc[s] - Lq[s]) + i                 absolute position of the query token
+ *     g = h / (Hq / Hkv)                      KV head serving this query head
+ *     k_j, v_j = cache[ block_table[s][j / B] ][ g ][ j % B ]   for j in [0, p]
+ *     x_j = scale * sum_d q[d] * k_j[d]
+ *     m   = max_j x_j ;  l = sum_j exp(x_j - m)
+ *     O   = sum_j exp(x_j - m) * v_j / l ;  lse = m + ln l
+ *
+ * Everything is evaluated in fp64 from the exact bf16 input values, keys in
+ * ascending order, with no blocking, fusion or reordering.
+ *
+ * Pins (tests, CPU only): brute-force dense masked attention on gathered
+ * contiguous K/V, the library scaled-dot-product routine on an identity block
+ * table, closed forms (Lc = 1, q = 0, constant V, dominant key) and invariants
+ * (page permutation, chunking, causal mask, batch order).
+ */
+#include <math.h>
+#include <stdint.h>
+#include <stdlib.h>
+#include <string.h>
+#ifdef _OPENMP
+#include <omp.h>
+#endif
+
+static double bf16_to_f64(uint16_t bits)
+{
+    uint32_t u = ((uint32_t)bits) << 16;
+    float f;
+    memcpy(&f, &u, sizeof f);
+    return (double)f;
+}
+
+/* Locate packed row r: which sequence owns it and which new-token index it is. */
+static int find_row(const int32_t *query_len, int32_t num_seqs, int64_t r, int32_t *seq, int32_t *idx)
+{
+    int64_t at = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        if (r < at + query_len[s]) {
+            *seq = s;
+            *idx = (int32_t)(r - at);
+            return 0;
+        }
+        at += query_len[s];
+    }
+    return -1;
+}
+
+/*
+ * rows == NULL: compute all T = sum(query_len) packed rows, outputs indexed by packed row.
+ * rows != NULL: compute only rows[0..n_rows), outputs indexed by position in that list.
+ * out     [n, Hq, D]  fp64
+ * lse     [n, Hq]     fp64 or NULL
+ * weights [n, Hq, weights_ld] fp64 or NULL: softmax weights of keys 0..p (rest zero-filled)
+ * Returns 0, or a negative code on invalid arguments.
+ */
+int cf_oracle_mixed_attention(
+    const uint16_t *q, const uint16_t *k_cache, const uint16_t *v_cache,
+    int64_t k_stride_block, int64_t k_stride_head, int64_t k_stride_token,
+    int64_t v_stride_block, int64_t v_stride_head, int64_t v_stride_token,
+    const int32_t *block_table, int32_t max_blocks_per_seq,
+    const int32_t *context_len, const int32_t *query_len, int32_t num_seqs,
+    int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t block_size,
+    double scale,
+    const int64_t *rows, int64_t n_rows,
+    double *out, double *lse, double *weights, int64_t weights_ld)
+{
+    if (num_q_heads <= 0 || num_kv_heads <= 0 || num_q_heads % num_kv_heads != 0) return -1;
+    if (head_dim <= 0 || block_size <= 0 || num_seqs < 0) return -1;
+    int64_t T = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        if (query_len[s] < 0 || query_len[s] > context_len[s]) return -2;
+        if ((int64_t)context_len[s] > (int64_t)max_blocks_per_seq * block_size) return -3;
+        T += query_len[s];
+    }
+    const int64_t n = rows ? n_rows : T;
+    const int32_t group = num_q_heads / num_kv_heads;
+    const int64_t work = n * num_q_heads;
+    int bad = 0;
+
+#pragma omp parallel for schedule(dynamic, 1)
+    for (int64_t w = 0; w < work; ++w) {
+        const int64_t slot = w / num_q_heads;
+        const int32_t h = (int32_t)(w % num_q_heads);
+        const int64_t r = rows ? rows[slot] : slot;
+        int32_t s, i;
+        if (find_row(query_len, num_seqs, r, &s, &i) != 0) {
+#pragma omp atomic write
+            bad = 1;
+            continue;
+        }
+        const int32_t p = context_len[s] - query_len[s] + i;
+        const int32_t g = h / group;
+        const uint16_t *qrow = q + (r * num_q_heads + h) * (int64_t)head_dim;
+        const int32_t *bt = block_table + (int64_t)s * max_blocks_per_seq;
+
+        double *x = (double *)malloc(sizeof(double) * (size_t)(p + 1));
+        double m = -INFINITY;
+        for (int32_t j = 0; j <= p; ++j) {
+            const uint16_t *kj = k_cache + (int64_t)bt[j / block_size] * k_stride_block
+                                 + (int64_t)g * k_stride_head + (int64_t)(j % block_size) * k_stride_token;
+            double dot = 0.0;
+            for (int32_t d = 0; d < head_dim; ++d) dot += bf16_to_f64(qrow[d]) * bf16_to_f64(kj[d]);
+            x[j] = scale * dot;
+            if (x[j] > m) m = x[j];
+        }
+        double l = 0.0;
+        for (int32_t j = 0; j <= p; ++j) {
+            x[j] = exp(x[j] - m);
+            l += x[j];
+        }
+        double *o = out + (slot * num_q_heads + h) * (int64_t)head_dim;
+        for (int32_t d = 0; d < head_dim; ++d) o[d] = 0.0;
+        for (int32_t j = 0; j <= p; ++j) {
+            const uint16_t *vj = v_cache + (int64_t)bt[j / block_size] * v_stride_block
+                                 + (int64_t)g * v_stride_head + (int64_t)(j % block_size) * v_stride_token;
+            for (int32_t d = 0; d < head_dim; ++d) o[d] += x[j] * bf16_to_f64(vj[d]);
+        }
+        for (int32_t d = 0; d < head_dim; ++d) o[d] /= l;
+        if (lse) lse[slot * num_q_heads + h] = m + log(l);
+        if (weights) {
+            double *wr = weights + (slot * num_q_heads + h) * weights_ld;
+            for (int64_t j = 0; j < weights_ld; ++j) wr[j] = (j <= p) ? x[j] / l : 0.0;
+        }
+        free(x);
+    }
+    return bad ? -4 : 0;
+}
+
+/*
+ * Scatter this iteration's new K/V rows into the paged cache: token i of sequence s
+ * goes to position P + i, i.e. page block_table[s][(P+i)/B], slot (P+i)%B
+ * (prefill "materializes" the KV cache, Section 2.1).  Pure byte copy.
+ */
+int cf_oracle_kv_append(
+    uint16_t *k_cache, uint16_t *v_cache,
+    int64_t k_stride_block, int64_t k_stride_head, int64_t k_stride_token,
+    int64_t v_stride_block, int64_t v_stride_head, int64_t v_stride_token,
+    const uint16_t *k_new, const uint16_t *v_new,
+    const int32_t *block_table, int32_t max_blocks_per_seq,
+    const int32_t *context_len, const int32_t *query_len, int32_t num_seqs,
+    int32_t num_kv_heads, int32_t head_dim, int32_t block_size)
+{
+    int64_t row = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        if (query_len[s] < 0 || query_len[s] > context_len[s]) return -2;
+        if ((int64_t)context_len[s] > (int64_t)max_blocks_per_seq * block_size) return -3;
+        const int32_t prefix = context_len[s] - query_len[s];
+        const int32_t *bt = block_table + (int64_t)s * max_blocks_per_seq;
+        for (int32_t i = 0; i < query_len[s]; ++i, ++row) {
+            const int32_t pos = prefix + i;
+            const int64_t blk = bt[pos / block_size];
+            const int64_t slot = pos % block_size;
+            for (int32_t g = 0; g < num_kv_heads; ++g) {
+                const int64_t src = (row * num_kv_heads + g) * (int64_t)head_dim;
+                memcpy(k_cache + blk * k_stride_block + g * k_stride_head + slot * k_stride_token,
+                       k_new + src, sizeof(uint16_t) * (size_t)head_dim);
+                memcpy(v_cache + blk * v_stride_block + g * v_stride_head + slot * v_stride_token,
+                       v_new + src, sizeof(uint16_t) * (size_t)head_dim);
+            }
+        }
+    }
+    return 0;
+}
+
+int cf_oracle_num_threads(void)
+{
+    int n = 1;
+#ifdef _OPENMP
+#pragma omp parallel
+    {
+#pragma omp master
+        n = omp_get_num_threads();
+    }
+#endif
+    return n;
+}

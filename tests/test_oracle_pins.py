@@ -1,0 +1,345 @@
+"""Pins for the CPU oracle: it is checked against things other than itself.
+
+The paper prints no worked attention value (it adds no kernels, Section 5), so the pins are:
+  * brute force: gather K/V into contiguous arrays, build the dense [Lq, Lc] mask, evaluate
+    softmax(QK^T * scale + mask) V with numpy matrices;
+  * a library routine: torch scaled_dot_product_attention in fp64 (with its own GQA head mapping);
+  * closed forms: Lc = 1, q = 0, constant V, V = 1, a dominant key;
+  * invariants: page permutation, chunking, decode == 1-token prefill, GQA == MHA with duplicated
+    KV heads, causal-mask / slack-slot / unassigned-page insensitivity, batch-order permutation.
+"""
+import math
+
+import numpy as np
+import pytest
+import torch
+
+import cf_synth as syn
+import oracle
+
+
+# ------------------------------------------------------------------ independent brute force
+def gather_contiguous(pool, block_row, n_tokens):
+    """[NB, Hkv, B, D] pool -> [Hkv, n_tokens, D] fp64 for one sequence."""
+    NB, H, B, D = pool.shape
+    nb = (n_tokens + B - 1) // B
+    pages = pool[block_row[:nb]]                                  # [nb, H, B, D]
+    flat = pages.transpose(1, 0, 2, 3).reshape(H, nb * B, D)[:, :n_tokens]
+    return syn.bf16_bits_to_f64(flat)
+
+
+def brute_force(batch, k_pool, v_pool, scale=None):
+    g = batch.geom
+    G = g.num_q_heads // g.num_kv_heads
+    scale = 1.0 / math.sqrt(g.head_dim) if scale is None else scale
+    qs = batch.q_start()
+    out = np.zeros((batch.total_q, g.num_q_heads, g.head_dim))
+    lse = np.zeros((batch.total_q, g.num_q_heads))
+    for s in range(batch.num_seqs):
+        Lq, Lc = int(batch.query_len[s]), int(batch.context_len[s])
+        if Lq == 0:
+            continue
+        K = gather_contiguous(k_pool, batch.block_table[s], Lc)
+        V = gather_contiguous(v_pool, batch.block_table[s], Lc)
+        Q = syn.bf16_bits_to_f64(batch.q[qs[s]:qs[s + 1]])          # [Lq, Hq, D]
+        mask = np.arange(Lc)[None, :] > (Lc - Lq + np.arange(Lq))[:, None]
+        for h in range(g.num_q_heads):
+            scores = Q[:, h, :] @ K[h // G].T * scale
+            scores[mask] = -np.inf
+            mx = scores.max(axis=1, keepdims=True)
+            e = np.exp(scores - mx)
+            out[qs[s]:qs[s + 1], h] = (e / e.sum(axis=1, keepdims=True)) @ V[h // G]
+            lse[qs[s]:qs[s + 1], h] = mx[:, 0] + np.log(e.sum(axis=1))
+    return out, lse
+
+
+def run_oracle(batch, k_pool, v_pool, append=True, **kw):
+    k, v = k_pool.copy(), v_pool.copy()
+    if append:
+        oracle.kv_append(k, v, batch.k_new, batch.v_new, batch.block_table, batch.context_len, batch.query_len)
+    return oracle.mixed_attention(batch.q, k, v, batch.block_table, batch.context_len, batch.query_len, **kw), (k, v)
+
+
+def small_scenario(seed, Hq, Hkv, D, prefix, qlens, NB=64, B=16, shuffle=False):
+    geom = syn.Geometry(Hq, Hkv, D, B, NB)
+    return syn.scenario_from_lengths("t", geom, seed, prefix, qlens, shuffle_seqs=shuffle)
+
+
+# ------------------------------------------------------------------ T1 brute force
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (4, 4, 32), (8, 1, 128), (6, 3, 16), (2, 2, 128)])
+def test_oracle_matches_brute_force(Hq, Hkv, D):
+    sc = small_scenario(11 + Hq, Hq, Hkv, D, prefix=[0, 5, 37, 16, 99, 0, 31], qlens=[[1, 1, 23, 16, 1, 40, 1]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    bo, blse = brute_force(b, k, v)
+    assert np.abs(o - bo).max() < 1e-12
+    assert np.abs(lse - blse).max() < 1e-12
+
+
+def test_oracle_matches_brute_force_config1():
+    sc = syn.config1_tiny()
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    bo, blse = brute_force(b, k, v)
+    assert np.abs(o - bo).max() < 1e-12
+    assert np.abs(lse - blse).max() < 1e-12
+    assert np.isfinite(o).all()
+
+
+def test_oracle_custom_scale_matches_brute_force():
+    sc = small_scenario(5, 4, 2, 32, prefix=[10, 3], qlens=[[7, 1]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool, scale=0.37)
+    bo, blse = brute_force(b, k, v, scale=0.37)
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - blse).max() < 1e-12
+
+
+# ------------------------------------------------------------------ T2 library special case
+@pytest.mark.parametrize("Hq,Hkv", [(8, 2), (4, 4), (8, 1)])
+def test_oracle_matches_torch_sdpa_identity_table(Hq, Hkv):
+    D, B, Lq, P = 64, 16, 37, 59
+    Lc = P + Lq
+    nb = (Lc + B - 1) // B
+    geom = syn.Geometry(Hq, Hkv, D, B, nb)
+    rng = np.random.default_rng(77)
+    k_pool, v_pool = syn.empty_pools(geom)
+    ident = np.arange(nb, dtype=np.int32)
+    syn.fill_prefix(rng, geom, k_pool, ident, Lc)
+    syn.fill_prefix(rng, geom, v_pool, ident, Lc)
+    q = syn.normal_bf16(rng, (Lq, Hq, D))
+    o, lse = oracle.mixed_attention(q, k_pool, v_pool, ident[None, :], [Lc], [Lq])
+
+    K = torch.from_numpy(gather_contiguous(k_pool, ident, Lc))[None]     # [1, Hkv, Lc, D]
+    V = torch.from_numpy(gather_contiguous(v_pool, ident, Lc))[None]
+    Q = torch.from_numpy(syn.bf16_bits_to_f64(q)).permute(1, 0, 2)[None]  # [1, Hq, Lq, D]
+    allow = torch.ones(Lq, Lc, dtype=torch.bool).tril(diagonal=P)
+    ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V, attn_mask=allow, enable_gqa=True)
+    ref = ref[0].permute(1, 0, 2).numpy()
+    assert np.abs(o - ref).max() < 1e-12
+
+
+# ------------------------------------------------------------------ T3 closed forms
+def _single_seq(Hq, Hkv, D, Lc, Lq, seed=3, NB=40, B=16):
+    sc = small_scenario(seed, Hq, Hkv, D, prefix=[Lc - Lq], qlens=[[Lq]], NB=NB, B=B)
+    b = sc.batches[0]
+    k, v = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(k, v, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    return b, k, v
+
+
+def test_context_length_one_returns_v0():
+    b, k, v = _single_seq(8, 2, 64, 1, 1)
+    o, lse = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len)
+    v0 = syn.bf16_bits_to_f64(v[b.block_table[0, 0], :, 0, :])            # [Hkv, D]
+    for h in range(8):
+        assert np.array_equal(o[0, h], v0[h // 4])
+    # lse = the single score itself
+    qf = syn.bf16_bits_to_f64(b.q)[0]
+    k0 = syn.bf16_bits_to_f64(k[b.block_table[0, 0], :, 0, :])
+    for h in range(8):
+        assert abs(lse[0, h] - (qf[h] @ k0[h // 4]) / 8.0) < 1e-13
+
+
+def test_zero_query_gives_mean_of_visible_values():
+    b, k, v = _single_seq(4, 2, 32, 45, 13)
+    q0 = np.zeros_like(b.q)
+    o, lse = oracle.mixed_attention(q0, k, v, b.block_table, b.context_len, b.query_len)
+    V = gather_contiguous(v, b.block_table[0], 45)
+    for i in range(13):
+        p = 45 - 13 + i
+        for h in range(4):
+            assert np.abs(o[i, h] - V[h // 2, :p + 1].mean(axis=0)).max() < 1e-13
+            assert abs(lse[i, h] - math.log(p + 1)) < 1e-13
+
+
+def test_equal_keys_give_mean_and_constant_v_is_returned():
+    b, k, v = _single_seq(4, 1, 32, 33, 5)
+    k2 = k.copy()
+    k2[...] = k[b.block_table[0, 0], 0, 0][None, None, None, :]             # every key identical
+    o, _ = oracle.mixed_attention(b.q, k2, v, b.block_table, b.context_len, b.query_len)
+    V = gather_contiguous(v, b.block_table[0], 33)
+    for i in range(5):
+        assert np.abs(o[i, 2] - V[0, :33 - 5 + i + 1].mean(axis=0)).max() < 1e-13
+    v2 = v.copy()
+    v2[...] = syn.f32_to_bf16_bits(np.float32(1.0))
+    o, _ = oracle.mixed_attention(b.q, k, v2, b.block_table, b.context_len, b.query_len)
+    assert np.abs(o - 1.0).max() < 1e-14
+
+
+def test_weights_rows_sum_to_one_and_respect_mask():
+    b, k, v = _single_seq(4, 2, 32, 50, 9)
+    o, lse, w = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, want_weights=50)
+    assert np.abs(w.sum(axis=-1) - 1.0).max() < 1e-14
+    for i in range(9):
+        p = 50 - 9 + i
+        assert (w[i, :, p + 1:] == 0).all() and (w[i, :, :p + 1] > 0).all()
+    # weights reproduce O as a plain weighted sum of gathered V
+    V = gather_contiguous(v, b.block_table[0], 50)
+    ref = np.einsum("ihj,hjd->ihd", w.reshape(9, 2, 2, 50).reshape(9, 4, 50)[:, [0, 1], :], V)  # heads 0,1 -> kv 0
+    assert np.abs(o[:, 0] - w[:, 0] @ V[0]).max() < 1e-13
+    assert np.abs(o[:, 3] - w[:, 3] @ V[1]).max() < 1e-13
+    del ref
+
+
+@pytest.mark.parametrize("jstar", [0, 15, 16, 40, 46])
+def test_dominant_key_selects_its_value(jstar):
+    Lc, Lq, D = 47, 1, 64
+    b, k, v = _single_seq(2, 1, D, Lc, Lq, seed=9)
+    # q = 8 * e_0 ; planted key = 64 * e_0 -> score 8*64/8 = 64 ; other keys have |k_0| <~ 5 -> score <~ 5
+    q = np.zeros_like(b.q)
+    q[0, :, 0] = syn.f32_to_bf16_bits(np.float32(8.0))
+    blk, slot = b.block_table[0, jstar // 16], jstar % 16
+    k[blk, 0, slot, :] = 0
+    k[blk, 0, slot, 0] = syn.f32_to_bf16_bits(np.float32(64.0))
+    o, _ = oracle.mixed_attention(q, k, v, b.block_table, b.context_len, b.query_len)
+    vj = syn.bf16_bits_to_f64(v[blk, 0, slot])
+    assert np.abs(o[0, 0] - vj).max() < 1e-15 * 1e3
+
+
+# ------------------------------------------------------------------ T4 invariants
+def test_page_permutation_leaves_output_bit_identical():
+    sc = small_scenario(21, 8, 2, 64, prefix=[20, 70, 0], qlens=[[1, 30, 17]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    perm = np.random.default_rng(0).permutation(sc.geom.num_blocks)
+    inv = np.empty_like(perm)
+    inv[perm] = np.arange(perm.size)
+    k2, v2 = k[perm], v[perm]                                   # new page i holds old page perm[i]
+    bt2 = np.where(b.block_table >= 0, inv[np.maximum(b.block_table, 0)], -1).astype(np.int32)
+    o2, lse2 = oracle.mixed_attention(b.q, k2, v2, bt2, b.context_len, b.query_len)
+    assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
+
+
+def test_chunking_invariance():
+    """A prompt cut into any bounded units gives the same rows (Section 4.4: units may be paused between)."""
+    Hq, Hkv, D, P, N = 4, 2, 32, 21, 90
+    one = small_scenario(31, Hq, Hkv, D, prefix=[P], qlens=[[N]], NB=16)
+    b1 = one.batches[0]
+    (o1, l1), (kf, vf) = run_oracle(b1, one.k_pool, one.v_pool)
+    for cuts in ([30, 30, 30], [1, 50, 39], [89, 1]):
+        k, v = one.k_pool.copy(), one.v_pool.copy()
+        at, have = 0, P
+        for c in cuts:
+            have += c
+            oracle.kv_append(k, v, b1.k_new[at:at + c], b1.v_new[at:at + c], b1.block_table, [have], [c])
+            o, l = oracle.mixed_attention(b1.q[at:at + c], k, v, b1.block_table, [have], [c])
+            assert np.array_equal(o, o1[at:at + c]) and np.array_equal(l, l1[at:at + c])
+            at += c
+        assert np.array_equal(k, kf) and np.array_equal(v, vf)
+
+
+def test_decode_equals_one_token_prefill_and_batch_order():
+    sc = small_scenario(41, 8, 4, 32, prefix=[12, 0, 33, 64], qlens=[[1, 9, 1, 16]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    qs = b.q_start()
+    order = [2, 0, 3, 1]
+    q2 = np.concatenate([b.q[qs[s]:qs[s + 1]] for s in order])
+    o2, lse2 = oracle.mixed_attention(q2, k, v, b.block_table[order], b.context_len[order], b.query_len[order])
+    at = 0
+    for s in order:
+        n = int(b.query_len[s])
+        assert np.array_equal(o2[at:at + n], o[qs[s]:qs[s + 1]])
+        assert np.array_equal(lse2[at:at + n], lse[qs[s]:qs[s + 1]])
+        at += n
+    # last row of a prefill chunk == the same token issued alone as a decode step
+    s = 3
+    o3, _ = oracle.mixed_attention(b.q[qs[s + 1] - 1:qs[s + 1]], k, v, b.block_table[s:s + 1], b.context_len[s:s + 1], [1])
+    assert np.array_equal(o3[0], o[qs[s + 1] - 1])
+
+
+def test_gqa_equals_mha_with_duplicated_kv_heads():
+    sc = small_scenario(51, 8, 2, 32, prefix=[19, 40], qlens=[[1, 11]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    k8, v8 = np.repeat(k, 4, axis=1), np.repeat(v, 4, axis=1)
+    o8, lse8 = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len)
+    assert np.array_equal(o, o8) and np.array_equal(lse, lse8)
+
+
+def test_invisible_positions_do_not_matter():
+    """Keys after the query position, slack slots of the last page, unassigned pages and the unused
+    tail of the block table may hold anything (NaN included)."""
+    sc = small_scenario(61, 4, 2, 32, prefix=[10, 37], qlens=[[1, 20]], NB=32)
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    assert np.isfinite(o).all()          # pools were NaN-filled outside the visible range already
+    k2, v2 = k.copy(), v.copy()
+    used = set(int(x) for x in b.block_table.ravel() if x >= 0)
+    for blk in range(32):
+        if blk not in used:
+            k2[blk] = 0x7F80             # +inf
+            v2[blk] = 0xFF80
+    # slack slots of the last page of seq 1 (Lc = 57 -> slots 9..15 of page 3)
+    last = b.block_table[1, 3]
+    k2[last, :, 9:, :] = 0x4000
+    v2[last, :, 9:, :] = 0x4000
+    bt2 = b.block_table.copy()
+    bt2[bt2 < 0] = 123456
+    o2, lse2 = oracle.mixed_attention(b.q, k2, v2, bt2, b.context_len, b.query_len)
+    assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
+    # changing keys at positions > p changes only later rows
+    qs = b.q_start()
+    k3 = k.copy()
+    pos = 37 + 10                        # visible to chunk rows i >= 10 only
+    k3[b.block_table[1, pos // 16], :, pos % 16, :] ^= 0x8000
+    o3, _ = oracle.mixed_attention(b.q, k3, v, b.block_table, b.context_len, b.query_len)
+    assert np.array_equal(o3[qs[1]:qs[1] + 10], o[qs[1]:qs[1] + 10])
+    assert not np.array_equal(o3[qs[1] + 10:], o[qs[1] + 10:])
+    assert np.array_equal(o3[:qs[1]], o[:qs[1]])
+
+
+def test_row_subset_matches_full_run():
+    sc = small_scenario(71, 4, 2, 32, prefix=[5, 80, 9], qlens=[[1, 50, 3]])
+    b = sc.batches[0]
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    rows = np.array([0, 1, 17, 50, 51, 53], dtype=np.int64)
+    o2, lse2 = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, rows=rows)
+    assert np.array_equal(o2, o[rows]) and np.array_equal(lse2, lse[rows])
+
+
+# ------------------------------------------------------------------ kv_append against a numpy scatter
+def test_kv_append_matches_python_scatter_and_touches_nothing_else():
+    sc = small_scenario(81, 4, 2, 32, prefix=[0, 15, 16, 37, 5], qlens=[[3, 1, 40, 0, 16]], NB=32)
+    b = sc.batches[0]
+    k, v = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(k, v, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    row = 0
+    for s in range(b.num_seqs):
+        P = int(b.context_len[s] - b.query_len[s])
+        for i in range(int(b.query_len[s])):
+            blk, slot = b.block_table[s, (P + i) // 16], (P + i) % 16
+            k_ref[blk, :, slot, :] = b.k_new[row]
+            v_ref[blk, :, slot, :] = b.v_new[row]
+            row += 1
+    assert np.array_equal(k, k_ref) and np.array_equal(v, v_ref)
+
+
+def test_oracle_rejects_bad_lengths():
+    sc = small_scenario(91, 4, 2, 32, prefix=[5], qlens=[[2]])
+    b = sc.batches[0]
+    with pytest.raises(ValueError):
+        oracle.mixed_attention(b.q, sc.k_pool, sc.v_pool, b.block_table, [1], [2])
+    with pytest.raises(ValueError):
+        oracle.mixed_attention(b.q, sc.k_pool, sc.v_pool, b.block_table[:, :0], [7], [2])
+
+
+# ------------------------------------------------------------------ error model used for the GPU tolerance
+def test_bf16_pipeline_error_is_inside_the_stated_tolerance():
+    """A numpy model of the obvious GPU scheme (fp32 scores, bf16 probabilities, fp32 accumulate, bf16
+    output) stays well inside max-abs 2e-2 / mean-abs 2e-3, so those bounds are attainable."""
+    rng = np.random.default_rng(5)
+    D = 128
+    for Lc in (2, 256, 4096):
+        q = syn.bf16_bits_to_f32(syn.normal_bf16(rng, (8, D)))
+        K = syn.bf16_bits_to_f32(syn.normal_bf16(rng, (Lc, D)))
+        V = syn.bf16_bits_to_f32(syn.normal_bf16(rng, (Lc, D)))
+        s = (q @ K.T) * np.float32(1 / math.sqrt(D))
+        e = np.exp(s - s.max(axis=1, keepdims=True)).astype(np.float32)
+        p16 = syn.bf16_bits_to_f32(syn.f32_to_bf16_bits(e))
+        o = syn.bf16_bits_to_f64(syn.f32_to_bf16_bits(((p16 @ V) / e.sum(axis=1, keepdims=True)).astype(np.float32)))
+        s64 = (q.astype(np.float64) @ K.astype(np.float64).T) / math.sqrt(D)
+        e64 = np.exp(s64 - s64.max(axis=1, keepdims=True))
+        o64 = (e64 / e64.sum(axis=1, keepdims=True)) @ V.astype(np.float64)
+        assert np.abs(o - o64).max() < 2e-2 and np.abs(o - o64).mean() < 2e-3
