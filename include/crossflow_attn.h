@@ -1,0 +1,142 @@
+/*
+ * crossflow_attn — mixed decode + chunked-prefill paged grouped-query attention for one B200.
+ *
+ * The workload is the one a Crossflow decode node produces (arxiv 2609.27085): the worker keeps
+ * a local prefill queue, reuses any resident prefix and "construct[s] a mixed prefill/decode
+ * batch" (Section 5); prefill is issued in bounded units that are revalidated between units
+ * (Section 4.4), so one call here is one unit of one layer: many one-token decode sequences
+ * plus a few prefill chunks, each chunk attending causally to its own new tokens and to an
+ * already-cached prefix.  The paper adds no model kernels (Section 5) and gives no formula;
+ * the arithmetic is textbook softmax attention over a paged KV cache:
+ *
+ *   sequence s, new-token row i in [0, query_len[s]), query head h:
+ *     p = context_len[s] - query_len[s] + i,  g = h / (num_q_heads / num_kv_heads)
+ *     x_j = softmax_scale * <q, k_j>  for j in [0, p],  k_j/v_j at page block_table[s][j / B], slot j % B, head g
+ *     out = sum_j softmax(x)_j * v_j ,  lse = ln sum_j exp(x_j)
+ *
+ * Conventions
+ *   - bf16 storage, fp32 accumulation, one fp32 -> bf16 rounding (nearest even) of the output.
+ *   - context_len[s] counts the visible KV tokens INCLUDING this call's query_len[s] new tokens.
+ *   - Rows of q / k_new / v_new / out are packed in sequence order: sequence s owns rows
+ *     [sum_{t<s} query_len[t], ... + query_len[s]).  Decode (query_len 1) and prefill
+ *     (query_len > 1) sequences may appear in any order; query_len 0 is legal (no rows).
+ *   - Block-table entries past ceil(context_len/B), cache slots past context_len and unassigned
+ *     pages are never read into the result (they may hold NaN).
+ *   - Pointers marked DEVICE must be device memory of the context's GPU and stay alive until the
+ *     stream has finished the enqueued work.  Pointers marked HOST are read before the call returns.
+ *   - All calls on one context must be issued on one stream (or be ordered by the caller): they
+ *     share the context's plan buffers and split-K workspace.
+ *   - Every entry point returns a cf_status; nothing throws.  Argument errors are detected on the
+ *     host BEFORE anything is enqueued.  There is no CPU fallback and no other backend: on a
+ *     device that is not compute capability 10.x cf_create returns CF_ERR_ARCH.
+ */
+#ifndef CROSSFLOW_ATTN_H
+#define CROSSFLOW_ATTN_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct cf_ctx cf_ctx; /* opaque; one per device; owns plan staging and split-K workspace */
+
+typedef enum {
+    CF_OK = 0,
+    CF_ERR_INVALID_ARG = 1,  /* null pointer, negative size, query_len > context_len, ... */
+    CF_ERR_UNSUPPORTED = 2,  /* head_dim / block_size / group size / stride outside the supported set */
+    CF_ERR_OUT_OF_RANGE = 3, /* context_len exceeds max_blocks_per_seq * block_size */
+    CF_ERR_WORKSPACE = 4,    /* fixed-size workspace too small for this batch */
+    CF_ERR_CUDA = 5,         /* a CUDA runtime call or launch failed */
+    CF_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (reported by cf_get_async_status) */
+    CF_ERR_ARCH = 7          /* device is not sm_100 */
+} cf_status;
+
+/* Geometry of the paged cache.  Strides are in ELEMENTS (bf16); head_dim is contiguous.
+ * The recommended layout is [num_blocks, num_kv_heads, block_size, head_dim]
+ * (stride_block = Hkv*B*D, stride_head = B*D, stride_token = D); [num_blocks, block_size,
+ * num_kv_heads, head_dim] is accepted too.  Strides must be multiples of 8 elements (16 bytes).
+ * Supported: head_dim 64 or 128; block_size 16; group size (Hq/Hkv) 1, 2, 4 or 8. */
+typedef struct {
+    int32_t num_q_heads, num_kv_heads, head_dim, block_size, num_blocks;
+    int64_t k_stride_block, k_stride_head, k_stride_token;
+    int64_t v_stride_block, v_stride_head, v_stride_token;
+    float softmax_scale; /* 0 -> 1/sqrt(head_dim) */
+} cf_cache_desc;
+
+/* Create a context on `device`.  workspace_bytes = 0: the split-K workspace starts at a default
+ * size and grows when a batch needs more (growth allocates and synchronises the device);
+ * workspace_bytes > 0: fixed size, a batch that needs more gets CF_ERR_WORKSPACE. */
+cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes);
+cf_status cf_destroy(cf_ctx* ctx);
+
+/* Section 2.1: prefill "materializes" the KV cache; decode appends one token per step.
+ * Copies row r of k_new / v_new (sequence s, new token i) to position P+i of sequence s:
+ * page block_table[s][(P+i)/B], slot (P+i)%B, P = context_len[s]-query_len[s].  Bit-exact byte move.
+ *   k_cache, v_cache : DEVICE, bf16 pools described by desc (written)
+ *   k_new, v_new     : DEVICE, bf16 [T, Hkv, D] contiguous, T = sum(query_len)
+ *   block_table      : DEVICE, int32 [num_seqs, max_blocks_per_seq]
+ *   context_len, query_len : HOST, int32 [num_seqs]
+ *   cuda_stream      : a cudaStream_t (NULL = default stream).  Asynchronous. */
+cf_status cf_kv_append(cf_ctx* ctx, const cf_cache_desc* desc, void* k_cache, void* v_cache,
+                       const void* k_new, const void* v_new,
+                       const int32_t* block_table, int32_t max_blocks_per_seq,
+                       const int32_t* context_len, const int32_t* query_len,
+                       int32_t num_seqs, void* cuda_stream);
+
+/* Section 5 (mixed prefill/decode batch) + Section 4.4 (one bounded unit): attention of every new
+ * token over its sequence's cached prefix and the new tokens up to itself.  Call after
+ * cf_kv_append with the same length arrays.  Launch sequence on the one stream: plan upload ->
+ * split-K decode -> combine -> chunked prefill (decode first, as decode latency is the protected
+ * quantity).  Decode and prefill write disjoint rows of `out`.
+ *   q    : DEVICE, bf16 [T, Hq, D] contiguous
+ *   out  : DEVICE, bf16 [T, Hq, D] contiguous (written)
+ *   lse  : DEVICE, fp32 [T, Hq] natural-log sum-exp of the scaled scores, or NULL
+ *   other arguments as in cf_kv_append (caches are read-only here).  Asynchronous. */
+cf_status cf_mixed_attention(cf_ctx* ctx, const cf_cache_desc* desc, const void* q,
+                             const void* k_cache, const void* v_cache,
+                             const int32_t* block_table, int32_t max_blocks_per_seq,
+                             const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                             void* out, float* lse, void* cuda_stream);
+
+/* One whole unit from HOST buffers: copies q, k_new, v_new (HOST, pinned memory recommended) to
+ * context-owned device staging, runs cf_kv_append + cf_mixed_attention, copies `out` back to
+ * out_host, all on cuda_stream.  The caches and the block table stay DEVICE pointers (they are the
+ * node's resident state).  Asynchronous; out_host is valid after the stream is synchronised. */
+cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
+                             const void* q_host, const void* k_new_host, const void* v_new_host,
+                             void* k_cache, void* v_cache,
+                             const int32_t* block_table, int32_t max_blocks_per_seq,
+                             const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                             void* out_host, void* cuda_stream);
+
+/* After the caller has synchronised the stream: CF_OK, or the first device-side finding
+ * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
+cf_status cf_get_async_status(cf_ctx* ctx);
+
+/* Per-kernel timing for benchmarks.  cf_set_timing(ctx, 1) makes every later cf_mixed_attention
+ * record CUDA events around its kernels; cf_get_last_timing synchronises on the last call's final
+ * event and returns milliseconds (0 for a kernel that was not launched) and the launch count. */
+cf_status cf_set_timing(cf_ctx* ctx, int enabled);
+cf_status cf_get_last_timing(cf_ctx* ctx, float* ms_decode, float* ms_combine, float* ms_prefill,
+                             int32_t* num_launches);
+
+/* Host planner, exposed for inspection and tests (no GPU needed).  Builds the plan that
+ * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.
+ *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}
+ *   combine_items : int32 [cap, 3] = {q_row, first_partial_slot, num_chunks}
+ *   prefill_items : int32 [cap, 4] = {seq, q_row_of_tile, first_row_in_chunk, num_rows}
+ *   counts        : int32 [4]      = {n_decode_items, n_combine_items, n_prefill_items, n_partial_slots}
+ * Any output pointer may be NULL. */
+cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                          int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                          int32_t* decode_items, int32_t* combine_items, int32_t* prefill_items,
+                          int32_t cap, int32_t* counts);
+
+const char* cf_status_string(cf_status s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* CROSSFLOW_ATTN_H */

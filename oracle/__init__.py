@@ -12,6 +12,7 @@ Inputs are numpy arrays; bf16 tensors are ``uint16`` bit patterns.
 from __future__ import annotations
 
 import ctypes
+import hashlib
 import math
 import os
 import subprocess
@@ -21,7 +22,19 @@ import numpy as np
 
 _HERE = os.path.dirname(os.path.abspath(__file__))
 _SRC = os.path.join(_HERE, "cf_oracle.c")
-_LIB = os.path.join(_HERE, "libcf_oracle.so")
+
+
+def _cpu_tag() -> str:
+    """The oracle is compiled -march=native, so the binary is keyed by the host's CPU flags."""
+    try:
+        with open("/proc/cpuinfo") as f:
+            flags = next((ln for ln in f if ln.startswith("flags")), "")
+    except OSError:
+        flags = ""
+    return hashlib.sha1(flags.encode()).hexdigest()[:10]
+
+
+_LIB = os.path.join(_HERE, f"libcf_oracle_{_cpu_tag()}.so")
 _lib = None
 
 

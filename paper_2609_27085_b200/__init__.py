@@ -1,0 +1,199 @@
+"""Thin Python binding of libcrossflow_attn.so (argument marshalling only).
+
+Every step of the path — KV append, split-K decode, combine, chunked prefill, the planner —
+runs inside the CUDA library; this module converts tensors to pointers and checks statuses.
+There is no CPU fallback: if the library is missing, loading raises.
+
+Names mirror the C ABI (``include/crossflow_attn.h``): ``cf_create``, ``cf_kv_append``,
+``cf_mixed_attention``, ``cf_mixed_step_host``, ``cf_get_async_status``, ``cf_set_timing``,
+``cf_get_last_timing``, ``cf_plan_inspect``, ``cf_status_string``.
+
+Device arguments may be torch tensors (their ``data_ptr()`` is used) or integer addresses; the
+length arrays are host ``int32`` numpy arrays (anything array-like is converted).
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libcrossflow_attn.so")
+
+CF_OK = 0
+CF_ERR_INVALID_ARG = 1
+CF_ERR_UNSUPPORTED = 2
+CF_ERR_OUT_OF_RANGE = 3
+CF_ERR_WORKSPACE = 4
+CF_ERR_CUDA = 5
+CF_ERR_TIMEOUT = 6
+CF_ERR_ARCH = 7
+
+EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host",
+           "cf_get_async_status", "cf_set_timing", "cf_get_last_timing", "cf_plan_inspect", "cf_status_string")
+
+
+class CacheDesc(ctypes.Structure):
+    """Mirror of ``cf_cache_desc``."""
+    _fields_ = [("num_q_heads", ctypes.c_int32), ("num_kv_heads", ctypes.c_int32), ("head_dim", ctypes.c_int32),
+                ("block_size", ctypes.c_int32), ("num_blocks", ctypes.c_int32),
+                ("k_stride_block", ctypes.c_int64), ("k_stride_head", ctypes.c_int64), ("k_stride_token", ctypes.c_int64),
+                ("v_stride_block", ctypes.c_int64), ("v_stride_head", ctypes.c_int64), ("v_stride_token", ctypes.c_int64),
+                ("softmax_scale", ctypes.c_float)]
+
+
+class CfError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        super().__init__(f"{where}: {cf_status_string(status)} ({status})")
+
+
+_lib = None
+
+
+def load_library() -> ctypes.CDLL:
+    """Loads the C-ABI library; raises if it has not been built (no fallback of any kind)."""
+    global _lib
+    if _lib is not None:
+        return _lib
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(f"{LIB_PATH} is missing: build it with `python -m paper_2609_27085_b200.build`")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i32, i32p, fp = ctypes.c_void_p, ctypes.c_int32, ctypes.POINTER(ctypes.c_int32), ctypes.POINTER(ctypes.c_float)
+    dp = ctypes.POINTER(CacheDesc)
+    lib.cf_create.argtypes = [ctypes.POINTER(vp), ctypes.c_int, ctypes.c_size_t]
+    lib.cf_destroy.argtypes = [vp]
+    lib.cf_kv_append.argtypes = [vp, dp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp]
+    lib.cf_mixed_attention.argtypes = [vp, dp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
+    lib.cf_mixed_step_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp]
+    lib.cf_get_async_status.argtypes = [vp]
+    lib.cf_set_timing.argtypes = [vp, ctypes.c_int]
+    lib.cf_get_last_timing.argtypes = [vp, fp, fp, fp, i32p]
+    lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
+    lib.cf_status_string.argtypes = [ctypes.c_int]
+    lib.cf_status_string.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name != "cf_status_string":
+            getattr(lib, name).restype = ctypes.c_int
+    _lib = lib
+    return lib
+
+
+def cf_status_string(status: int) -> str:
+    return load_library().cf_status_string(int(status)).decode()
+
+
+def _check(status: int, where: str) -> None:
+    if status != CF_OK:
+        raise CfError(status, where)
+
+
+def _dev(x) -> Optional[int]:
+    """Device address of a torch tensor, or an integer address, or None."""
+    if x is None:
+        return None
+    if hasattr(x, "data_ptr"):
+        return int(x.data_ptr())
+    return int(x)
+
+
+def _host_i32(x) -> np.ndarray:
+    return np.ascontiguousarray(x, dtype=np.int32)
+
+
+def _stream(stream) -> Optional[int]:
+    if stream is None:
+        return None
+    return int(getattr(stream, "cuda_stream", stream)) or None
+
+
+def make_desc(num_q_heads: int, num_kv_heads: int, head_dim: int, block_size: int, num_blocks: int,
+              k_strides: Optional[Tuple[int, int, int]] = None, v_strides: Optional[Tuple[int, int, int]] = None,
+              softmax_scale: float = 0.0) -> CacheDesc:
+    """Descriptor for pools laid out [num_blocks, num_kv_heads, block_size, head_dim] unless
+    (block, head, token) element strides are given."""
+    default = (num_kv_heads * block_size * head_dim, block_size * head_dim, head_dim)
+    ks = k_strides or default
+    vs = v_strides or default
+    return CacheDesc(num_q_heads, num_kv_heads, head_dim, block_size, num_blocks,
+                     ks[0], ks[1], ks[2], vs[0], vs[1], vs[2], softmax_scale)
+
+
+def cf_create(device: int = 0, workspace_bytes: int = 0) -> ctypes.c_void_p:
+    lib = load_library()
+    ctx = ctypes.c_void_p()
+    _check(lib.cf_create(ctypes.byref(ctx), int(device), int(workspace_bytes)), "cf_create")
+    return ctx
+
+
+def cf_destroy(ctx) -> None:
+    _check(load_library().cf_destroy(ctx), "cf_destroy")
+
+
+def cf_kv_append(ctx, desc: CacheDesc, k_cache, v_cache, k_new, v_new, block_table, max_blocks_per_seq: int,
+                 context_len, query_len, stream=None, check: bool = True) -> int:
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    st = load_library().cf_kv_append(ctx, ctypes.byref(desc), _dev(k_cache), _dev(v_cache), _dev(k_new), _dev(v_new),
+                                     _dev(block_table), int(max_blocks_per_seq), lc.ctypes.data, lq.ctypes.data,
+                                     int(lc.shape[0]), _stream(stream))
+    if check:
+        _check(st, "cf_kv_append")
+    return st
+
+
+def cf_mixed_attention(ctx, desc: CacheDesc, q, k_cache, v_cache, block_table, max_blocks_per_seq: int,
+                       context_len, query_len, out, lse=None, stream=None, check: bool = True) -> int:
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    st = load_library().cf_mixed_attention(ctx, ctypes.byref(desc), _dev(q), _dev(k_cache), _dev(v_cache),
+                                           _dev(block_table), int(max_blocks_per_seq), lc.ctypes.data, lq.ctypes.data,
+                                           int(lc.shape[0]), _dev(out), _dev(lse), _stream(stream))
+    if check:
+        _check(st, "cf_mixed_attention")
+    return st
+
+
+def cf_mixed_step_host(ctx, desc: CacheDesc, q_host, k_new_host, v_new_host, k_cache, v_cache, block_table,
+                       max_blocks_per_seq: int, context_len, query_len, out_host, stream=None, check: bool = True) -> int:
+    """q_host / k_new_host / v_new_host / out_host: host tensors (pinned recommended) or addresses."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    st = load_library().cf_mixed_step_host(ctx, ctypes.byref(desc), _dev(q_host), _dev(k_new_host), _dev(v_new_host),
+                                           _dev(k_cache), _dev(v_cache), _dev(block_table), int(max_blocks_per_seq),
+                                           lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]), _dev(out_host),
+                                           _stream(stream))
+    if check:
+        _check(st, "cf_mixed_step_host")
+    return st
+
+
+def cf_get_async_status(ctx) -> int:
+    return int(load_library().cf_get_async_status(ctx))
+
+
+def cf_set_timing(ctx, enabled: bool) -> None:
+    _check(load_library().cf_set_timing(ctx, int(bool(enabled))), "cf_set_timing")
+
+
+def cf_get_last_timing(ctx) -> Tuple[float, float, float, int]:
+    """(ms_decode, ms_combine, ms_prefill, num_launches) of the last cf_mixed_attention."""
+    a, b, c, n = ctypes.c_float(), ctypes.c_float(), ctypes.c_float(), ctypes.c_int32()
+    _check(load_library().cf_get_last_timing(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
+           "cf_get_last_timing")
+    return a.value, b.value, c.value, n.value
+
+
+def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148,
+                    cap: int = 1 << 16, check: bool = True):
+    """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,4], n_partial_slots)."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    dec = np.zeros((cap, 6), dtype=np.int32)
+    comb = np.zeros((cap, 3), dtype=np.int32)
+    pre = np.zeros((cap, 4), dtype=np.int32)
+    counts = np.zeros(4, dtype=np.int32)
+    st = load_library().cf_plan_inspect(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
+                                        int(max_blocks_per_seq), int(num_sms), dec.ctypes.data, comb.ctypes.data,
+                                        pre.ctypes.data, cap, counts.ctypes.data)
+    if check:
+        _check(st, "cf_plan_inspect")
+    return st, dec[:counts[0]], comb[:counts[1]], pre[:counts[2]], int(counts[3])

@@ -1,0 +1,485 @@
+// C ABI of the library: context, plan upload and the launch sequence.
+// See include/crossflow_attn.h for the contract of every entry point.
+#include <cmath>
+#include <cstdio>
+#include <cstdlib>
+#include <cstring>
+#include <new>
+
+#include "../../include/crossflow_attn.h"
+#include "kernels.h"
+#include "plan.h"
+
+namespace cf {
+
+static constexpr int kRing = 4;                         // plan slots in flight
+static constexpr size_t kDefaultWorkspace = 64u << 20;  // split-K partials
+static constexpr size_t kDefaultPlanBytes = 1u << 20;
+
+struct PlanSlot {
+    uint8_t* host = nullptr;   // pinned
+    uint8_t* dev = nullptr;
+    cudaEvent_t done = nullptr;
+    bool used = false;
+};
+
+}  // namespace cf
+
+struct cf_ctx {
+    int device = 0;
+    int num_sms = 0;
+    cf::PlanConfig cfg;
+    cf::PlanSlot slots[cf::kRing];
+    size_t plan_bytes = 0;
+    int next_slot = 0;
+    float* workspace = nullptr;
+    size_t workspace_bytes = 0;
+    bool workspace_fixed = false;
+    uint32_t* err_dev = nullptr;
+    // host-staged step
+    uint8_t* stage_dev = nullptr;
+    size_t stage_bytes = 0;
+    // timing
+    bool timing = false;
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ev_valid = false;
+    bool ran[3] = {false, false, false};
+    int launches = 0;
+};
+
+namespace cf {
+
+static int env_int(const char* name, int fallback)
+{
+    const char* v = std::getenv(name);
+    if (!v || !*v) return fallback;
+    char* end = nullptr;
+    long x = std::strtol(v, &end, 10);
+    return (end && *end == 0 && x > 0 && x < (1 << 20)) ? (int)x : fallback;
+}
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = false;
+    explicit DeviceGuard(int dev)
+    {
+        if (cudaGetDevice(&prev) != cudaSuccess) return;
+        ok = (prev == dev) || cudaSetDevice(dev) == cudaSuccess;
+    }
+    ~DeviceGuard()
+    {
+        if (ok && prev >= 0) cudaSetDevice(prev);
+    }
+};
+
+static size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+static cf_status ensure_plan_capacity(cf_ctx* c, size_t need)
+{
+    if (need <= c->plan_bytes) return CF_OK;
+    size_t nb = c->plan_bytes ? c->plan_bytes : kDefaultPlanBytes;
+    while (nb < need) nb *= 2;
+    if (cudaDeviceSynchronize() != cudaSuccess) return CF_ERR_CUDA;
+    for (int i = 0; i < kRing; ++i) {
+        PlanSlot& s = c->slots[i];
+        if (s.host) cudaFreeHost(s.host);
+        if (s.dev) cudaFree(s.dev);
+        s.host = s.dev = nullptr;
+        s.used = false;
+        if (cudaMallocHost((void**)&s.host, nb) != cudaSuccess) return CF_ERR_CUDA;
+        if (cudaMalloc((void**)&s.dev, nb) != cudaSuccess) return CF_ERR_CUDA;
+    }
+    c->plan_bytes = nb;
+    return CF_OK;
+}
+
+static cf_status ensure_workspace(cf_ctx* c, size_t need)
+{
+    if (need <= c->workspace_bytes) return CF_OK;
+    if (c->workspace_fixed) return CF_ERR_WORKSPACE;
+    if (cudaDeviceSynchronize() != cudaSuccess) return CF_ERR_CUDA;
+    if (c->workspace) cudaFree(c->workspace);
+    c->workspace = nullptr;
+    c->workspace_bytes = 0;
+    size_t nb = align_up(need + need / 4, 1u << 20);
+    if (cudaMalloc((void**)&c->workspace, nb) != cudaSuccess) return CF_ERR_CUDA;
+    c->workspace_bytes = nb;
+    return CF_OK;
+}
+
+// Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
+struct PlanLayout {
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, total;
+};
+
+static PlanLayout layout_of(int32_t S, const Plan& pl)
+{
+    PlanLayout L;
+    size_t at = 0;
+    L.off_qstart = at; at = align_up(at + sizeof(int32_t) * ((size_t)S + 1), 16);
+    L.off_ctx = at;    at = align_up(at + sizeof(int32_t) * (size_t)S, 16);
+    L.off_qlen = at;   at = align_up(at + sizeof(int32_t) * (size_t)S, 16);
+    L.off_dec = at;    at = align_up(at + sizeof(DecodeItem) * pl.decode.size(), 16);
+    L.off_comb = at;   at = align_up(at + sizeof(CombineItem) * pl.combine.size(), 16);
+    L.off_pre = at;    at = align_up(at + sizeof(PrefillItem) * pl.prefill.size(), 16);
+    L.total = at ? at : 16;
+    return L;
+}
+
+// Copies the plan into the next pinned slot and enqueues its upload.  Returns the device base.
+static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, const int32_t* query_len,
+                             const Plan& pl, cudaStream_t stream, PlanLayout* L, uint8_t** dev_base, PlanSlot** slot_out)
+{
+    *L = layout_of(S, pl);
+    cf_status st = ensure_plan_capacity(c, L->total);
+    if (st != CF_OK) return st;
+    PlanSlot& s = c->slots[c->next_slot];
+    c->next_slot = (c->next_slot + 1) % kRing;
+    if (s.used && cudaEventSynchronize(s.done) != cudaSuccess) return CF_ERR_CUDA;   // slot still in flight
+    std::memcpy(s.host + L->off_qstart, pl.q_start.data(), sizeof(int32_t) * ((size_t)S + 1));
+    if (S > 0) {
+        std::memcpy(s.host + L->off_ctx, context_len, sizeof(int32_t) * (size_t)S);
+        std::memcpy(s.host + L->off_qlen, query_len, sizeof(int32_t) * (size_t)S);
+    }
+    if (!pl.decode.empty()) std::memcpy(s.host + L->off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
+    if (!pl.combine.empty()) std::memcpy(s.host + L->off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
+    if (!pl.prefill.empty()) std::memcpy(s.host + L->off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
+    if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    *dev_base = s.dev;
+    *slot_out = &s;
+    return CF_OK;
+}
+
+static cf_status finish_slot(PlanSlot* s, cudaStream_t stream)
+{
+    if (cudaEventRecord(s->done, stream) != cudaSuccess) return CF_ERR_CUDA;
+    s->used = true;
+    return CF_OK;
+}
+
+static float scale_log2_of(const cf_cache_desc* d)
+{
+    const float sc = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / std::sqrt((float)d->head_dim);
+    return sc * 1.4426950408889634f;
+}
+
+}  // namespace cf
+
+using namespace cf;
+
+extern "C" {
+
+const char* cf_status_string(cf_status s)
+{
+    switch (s) {
+        case CF_OK: return "CF_OK";
+        case CF_ERR_INVALID_ARG: return "CF_ERR_INVALID_ARG";
+        case CF_ERR_UNSUPPORTED: return "CF_ERR_UNSUPPORTED";
+        case CF_ERR_OUT_OF_RANGE: return "CF_ERR_OUT_OF_RANGE";
+        case CF_ERR_WORKSPACE: return "CF_ERR_WORKSPACE";
+        case CF_ERR_CUDA: return "CF_ERR_CUDA";
+        case CF_ERR_TIMEOUT: return "CF_ERR_TIMEOUT";
+        case CF_ERR_ARCH: return "CF_ERR_ARCH";
+    }
+    return "CF_ERR_UNKNOWN";
+}
+
+cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
+{
+    if (!out) return CF_ERR_INVALID_ARG;
+    *out = nullptr;
+    int count = 0;
+    if (cudaGetDeviceCount(&count) != cudaSuccess || device < 0 || device >= count) {
+        cudaGetLastError();
+        return count == 0 ? CF_ERR_CUDA : CF_ERR_INVALID_ARG;
+    }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, device) != cudaSuccess) return CF_ERR_CUDA;
+    if (prop.major != 10) return CF_ERR_ARCH;
+    DeviceGuard guard(device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cf_ctx* c = new (std::nothrow) cf_ctx();
+    if (!c) return CF_ERR_CUDA;
+    c->device = device;
+    c->num_sms = prop.multiProcessorCount;
+    c->cfg.num_sms = c->num_sms;
+    c->cfg.decode_waves = env_int("CF_DECODE_WAVES", c->cfg.decode_waves);
+    c->cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", c->cfg.decode_min_chunk_pages);
+    c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    bool ok = true;
+    for (int i = 0; i < kRing && ok; ++i)
+        ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
+    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
+    ok = ok && ensure_plan_capacity(c, kDefaultPlanBytes) == CF_OK;
+    c->workspace_fixed = false;
+    ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
+    c->workspace_fixed = workspace_bytes != 0;
+    ok = ok && cudaMalloc((void**)&c->err_dev, sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(c->err_dev, 0, sizeof(uint32_t)) == cudaSuccess;
+    if (!ok) {
+        cf_destroy(c);
+        return CF_ERR_CUDA;
+    }
+    *out = c;
+    return CF_OK;
+}
+
+cf_status cf_destroy(cf_ctx* c)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    cudaDeviceSynchronize();
+    for (int i = 0; i < kRing; ++i) {
+        if (c->slots[i].host) cudaFreeHost(c->slots[i].host);
+        if (c->slots[i].dev) cudaFree(c->slots[i].dev);
+        if (c->slots[i].done) cudaEventDestroy(c->slots[i].done);
+    }
+    for (int i = 0; i < 4; ++i)
+        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    if (c->workspace) cudaFree(c->workspace);
+    if (c->err_dev) cudaFree(c->err_dev);
+    if (c->stage_dev) cudaFree(c->stage_dev);
+    delete c;
+    return CF_OK;
+}
+
+cf_status cf_kv_append(cf_ctx* c, const cf_cache_desc* desc, void* k_cache, void* v_cache,
+                       const void* k_new, const void* v_new,
+                       const int32_t* block_table, int32_t max_blocks_per_seq,
+                       const int32_t* context_len, const int32_t* query_len,
+                       int32_t num_seqs, void* cuda_stream)
+{
+    if (!c || !desc) return CF_ERR_INVALID_ARG;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    Plan pl;
+    st = validate_lengths(desc, context_len, query_len, num_seqs, max_blocks_per_seq, &pl);
+    if (st != CF_OK) return st;
+    if (pl.total_q == 0) return CF_OK;
+    if (!k_cache || !v_cache || !k_new || !v_new || !block_table) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    PlanLayout L;
+    uint8_t* base = nullptr;
+    PlanSlot* slot = nullptr;
+    st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
+    if (st != CF_OK) return st;
+    AppendParams p;
+    p.k_cache = (__nv_bfloat16*)k_cache;
+    p.v_cache = (__nv_bfloat16*)v_cache;
+    p.k_new = (const __nv_bfloat16*)k_new;
+    p.v_new = (const __nv_bfloat16*)v_new;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks_per_seq;
+    p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
+    p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
+    p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = num_seqs; p.total_rows = pl.total_q;
+    p.q_start = (const int32_t*)(base + L.off_qstart);
+    p.context_len = (const int32_t*)(base + L.off_ctx);
+    p.query_len = (const int32_t*)(base + L.off_qlen);
+    const cudaError_t e = launch_kv_append(p, stream);
+    const cf_status fs = finish_slot(slot, stream);
+    if (e != cudaSuccess) return CF_ERR_CUDA;
+    return fs;
+}
+
+cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q,
+                             const void* k_cache, const void* v_cache,
+                             const int32_t* block_table, int32_t max_blocks_per_seq,
+                             const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                             void* out, float* lse, void* cuda_stream)
+{
+    if (!c || !desc) return CF_ERR_INVALID_ARG;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    Plan pl;
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, c->cfg, &pl);
+    if (st != CF_OK) return st;
+    c->ev_valid = false;
+    c->launches = 0;
+    if (pl.total_q == 0) return CF_OK;
+    if (!q || !k_cache || !v_cache || !block_table || !out) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+
+    const int Hq = desc->num_q_heads, D = desc->head_dim;
+    const size_t part_o_bytes = align_up((size_t)pl.n_part_slots * Hq * D * sizeof(float), 256);
+    const size_t part_ml_bytes = align_up((size_t)pl.n_part_slots * Hq * 2 * sizeof(float), 256);
+    st = ensure_workspace(c, part_o_bytes + part_ml_bytes);
+    if (st != CF_OK) return st;
+
+    PlanLayout L;
+    uint8_t* base = nullptr;
+    PlanSlot* slot = nullptr;
+    st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
+    if (st != CF_OK) return st;
+
+    AttnParams p;
+    p.q = (const __nv_bfloat16*)q;
+    p.k_cache = (const __nv_bfloat16*)k_cache;
+    p.v_cache = (const __nv_bfloat16*)v_cache;
+    p.out = (__nv_bfloat16*)out;
+    p.lse = lse;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks_per_seq;
+    p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
+    p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
+    p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
+    p.scale_log2 = scale_log2_of(desc);
+    p.q_start = (const int32_t*)(base + L.off_qstart);
+    p.context_len = (const int32_t*)(base + L.off_ctx);
+    p.query_len = (const int32_t*)(base + L.off_qlen);
+    p.dec_items = (const DecodeItem*)(base + L.off_dec);
+    p.comb_items = (const CombineItem*)(base + L.off_comb);
+    p.pre_items = (const PrefillItem*)(base + L.off_pre);
+    p.part_o = c->workspace;
+    p.part_ml = (float*)((uint8_t*)c->workspace + part_o_bytes);
+    p.err = c->err_dev;
+
+    cudaError_t e = cudaSuccess;
+    const bool t = c->timing;
+    c->ran[0] = !pl.decode.empty();
+    c->ran[1] = !pl.combine.empty();
+    c->ran[2] = !pl.prefill.empty();
+    if (t) cudaEventRecord(c->ev[0], stream);
+    if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
+    if (t) cudaEventRecord(c->ev[1], stream);
+    if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
+    if (t) cudaEventRecord(c->ev[2], stream);
+    if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
+    if (t) cudaEventRecord(c->ev[3], stream);
+    c->ev_valid = t;
+    c->launches = (int)c->ran[0] + (int)c->ran[1] + (int)c->ran[2];
+    const cf_status fs = finish_slot(slot, stream);
+    if (e != cudaSuccess) return CF_ERR_CUDA;
+    return fs;
+}
+
+cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
+                             const void* q_host, const void* k_new_host, const void* v_new_host,
+                             void* k_cache, void* v_cache,
+                             const int32_t* block_table, int32_t max_blocks_per_seq,
+                             const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                             void* out_host, void* cuda_stream)
+{
+    if (!c || !desc) return CF_ERR_INVALID_ARG;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    Plan pl;
+    st = validate_lengths(desc, context_len, query_len, num_seqs, max_blocks_per_seq, &pl);
+    if (st != CF_OK) return st;
+    if (pl.total_q == 0) return CF_OK;
+    if (!q_host || !k_new_host || !v_new_host || !out_host) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    const size_t T = (size_t)pl.total_q;
+    const size_t q_bytes = align_up(T * desc->num_q_heads * desc->head_dim * 2, 256);
+    const size_t kv_bytes = align_up(T * desc->num_kv_heads * desc->head_dim * 2, 256);
+    const size_t need = 2 * q_bytes + 2 * kv_bytes;
+    if (need > c->stage_bytes) {
+        if (cudaDeviceSynchronize() != cudaSuccess) return CF_ERR_CUDA;
+        if (c->stage_dev) cudaFree(c->stage_dev);
+        c->stage_dev = nullptr;
+        c->stage_bytes = 0;
+        if (cudaMalloc((void**)&c->stage_dev, need) != cudaSuccess) return CF_ERR_CUDA;
+        c->stage_bytes = need;
+    }
+    uint8_t* dq = c->stage_dev;
+    uint8_t* dk = dq + q_bytes;
+    uint8_t* dv = dk + kv_bytes;
+    uint8_t* dout = dv + kv_bytes;
+    const size_t qb = T * desc->num_q_heads * desc->head_dim * 2, kb = T * desc->num_kv_heads * desc->head_dim * 2;
+    if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    st = cf_kv_append(c, desc, k_cache, v_cache, dk, dv, block_table, max_blocks_per_seq, context_len, query_len,
+                      num_seqs, cuda_stream);
+    if (st != CF_OK) return st;
+    st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
+                            num_seqs, dout, nullptr, cuda_stream);
+    if (st != CF_OK) return st;
+    if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return CF_ERR_CUDA;
+    return CF_OK;
+}
+
+cf_status cf_get_async_status(cf_ctx* c)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    uint32_t w = 0;
+    if (cudaMemcpy(&w, c->err_dev, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess) return CF_ERR_CUDA;
+    if (w == 0) return CF_OK;
+    cudaMemset(c->err_dev, 0, sizeof w);
+    return CF_ERR_TIMEOUT;
+}
+
+cf_status cf_set_timing(cf_ctx* c, int enabled)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    c->timing = enabled != 0;
+    c->ev_valid = false;
+    return CF_OK;
+}
+
+cf_status cf_get_last_timing(cf_ctx* c, float* ms_decode, float* ms_combine, float* ms_prefill, int32_t* num_launches)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    float t[3] = {0.f, 0.f, 0.f};
+    if (c->ev_valid) {
+        DeviceGuard guard(c->device);
+        if (cudaEventSynchronize(c->ev[3]) != cudaSuccess) return CF_ERR_CUDA;
+        for (int i = 0; i < 3; ++i)
+            if (c->ran[i] && cudaEventElapsedTime(&t[i], c->ev[i], c->ev[i + 1]) != cudaSuccess) return CF_ERR_CUDA;
+    }
+    if (ms_decode) *ms_decode = t[0];
+    if (ms_combine) *ms_combine = t[1];
+    if (ms_prefill) *ms_prefill = t[2];
+    if (num_launches) *num_launches = c->launches;
+    return CF_OK;
+}
+
+cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                          int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                          int32_t* decode_items, int32_t* combine_items, int32_t* prefill_items,
+                          int32_t cap, int32_t* counts)
+{
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    PlanConfig cfg;
+    cfg.num_sms = num_sms > 0 ? num_sms : 148;
+    cfg.decode_waves = env_int("CF_DECODE_WAVES", cfg.decode_waves);
+    cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
+    cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    Plan pl;
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
+    if (st != CF_OK) return st;
+    if (cap < 0) cap = 0;
+    if (decode_items)
+        for (size_t i = 0; i < pl.decode.size() && i < (size_t)cap; ++i) {
+            const DecodeItem& d = pl.decode[i];
+            int32_t* o = decode_items + 6 * i;
+            o[0] = d.seq; o[1] = d.q_row; o[2] = d.kv_begin; o[3] = d.kv_end; o[4] = d.part_slot; o[5] = d.chunk;
+        }
+    if (combine_items)
+        for (size_t i = 0; i < pl.combine.size() && i < (size_t)cap; ++i) {
+            int32_t* o = combine_items + 3 * i;
+            o[0] = pl.combine[i].q_row; o[1] = pl.combine[i].part_first; o[2] = pl.combine[i].n_chunks;
+        }
+    if (prefill_items)
+        for (size_t i = 0; i < pl.prefill.size() && i < (size_t)cap; ++i) {
+            int32_t* o = prefill_items + 4 * i;
+            o[0] = pl.prefill[i].seq; o[1] = pl.prefill[i].q_row0; o[2] = pl.prefill[i].row0; o[3] = pl.prefill[i].n_rows;
+        }
+    if (counts) {
+        counts[0] = (int32_t)pl.decode.size();
+        counts[1] = (int32_t)pl.combine.size();
+        counts[2] = (int32_t)pl.prefill.size();
+        counts[3] = pl.n_part_slots;
+    }
+    return CF_OK;
+}
+
+}  // extern "C"

@@ -1,0 +1,292 @@
+// Split-K decode attention over the paged KV cache (HBM-bound).
+//
+// One CTA serves one (decode sequence, KV chunk, KV head).  The G query heads that share the KV
+// head ride along as the N dimension of the tensor-core tiles, so every K/V byte is read from HBM
+// exactly once.  Each warp walks its own pages (page = 16 tokens) through a private cp.async ring;
+// there is no block-wide barrier in the main loop.
+//
+// Orientation.  With only G <= 8 query rows, the usual S = Q K^T wastes the 16-row MMA tile.  The
+// kernel computes the transposes instead:
+//     S^T[token, head] = K[token, :] . Q[head, :]        A = K page (16 x D),   B = Q^T (D x 8)
+//     O^T[d, head]    += V^T[d, token] . P^T[token, head] A = V^T via ldmatrix.trans, B = P^T
+// so one m16n8k16 covers a whole page against all (up to 8) heads with no padding rows, and the
+// probabilities move from accumulator layout to B-operand layout with one movmatrix per 8 tokens.
+// Softmax runs per head (a column of S^T): running max in the log2 domain, un-normalised sums.
+//
+// Output: a sequence with a single chunk writes bf16 `out` (and lse) directly; otherwise the CTA
+// writes an fp32 partial (o, m, l) that the combine kernel merges in fixed chunk order.
+#include "device_common.cuh"
+#include "kernels.h"
+
+namespace cf {
+
+template <int D, int NWARPS, int NSTAGE>
+__global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const AttnParams p)
+{
+    constexpr int CPR = D / 8;                  // 16-byte chunks per token row
+    constexpr int PAGE_BYTES = 16 * D * 2;      // one (page, head) of K or of V
+    constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+    constexpr int WARP_BYTES = NSTAGE * STAGE_BYTES;
+    constexpr int KSTEPS = D / 16;
+    constexpr int DP = D + 4;                   // padded row of the merge buffer (bank-conflict free)
+    extern __shared__ __align__(1024) uint8_t smem[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const DecodeItem it = p.dec_items[item_id];
+    const int G = p.G;
+
+    // ---- Q^T fragments (B operand): thread holds Q[head = lane/4][d = 16*ks + 2*(lane%4) + {0,1} (+8)]
+    uint32_t qf[KSTEPS][2];
+    {
+        const int head = lane >> 2;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(
+            p.q + ((int64_t)it.q_row * p.Hq + (int64_t)kvh * G + head) * D);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            qf[ks][0] = head < G ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+            qf[ks][1] = head < G ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+        }
+    }
+
+    const int first_page = it.kv_begin >> 4;
+    const int n_pages = (it.kv_end - it.kv_begin + 15) >> 4;
+    const int my_n = n_pages > warp ? (n_pages - warp + NWARPS - 1) / NWARPS : 0;
+    const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks + first_page + warp;
+    const uint32_t wbase = smem_u32(smem) + warp * WARP_BYTES;
+    const __nv_bfloat16* kbase = p.k_cache + (int64_t)kvh * p.ks_head;
+    const __nv_bfloat16* vbase = p.v_cache + (int64_t)kvh * p.vs_head;
+
+    int cache_base = 0;
+    int32_t pid_cache = (lane < my_n) ? __ldg(bt + lane * NWARPS) : 0;
+
+    auto issue = [&](int i) {
+        if (i - cache_base == 32) {             // refill the per-lane page-id cache
+            cache_base = i;
+            pid_cache = (i + lane < my_n) ? __ldg(bt + (i + lane) * NWARPS) : 0;
+        }
+        const int32_t pid = __shfl_sync(0xffffffffu, pid_cache, i - cache_base);
+        const int tok0 = it.kv_begin + (i * NWARPS + warp) * 16;
+        const uint32_t sbase = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const __nv_bfloat16* kp = kbase + (int64_t)pid * p.ks_block;
+        const __nv_bfloat16* vp = vbase + (int64_t)pid * p.vs_block;
+#pragma unroll
+        for (int r = 0; r < (16 * CPR) / 32; ++r) {
+            const int id = r * 32 + lane;
+            const int t = id / CPR, c = id % CPR;
+            const bool ok = tok0 + t < it.kv_end;     // slack slots of the last page are zero-filled
+            const int tt = ok ? t : 0;
+            cp_async16(sbase + tile_off<16>(t, c), kp + tt * p.ks_token + c * 8, ok ? 16 : 0);
+            cp_async16(sbase + PAGE_BYTES + tile_off<16>(t, c), vp + tt * p.vs_token + c * 8, ok ? 16 : 0);
+        }
+    };
+
+    float o[KSTEPS][4];
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (s < my_n) issue(s);
+        cp_async_commit();
+    }
+
+    for (int i = 0; i < my_n; ++i) {
+        cp_async_wait<NSTAGE - 2>();
+        __syncwarp();
+        if (i + NSTAGE - 1 < my_n) issue(i + NSTAGE - 1);
+        cp_async_commit();
+
+        const uint32_t sK = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const uint32_t sV = sK + PAGE_BYTES;
+        const int tok0 = it.kv_begin + (i * NWARPS + warp) * 16;
+
+        // S^T = K Q^T ; two accumulators break the dependent MMA chain
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+        {
+            const int t = (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                uint32_t a[4];
+                ldmatrix_x4(a, sK + tile_off<16>(t, 2 * ks + (lane >> 4)));
+                if (ks & 1) mma_bf16_16816(s1, a, qf[ks][0], qf[ks][1]);
+                else        mma_bf16_16816(s0, a, qf[ks][0], qf[ks][1]);
+            }
+        }
+        float s[4];
+        const int tA = tok0 + (lane >> 2);
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const bool ok = (tA + (e >> 1) * 8) < it.kv_end;
+            s[e] = ok ? (s0[e] + s1[e]) * p.scale_log2 : -INFINITY;
+        }
+        // per-head (column) max over the 16 tokens of the page: 2 local rows, 8 lane groups
+        float alpha[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float mx = fmaxf(s[j], s[2 + j]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float mnew = fmaxf(m_run[j], mx);      // finite: a page always has a visible token
+            alpha[j] = fast_exp2(m_run[j] - mnew);
+            m_run[j] = mnew;
+            s[j] = fast_exp2(s[j] - mnew);
+            s[2 + j] = fast_exp2(s[2 + j] - mnew);
+            l_run[j] = l_run[j] * alpha[j] + s[j] + s[2 + j];
+        }
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt) {
+            o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1];
+            o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1];
+        }
+        // P^T as B operand: transpose the two 8x8 (token x head) blocks
+        const uint32_t pb0 = movmatrix_trans(pack_bf16(s[0], s[1]));
+        const uint32_t pb1 = movmatrix_trans(pack_bf16(s[2], s[3]));
+        {
+            const int t = (lane & 7) + (lane >> 4) * 8;
+#pragma unroll
+            for (int mt = 0; mt < KSTEPS; ++mt) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, sV + tile_off<16>(t, 2 * mt + ((lane >> 3) & 1)));
+                mma_bf16_16816(o[mt], a, pb0, pb1);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+    // ---- reduce the sums over the 8 lane groups, then merge the warps through shared memory
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 4);
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 8);
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 16);
+    }
+    __syncthreads();                                  // every warp is done with its ring
+    float* mo = reinterpret_cast<float*>(smem);       // [NWARPS][8][DP]
+    float* mm = mo + NWARPS * 8 * DP;                 // [NWARPS][8]
+    float* ml = mm + NWARPS * 8;                      // [NWARPS][8]
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int d = mt * 16 + (lane >> 2) + (e >> 1) * 8;
+            const int head = 2 * (lane & 3) + (e & 1);
+            mo[(warp * 8 + head) * DP + d] = o[mt][e];
+        }
+    if (lane < 4) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            mm[warp * 8 + 2 * lane + j] = m_run[j];
+            ml[warp * 8 + 2 * lane + j] = l_run[j];
+        }
+    }
+    __syncthreads();
+
+    for (int idx = threadIdx.x; idx < G * (D / 2); idx += NWARPS * 32) {
+        const int head = idx / (D / 2), d = (idx % (D / 2)) * 2;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) M = fmaxf(M, mm[w * 8 + head]);
+        float L = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) {
+            const float f = fast_exp2(mm[w * 8 + head] - M);   // idle warps: 2^(-inf) = 0
+            L += ml[w * 8 + head] * f;
+            o0 += mo[(w * 8 + head) * DP + d] * f;
+            o1 += mo[(w * 8 + head) * DP + d + 1] * f;
+        }
+        const int hq = kvh * G + head;
+        if (it.part_slot < 0) {
+            const float inv = 1.f / L;
+            *reinterpret_cast<__nv_bfloat162*>(p.out + ((int64_t)it.q_row * p.Hq + hq) * D + d) =
+                __floats2bfloat162_rn(o0 * inv, o1 * inv);
+            if (p.lse && d == 0) p.lse[(int64_t)it.q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
+        } else {
+            const int64_t pr = (int64_t)it.part_slot * p.Hq + hq;
+            *reinterpret_cast<float2*>(p.part_o + pr * D + d) = make_float2(o0, o1);
+            if (d == 0) *reinterpret_cast<float2*>(p.part_ml + pr * 2) = make_float2(M, L);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Combine: merges the partials of a split sequence in fixed chunk order (deterministic).
+//   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
+// grid (n_combine_items, Hq), D/4 threads, one float4 of the head each.
+template <int D>
+__global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
+{
+    const CombineItem it = p.comb_items[blockIdx.x];
+    const int hq = blockIdx.y;
+    const int d = threadIdx.x * 4;
+    float M = -INFINITY;
+    for (int c = 0; c < it.n_chunks; ++c)
+        M = fmaxf(M, __ldg(p.part_ml + ((int64_t)(it.part_first + c) * p.Hq + hq) * 2));
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c = 0; c < it.n_chunks; ++c) {
+        const int64_t pr = (int64_t)(it.part_first + c) * p.Hq + hq;
+        const float2 ml = __ldg(reinterpret_cast<const float2*>(p.part_ml + pr * 2));
+        const float f = fast_exp2(ml.x - M);
+        const float4 v = __ldg(reinterpret_cast<const float4*>(p.part_o + pr * D + d));
+        L += ml.y * f;
+        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+    }
+    const float inv = 1.f / L;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t*>(&lo);
+    packed.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p.out + ((int64_t)it.q_row * p.Hq + hq) * D + d) = packed;
+    if (p.lse && threadIdx.x == 0) p.lse[(int64_t)it.q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
+}
+
+// ---------------------------------------------------------------------------------------------
+static constexpr int kDecWarps = 4;
+static constexpr int kDecStages = 3;
+
+template <int D>
+static size_t decode_smem_bytes()
+{
+    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * D * 2;
+    const size_t merge = (size_t)kDecWarps * 8 * (D + 4) * 4 + (size_t)kDecWarps * 8 * 4 * 2;
+    return ring > merge ? ring : merge;
+}
+
+template <int D>
+static cudaError_t launch_decode_t(const AttnParams& p, int n_items, cudaStream_t stream)
+{
+    auto kern = decode_splitk_kernel<D, kDecWarps, kDecStages>;
+    const size_t smem = decode_smem_bytes<D>();
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    kern<<<n_items * p.Hkv, kDecWarps * 32, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    return head_dim == 128 ? launch_decode_t<128>(p, n_items, stream) : launch_decode_t<64>(p, n_items, stream);
+}
+
+cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    dim3 grid(n_items, p.Hq);
+    if (head_dim == 128) combine_kernel<128><<<grid, 32, 0, stream>>>(p);
+    else combine_kernel<64><<<grid, 16, 0, stream>>>(p);
+    return cudaGetLastError();
+}
+
+}  // namespace cf

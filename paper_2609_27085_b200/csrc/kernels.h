@@ -1,0 +1,31 @@
+// Host-callable launchers of the CUDA kernels (one translation unit per kernel family).
+#pragma once
+#include <cuda_runtime.h>
+
+#include "device_common.cuh"
+
+namespace cf {
+
+struct AppendParams {
+    __nv_bfloat16* k_cache;
+    __nv_bfloat16* v_cache;
+    const __nv_bfloat16* k_new;
+    const __nv_bfloat16* v_new;
+    const int32_t* block_table;
+    int32_t max_blocks;
+    int64_t ks_block, ks_head, ks_token;
+    int64_t vs_block, vs_head, vs_token;
+    int32_t Hkv, D, num_seqs, total_rows;
+    const int32_t* context_len;
+    const int32_t* query_len;
+    const int32_t* q_start;
+};
+
+cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
+cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
+cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
+// mma.sync chunked prefill; tile height must equal kPrefillMmaTileRows
+constexpr int kPrefillMmaTileRows = 64;
+cudaError_t launch_prefill_mma(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
+
+}  // namespace cf

@@ -1,0 +1,118 @@
+#include "plan.h"
+
+#include <algorithm>
+
+namespace cf {
+
+cf_status validate_desc(const cf_cache_desc* d)
+{
+    if (!d) return CF_ERR_INVALID_ARG;
+    if (d->num_q_heads <= 0 || d->num_kv_heads <= 0 || d->num_blocks <= 0) return CF_ERR_INVALID_ARG;
+    if (d->num_q_heads % d->num_kv_heads != 0) return CF_ERR_INVALID_ARG;
+    const int g = d->num_q_heads / d->num_kv_heads;
+    if (d->head_dim != 64 && d->head_dim != 128) return CF_ERR_UNSUPPORTED;
+    if (d->block_size != 16) return CF_ERR_UNSUPPORTED;
+    if (g != 1 && g != 2 && g != 4 && g != 8) return CF_ERR_UNSUPPORTED;
+    const int64_t st[6] = {d->k_stride_block, d->k_stride_head, d->k_stride_token,
+                           d->v_stride_block, d->v_stride_head, d->v_stride_token};
+    for (int i = 0; i < 6; ++i) {
+        if (st[i] <= 0) return CF_ERR_INVALID_ARG;
+        if (st[i] % 8 != 0) return CF_ERR_UNSUPPORTED;
+    }
+    if (d->k_stride_token < d->head_dim || d->v_stride_token < d->head_dim) return CF_ERR_INVALID_ARG;
+    if (!(d->softmax_scale >= 0.0f)) return CF_ERR_INVALID_ARG;   // also rejects NaN
+    return CF_OK;
+}
+
+cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
+                           int32_t num_seqs, int32_t max_blocks_per_seq, Plan* plan)
+{
+    if (num_seqs < 0 || max_blocks_per_seq < 0) return CF_ERR_INVALID_ARG;
+    if (num_seqs > 0 && (!context_len || !query_len)) return CF_ERR_INVALID_ARG;
+    plan->q_start.assign((size_t)num_seqs + 1, 0);
+    int64_t total = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int32_t lq = query_len[s], lc = context_len[s];
+        if (lq < 0 || lc < 0 || lq > lc) return CF_ERR_INVALID_ARG;
+        if ((int64_t)lc > (int64_t)max_blocks_per_seq * d->block_size) return CF_ERR_OUT_OF_RANGE;
+        total += lq;
+        if (total > (int64_t)1 << 30) return CF_ERR_OUT_OF_RANGE;
+        plan->q_start[(size_t)s + 1] = (int32_t)total;
+    }
+    plan->total_q = (int32_t)total;
+    return CF_OK;
+}
+
+cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
+                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan)
+{
+    *plan = Plan();
+    cf_status st = validate_lengths(d, context_len, query_len, num_seqs, max_blocks_per_seq, plan);
+    if (st != CF_OK) return st;
+    const int32_t B = d->block_size;
+
+    // ---- decode: near-equal KV chunks, sized so that (chunks x kv heads) fills the machine a few times
+    int64_t total_pages = 0;
+    for (int32_t s = 0; s < num_seqs; ++s)
+        if (query_len[s] == 1) {
+            total_pages += (context_len[s] + B - 1) / B;
+            ++plan->n_decode_seqs;
+        } else if (query_len[s] > 1) {
+            ++plan->n_prefill_seqs;
+        }
+    const int64_t slots = (int64_t)std::max(1, cfg.num_sms) * std::max(1, cfg.decode_ctas_per_sm)
+                          * std::max(1, cfg.decode_waves);
+    const int32_t quantum = std::max(1, cfg.decode_page_quantum);
+    int64_t target = (total_pages * d->num_kv_heads + slots - 1) / slots;
+    target = std::max<int64_t>(target, cfg.decode_min_chunk_pages);
+    target = (target + quantum - 1) / quantum * quantum;
+
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        if (query_len[s] != 1) continue;
+        const int32_t lc = context_len[s];
+        const int64_t pages = (lc + B - 1) / B;
+        int64_t n = (pages + target - 1) / target;
+        int64_t per = (pages + n - 1) / n;
+        per = (per + quantum - 1) / quantum * quantum;
+        n = (pages + per - 1) / per;
+        int32_t first = -1;
+        if (n > 1) {
+            first = plan->n_part_slots;
+            plan->combine.push_back(CombineItem{plan->q_start[s], first, (int32_t)n});
+            plan->n_part_slots += (int32_t)n;
+        }
+        for (int64_t c = 0; c < n; ++c) {
+            DecodeItem it;
+            it.seq = s;
+            it.q_row = plan->q_start[s];
+            it.kv_begin = (int32_t)(c * per * B);
+            it.kv_end = (int32_t)std::min<int64_t>((c + 1) * per * B, lc);
+            it.part_slot = n > 1 ? first + (int32_t)c : -1;
+            it.chunk = (int32_t)c;
+            plan->decode.push_back(it);
+        }
+    }
+    std::stable_sort(plan->decode.begin(), plan->decode.end(), [](const DecodeItem& a, const DecodeItem& b) {
+        return (a.kv_end - a.kv_begin) > (b.kv_end - b.kv_begin);
+    });
+
+    // ---- prefill: q tiles of every chunk, the tile with the longest visible KV range first
+    const int32_t tr = std::max(1, cfg.prefill_tile_rows);
+    struct Keyed { int64_t extent; PrefillItem it; };
+    std::vector<Keyed> tiles;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int32_t lq = query_len[s];
+        if (lq <= 1) continue;
+        const int32_t prefix = context_len[s] - lq;
+        for (int32_t r0 = 0; r0 < lq; r0 += tr) {
+            const int32_t n = std::min(tr, lq - r0);
+            tiles.push_back(Keyed{(int64_t)prefix + r0 + n, PrefillItem{s, plan->q_start[s] + r0, r0, n}});
+        }
+    }
+    std::stable_sort(tiles.begin(), tiles.end(), [](const Keyed& a, const Keyed& b) { return a.extent > b.extent; });
+    plan->prefill.reserve(tiles.size());
+    for (const Keyed& k : tiles) plan->prefill.push_back(k.it);
+    return CF_OK;
+}
+
+}  // namespace cf

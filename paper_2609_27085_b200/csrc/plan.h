@@ -1,0 +1,65 @@
+// Host planner: turns the per-sequence lengths of one mixed batch into work items for the
+// split-K decode kernel, the combine kernel and the chunked-prefill kernel.
+// The batch is the one the paper's decode worker builds from its resident decode sequences plus
+// its local prefill queue (Section 5); the planner only partitions work, it does no arithmetic
+// on tensor data.
+#pragma once
+#include <cstdint>
+#include <vector>
+
+#include "../../include/crossflow_attn.h"
+
+namespace cf {
+
+struct DecodeItem {        // one (decode sequence, KV chunk); the kernel adds the KV-head index
+    int32_t seq;
+    int32_t q_row;         // packed row of the sequence's single query token
+    int32_t kv_begin;      // first visible token of the chunk (multiple of block_size)
+    int32_t kv_end;        // one past the last token (== context_len for the last chunk)
+    int32_t part_slot;     // partial slot to write, or -1: the only chunk, write `out` directly
+    int32_t chunk;         // index of this chunk within its sequence
+};
+
+struct CombineItem {       // one decode sequence that was split
+    int32_t q_row;
+    int32_t part_first;    // its chunks occupy slots [part_first, part_first + n_chunks)
+    int32_t n_chunks;
+};
+
+struct PrefillItem {       // one q tile of one prefill chunk; the kernel adds the head index
+    int32_t seq;
+    int32_t q_row0;        // packed row of the tile's first row
+    int32_t row0;          // index of that row inside the chunk (0-based)
+    int32_t n_rows;        // rows in this tile (<= tile height)
+};
+
+struct PlanConfig {
+    int32_t num_sms = 148;
+    int32_t decode_ctas_per_sm = 2;   // resident decode CTAs per SM the kernel is built for
+    int32_t decode_waves = 4;         // target number of CTA waves (load balance vs. partial traffic)
+    int32_t decode_min_chunk_pages = 32;
+    int32_t decode_page_quantum = 4;  // chunk lengths are multiples of this many pages (warps per CTA)
+    int32_t prefill_tile_rows = 64;
+};
+
+struct Plan {
+    std::vector<int32_t> q_start;     // [S+1] exclusive prefix sum of query_len
+    std::vector<DecodeItem> decode;   // longest chunk first
+    std::vector<CombineItem> combine;
+    std::vector<PrefillItem> prefill; // longest KV extent first
+    int32_t n_part_slots = 0;
+    int32_t total_q = 0;
+    int32_t n_decode_seqs = 0;
+    int32_t n_prefill_seqs = 0;
+};
+
+// Validates geometry (supported head_dim / block_size / group / strides).
+cf_status validate_desc(const cf_cache_desc* d);
+// Validates lengths against the block-table width; fills q_start/total_q.
+cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
+                           int32_t num_seqs, int32_t max_blocks_per_seq, Plan* plan);
+// Full plan (calls validate_lengths).
+cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
+                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan);
+
+}  // namespace cf

@@ -1,0 +1,132 @@
+"""CPU-only checks of the C-ABI library: it loads, exports every declared symbol, rejects bad
+arguments on the host before touching a device, and its planner covers every token exactly once."""
+import ctypes
+import os
+import re
+
+import numpy as np
+import pytest
+
+import cf_synth as syn
+import paper_2609_27085_b200 as cf
+from paper_2609_27085_b200 import build as cf_build
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+@pytest.fixture(scope="module", autouse=True)
+def _built():
+    cf_build.build()
+
+
+def test_library_exports_every_declared_symbol():
+    header = open(os.path.join(ROOT, "include", "crossflow_attn.h")).read()
+    declared = set(re.findall(r"\b(cf_[a-z_]+)\s*\(", header))
+    assert declared == set(cf.EXPORTS)
+    lib = cf.load_library()
+    for name in declared:
+        assert hasattr(lib, name), name
+
+
+def test_status_strings():
+    assert cf.cf_status_string(cf.CF_OK) == "CF_OK"
+    assert cf.cf_status_string(cf.CF_ERR_TIMEOUT) == "CF_ERR_TIMEOUT"
+    assert cf.cf_status_string(99) == "CF_ERR_UNKNOWN"
+
+
+def _plan(desc, lc, lq, max_blocks=4096, sms=148, check=True):
+    return cf.cf_plan_inspect(desc, lc, lq, max_blocks, sms, check=check)
+
+
+def test_desc_validation():
+    ok = cf.make_desc(32, 8, 128, 16, 1024)
+    assert _plan(ok, [5], [1])[0] == cf.CF_OK
+    for bad, want in [
+        (cf.make_desc(32, 8, 96, 16, 1024), cf.CF_ERR_UNSUPPORTED),      # head_dim
+        (cf.make_desc(32, 8, 128, 32, 1024), cf.CF_ERR_UNSUPPORTED),     # block_size
+        (cf.make_desc(48, 8, 128, 16, 1024), cf.CF_ERR_UNSUPPORTED),     # group 6
+        (cf.make_desc(30, 8, 128, 16, 1024), cf.CF_ERR_INVALID_ARG),     # Hq % Hkv
+        (cf.make_desc(32, 8, 128, 16, 1024, k_strides=(16388, 2048, 128)), cf.CF_ERR_UNSUPPORTED),  # 16-byte rule
+        (cf.make_desc(32, 8, 128, 16, 1024, v_strides=(16384, 2048, 64)), cf.CF_ERR_INVALID_ARG),
+        (cf.make_desc(32, 8, 128, 16, 1024, softmax_scale=-1.0), cf.CF_ERR_INVALID_ARG),
+    ]:
+        assert _plan(bad, [5], [1], check=False)[0] == want
+
+
+def test_length_validation():
+    d = cf.make_desc(8, 2, 64, 16, 64)
+    assert _plan(d, [5], [6], check=False)[0] == cf.CF_ERR_INVALID_ARG        # Lq > Lc
+    assert _plan(d, [5], [-1], check=False)[0] == cf.CF_ERR_INVALID_ARG
+    assert _plan(d, [65], [1], max_blocks=4, check=False)[0] == cf.CF_ERR_OUT_OF_RANGE
+    assert _plan(d, [64], [1], max_blocks=4, check=False)[0] == cf.CF_OK
+    st, dec, comb, pre, parts = _plan(d, [0, 7], [0, 0])                      # nothing to do
+    assert st == cf.CF_OK and len(dec) == len(comb) == len(pre) == 0 and parts == 0
+
+
+def _check_plan(geom, lc, lq, sms=148):
+    d = cf.make_desc(geom.num_q_heads, geom.num_kv_heads, geom.head_dim, geom.block_size, geom.num_blocks)
+    lc, lq = np.asarray(lc, dtype=np.int32), np.asarray(lq, dtype=np.int32)
+    st, dec, comb, pre, parts = _plan(d, lc, lq, max_blocks=1 << 20, sms=sms)
+    qs = np.concatenate([[0], np.cumsum(lq)])
+    # decode: chunks of each Lq == 1 sequence tile [0, Lc) exactly, in page multiples, none empty
+    slots_seen = set()
+    for s in np.nonzero(lq == 1)[0]:
+        mine = dec[dec[:, 0] == s]
+        mine = mine[np.argsort(mine[:, 5])]
+        assert len(mine) >= 1 and mine[0, 2] == 0 and mine[-1, 3] == lc[s]
+        assert (mine[:, 1] == qs[s]).all()
+        assert (mine[1:, 2] == mine[:-1, 3]).all() and (mine[:, 2] % 16 == 0).all() and (mine[:, 3] > mine[:, 2]).all()
+        assert list(mine[:, 5]) == list(range(len(mine)))
+        if len(mine) == 1:
+            assert mine[0, 4] == -1
+        else:
+            c = comb[comb[:, 0] == qs[s]]
+            assert len(c) == 1 and c[0, 2] == len(mine)
+            assert list(mine[:, 4]) == list(range(c[0, 1], c[0, 1] + len(mine)))
+            slots_seen.update(int(x) for x in mine[:, 4])
+    assert set(int(s) for s in dec[:, 0]) == set(int(s) for s in np.nonzero(lq == 1)[0])
+    assert slots_seen == set(range(parts))
+    lens = dec[:, 3] - dec[:, 2]
+    assert (np.diff(lens) <= 0).all()                                      # longest first
+    # prefill: tiles of each Lq > 1 sequence cover its rows exactly once
+    for s in np.nonzero(lq > 1)[0]:
+        mine = pre[pre[:, 0] == s]
+        mine = mine[np.argsort(mine[:, 2])]
+        assert mine[0, 2] == 0 and (mine[:, 1] == qs[s] + mine[:, 2]).all()
+        assert (mine[1:, 2] == mine[:-1, 2] + mine[:-1, 3]).all() and mine[-1, 2] + mine[-1, 3] == lq[s]
+    assert set(int(s) for s in pre[:, 0]) == set(int(s) for s in np.nonzero(lq > 1)[0])
+    ext = (lc - lq)[pre[:, 0]] + pre[:, 2] + pre[:, 3]
+    assert (np.diff(ext) <= 0).all()
+    return dec, comb, pre, parts
+
+
+def test_plan_covers_the_five_configs():
+    g4, g8 = syn.GEOM_G4, syn.GEOM_G8
+    _check_plan(syn.GEOM_TINY, [256] * 5, [128, 1, 1, 1, 1])
+    dec, *_ = _check_plan(g4, syn.config2_lengths(), [1] * 64)
+    assert 148 * 2 <= len(dec) * 8 <= 148 * 2 * 8          # a few waves of CTAs, not thousands
+    _check_plan(g4, [6144 + 512, 6144 + 512] + list(syn.config3_lengths()), [512, 512] + [1] * 48)
+    dec, *_ = _check_plan(g4, [24576 + 2048] + list(syn.config4_lengths()), [2048] + [1] * 16)
+    assert len(dec) * 8 >= 148 * 2                          # 16 x 8 pairs alone would leave SMs idle
+    _check_plan(g8, [4096 + 8192] + list(syn.config5_lengths()), [8192] + [1] * 256)
+
+
+def test_plan_random_batches():
+    rng = np.random.default_rng(0)
+    for _ in range(50):
+        S = int(rng.integers(1, 40))
+        lq = rng.choice([0, 1, 1, 1, 2, 17, 64, 65, 300], size=S)
+        lc = lq + rng.integers(0, 5000, size=S)
+        _check_plan(syn.GEOM_G4, lc, lq, sms=int(rng.choice([1, 4, 148])))
+
+
+def test_calls_without_a_device_fail_with_a_status():
+    """On a machine with no GPU the entry points report an error code; nothing falls back to the CPU."""
+    import torch
+    if torch.cuda.is_available():
+        pytest.skip("device present")
+    ctx = ctypes.c_void_p()
+    st = cf.load_library().cf_create(ctypes.byref(ctx), 0, 0)
+    assert st in (cf.CF_ERR_CUDA, cf.CF_ERR_INVALID_ARG) and not ctx.value
+    with pytest.raises(cf.CfError):
+        cf.cf_create(0)

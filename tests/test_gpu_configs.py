@@ -1,0 +1,28 @@
+"""GPU parity at the full sizes of the five workload configurations, in the launch configuration
+the benchmark times.  Decode rows are all checked; prefill rows are checked on a deterministic
+sample (first and last row of every 128-row tile plus every 7th row, thinned to a cap) because
+the fp64 oracle needs ~1 TFLOP per iteration for the long chunks."""
+import pytest
+
+import cf_synth as syn
+from harness import run_and_check
+
+pytestmark = pytest.mark.gpu
+
+
+def test_config2_decode_only_full_size():
+    print(run_and_check(syn.config2_decode_only(), check_append=True))
+
+
+def test_config3_chat_all_iterations():
+    print(run_and_check(syn.config3_chat(), max_prefill_rows=24, check_append=False))
+
+
+def test_config4_agentic_first_and_last_iteration():
+    sc = syn.config4_agentic()
+    print(run_and_check(sc, max_prefill_rows=12, check_append=False))
+
+
+@pytest.mark.parametrize("budget,n", [(0, 0), (512, 4), (2048, 3), (8192, 1)])
+def test_config5_sweep_points(budget, n):
+    print(run_and_check(syn.config5_sweep_point(budget, n), max_prefill_rows=8, check_append=False))

@@ -1,0 +1,203 @@
+"""GPU parity: the CUDA library (through its C ABI) against the CPU oracle, element by element,
+on seeded inputs that span several tiles, ragged tails and the degenerate cases."""
+import numpy as np
+import pytest
+import torch
+
+import cf_synth as syn
+import oracle
+import paper_2609_27085_b200 as cf
+from harness import GpuScenario, compare, run_and_check, to_dev_bf16, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def small(seed, Hq, Hkv, D, prefix, qlens, NB=2048, shuffle=False):
+    return syn.scenario_from_lengths("t", syn.Geometry(Hq, Hkv, D, 16, NB), seed, prefix, qlens, shuffle_seqs=shuffle)
+
+
+def test_config1_tiny():
+    stats = run_and_check(syn.config1_tiny())
+    print(stats)
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (8, 8, 128), (8, 4, 128), (32, 8, 128), (64, 8, 128), (16, 2, 64), (8, 1, 64)])
+def test_decode_only_ragged(Hq, Hkv, D):
+    lens = [1, 2, 15, 16, 17, 31, 33, 63, 64, 65, 127, 129, 255, 700, 1023, 1025, 2500, 4097, 9000]
+    run_and_check(small(3, Hq, Hkv, D, [l - 1 for l in lens], [[1] * len(lens)]))
+
+
+@pytest.mark.parametrize("Hq,Hkv,D", [(8, 2, 64), (4, 4, 128), (32, 8, 128), (16, 2, 128)])
+def test_prefill_only_ragged(Hq, Hkv, D):
+    prefix = [0, 0, 5, 16, 63, 64, 100, 1000, 0, 333]
+    qlen = [2, 64, 65, 17, 1, 128, 129, 200, 300, 31]
+    run_and_check(small(5, Hq, Hkv, D, prefix, [qlen]))
+
+
+def test_mixed_shuffled_order_with_empty_sequences():
+    prefix = [10, 0, 500, 77, 0, 2000, 31, 640, 5, 1]
+    qlen = [1, 90, 1, 0, 1, 1, 130, 1, 0, 64]
+    run_and_check(small(7, 32, 8, 128, prefix, [qlen], shuffle=True))
+
+
+def test_multi_iteration_chunked_prefill_with_growing_decodes():
+    prefix = [300, 40, 999, 0]
+    qlens = [[100, 1, 1, 64], [37, 1, 1, 64], [200, 1, 1, 1]]
+    run_and_check(small(9, 8, 2, 64, prefix, qlens))
+    run_and_check(small(9, 32, 8, 128, prefix, qlens))
+
+
+def test_nhd_layout_and_custom_scale():
+    prefix = [10, 700, 0, 2047]
+    qlen = [1, 1, 80, 1]
+    run_and_check(small(11, 32, 8, 128, prefix, [qlen]), layout="NHD")
+    run_and_check(small(11, 8, 2, 64, prefix, [qlen]), layout="NHD", softmax_scale=0.2)
+
+
+def test_long_split_decode_uses_partials_and_combine():
+    sc = small(13, 32, 8, 128, [40000 - 1, 123], [[1, 1]], NB=4096)
+    d = cf.make_desc(32, 8, 128, 16, 4096)
+    _, dec, comb, _, parts = cf.cf_plan_inspect(d, sc.batches[0].context_len, sc.batches[0].query_len, sc.batches[0].max_blocks)
+    assert parts >= 2 and len(comb) == 1
+    run_and_check(sc)
+
+
+def test_chunking_invariance_on_gpu():
+    """One 300-token unit vs. three ragged units (Section 4.4): same rows within tolerance, and both match the oracle."""
+    one = small(15, 8, 2, 64, [77], [[300]])
+    cut = small(15, 8, 2, 64, [77], [[300]])
+    b = one.batches[0]
+    g1 = GpuScenario(one)
+    g1.append(b)
+    o_full, _ = g1.attend(b)
+    g1.close()
+    g2 = GpuScenario(cut)
+    at, have = 0, 77
+    outs = []
+    for c in (130, 1, 169):
+        have += c
+        part = syn.Batch(b.geom, np.array([have], np.int32), np.array([c], np.int32), b.block_table,
+                         b.q[at:at + c], b.k_new[at:at + c], b.v_new[at:at + c])
+        g2.append(part)
+        outs.append(g2.attend(part)[0])
+        at += c
+    g2.close()
+    o_cut = np.concatenate(outs)
+    diff = np.abs(syn.bf16_bits_to_f64(o_full) - syn.bf16_bits_to_f64(o_cut))
+    assert diff.max() <= 2e-2 and diff.mean() <= 2e-3
+
+
+def test_determinism_and_unrelated_calls():
+    sc = small(17, 32, 8, 128, [5000, 20, 300], [[1, 1, 150]])
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    first, lse0 = g.attend(b)
+    other = small(18, 8, 2, 64, [900], [[1]])
+    g_other = GpuScenario(other, ctx=g.ctx)
+    g_other.append(other.batches[0])
+    g_other.attend(other.batches[0])
+    for _ in range(10):
+        o, lse = g.attend(b)
+        assert np.array_equal(o, first) and np.array_equal(lse, lse0)
+    g.close()
+
+
+@pytest.mark.parametrize("kind", ["decode", "prefill"])
+def test_spike_keys(kind):
+    """A key planted 40+ above the rest must be found wherever it sits: page edges, chunk edges,
+    the prefix/chunk boundary, the diagonal; a key just past the diagonal must have no effect."""
+    Hq, Hkv, D = 8, 2, 128
+    if kind == "decode":
+        Lc, Lq = 20000, 1
+    else:
+        Lc, Lq = 1500, 200
+    P = Lc - Lq
+    sc = small(19, Hq, Hkv, D, [P], [[Lq]], NB=2048)
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    d = cf.make_desc(Hq, Hkv, D, 16, 2048)
+    _, dec, _, _, _ = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks)
+    edges = sorted(set(int(x) for x in dec[:, 2]) | set(int(x) for x in dec[:, 3]))
+    cand = {0, 15, 16, 63, 64, 127, 128, P - 1, P, Lc - 2, Lc - 1}
+    for e in edges:
+        cand.update({e - 1, e, e + 1})
+    cand = sorted(j for j in cand if 0 <= j < Lc)
+    k0 = g.k.clone()
+    big = torch.zeros(D, dtype=torch.bfloat16, device="cuda")
+    big[0] = 96.0
+    q = b.q.copy()
+    q[:, :, 0] = syn.f32_to_bf16_bits(np.float32(8.0))       # every row: score of the planted key = 8*96/sqrt(128) ~ 68
+    bq = syn.Batch(b.geom, b.context_len, b.query_len, b.block_table, q, b.k_new, b.v_new)
+    v_host = to_host_bits(g.v)
+    for j in cand:
+        g.k.copy_(k0)
+        blk, slot = int(b.block_table[0, j // 16]), j % 16
+        g.k[blk, :, slot, :] = big
+        o, _ = g.attend(bq, want_lse=False)
+        o = syn.bf16_bits_to_f64(o)                          # [Lq, Hq, D]
+        vj = syn.bf16_bits_to_f64(v_host[blk, :, slot, :])   # [Hkv, D]
+        for i in ([0] if Lq == 1 else [0, 1, Lq // 2, Lq - 2, Lq - 1]):
+            p = P + i
+            want = np.repeat(vj, Hq // Hkv, axis=0)
+            if j <= p:
+                assert np.abs(o[i] - want).max() <= 2e-2, (kind, j, i)
+            else:
+                assert np.abs(o[i] - want).max() > 0.5, (kind, j, i)   # invisible key: output is the ordinary average
+    g.close()
+
+
+def test_abi_rejects_bad_arguments_without_launching():
+    sc = small(21, 8, 2, 64, [10], [[1]])
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    bt = torch.from_numpy(b.block_table).cuda()
+    q = to_dev_bf16(b.q)
+    out = torch.zeros_like(q)
+    A = dict(check=False)
+    assert cf.cf_mixed_attention(g.ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, [5], [6], out, **A) == cf.CF_ERR_INVALID_ARG
+    assert cf.cf_mixed_attention(g.ctx, g.desc, q, g.k, g.v, bt, 0, [11], [1], out, **A) == cf.CF_ERR_OUT_OF_RANGE
+    assert cf.cf_mixed_attention(g.ctx, g.desc, None, g.k, g.v, bt, b.max_blocks, [11], [1], out, **A) == cf.CF_ERR_INVALID_ARG
+    assert cf.cf_mixed_attention(g.ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, [11], [1], None, **A) == cf.CF_ERR_INVALID_ARG
+    bad = cf.make_desc(8, 2, 96, 16, 2048)
+    assert cf.cf_mixed_attention(g.ctx, bad, q, g.k, g.v, bt, b.max_blocks, [11], [1], out, **A) == cf.CF_ERR_UNSUPPORTED
+    assert cf.cf_kv_append(g.ctx, g.desc, g.k, g.v, None, None, bt, b.max_blocks, [11], [1], **A) == cf.CF_ERR_INVALID_ARG
+    assert cf.cf_kv_append(g.ctx, g.desc, g.k, g.v, q, q, bt, b.max_blocks, [11], [12], **A) == cf.CF_ERR_INVALID_ARG
+    torch.cuda.synchronize()
+    assert (out == 0).all()
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    g.close()
+
+
+def test_fixed_workspace_too_small_is_reported():
+    sc = small(23, 32, 8, 128, [60000], [[1]], NB=4096)
+    b = sc.batches[0]
+    ctx = cf.cf_create(0, workspace_bytes=4096)
+    g = GpuScenario(sc, ctx=ctx)
+    bt = torch.from_numpy(b.block_table).cuda()
+    q = to_dev_bf16(b.q)
+    out = torch.zeros_like(q)
+    st = cf.cf_mixed_attention(ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len, out, check=False)
+    assert st == cf.CF_ERR_WORKSPACE
+    cf.cf_destroy(ctx)
+
+
+def test_host_step_matches_device_step():
+    sc = small(25, 32, 8, 128, [100, 3000, 50], [[70, 1, 1]])
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    bt = torch.from_numpy(b.block_table).cuda()
+    qh = torch.from_numpy(b.q.view(np.int16)).pin_memory()
+    kh = torch.from_numpy(b.k_new.view(np.int16)).pin_memory()
+    vh = torch.from_numpy(b.v_new.view(np.int16)).pin_memory()
+    oh = torch.zeros_like(qh).pin_memory()
+    cf.cf_mixed_step_host(g.ctx, g.desc, qh, kh, vh, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len, oh)
+    torch.cuda.synchronize()
+    o_dev, _ = g.attend(b, want_lse=False)          # caches were appended by the host step
+    assert np.array_equal(oh.numpy().view(np.uint16), o_dev)
+    k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
+    compare(o_dev, None, ref_o, ref_lse)
+    g.close()
