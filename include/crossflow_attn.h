@@ -115,12 +115,16 @@ cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
  * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
 cf_status cf_get_async_status(cf_ctx* ctx);
 
-/* Per-kernel timing for benchmarks.  cf_set_timing(ctx, 1) makes every later cf_mixed_attention
- * record CUDA events around its kernels; cf_get_last_timing synchronises on the last call's final
- * event and returns milliseconds (0 for a kernel that was not launched) and the launch count. */
+/* Per-kernel timing for benchmarks.  After cf_set_timing(ctx, 1) every cf_mixed_attention records
+ * CUDA events around its kernels on the caller's stream (no host synchronisation).
+ * cf_get_timing_sums waits for the last timed call, returns the summed milliseconds of each
+ * kernel over all calls timed since the previous cf_get_timing_sums / cf_set_timing (0 for a
+ * kernel that never ran) and the number of calls, and resets the sums. */
 cf_status cf_set_timing(cf_ctx* ctx, int enabled);
-cf_status cf_get_last_timing(cf_ctx* ctx, float* ms_decode, float* ms_combine, float* ms_prefill,
-                             int32_t* num_launches);
+cf_status cf_get_timing_sums(cf_ctx* ctx, float* ms_decode, float* ms_combine, float* ms_prefill,
+                             int32_t* num_calls);
+/* Number of kernels the last cf_mixed_attention launched (decode, combine, prefill: 0..3). */
+cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
 
 /* Host planner, exposed for inspection and tests (no GPU needed).  Builds the plan that
  * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.

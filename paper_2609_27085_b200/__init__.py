@@ -6,7 +6,7 @@ There is no CPU fallback: if the library is missing, loading raises.
 
 Names mirror the C ABI (``include/crossflow_attn.h``): ``cf_create``, ``cf_kv_append``,
 ``cf_mixed_attention``, ``cf_mixed_step_host``, ``cf_get_async_status``, ``cf_set_timing``,
-``cf_get_last_timing``, ``cf_plan_inspect``, ``cf_status_string``.
+``cf_get_timing_sums``, ``cf_get_last_launch_count``, ``cf_plan_inspect``, ``cf_status_string``.
 
 Device arguments may be torch tensors (their ``data_ptr()`` is used) or integer addresses; the
 length arrays are host ``int32`` numpy arrays (anything array-like is converted).
@@ -32,7 +32,8 @@ CF_ERR_TIMEOUT = 6
 CF_ERR_ARCH = 7
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host",
-           "cf_get_async_status", "cf_set_timing", "cf_get_last_timing", "cf_plan_inspect", "cf_status_string")
+           "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
+           "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -70,7 +71,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_mixed_step_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp]
     lib.cf_get_async_status.argtypes = [vp]
     lib.cf_set_timing.argtypes = [vp, ctypes.c_int]
-    lib.cf_get_last_timing.argtypes = [vp, fp, fp, fp, i32p]
+    lib.cf_get_timing_sums.argtypes = [vp, fp, fp, fp, i32p]
+    lib.cf_get_last_launch_count.argtypes = [vp, i32p]
     lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.cf_status_string.argtypes = [ctypes.c_int]
     lib.cf_status_string.restype = ctypes.c_char_p
@@ -175,12 +177,18 @@ def cf_set_timing(ctx, enabled: bool) -> None:
     _check(load_library().cf_set_timing(ctx, int(bool(enabled))), "cf_set_timing")
 
 
-def cf_get_last_timing(ctx) -> Tuple[float, float, float, int]:
-    """(ms_decode, ms_combine, ms_prefill, num_launches) of the last cf_mixed_attention."""
+def cf_get_timing_sums(ctx) -> Tuple[float, float, float, int]:
+    """(ms_decode, ms_combine, ms_prefill, num_calls) summed over the calls timed since the last query."""
     a, b, c, n = ctypes.c_float(), ctypes.c_float(), ctypes.c_float(), ctypes.c_int32()
-    _check(load_library().cf_get_last_timing(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
-           "cf_get_last_timing")
+    _check(load_library().cf_get_timing_sums(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
+           "cf_get_timing_sums")
     return a.value, b.value, c.value, n.value
+
+
+def cf_get_last_launch_count(ctx) -> int:
+    n = ctypes.c_int32()
+    _check(load_library().cf_get_last_launch_count(ctx, ctypes.byref(n)), "cf_get_last_launch_count")
+    return n.value
 
 
 def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148,

@@ -5,6 +5,7 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "../../include/crossflow_attn.h"
 #include "kernels.h"
@@ -15,6 +16,11 @@ namespace cf {
 static constexpr int kRing = 4;                         // plan slots in flight
 static constexpr size_t kDefaultWorkspace = 64u << 20;  // split-K partials
 static constexpr size_t kDefaultPlanBytes = 1u << 20;
+
+struct TimedCall {
+    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
+    bool ran[3] = {false, false, false};
+};
 
 struct PlanSlot {
     uint8_t* host = nullptr;   // pinned
@@ -39,11 +45,10 @@ struct cf_ctx {
     // host-staged step
     uint8_t* stage_dev = nullptr;
     size_t stage_bytes = 0;
-    // timing
+    // timing: one quad of events per timed call since the last cf_get_timing_sums
     bool timing = false;
-    cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
-    bool ev_valid = false;
-    bool ran[3] = {false, false, false};
+    std::vector<cf::TimedCall> timed;
+    size_t timed_used = 0;
     int launches = 0;
 };
 
@@ -209,7 +214,6 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
-    for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&c->ev[i]) == cudaSuccess;
     ok = ok && ensure_plan_capacity(c, kDefaultPlanBytes) == CF_OK;
     c->workspace_fixed = false;
     ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
@@ -234,8 +238,9 @@ cf_status cf_destroy(cf_ctx* c)
         if (c->slots[i].dev) cudaFree(c->slots[i].dev);
         if (c->slots[i].done) cudaEventDestroy(c->slots[i].done);
     }
-    for (int i = 0; i < 4; ++i)
-        if (c->ev[i]) cudaEventDestroy(c->ev[i]);
+    for (cf::TimedCall& tc : c->timed)
+        for (int i = 0; i < 4; ++i)
+            if (tc.ev[i]) cudaEventDestroy(tc.ev[i]);
     if (c->workspace) cudaFree(c->workspace);
     if (c->err_dev) cudaFree(c->err_dev);
     if (c->stage_dev) cudaFree(c->stage_dev);
@@ -296,7 +301,6 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, c->cfg, &pl);
     if (st != CF_OK) return st;
-    c->ev_valid = false;
     c->launches = 0;
     if (pl.total_q == 0) return CF_OK;
     if (!q || !k_cache || !v_cache || !block_table || !out) return CF_ERR_INVALID_ARG;
@@ -339,19 +343,28 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     p.err = c->err_dev;
 
     cudaError_t e = cudaSuccess;
-    const bool t = c->timing;
-    c->ran[0] = !pl.decode.empty();
-    c->ran[1] = !pl.combine.empty();
-    c->ran[2] = !pl.prefill.empty();
-    if (t) cudaEventRecord(c->ev[0], stream);
+    TimedCall* tc = nullptr;
+    if (c->timing) {
+        if (c->timed_used == c->timed.size()) {
+            TimedCall fresh;
+            bool ok = true;
+            for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&fresh.ev[i]) == cudaSuccess;
+            if (!ok) return CF_ERR_CUDA;
+            c->timed.push_back(fresh);
+        }
+        tc = &c->timed[c->timed_used++];
+        tc->ran[0] = !pl.decode.empty();
+        tc->ran[1] = !pl.combine.empty();
+        tc->ran[2] = !pl.prefill.empty();
+    }
+    if (tc) cudaEventRecord(tc->ev[0], stream);
     if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
-    if (t) cudaEventRecord(c->ev[1], stream);
+    if (tc) cudaEventRecord(tc->ev[1], stream);
     if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
-    if (t) cudaEventRecord(c->ev[2], stream);
+    if (tc) cudaEventRecord(tc->ev[2], stream);
     if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
-    if (t) cudaEventRecord(c->ev[3], stream);
-    c->ev_valid = t;
-    c->launches = (int)c->ran[0] + (int)c->ran[1] + (int)c->ran[2];
+    if (tc) cudaEventRecord(tc->ev[3], stream);
+    c->launches = (int)!pl.decode.empty() + (int)!pl.combine.empty() + (int)!pl.prefill.empty();
     const cf_status fs = finish_slot(slot, stream);
     if (e != cudaSuccess) return CF_ERR_CUDA;
     return fs;
@@ -420,24 +433,38 @@ cf_status cf_set_timing(cf_ctx* c, int enabled)
 {
     if (!c) return CF_ERR_INVALID_ARG;
     c->timing = enabled != 0;
-    c->ev_valid = false;
+    c->timed_used = 0;
     return CF_OK;
 }
 
-cf_status cf_get_last_timing(cf_ctx* c, float* ms_decode, float* ms_combine, float* ms_prefill, int32_t* num_launches)
+cf_status cf_get_timing_sums(cf_ctx* c, float* ms_decode, float* ms_combine, float* ms_prefill, int32_t* num_calls)
 {
     if (!c) return CF_ERR_INVALID_ARG;
-    float t[3] = {0.f, 0.f, 0.f};
-    if (c->ev_valid) {
+    double t[3] = {0., 0., 0.};
+    const size_t n = c->timed_used;
+    if (n > 0) {
         DeviceGuard guard(c->device);
-        if (cudaEventSynchronize(c->ev[3]) != cudaSuccess) return CF_ERR_CUDA;
-        for (int i = 0; i < 3; ++i)
-            if (c->ran[i] && cudaEventElapsedTime(&t[i], c->ev[i], c->ev[i + 1]) != cudaSuccess) return CF_ERR_CUDA;
+        if (cudaEventSynchronize(c->timed[n - 1].ev[3]) != cudaSuccess) return CF_ERR_CUDA;
+        for (size_t k = 0; k < n; ++k)
+            for (int i = 0; i < 3; ++i) {
+                float ms = 0.f;
+                if (c->timed[k].ran[i] && cudaEventElapsedTime(&ms, c->timed[k].ev[i], c->timed[k].ev[i + 1]) != cudaSuccess)
+                    return CF_ERR_CUDA;
+                t[i] += ms;
+            }
     }
-    if (ms_decode) *ms_decode = t[0];
-    if (ms_combine) *ms_combine = t[1];
-    if (ms_prefill) *ms_prefill = t[2];
-    if (num_launches) *num_launches = c->launches;
+    c->timed_used = 0;
+    if (ms_decode) *ms_decode = (float)t[0];
+    if (ms_combine) *ms_combine = (float)t[1];
+    if (ms_prefill) *ms_prefill = (float)t[2];
+    if (num_calls) *num_calls = (int32_t)n;
+    return CF_OK;
+}
+
+cf_status cf_get_last_launch_count(cf_ctx* c, int32_t* num_launches)
+{
+    if (!c || !num_launches) return CF_ERR_INVALID_ARG;
+    *num_launches = c->launches;
     return CF_OK;
 }
 
