@@ -126,6 +126,31 @@ cf_status cf_get_timing_sums(cf_ctx* ctx, float* ms_decode, float* ms_combine, f
 /* Number of kernels the last cf_mixed_attention launched (decode, combine, prefill: 0..3). */
 cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
 
+/* Decode attention that allocates nothing (the paper has no counterpart; this serves callers that
+ * must not allocate).  Some integrators cannot call cudaMalloc where they need attention: a plugin
+ * that is handed only its input and output buffers, a process whose whole GPU is owned by another
+ * framework's caching allocator, a latency-critical loop that must stay off the driver's allocator
+ * lock.  This entry point needs no cf_ctx: the split-K scratch (work items and fp32 partials) is a
+ * fixed 16 MiB array inside the library's device image, resident on every GPU that loads the library
+ * until the process exits.  It calls no cudaMalloc / cudaFree / cudaMallocHost and no allocating
+ * library routine; the host plan lives on the stack (about 110 KB).
+ *   Every sequence decodes exactly one token: q / out are bf16 [num_seqs, Hq, D], lse fp32
+ *   [num_seqs, Hq] or NULL, context_len HOST int32 [num_seqs] (>= 1, includes the new token);
+ *   caches, block_table and desc as in cf_mixed_attention.  Runs on the CURRENT device.
+ *   Limits: num_seqs <= 1024, <= 4096 KV chunks, and partials (chunks of split sequences x Hq x
+ *   (D+2) x 4 bytes) + 128 KiB <= 16 MiB; anything larger returns CF_ERR_WORKSPACE and enqueues nothing.
+ *   The first call on a device resolves the array's address and sets kernel attributes; make that
+ *   call before any stream capture begins.  All calls share the one array and it keeps the previous
+ *   call's contents (nothing in it has to start at zero: every partial that is read is written first
+ *   by the same call), so two calls whose GPU work overlaps - different streams, or different host
+ *   threads - race; keep them on one stream or order them yourself.  Results are identical to
+ *   cf_mixed_attention on the same all-decode batch. */
+cf_status cf_decode_attention_static(const cf_cache_desc* desc, const void* q,
+                                     const void* k_cache, const void* v_cache,
+                                     const int32_t* block_table, int32_t max_blocks_per_seq,
+                                     const int32_t* context_len, int32_t num_seqs,
+                                     void* out, float* lse, void* cuda_stream);
+
 /* Host planner, exposed for inspection and tests (no GPU needed).  Builds the plan that
  * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.
  *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}

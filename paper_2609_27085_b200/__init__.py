@@ -6,7 +6,7 @@ There is no CPU fallback: if the library is missing, loading raises.
 
 Names mirror the C ABI (``include/crossflow_attn.h``): ``cf_create``, ``cf_kv_append``,
 ``cf_mixed_attention``, ``cf_mixed_step_host``, ``cf_get_async_status``, ``cf_set_timing``,
-``cf_get_timing_sums``, ``cf_get_last_launch_count``, ``cf_plan_inspect``, ``cf_status_string``.
+``cf_get_timing_sums``, ``cf_get_last_launch_count``, ``cf_plan_inspect``, ``cf_decode_attention_static``, ``cf_status_string``.
 
 Device arguments may be torch tensors (their ``data_ptr()`` is used) or integer addresses; the
 length arrays are host ``int32`` numpy arrays (anything array-like is converted).
@@ -33,7 +33,7 @@ CF_ERR_ARCH = 7
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
-           "cf_status_string")
+           "cf_decode_attention_static", "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -74,6 +74,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_get_timing_sums.argtypes = [vp, fp, fp, fp, i32p]
     lib.cf_get_last_launch_count.argtypes = [vp, i32p]
     lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
+    lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_status_string.argtypes = [ctypes.c_int]
     lib.cf_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -205,3 +206,19 @@ def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq:
     if check:
         _check(st, "cf_plan_inspect")
     return st, dec[:counts[0]], comb[:counts[1]], pre[:counts[2]], int(counts[3])
+
+
+def cf_decode_attention_static(desc: CacheDesc, q, k_cache, v_cache, block_table, max_blocks_per_seq: int,
+                               context_len, out, lse=None, stream=None, check: bool = True) -> int:
+    """All-decode attention for callers that must not allocate device memory (a plugin that only
+    receives its buffers, a process whose GPU memory belongs to another allocator): no context, the
+    split-K scratch is a fixed 16 MiB array inside the library.  One query token per sequence;
+    runs on the current device; calls sharing the array must not overlap on the GPU.  Batches beyond
+    the fixed limits return CF_ERR_WORKSPACE."""
+    lc = _host_i32(context_len)
+    st = load_library().cf_decode_attention_static(ctypes.byref(desc), _dev(q), _dev(k_cache), _dev(v_cache),
+                                                   _dev(block_table), int(max_blocks_per_seq), lc.ctypes.data,
+                                                   int(lc.shape[0]), _dev(out), _dev(lse), _stream(stream))
+    if check:
+        _check(st, "cf_decode_attention_static")
+    return st

@@ -290,3 +290,155 @@ cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaS
 }
 
 }  // namespace cf
+
+// =============================================================================================
+// Allocation-free decode entry point.
+//
+// Some callers cannot allocate device memory at the point where they need attention: code that
+// runs inside another framework's memory plan (every byte of the GPU already handed to a caching
+// allocator), real-time loops that must not hit the driver's allocator lock, or plugins that are
+// only given input and output buffers.  For them the split-K scratch (plan items and fp32
+// partials) lives in a fixed array in the library's own device image instead of a cf_ctx
+// workspace.  Every GPU that loads the library holds the array until the process exits.
+//
+// The array's name is a host-side handle in host code, not a device address; the address comes
+// from cudaGetSymbolAddress, taken once per device (with that device current) on the first call.
+// =============================================================================================
+namespace {
+
+constexpr size_t kStaticScratchBytes = (size_t)16 << 20;          // whole array
+constexpr size_t kStaticPlanBytes = (size_t)128 << 10;            // items + combine items
+constexpr int kStaticMaxSeqs = 1024;
+constexpr int kStaticMaxItems = 4096;
+constexpr int kMaxDevices = 64;
+
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+struct StaticSetup {
+    bool ready = false;
+    unsigned char* base = nullptr;   // device address of g_static_scratch on this device
+    int num_sms = 0;
+};
+StaticSetup g_static_setup[kMaxDevices];
+
+struct StaticPlan {                  // fixed capacity, lives on the caller's stack
+    cf::DecodeItem items[kStaticMaxItems];
+    cf::CombineItem comb[kStaticMaxSeqs];
+    int n_items = 0, n_comb = 0, n_slots = 0;
+};
+
+}  // namespace
+
+extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const void* q,
+                                                const void* k_cache, const void* v_cache,
+                                                const int32_t* block_table, int32_t max_blocks_per_seq,
+                                                const int32_t* context_len, int32_t num_seqs,
+                                                void* out, float* lse, void* cuda_stream)
+{
+    using namespace cf;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    if (num_seqs < 0 || max_blocks_per_seq < 0) return CF_ERR_INVALID_ARG;
+    if (num_seqs == 0) return CF_OK;
+    if (!q || !k_cache || !v_cache || !block_table || !context_len || !out) return CF_ERR_INVALID_ARG;
+    if (num_seqs > kStaticMaxSeqs) return CF_ERR_WORKSPACE;
+
+    // ---- once per device: resolve the scratch address, read the SM count (no allocation)
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CF_ERR_CUDA;
+    StaticSetup& su = g_static_setup[dev];
+    if (!su.ready) {
+        int major = 0, sms = 0;
+        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return CF_ERR_CUDA;
+        if (major != 10) return CF_ERR_ARCH;
+        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CF_ERR_CUDA;
+        void* ptr = nullptr;
+        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return CF_ERR_CUDA;
+        su.base = static_cast<unsigned char*>(ptr);
+        su.num_sms = sms;
+        su.ready = true;
+    }
+
+    // ---- plan: same chunking rule as the context path, into fixed-capacity arrays
+    const int32_t B = desc->block_size, Hq = desc->num_q_heads, D = desc->head_dim;
+    PlanConfig cfg;
+    cfg.num_sms = su.num_sms;
+    int64_t total_pages = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int32_t lc = context_len[s];
+        if (lc < 1) return CF_ERR_INVALID_ARG;                       // every sequence decodes one token
+        if ((int64_t)lc > (int64_t)max_blocks_per_seq * B) return CF_ERR_OUT_OF_RANGE;
+        total_pages += (lc + B - 1) / B;
+    }
+    const int64_t slots = (int64_t)cfg.num_sms * cfg.decode_ctas_per_sm * cfg.decode_waves;
+    const int32_t quantum = cfg.decode_page_quantum;
+    int64_t target = (total_pages * desc->num_kv_heads + slots - 1) / slots;
+    if (target < cfg.decode_min_chunk_pages) target = cfg.decode_min_chunk_pages;
+    target = (target + quantum - 1) / quantum * quantum;
+
+    StaticPlan pl;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int32_t lc = context_len[s];
+        const int64_t pages = (lc + B - 1) / B;
+        int64_t n = (pages + target - 1) / target;
+        int64_t per = (pages + n - 1) / n;
+        per = (per + quantum - 1) / quantum * quantum;
+        n = (pages + per - 1) / per;
+        if (pl.n_items + n > kStaticMaxItems) return CF_ERR_WORKSPACE;
+        int32_t first = -1;
+        if (n > 1) {
+            first = pl.n_slots;
+            pl.comb[pl.n_comb++] = CombineItem{s, first, (int32_t)n};
+            pl.n_slots += (int32_t)n;
+        }
+        for (int64_t c = 0; c < n; ++c) {
+            DecodeItem& it = pl.items[pl.n_items++];
+            it.seq = s;
+            it.q_row = s;
+            it.kv_begin = (int32_t)(c * per * B);
+            it.kv_end = (int32_t)(((c + 1) * per * B < lc) ? (c + 1) * per * B : lc);
+            it.part_slot = n > 1 ? first + (int32_t)c : -1;
+            it.chunk = (int32_t)c;
+        }
+    }
+    const size_t items_bytes = sizeof(DecodeItem) * (size_t)pl.n_items;
+    const size_t comb_off = (items_bytes + 255) / 256 * 256;
+    const size_t comb_bytes = sizeof(CombineItem) * (size_t)pl.n_comb;
+    if (comb_off + comb_bytes > kStaticPlanBytes) return CF_ERR_WORKSPACE;
+    const size_t part_o_bytes = ((size_t)pl.n_slots * Hq * D * sizeof(float) + 255) / 256 * 256;
+    const size_t part_ml_bytes = (size_t)pl.n_slots * Hq * 2 * sizeof(float);
+    if (kStaticPlanBytes + part_o_bytes + part_ml_bytes > kStaticScratchBytes) return CF_ERR_WORKSPACE;
+
+    // Pageable-source copies: the runtime stages the bytes before returning, so the stack arrays
+    // may go out of scope as soon as this function returns.
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    if (cudaMemcpyAsync(su.base, pl.items, items_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (comb_bytes &&
+        cudaMemcpyAsync(su.base + comb_off, pl.comb, comb_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
+        return CF_ERR_CUDA;
+
+    AttnParams p;
+    p.q = (const __nv_bfloat16*)q;
+    p.k_cache = (const __nv_bfloat16*)k_cache;
+    p.v_cache = (const __nv_bfloat16*)v_cache;
+    p.out = (__nv_bfloat16*)out;
+    p.lse = lse;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks_per_seq;
+    p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
+    p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
+    p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
+    p.scale_log2 = (desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf((float)D)) * 1.4426950408889634f;
+    p.context_len = nullptr; p.query_len = nullptr; p.q_start = nullptr;   // not read by these two kernels
+    p.dec_items = reinterpret_cast<const DecodeItem*>(su.base);
+    p.comb_items = reinterpret_cast<const CombineItem*>(su.base + comb_off);
+    p.pre_items = nullptr;
+    // Partials need no clearing: every slot the combine kernel reads is fully written by its decode CTA
+    // in the same call.
+    p.part_o = reinterpret_cast<float*>(su.base + kStaticPlanBytes);
+    p.part_ml = reinterpret_cast<float*>(su.base + kStaticPlanBytes + part_o_bytes);
+    p.err = nullptr;
+    if (launch_decode(p, D, pl.n_items, stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (launch_combine(p, D, pl.n_comb, stream) != cudaSuccess) return CF_ERR_CUDA;
+    return CF_OK;
+}
