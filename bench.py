@@ -405,15 +405,49 @@ def write_report(torch, cf, ctx, stream, peaks):
               file=sys.stderr, flush=True)
 
 
+def small_case(name: str) -> syn.Scenario:
+    """Reduced workloads for profiler captures (inputs still larger than L2 for the decode case,
+    under 1.5 GB on the device)."""
+    if name == "decode_small":
+        geom = syn.Geometry(32, 8, 128, 16, 16384)
+        lens = syn.uniform_int(np.random.default_rng(42), 32, 2048, 6144)
+        return syn.scenario_from_lengths(name, geom, 43, lens - 1, [[1] * 32])
+    if name == "prefill_small":
+        geom = syn.Geometry(32, 8, 128, 16, 4096)
+        return syn.scenario_from_lengths(name, geom, 44, [3072], [[1024]])
+    raise SystemExit(f"unknown case {name}")
+
+
+def run_case(args):
+    """Runs one reduced workload for `warmup + steps` steps and prints its per-kernel times."""
+    import torch
+    import paper_2609_27085_b200 as cf
+    torch.cuda.set_device(0)
+    peaks = load_peaks()
+    ctx = cf.cf_create(0)
+    wl = DeviceWorkload(small_case(args.case), torch, cf, ctx)
+    stream = torch.cuda.current_stream()
+    for i in range(args.warmup):
+        wl.step(i, stream)
+    kern, launches = measure_kernels(torch, cf, wl, args.steps, stream, peaks)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": args.case, "steps": args.steps, "kernels": kern, "gpu_launches": launches}), flush=True)
+    del wl
+    cf.cf_destroy(ctx)
+
+
 def main():
     ap = argparse.ArgumentParser()
+    ap.add_argument("--case", default=None, help="run a reduced workload (decode_small | prefill_small) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--report", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.case:
+        run_case(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
