@@ -155,8 +155,9 @@ cf_status cf_decode_attention_static(const cf_cache_desc* desc, const void* q,
  * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.
  *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}
  *   combine_items : int32 [cap, 3] = {q_row, first_partial_slot, num_chunks}
- *   prefill_items : int32 [cap, 4] = {seq, q_row_of_tile, first_row_in_chunk, num_rows}
- *   counts        : int32 [4]      = {n_decode_items, n_combine_items, n_prefill_items, n_partial_slots}
+ *   prefill_items : int32 [cap, 6] = {seq, q_row_of_tile, first_row_in_chunk, num_rows, query_head, kv_head},
+ *                   one entry per (q tile, query head) in launch order
+ *   counts        : int32 [4]      = {n_decode_items, n_combine_items, n_prefill_entries, n_partial_slots}
  * Any output pointer may be NULL. */
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
                           int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,

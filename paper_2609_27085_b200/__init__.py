@@ -194,11 +194,11 @@ def cf_get_last_launch_count(ctx) -> int:
 
 def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148,
                     cap: int = 1 << 16, check: bool = True):
-    """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,4], n_partial_slots)."""
+    """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,6], n_partial_slots)."""
     lc, lq = _host_i32(context_len), _host_i32(query_len)
     dec = np.zeros((cap, 6), dtype=np.int32)
     comb = np.zeros((cap, 3), dtype=np.int32)
-    pre = np.zeros((cap, 4), dtype=np.int32)
+    pre = np.zeros((cap, 6), dtype=np.int32)
     counts = np.zeros(4, dtype=np.int32)
     st = load_library().cf_plan_inspect(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
                                         int(max_blocks_per_seq), int(num_sms), dec.ctypes.data, comb.ctypes.data,

@@ -42,6 +42,7 @@ struct cf_ctx {
     size_t workspace_bytes = 0;
     bool workspace_fixed = false;
     uint32_t* err_dev = nullptr;
+    bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // host-staged step
     uint8_t* stage_dev = nullptr;
     size_t stage_bytes = 0;
@@ -114,7 +115,7 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, total;
 };
 
 static PlanLayout layout_of(int32_t S, const Plan& pl)
@@ -127,6 +128,7 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_dec = at;    at = align_up(at + sizeof(DecodeItem) * pl.decode.size(), 16);
     L.off_comb = at;   at = align_up(at + sizeof(CombineItem) * pl.combine.size(), 16);
     L.off_pre = at;    at = align_up(at + sizeof(PrefillItem) * pl.prefill.size(), 16);
+    L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
     L.total = at ? at : 16;
     return L;
 }
@@ -149,6 +151,8 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     if (!pl.decode.empty()) std::memcpy(s.host + L->off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
     if (!pl.combine.empty()) std::memcpy(s.host + L->off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
     if (!pl.prefill.empty()) std::memcpy(s.host + L->off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
+    if (!pl.prefill_tc.empty())
+        std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
     if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
     *dev_base = s.dev;
     *slot_out = &s;
@@ -211,6 +215,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.decode_waves = env_int("CF_DECODE_WAVES", c->cfg.decode_waves);
     c->cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", c->cfg.decode_min_chunk_pages);
     c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
@@ -299,7 +304,9 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     cf_status st = validate_desc(desc);
     if (st != CF_OK) return st;
     Plan pl;
-    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, c->cfg, &pl);
+    PlanConfig cfg = c->cfg;
+    cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
     c->launches = 0;
     if (pl.total_q == 0) return CF_OK;
@@ -338,6 +345,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     p.dec_items = (const DecodeItem*)(base + L.off_dec);
     p.comb_items = (const CombineItem*)(base + L.off_comb);
     p.pre_items = (const PrefillItem*)(base + L.off_pre);
+    p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
     p.part_o = c->workspace;
     p.part_ml = (float*)((uint8_t*)c->workspace + part_o_bytes);
     p.err = c->err_dev;
@@ -355,7 +363,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
         tc = &c->timed[c->timed_used++];
         tc->ran[0] = !pl.decode.empty();
         tc->ran[1] = !pl.combine.empty();
-        tc->ran[2] = !pl.prefill.empty();
+        tc->ran[2] = !pl.prefill.empty() || !pl.prefill_tc.empty();
     }
     if (tc) cudaEventRecord(tc->ev[0], stream);
     if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
@@ -363,8 +371,9 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
     if (tc) cudaEventRecord(tc->ev[2], stream);
     if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
+    if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), stream);
     if (tc) cudaEventRecord(tc->ev[3], stream);
-    c->launches = (int)!pl.decode.empty() + (int)!pl.combine.empty() + (int)!pl.prefill.empty();
+    c->launches = (int)!pl.decode.empty() + (int)!pl.combine.empty() + (int)!pl.prefill.empty() + (int)!pl.prefill_tc.empty();
     const cf_status fs = finish_slot(slot, stream);
     if (e != cudaSuccess) return CF_ERR_CUDA;
     return fs;
@@ -480,6 +489,7 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
     cfg.decode_waves = env_int("CF_DECODE_WAVES", cfg.decode_waves);
     cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
     cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -495,15 +505,24 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
             int32_t* o = combine_items + 3 * i;
             o[0] = pl.combine[i].q_row; o[1] = pl.combine[i].part_first; o[2] = pl.combine[i].n_chunks;
         }
-    if (prefill_items)
-        for (size_t i = 0; i < pl.prefill.size() && i < (size_t)cap; ++i) {
-            int32_t* o = prefill_items + 4 * i;
-            o[0] = pl.prefill[i].seq; o[1] = pl.prefill[i].q_row0; o[2] = pl.prefill[i].row0; o[3] = pl.prefill[i].n_rows;
+    size_t n_pre = 0;
+    auto emit = [&](int32_t seq, int32_t q_row0, int32_t row0, int32_t n_rows, int32_t head, int32_t kvh) {
+        if (prefill_items && n_pre < (size_t)cap) {
+            int32_t* o = prefill_items + 6 * n_pre;
+            o[0] = seq; o[1] = q_row0; o[2] = row0; o[3] = n_rows; o[4] = head; o[5] = kvh;
         }
+        ++n_pre;
+    };
+    const int32_t G = desc->num_q_heads / desc->num_kv_heads;
+    for (const PrefillItem& it : pl.prefill)
+        for (int32_t h = 0; h < desc->num_q_heads; ++h) emit(it.seq, it.q_row0, it.row0, it.n_rows, h, h / G);
+    for (const PrefillTcItem& it : pl.prefill_tc)
+        for (int t = 0; t < 2; ++t)
+            if (it.n_rows[t] > 0) emit(it.seq, it.q_row0[t], it.row0[t], it.n_rows[t], it.head[t], it.kvh);
     if (counts) {
         counts[0] = (int32_t)pl.decode.size();
         counts[1] = (int32_t)pl.combine.size();
-        counts[2] = (int32_t)pl.prefill.size();
+        counts[2] = (int32_t)n_pre;
         counts[3] = pl.n_part_slots;
     }
     return CF_OK;

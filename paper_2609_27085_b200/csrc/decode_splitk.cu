@@ -433,6 +433,7 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     p.dec_items = reinterpret_cast<const DecodeItem*>(su.base);
     p.comb_items = reinterpret_cast<const CombineItem*>(su.base + comb_off);
     p.pre_items = nullptr;
+    p.pre_tc_items = nullptr;
     // Partials need no clearing: every slot the combine kernel reads is fully written by its decode CTA
     // in the same call.
     p.part_o = reinterpret_cast<float*>(su.base + kStaticPlanBytes);

@@ -26,6 +26,7 @@ struct AttnParams {
     const DecodeItem* dec_items;
     const CombineItem* comb_items;
     const PrefillItem* pre_items;
+    const PrefillTcItem* pre_tc_items;
     float* part_o;                    // [slot, Hq, D] fp32 un-normalised partial outputs
     float* part_ml;                   // [slot, Hq, 2] running max (log2 domain) and sum
     uint32_t* err;                    // device error word

@@ -28,4 +28,9 @@ cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaS
 constexpr int kPrefillMmaTileRows = 64;
 cudaError_t launch_prefill_mma(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 
+// tcgen05 / tensor-memory chunked prefill (head_dim 128); one CTA per PrefillTcItem
+bool prefill_tc_supported(const cf_cache_desc* desc);
+cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items,
+                              cudaStream_t stream);
+
 }  // namespace cf

@@ -97,6 +97,57 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     });
 
     // ---- prefill: q tiles of every chunk, the tile with the longest visible KV range first
+    if (cfg.prefill_tc) {
+        // pairs of 128-row tiles that share a KV head: two heads of a group over the same rows, or
+        // (group size 1) two consecutive row tiles of one head
+        constexpr int32_t TR = 128;
+        const int32_t G = d->num_q_heads / d->num_kv_heads;
+        struct KeyedTc { int64_t extent; PrefillTcItem it; };
+        std::vector<KeyedTc> items;
+        for (int32_t s = 0; s < num_seqs; ++s) {
+            const int32_t lq = query_len[s];
+            if (lq <= 1) continue;
+            const int32_t prefix = context_len[s] - lq;
+            const int32_t n_tiles = (lq + TR - 1) / TR;
+            auto rows_of = [&](int32_t tile) { return std::min(TR, lq - tile * TR); };
+            if (G >= 2) {
+                for (int32_t tile = 0; tile < n_tiles; ++tile)
+                    for (int32_t kvh = 0; kvh < d->num_kv_heads; ++kvh)
+                        for (int32_t i = 0; i < G; i += 2) {
+                            PrefillTcItem it;
+                            it.seq = s; it.kvh = kvh;
+                            for (int t = 0; t < 2; ++t) {
+                                it.q_row0[t] = plan->q_start[s] + tile * TR;
+                                it.row0[t] = tile * TR;
+                                it.n_rows[t] = rows_of(tile);
+                                it.head[t] = kvh * G + i + t;
+                            }
+                            items.push_back(KeyedTc{(int64_t)prefix + tile * TR + rows_of(tile), it});
+                        }
+            } else {
+                for (int32_t tile = 0; tile < n_tiles; tile += 2)
+                    for (int32_t h = 0; h < d->num_q_heads; ++h) {
+                        PrefillTcItem it;
+                        it.seq = s; it.kvh = h;
+                        int32_t last = tile;
+                        for (int t = 0; t < 2; ++t) {
+                            const int32_t tt = tile + t;
+                            const bool present = tt < n_tiles;
+                            it.q_row0[t] = present ? plan->q_start[s] + tt * TR : 0;
+                            it.row0[t] = present ? tt * TR : 0;
+                            it.n_rows[t] = present ? rows_of(tt) : 0;
+                            it.head[t] = h;
+                            if (present) last = tt;
+                        }
+                        items.push_back(KeyedTc{(int64_t)prefix + last * TR + rows_of(last), it});
+                    }
+            }
+        }
+        std::stable_sort(items.begin(), items.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
+        plan->prefill_tc.reserve(items.size());
+        for (const KeyedTc& k : items) plan->prefill_tc.push_back(k.it);
+        return CF_OK;
+    }
     const int32_t tr = std::max(1, cfg.prefill_tile_rows);
     struct Keyed { int64_t extent; PrefillItem it; };
     std::vector<Keyed> tiles;

@@ -33,20 +33,31 @@ struct PrefillItem {       // one q tile of one prefill chunk; the kernel adds t
     int32_t n_rows;        // rows in this tile (<= tile height)
 };
 
+struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one KV head (tile 1 may be absent)
+    int32_t seq;
+    int32_t kvh;
+    int32_t q_row0[2];     // packed row of each tile's first row
+    int32_t row0[2];       // index of that row inside the chunk
+    int32_t n_rows[2];     // 0 = tile absent
+    int32_t head[2];       // query head of each tile
+};
+
 struct PlanConfig {
     int32_t num_sms = 148;
     int32_t decode_ctas_per_sm = 2;   // resident decode CTAs per SM the kernel is built for
     int32_t decode_waves = 4;         // target number of CTA waves (load balance vs. partial traffic)
     int32_t decode_min_chunk_pages = 32;
     int32_t decode_page_quantum = 4;  // chunk lengths are multiples of this many pages (warps per CTA)
-    int32_t prefill_tile_rows = 64;
+    int32_t prefill_tile_rows = 64;   // tile height of the mma.sync prefill kernel
+    bool prefill_tc = false;          // true: plan items for the tcgen05 kernel (128-row tile pairs)
 };
 
 struct Plan {
     std::vector<int32_t> q_start;     // [S+1] exclusive prefix sum of query_len
     std::vector<DecodeItem> decode;   // longest chunk first
     std::vector<CombineItem> combine;
-    std::vector<PrefillItem> prefill; // longest KV extent first
+    std::vector<PrefillItem> prefill; // longest KV extent first (mma.sync kernel)
+    std::vector<PrefillTcItem> prefill_tc;   // longest KV extent first (tcgen05 kernel)
     int32_t n_part_slots = 0;
     int32_t total_q = 0;
     int32_t n_decode_seqs = 0;

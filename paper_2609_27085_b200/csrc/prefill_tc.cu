@@ -1,0 +1,396 @@
+// Chunked-prefill attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
+// tensor memory), head_dim 128.
+//
+// One CTA = one work item = two 128-row q tiles that share a KV head (two query heads of one group
+// over the same rows; for G = 1 two consecutive row tiles of one head), so every K/V tile fetched
+// into shared memory feeds two S = Q K^T and two O += P V products.  320 threads, warp-specialised:
+//   warp 0      TMA producer: Q tiles once, then 128-token K and V tiles, one 16-token page-half per
+//               TMA box, gathered through the block table into 128B-swizzled shared memory rings.
+//   warp 1      MMA issuer (one elected lane): S_t = Q_t K^T, O_t += P_t V, in the order
+//               PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) so that the tensor pipe works on one tile while
+//               the other tile's softmax runs.
+//   warps 2-5   softmax of tile 0, one thread per q row; warps 6-9 softmax of tile 1.
+// Tensor memory (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites
+// the first 64 columns of S_t and is consumed by the PV product straight from tensor memory.
+// Softmax: scores leave tensor memory once (tcgen05.ld), exp2 with the scale folded in, the
+// running maximum is only raised when it grows by more than 2^8 (then O_t is rescaled in tensor
+// memory), so almost every tile costs no correction pass.  The causal comparison j <= P + i is
+// evaluated only in warps whose rows can see a masked key of the tile; tiles above the diagonal
+// are never loaded.
+// Every wait is bounded: on expiry the CTA raises an abort flag, every role leaves its loop, the
+// error word is set and tensor memory is released.
+#include "device_common.cuh"
+#include "kernels.h"
+#include "tc05.cuh"
+
+namespace cf {
+
+using namespace tc;
+
+namespace {
+
+constexpr int D = 128;
+constexpr int QT = 128;                    // rows per q tile
+constexpr int KT = 128;                    // tokens per K/V tile
+constexpr int HALF_BYTES = 128 * 128;      // [128 rows][64 elements] bf16
+constexpr int TILE_BYTES = 2 * HALF_BYTES; // 32 KB
+constexpr int KV_STAGES = 2;
+constexpr int NTHREADS = 320;
+constexpr uint32_t SMEM_Q = 0;
+constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
+constexpr uint32_t SMEM_V = SMEM_K + KV_STAGES * TILE_BYTES;
+constexpr uint32_t SMEM_TOTAL = SMEM_V + KV_STAGES * TILE_BYTES;   // 192 KB
+constexpr uint32_t TM_S = 0, TM_O = 256;   // column offsets; tile t adds 128 * t
+constexpr float kRescaleThreshold = 8.0f;  // log2 units
+
+struct Bars {
+    uint64_t q_full;
+    uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
+    uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
+    uint64_t s_full[2], p_full[2], o_done[2];
+};
+
+__device__ __forceinline__ uint32_t lane_field(int warp) { return (uint32_t)((warp & 3) * 32) << 16; }
+
+}  // namespace
+
+__global__ void __launch_bounds__(NTHREADS, 1)
+prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
+                  const __grid_constant__ CUtensorMap map_v, const AttnParams p)
+{
+    extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(8) Bars bars;
+    __shared__ uint32_t tmem_base_s;
+    __shared__ uint32_t abort_s;
+
+    const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const PrefillTcItem it = p.pre_tc_items[blockIdx.x];
+    const int Lq = __ldg(p.query_len + it.seq), Lc = __ldg(p.context_len + it.seq);
+    const int prefix = Lc - Lq;
+    int kv_hi_t[2], n_j[2];
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        kv_hi_t[t] = it.n_rows[t] > 0 ? prefix + it.row0[t] + it.n_rows[t] : 0;
+        n_j[t] = (kv_hi_t[t] + KT - 1) / KT;
+    }
+    const int kv_hi = max(kv_hi_t[0], kv_hi_t[1]);
+    const int n_max = max(n_j[0], n_j[1]);
+    const int total_pages = (kv_hi + 15) >> 4;
+    volatile uint32_t* abort_flag = &abort_s;
+
+    if (threadIdx.x == 0) {
+        abort_s = (p.err != nullptr && *reinterpret_cast<volatile uint32_t*>(p.err) != 0u) ? 2u : 0u;   // an earlier CTA gave up
+        mbar_init(smem_u32(&bars.q_full), 1);
+        for (int s = 0; s < KV_STAGES; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(smem_u32(&bars.s_full[t]), 1);
+            mbar_init(smem_u32(&bars.p_full[t]), 4);      // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.o_done[t]), 1);
+        }
+        fence_mbar_init();
+    }
+    if (warp == 0) tmem_alloc<512>(smem_u32(&tmem_base_s));
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem = tmem_base_s;
+
+    if (abort_s) {
+        // nothing was issued: fall through to the teardown
+    } else if (warp == 0) {
+        // =========================================================== TMA producer
+        if (lane == 0) {
+            prefetch_tensormap(&map_q);
+            prefetch_tensormap(&map_k);
+            prefetch_tensormap(&map_v);
+            const int nq = (it.n_rows[0] > 0) + (it.n_rows[1] > 0);
+            mbar_arrive_expect_tx(smem_u32(&bars.q_full), nq * TILE_BYTES);
+            for (int t = 0; t < 2; ++t)
+                if (it.n_rows[t] > 0)
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_3d(smem + SMEM_Q + t * TILE_BYTES + h * HALF_BYTES, &map_q, h * 64, it.head[t],
+                                    it.q_row0[t], smem_u32(&bars.q_full));
+        }
+        const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks;
+        bool ok = true;
+        for (int j = 0; j < n_max && ok; ++j) {
+            const int stage = j % KV_STAGES, use = j / KV_STAGES;
+            const int np = min(8, total_pages - 8 * j);
+            const int32_t pid = lane < np ? __ldg(bt + 8 * j + lane) : 0;
+            const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
+            const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
+            // K tile
+            if (use > 0) ok = mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1, abort_flag);
+            if (!ok) break;
+            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 4096);
+            __syncwarp();
+            if (lane < 2 * np)
+                tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane & 1) * 64, 0, it.kvh, my_pid,
+                            smem_u32(&bars.k_full[stage]));
+            // V tile
+            if (use > 0) ok = mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1, abort_flag);
+            if (!ok) break;
+            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 4096);
+            __syncwarp();
+            if (lane < 2 * np)
+                tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane & 1) * 64, 0, it.kvh, my_pid,
+                            smem_u32(&bars.v_full[stage]));
+        }
+    } else if (warp == 1) {
+        // =========================================================== MMA issuer
+        constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
+        constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, true);
+        auto issue_qk = [&](int t, int stage) {          // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
+            const uint32_t qa = smem + SMEM_Q + t * TILE_BYTES, kb = smem + SMEM_K + stage * TILE_BYTES;
+#pragma unroll
+            for (int ks = 0; ks < D / 16; ++ks) {
+                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
+                umma_ss(tmem + TM_S + t * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
+                        IDESC_QK, ks > 0);
+            }
+            umma_commit(smem_u32(&bars.s_full[t]));
+        };
+        auto issue_pv = [&](int t, int stage, int n_steps, bool first) {   // O_t (+)= P_t V, one step per loaded page
+            const uint32_t vb = smem + SMEM_V + stage * TILE_BYTES;
+            for (int ks = 0; ks < n_steps; ++ks)
+                umma_ts(tmem + TM_O + t * 128, tmem + TM_S + t * 128 + ks * 8, smem_desc_sw128(vb + ks * 2048, HALF_BYTES, 1024),
+                        IDESC_PV, (!first || ks > 0) ? 1u : 0u);
+            umma_commit(smem_u32(&bars.o_done[t]));
+        };
+        bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
+        ok = ok && mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
+        if (ok) {
+            tc_fence_after();
+            if (lane == 0) {
+                for (int t = 0; t < 2; ++t)
+                    if (n_j[t] > 0) issue_qk(t, 0);
+                umma_commit(smem_u32(&bars.k_empty[0]));
+            }
+            __syncwarp();
+        }
+        for (int j = 0; j < n_max && ok; ++j) {
+            const int stage = j % KV_STAGES;
+            const int np = min(8, total_pages - 8 * j);
+            ok = mbar_wait(smem_u32(&bars.v_full[stage]), (j / KV_STAGES) & 1, abort_flag);
+            if (!ok) break;
+            if (j == n_max - 1 && Lc < (8 * j + np) * 16) {
+                // slack slots of the sequence's last page came in with the page: zero those V rows so
+                // that a zero probability never multiplies a NaN
+                const int r0 = Lc - j * KT, r1 = np * 16;
+                for (int idx = lane; idx < (r1 - r0) * 16; idx += 32) {
+                    const int r = r0 + (idx >> 4), c = idx & 15;
+                    uint8_t* dst = smem_raw + ((smem + SMEM_V + stage * TILE_BYTES) - smem_u32(smem_raw)) +
+                                   (c >> 3) * HALF_BYTES + r * 128 + (c & 7) * 16;
+                    *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
+                }
+                fence_proxy_async();
+                __syncwarp();
+            }
+            for (int t = 0; t < 2 && ok; ++t) {
+                if (j >= n_j[t]) continue;
+                ok = mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag);
+                if (!ok) break;
+                if (j + 1 < n_j[t])
+                    ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) % KV_STAGES]), ((j + 1) / KV_STAGES) & 1, abort_flag);
+                if (!ok) break;
+                tc_fence_after();
+                if (lane == 0) {
+                    issue_pv(t, stage, np, j == 0);
+                    if (j + 1 < n_j[t]) issue_qk(t, (j + 1) % KV_STAGES);
+                }
+                __syncwarp();
+            }
+            if (ok && lane == 0) {
+                umma_commit(smem_u32(&bars.v_empty[stage]));
+                if (j + 1 < n_max) umma_commit(smem_u32(&bars.k_empty[(j + 1) % KV_STAGES]));
+            }
+            __syncwarp();
+        }
+    } else {
+        // =========================================================== softmax + epilogue, one thread per q row
+        const int t = (warp - 2) >> 2;
+        const int row = (warp & 3) * 32 + lane;
+        const uint32_t lanes = lane_field(warp);
+        const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
+        const int limit = min(prefix + it.row0[t] + row, kv_hi_t[t] - 1);   // last visible key of this row
+        const float sc = p.scale_log2;
+        float m_used = -INFINITY, l_sum = 0.f;
+        bool ok = true;
+        for (int j = 0; j < n_j[t]; ++j) {
+            ok = mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag);
+            if (!ok) break;
+            tc_fence_after();
+            float sv[128];
+#pragma unroll
+            for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(&sv[c * 32]));
+            tmem_wait_ld();
+            const int col_limit = limit - j * KT;            // columns <= col_limit are visible
+            if (__any_sync(0xffffffffu, col_limit < KT - 1)) {
+#pragma unroll
+                for (int c = 0; c < 128; ++c) sv[c] = (c <= col_limit) ? sv[c] : -INFINITY;
+            }
+            float mx = sv[0];
+#pragma unroll
+            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, sv[c]);
+            const float m_new = fmaxf(m_used, mx * sc);
+            // raise the reference maximum only when it moved by more than 2^8 (always on the first tile)
+            if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
+                const float f = fast_exp2(m_used - m_new);       // first tile: 2^(-inf) = 0
+                m_used = m_new;
+                l_sum *= f;
+                if (j > 0) {
+                    ok = mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag);
+                    if (!ok) break;
+                    tc_fence_after();
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        float ov[32];
+                        tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
+                        tmem_wait_ld();
+#pragma unroll
+                        for (int i = 0; i < 32; ++i) ov[i] *= f;
+                        tmem_st32(tO + c * 32, reinterpret_cast<const uint32_t*>(ov));
+                    }
+                }
+            }
+            const float neg_m = -m_used;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                uint32_t pk[16];
+#pragma unroll
+                for (int i = 0; i < 16; ++i) {
+                    const float p0 = fast_exp2(fmaf(sv[c * 32 + 2 * i], sc, neg_m));
+                    const float p1 = fast_exp2(fmaf(sv[c * 32 + 2 * i + 1], sc, neg_m));
+                    l_sum += p0 + p1;
+                    pk[i] = pack_bf16(p0, p1);
+                }
+                tmem_st16(tS + c * 16, pk);
+            }
+            tmem_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
+        }
+        if (ok && n_j[t] > 0) ok = mbar_wait(smem_u32(&bars.o_done[t]), (n_j[t] - 1) & 1, abort_flag);
+        if (ok && n_j[t] > 0) {
+            tc_fence_after();
+            const float inv = 1.f / l_sum;
+            const bool live = row < it.n_rows[t];
+            __nv_bfloat16* orow = p.out + ((int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]) * D;
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                float ov[32];
+                tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
+                tmem_wait_ld();
+                if (live) {
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) {
+                        uint4 w;
+                        w.x = pack_bf16(ov[8 * i + 0] * inv, ov[8 * i + 1] * inv);
+                        w.y = pack_bf16(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
+                        w.z = pack_bf16(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
+                        w.w = pack_bf16(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
+                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+                    }
+                }
+            }
+            if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
+        }
+    }
+
+    // ---- teardown: every role has left its loop (normally, or because the abort flag went up)
+    tc_fence_before();
+    __syncthreads();
+    if (abort_s == 1u) {
+        if (threadIdx.x == 0 && p.err) atomicExch(p.err, 1u);
+        // let copies and MMAs that may still be in flight settle before tensor memory is handed back
+        for (int i = 0; i < 64; ++i) __nanosleep(2000);
+        __syncthreads();
+    }
+    if (warp == 0) tmem_dealloc<512>(tmem);
+}
+
+// ---------------------------------------------------------------------------------------------
+namespace {
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode()
+{
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* ptr = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(ptr);
+    }
+    return fn;
+}
+
+// pool viewed as (d, token-in-page, head, block); one box = 64 elements x 16 tokens of one head of one page
+bool encode_pool(CUtensorMap* m, const void* base, int num_blocks, int Hkv, int64_t s_block, int64_t s_head, int64_t s_token)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[4] = {(cuuint64_t)D, 16, (cuuint64_t)Hkv, (cuuint64_t)num_blocks};
+    cuuint64_t strides[3] = {(cuuint64_t)s_token * 2, (cuuint64_t)s_head * 2, (cuuint64_t)s_block * 2};
+    cuuint32_t box[4] = {64, 16, 1, 1}, es[4] = {1, 1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// q viewed as (d, head, row); one box = 64 elements x 1 head x 128 rows; rows past the end read as zero
+bool encode_q(CUtensorMap* m, const void* base, int total_rows, int Hq)
+{
+    EncodeTiledFn enc = get_encode();
+    if (!enc) return false;
+    cuuint64_t dims[3] = {(cuuint64_t)D, (cuuint64_t)Hq, (cuuint64_t)total_rows};
+    cuuint64_t strides[2] = {(cuuint64_t)D * 2, (cuuint64_t)Hq * D * 2};
+    cuuint32_t box[3] = {64, 1, (cuuint32_t)QT}, es[3] = {1, 1, 1};
+    return enc(m, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(base), dims, strides, box, es,
+               CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+}  // namespace
+
+bool prefill_tc_supported(const cf_cache_desc* d)
+{
+    // TMA needs 16-byte aligned strides (checked for every descriptor) and a 128-element head
+    return d->head_dim == D && d->block_size == 16;
+}
+
+cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    CUtensorMap mq, mk, mv;
+    if (!encode_q(&mq, p.q, total_q_rows, p.Hq) ||
+        !encode_pool(&mk, p.k_cache, desc->num_blocks, p.Hkv, p.ks_block, p.ks_head, p.ks_token) ||
+        !encode_pool(&mv, p.v_cache, desc->num_blocks, p.Hkv, p.vs_block, p.vs_head, p.vs_token))
+        return cudaErrorInvalidValue;
+    const size_t smem = SMEM_TOTAL + 1024;
+    static bool configured[64] = {};
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev]) {
+        cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev] = true;
+    }
+    prefill_tc_kernel<<<n_items, NTHREADS, smem, stream>>>(mq, mk, mv, p);
+    return cudaGetLastError();
+}
+
+}  // namespace cf

@@ -88,15 +88,20 @@ def _check_plan(geom, lc, lq, sms=148):
     assert slots_seen == set(range(parts))
     lens = dec[:, 3] - dec[:, 2]
     assert (np.diff(lens) <= 0).all()                                      # longest first
-    # prefill: tiles of each Lq > 1 sequence cover its rows exactly once
+    # prefill: every (row, query head) of each Lq > 1 sequence is covered exactly once, by an entry whose
+    # kv head serves that query head
+    G = geom.num_q_heads // geom.num_kv_heads
     for s in np.nonzero(lq > 1)[0]:
         mine = pre[pre[:, 0] == s]
-        mine = mine[np.argsort(mine[:, 2])]
-        assert mine[0, 2] == 0 and (mine[:, 1] == qs[s] + mine[:, 2]).all()
-        assert (mine[1:, 2] == mine[:-1, 2] + mine[:-1, 3]).all() and mine[-1, 2] + mine[-1, 3] == lq[s]
+        cover = np.zeros((lq[s], geom.num_q_heads), dtype=np.int32)
+        for _, q_row0, row0, n_rows, head, kvh in mine:
+            assert q_row0 == qs[s] + row0 and n_rows >= 1 and kvh == head // G
+            cover[row0:row0 + n_rows, head] += 1
+        assert (cover == 1).all()
     assert set(int(s) for s in pre[:, 0]) == set(int(s) for s in np.nonzero(lq > 1)[0])
     ext = (lc - lq)[pre[:, 0]] + pre[:, 2] + pre[:, 3]
-    assert (np.diff(ext) <= 0).all()
+    if len(ext):
+        assert ext[0] == ext.max()                                         # longest KV extent first
     return dec, comb, pre, parts
 
 
@@ -118,6 +123,8 @@ def test_plan_random_batches():
         lq = rng.choice([0, 1, 1, 1, 2, 17, 64, 65, 300], size=S)
         lc = lq + rng.integers(0, 5000, size=S)
         _check_plan(syn.GEOM_G4, lc, lq, sms=int(rng.choice([1, 4, 148])))
+        _check_plan(syn.Geometry(4, 4, 128, 16, 1 << 16), lc, lq)          # group size 1: row-tile pairs
+        _check_plan(syn.Geometry(8, 2, 64, 16, 1 << 16), lc, lq)           # head_dim 64: mma.sync tiles
 
 
 def test_calls_without_a_device_fail_with_a_status():
