@@ -3,13 +3,14 @@
 //
 // One CTA = one work item = two 128-row q tiles that share a KV head (two query heads of one group
 // over the same rows; for G = 1 two consecutive row tiles of one head), so every K/V tile fetched
-// into shared memory feeds two S = Q K^T and two O += P V products.  320 threads, warp-specialised:
+// into shared memory feeds two S = Q K^T and two O += P V products.  384 threads, warp-specialised
+// (the first warpgroup hands most of its registers to the two softmax warpgroups with setmaxnreg):
 //   warp 0      TMA producer: Q tiles once, then 128-token K and V tiles, one 16-token page-half per
 //               TMA box, gathered through the block table into 128B-swizzled shared memory rings.
 //   warp 1      MMA issuer (one elected lane): S_t = Q_t K^T, O_t += P_t V, in the order
 //               PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) so that the tensor pipe works on one tile while
 //               the other tile's softmax runs.
-//   warps 2-5   softmax of tile 0, one thread per q row; warps 6-9 softmax of tile 1.
+//   warps 4-7   softmax of tile 0, one thread per q row; warps 8-11 softmax of tile 1.
 // Tensor memory (512 columns): S_0 | S_1 | O_0 | O_1, 128 fp32 columns each; P_t (bf16) overwrites
 // the first 64 columns of S_t and is consumed by the PV product straight from tensor memory.
 // Softmax: scores leave tensor memory once (tcgen05.ld), exp2 with the scale folded in, the
@@ -35,7 +36,8 @@ constexpr int KT = 128;                    // tokens per K/V tile
 constexpr int HALF_BYTES = 128 * 128;      // [128 rows][64 elements] bf16
 constexpr int TILE_BYTES = 2 * HALF_BYTES; // 32 KB
 constexpr int KV_STAGES = 2;
-constexpr int NTHREADS = 320;
+constexpr int NTHREADS = 384;
+constexpr int REGS_ROLE = 48, REGS_SOFTMAX = 224;   // 4*32*48 + 8*32*224 <= 64K registers
 constexpr uint32_t SMEM_Q = 0;
 constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
 constexpr uint32_t SMEM_V = SMEM_K + KV_STAGES * TILE_BYTES;
@@ -51,6 +53,14 @@ struct Bars {
 };
 
 __device__ __forceinline__ uint32_t lane_field(int warp) { return (uint32_t)((warp & 3) * 32) << 16; }
+template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
+template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
+__device__ __forceinline__ float max3(float a, float b, float c)
+{
+    float d;
+    asm("max.f32 %0, %1, %2, %3;" : "=f"(d) : "f"(a), "f"(b), "f"(c));
+    return d;
+}
 
 }  // namespace
 
@@ -101,9 +111,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
 
-    if (abort_s) {
-        // nothing was issued: fall through to the teardown
-    } else if (warp == 0) {
+    const bool live_cta = abort_s == 0;       // otherwise nothing is issued: fall through to the teardown
+    if (warp < 4) {
+      reg_dec<REGS_ROLE>();
+      if (!live_cta || warp >= 2) {
+        // spare warps of the first warpgroup
+      } else if (warp == 0) {
         // =========================================================== TMA producer
         if (lane == 0) {
             prefetch_tensormap(&map_q);
@@ -212,9 +225,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
             __syncwarp();
         }
+      }
     } else {
+      reg_inc<REGS_SOFTMAX>();
+      if (live_cta) {
         // =========================================================== softmax + epilogue, one thread per q row
-        const int t = (warp - 2) >> 2;
+        const int t = (warp - 4) >> 2;
         const int row = (warp & 3) * 32 + lane;
         const uint32_t lanes = lane_field(warp);
         const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
@@ -235,9 +251,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                 for (int c = 0; c < 128; ++c) sv[c] = (c <= col_limit) ? sv[c] : -INFINITY;
             }
-            float mx = sv[0];
+            float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
-            for (int c = 1; c < 128; ++c) mx = fmaxf(mx, sv[c]);
+            for (int c = 4; c < 128; c += 8) {
+                mx4[(c >> 3) & 3] = max3(mx4[(c >> 3) & 3], sv[c], sv[c + 1]);
+                mx4[((c >> 3) + 1) & 3] = max3(mx4[((c >> 3) + 1) & 3], sv[c + 2], sv[c + 3]);
+                if (c + 4 < 128) {
+                    mx4[((c >> 3) + 2) & 3] = max3(mx4[((c >> 3) + 2) & 3], sv[c + 4], sv[c + 5]);
+                    mx4[((c >> 3) + 3) & 3] = max3(mx4[((c >> 3) + 3) & 3], sv[c + 6], sv[c + 7]);
+                }
+            }
+            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
             const float m_new = fmaxf(m_used, mx * sc);
             // raise the reference maximum only when it moved by more than 2^8 (always on the first tile)
             if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
@@ -260,6 +284,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
             }
             const float neg_m = -m_used;
+            float acc[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 uint32_t pk[16];
@@ -267,11 +292,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 for (int i = 0; i < 16; ++i) {
                     const float p0 = fast_exp2(fmaf(sv[c * 32 + 2 * i], sc, neg_m));
                     const float p1 = fast_exp2(fmaf(sv[c * 32 + 2 * i + 1], sc, neg_m));
-                    l_sum += p0 + p1;
+                    acc[i & 3] += p0 + p1;
                     pk[i] = pack_bf16(p0, p1);
                 }
                 tmem_st16(tS + c * 16, pk);
             }
+            l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -302,6 +328,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
             if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
         }
+      }
     }
 
     // ---- teardown: every role has left its loop (normally, or because the abort flag went up)
