@@ -37,13 +37,17 @@ constexpr int HALF_BYTES = 128 * 128;      // [128 rows][64 elements] bf16
 constexpr int TILE_BYTES = 2 * HALF_BYTES; // 32 KB
 constexpr int KV_STAGES = 2;
 constexpr int NTHREADS = 384;
-constexpr int REGS_ROLE = 48, REGS_SOFTMAX = 224;   // 4*32*48 + 8*32*224 <= 64K registers
+// Register hand-over (setmaxnreg).  The kernel launches with LAUNCH_REGS registers per thread; the
+// first warpgroup shrinks to REGS_ROLE and the two softmax warpgroups grow to REGS_SOFTMAX.  A grow
+// request blocks until the CTA's pool holds enough released registers, so the released amount MUST
+// cover the growth or the kernel never returns; the launcher also checks the compiled register count.
+constexpr int LAUNCH_REGS = 168, REGS_ROLE = 88, REGS_SOFTMAX = 208;
+static_assert(4 * (LAUNCH_REGS - REGS_ROLE) >= 8 * (REGS_SOFTMAX - LAUNCH_REGS), "setmaxnreg.inc would block forever");
 constexpr uint32_t SMEM_Q = 0;
 constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
 constexpr uint32_t SMEM_V = SMEM_K + KV_STAGES * TILE_BYTES;
 constexpr uint32_t SMEM_TOTAL = SMEM_V + KV_STAGES * TILE_BYTES;   // 192 KB
 constexpr uint32_t TM_S = 0, TM_O = 256;   // column offsets; tile t adds 128 * t
-constexpr float kRescaleThreshold = 8.0f;  // log2 units
 
 struct Bars {
     uint64_t q_full;
@@ -159,22 +163,57 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // =========================================================== MMA issuer
         constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
         constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, true);
-        auto issue_qk = [&](int t, int stage) {          // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
-            const uint32_t qa = smem + SMEM_Q + t * TILE_BYTES, kb = smem + SMEM_K + stage * TILE_BYTES;
+        // descriptors are built once; each MMA advances the address field with one add
+        constexpr uint32_t HI = desc_hi_sw128(1024);
+        const uint32_t q_lo[2] = {desc_lo_sw128(smem + SMEM_Q, 16), desc_lo_sw128(smem + SMEM_Q + TILE_BYTES, 16)};
+        const uint32_t k_lo[KV_STAGES] = {desc_lo_sw128(smem + SMEM_K, 16), desc_lo_sw128(smem + SMEM_K + TILE_BYTES, 16)};
+        const uint32_t v_lo[KV_STAGES] = {desc_lo_sw128(smem + SMEM_V, HALF_BYTES), desc_lo_sw128(smem + SMEM_V + TILE_BYTES, HALF_BYTES)};
+        const uint32_t bar_s[2] = {smem_u32(&bars.s_full[0]), smem_u32(&bars.s_full[1])};
+        const uint32_t bar_o[2] = {smem_u32(&bars.o_done[0]), smem_u32(&bars.o_done[1])};
+        // The issuing lane shares its scheduler with two softmax warps and runs at only about one
+        // instruction per 10 cycles, while a 128x128x16 MMA lasts 64 cycles: every operand of a batch
+        // is therefore put in registers before the wait, so that the batch itself is MMAs back to back.
+        struct QkOps { uint64_t a[8], b[8]; };
+        struct PvOps { uint32_t a[8]; uint64_t b[8]; };
+        auto d64 = [](uint32_t lo) { return ((uint64_t)HI << 32) | lo; };
+        auto make_qk = [&](int t, int stage) {
+            QkOps o;
 #pragma unroll
-            for (int ks = 0; ks < D / 16; ++ks) {
-                const uint32_t off = (ks >> 2) * HALF_BYTES + (ks & 3) * 32;
-                umma_ss(tmem + TM_S + t * 128, smem_desc_sw128(qa + off, 16, 1024), smem_desc_sw128(kb + off, 16, 1024),
-                        IDESC_QK, ks > 0);
+            for (int ks = 0; ks < 8; ++ks) {
+                const uint32_t off = (uint32_t)(((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4);
+                o.a[ks] = d64(q_lo[t] + off);
+                o.b[ks] = d64(k_lo[stage] + off);
             }
-            umma_commit(smem_u32(&bars.s_full[t]));
+            return o;
         };
-        auto issue_pv = [&](int t, int stage, int n_steps, bool first) {   // O_t (+)= P_t V, one step per loaded page
-            const uint32_t vb = smem + SMEM_V + stage * TILE_BYTES;
-            for (int ks = 0; ks < n_steps; ++ks)
-                umma_ts(tmem + TM_O + t * 128, tmem + TM_S + t * 128 + ks * 8, smem_desc_sw128(vb + ks * 2048, HALF_BYTES, 1024),
-                        IDESC_PV, (!first || ks > 0) ? 1u : 0u);
-            umma_commit(smem_u32(&bars.o_done[t]));
+        auto make_pv = [&](int t, int stage) {
+            PvOps o;
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks) {
+                o.a[ks] = tmem + TM_S + t * 128 + ks * 8;
+                o.b[ks] = d64(v_lo[stage] + ks * (2048 >> 4));
+            }
+            return o;
+        };
+        auto issue_qk = [&](int t, const QkOps& o) {     // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
+            const uint32_t dS = tmem + TM_S + t * 128;
+            umma_ss(dS, o.a[0], o.b[0], IDESC_QK, 0u);
+#pragma unroll
+            for (int ks = 1; ks < 8; ++ks) umma_ss(dS, o.a[ks], o.b[ks], IDESC_QK, 1u);
+            umma_commit(bar_s[t]);
+        };
+        auto issue_pv = [&](int t, const PvOps& o, int n_steps, uint32_t acc0) {   // O_t (+)= P_t V, one step per loaded page
+            const uint32_t dO = tmem + TM_O + t * 128;
+            umma_ts(dO, o.a[0], o.b[0], IDESC_PV, acc0);
+            if (n_steps == 8) {
+#pragma unroll
+                for (int ks = 1; ks < 8; ++ks) umma_ts(dO, o.a[ks], o.b[ks], IDESC_PV, 1u);
+            } else {
+#pragma unroll
+                for (int ks = 1; ks < 8; ++ks)
+                    if (ks < n_steps) umma_ts(dO, o.a[ks], o.b[ks], IDESC_PV, 1u);
+            }
+            umma_commit(bar_o[t]);
         };
         bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
         ok = ok && mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
@@ -182,7 +221,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tc_fence_after();
             if (lane == 0) {
                 for (int t = 0; t < 2; ++t)
-                    if (n_j[t] > 0) issue_qk(t, 0);
+                    if (n_j[t] > 0) issue_qk(t, make_qk(t, 0));
                 umma_commit(smem_u32(&bars.k_empty[0]));
             }
             __syncwarp();
@@ -207,15 +246,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
             for (int t = 0; t < 2 && ok; ++t) {
                 if (j >= n_j[t]) continue;
-                ok = mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag);
-                if (!ok) break;
-                if (j + 1 < n_j[t])
+                const bool more = j + 1 < n_j[t];
+                const PvOps pv = make_pv(t, stage);
+                const QkOps qk = make_qk(t, (j + 1) % KV_STAGES);
+                const uint32_t acc0 = j > 0 ? 1u : 0u;
+                if (more)
                     ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) % KV_STAGES]), ((j + 1) / KV_STAGES) & 1, abort_flag);
+                if (!ok) break;
+                ok = mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag);
                 if (!ok) break;
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_pv(t, stage, np, j == 0);
-                    if (j + 1 < n_j[t]) issue_qk(t, (j + 1) % KV_STAGES);
+                    issue_pv(t, pv, np, acc0);
+                    if (more) issue_qk(t, qk);
                 }
                 __syncwarp();
             }
@@ -251,22 +294,58 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                 for (int c = 0; c < 128; ++c) sv[c] = (c <= col_limit) ? sv[c] : -INFINITY;
             }
-            float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
+            if (j == 0) {
+                // first tile: exact row maximum (key 0 is visible to every row, so it is finite)
+                float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
-            for (int c = 4; c < 128; c += 8) {
-                mx4[(c >> 3) & 3] = max3(mx4[(c >> 3) & 3], sv[c], sv[c + 1]);
-                mx4[((c >> 3) + 1) & 3] = max3(mx4[((c >> 3) + 1) & 3], sv[c + 2], sv[c + 3]);
-                if (c + 4 < 128) {
-                    mx4[((c >> 3) + 2) & 3] = max3(mx4[((c >> 3) + 2) & 3], sv[c + 4], sv[c + 5]);
-                    mx4[((c >> 3) + 3) & 3] = max3(mx4[((c >> 3) + 3) & 3], sv[c + 6], sv[c + 7]);
+                for (int c = 4; c < 128; c += 8) {
+                    mx4[0] = max3(mx4[0], sv[c], sv[c + 1]);
+                    mx4[1] = max3(mx4[1], sv[c + 2], sv[c + 3]);
+                    if (c + 4 < 128) {
+                        mx4[2] = max3(mx4[2], sv[c + 4], sv[c + 5]);
+                        mx4[3] = max3(mx4[3], sv[c + 6], sv[c + 7]);
+                    }
                 }
+                m_used = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
             }
-            const float mx = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3]));
-            const float m_new = fmaxf(m_used, mx * sc);
-            // raise the reference maximum only when it moved by more than 2^8 (always on the first tile)
-            if (__any_sync(0xffffffffu, m_new > m_used + kRescaleThreshold)) {
-                const float f = fast_exp2(m_used - m_new);       // first tile: 2^(-inf) = 0
-                m_used = m_new;
+            // Optimistic pass: exponentials against the current reference maximum, packed two per
+            // FMA-pipe instruction.  Whether the reference has to be raised is read off the tile's row
+            // sum (a probability above 2^8 makes it exceed 2^15 long before anything can overflow); only
+            // then is the exact maximum taken, O_t rescaled in tensor memory and the pass repeated.
+            float2 acc2[4];
+            auto exp_pass = [&](const float neg_m) {
+                const float2 sc2 = make_float2(sc, sc), nm2 = make_float2(neg_m, neg_m);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc2[i] = make_float2(0.f, 0.f);
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    uint32_t pk[16];
+#pragma unroll
+                    for (int i = 0; i < 16; ++i) {
+                        const float2 x = fma2(make_float2(sv[c * 32 + 2 * i], sv[c * 32 + 2 * i + 1]), sc2, nm2);
+                        const float2 pr = make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        acc2[i & 3] = add2(acc2[i & 3], pr);
+                        pk[i] = pack_bf16(pr.x, pr.y);
+                    }
+                    tmem_st16(tS + c * 16, pk);
+                }
+                const float2 a01 = add2(acc2[0], acc2[1]), a23 = add2(acc2[2], acc2[3]);
+                return (a01.x + a01.y) + (a23.x + a23.y);
+            };
+            float tile_sum = exp_pass(-m_used);
+            if (__any_sync(0xffffffffu, !(tile_sum <= 32768.f))) {
+                float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
+#pragma unroll
+                for (int c = 4; c < 128; c += 4) {
+                    mx4[0] = fmaxf(mx4[0], sv[c]);
+                    mx4[1] = fmaxf(mx4[1], sv[c + 1]);
+                    mx4[2] = fmaxf(mx4[2], sv[c + 2]);
+                    mx4[3] = fmaxf(mx4[3], sv[c + 3]);
+                }
+                const float rise = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc - m_used;
+                const float d = fmaxf(rise, 0.f);            // rows that did not rise keep their reference
+                const float f = fast_exp2(-d);
+                m_used += d;
                 l_sum *= f;
                 if (j > 0) {
                     ok = mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag);
@@ -282,22 +361,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         tmem_st32(tO + c * 32, reinterpret_cast<const uint32_t*>(ov));
                     }
                 }
+                tmem_wait_st();
+                tile_sum = exp_pass(-m_used);
             }
-            const float neg_m = -m_used;
-            float acc[4] = {0.f, 0.f, 0.f, 0.f};
-#pragma unroll
-            for (int c = 0; c < 4; ++c) {
-                uint32_t pk[16];
-#pragma unroll
-                for (int i = 0; i < 16; ++i) {
-                    const float p0 = fast_exp2(fmaf(sv[c * 32 + 2 * i], sc, neg_m));
-                    const float p1 = fast_exp2(fmaf(sv[c * 32 + 2 * i + 1], sc, neg_m));
-                    acc[i & 3] += p0 + p1;
-                    pk[i] = pack_bf16(p0, p1);
-                }
-                tmem_st16(tS + c * 16, pk);
-            }
-            l_sum += (acc[0] + acc[1]) + (acc[2] + acc[3]);
+            l_sum += tile_sum;
             tmem_wait_st();
             tc_fence_before();
             __syncwarp();
@@ -408,6 +475,12 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
         !encode_pool(&mv, p.v_cache, desc->num_blocks, p.Hkv, p.vs_block, p.vs_head, p.vs_token))
         return cudaErrorInvalidValue;
     const size_t smem = SMEM_TOTAL + 1024;
+    static int regs_ok = -1;
+    if (regs_ok < 0) {
+        cudaFuncAttributes fa;
+        regs_ok = (cudaFuncGetAttributes(&fa, prefill_tc_kernel) == cudaSuccess && fa.numRegs == LAUNCH_REGS) ? 1 : 0;
+    }
+    if (!regs_ok) return cudaErrorLaunchOutOfResources;   // the register hand-over arithmetic would not hold
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
