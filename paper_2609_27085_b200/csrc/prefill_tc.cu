@@ -20,6 +20,8 @@
 // are never loaded.
 // Every wait is bounded: on expiry the CTA raises an abort flag, every role leaves its loop, the
 // error word is set and tensor memory is released.
+#include <type_traits>
+
 #include "device_common.cuh"
 #include "kernels.h"
 #include "tc05.cuh"
@@ -41,7 +43,7 @@ constexpr int NTHREADS = 384;
 // first warpgroup shrinks to REGS_ROLE and the two softmax warpgroups grow to REGS_SOFTMAX.  A grow
 // request blocks until the CTA's pool holds enough released registers, so the released amount MUST
 // cover the growth or the kernel never returns; the launcher also checks the compiled register count.
-constexpr int LAUNCH_REGS = 168, REGS_ROLE = 88, REGS_SOFTMAX = 208;
+constexpr int LAUNCH_REGS = 168, REGS_ROLE = 136, REGS_SOFTMAX = 184;
 static_assert(4 * (LAUNCH_REGS - REGS_ROLE) >= 8 * (REGS_SOFTMAX - LAUNCH_REGS), "setmaxnreg.inc would block forever");
 constexpr uint32_t SMEM_Q = 0;
 constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
@@ -163,110 +165,106 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // =========================================================== MMA issuer
         constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
         constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, true);
-        // descriptors are built once; each MMA advances the address field with one add
-        constexpr uint32_t HI = desc_hi_sw128(1024);
-        const uint32_t q_lo[2] = {desc_lo_sw128(smem + SMEM_Q, 16), desc_lo_sw128(smem + SMEM_Q + TILE_BYTES, 16)};
-        const uint32_t k_lo[KV_STAGES] = {desc_lo_sw128(smem + SMEM_K, 16), desc_lo_sw128(smem + SMEM_K + TILE_BYTES, 16)};
-        const uint32_t v_lo[KV_STAGES] = {desc_lo_sw128(smem + SMEM_V, HALF_BYTES), desc_lo_sw128(smem + SMEM_V + TILE_BYTES, HALF_BYTES)};
-        const uint32_t bar_s[2] = {smem_u32(&bars.s_full[0]), smem_u32(&bars.s_full[1])};
-        const uint32_t bar_o[2] = {smem_u32(&bars.o_done[0]), smem_u32(&bars.o_done[1])};
-        // The issuing lane shares its scheduler with two softmax warps and runs at only about one
-        // instruction per 10 cycles, while a 128x128x16 MMA lasts 64 cycles: every operand of a batch
-        // is therefore put in registers before the wait, so that the batch itself is MMAs back to back.
-        struct QkOps { uint64_t a[8], b[8]; };
-        struct PvOps { uint32_t a[8]; uint64_t b[8]; };
-        auto d64 = [](uint32_t lo) { return ((uint64_t)HI << 32) | lo; };
-        auto make_qk = [&](int t, int stage) {
-            QkOps o;
+        constexpr uint64_t HI64 = (uint64_t)desc_hi_sw128(1024) << 32;
+        // The issuing lane shares its scheduler with two softmax warps and gets roughly one issue
+        // slot in ten, while a 128x128x16 MMA lasts only 64 cycles.  Every shared-memory descriptor
+        // (q tile x k-step, K/V stage x k-step) is therefore built once and kept in registers, and the
+        // tile / stage indices are compile-time, so that a batch is MMAs back to back.
+        uint64_t qd[2][8], kd[KV_STAGES][8], vd[KV_STAGES][8];
+#pragma unroll
+        for (int i = 0; i < 2; ++i)
 #pragma unroll
             for (int ks = 0; ks < 8; ++ks) {
                 const uint32_t off = (uint32_t)(((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4);
-                o.a[ks] = d64(q_lo[t] + off);
-                o.b[ks] = d64(k_lo[stage] + off);
+                qd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_Q + i * TILE_BYTES, 16) + off);
+                kd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_K + i * TILE_BYTES, 16) + off);
+                vd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_V + i * TILE_BYTES, HALF_BYTES) + ks * (2048 >> 4));
             }
-            return o;
-        };
-        auto make_pv = [&](int t, int stage) {
-            PvOps o;
-#pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
-                o.a[ks] = tmem + TM_S + t * 128 + ks * 8;
-                o.b[ks] = d64(v_lo[stage] + ks * (2048 >> 4));
-            }
-            return o;
-        };
-        auto issue_qk = [&](int t, const QkOps& o) {     // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
+        const uint32_t bar_s[2] = {smem_u32(&bars.s_full[0]), smem_u32(&bars.s_full[1])};
+        const uint32_t bar_o[2] = {smem_u32(&bars.o_done[0]), smem_u32(&bars.o_done[1])};
+        const uint32_t bar_p[2] = {smem_u32(&bars.p_full[0]), smem_u32(&bars.p_full[1])};
+        auto issue_qk = [&](auto T, auto S) {             // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
+            constexpr int t = decltype(T)::value, st = decltype(S)::value;
             const uint32_t dS = tmem + TM_S + t * 128;
-            umma_ss(dS, o.a[0], o.b[0], IDESC_QK, 0u);
+            umma_ss(dS, qd[t][0], kd[st][0], IDESC_QK, 0u);
 #pragma unroll
-            for (int ks = 1; ks < 8; ++ks) umma_ss(dS, o.a[ks], o.b[ks], IDESC_QK, 1u);
+            for (int ks = 1; ks < 8; ++ks) umma_ss(dS, qd[t][ks], kd[st][ks], IDESC_QK, 1u);
             umma_commit(bar_s[t]);
         };
-        auto issue_pv = [&](int t, const PvOps& o, int n_steps, uint32_t acc0) {   // O_t (+)= P_t V, one step per loaded page
-            const uint32_t dO = tmem + TM_O + t * 128;
-            umma_ts(dO, o.a[0], o.b[0], IDESC_PV, acc0);
+        auto issue_pv = [&](auto T, auto S, int n_steps, uint32_t acc0) {   // O_t (+)= P_t V, one step per loaded page
+            constexpr int t = decltype(T)::value, st = decltype(S)::value;
+            const uint32_t dO = tmem + TM_O + t * 128, aP = tmem + TM_S + t * 128;
+            umma_ts(dO, aP, vd[st][0], IDESC_PV, acc0);
             if (n_steps == 8) {
 #pragma unroll
-                for (int ks = 1; ks < 8; ++ks) umma_ts(dO, o.a[ks], o.b[ks], IDESC_PV, 1u);
+                for (int ks = 1; ks < 8; ++ks) umma_ts(dO, aP + ks * 8, vd[st][ks], IDESC_PV, 1u);
             } else {
 #pragma unroll
                 for (int ks = 1; ks < 8; ++ks)
-                    if (ks < n_steps) umma_ts(dO, o.a[ks], o.b[ks], IDESC_PV, 1u);
+                    if (ks < n_steps) umma_ts(dO, aP + ks * 8, vd[st][ks], IDESC_PV, 1u);
             }
             umma_commit(bar_o[t]);
         };
+        using I0 = std::integral_constant<int, 0>;
+        using I1 = std::integral_constant<int, 1>;
         bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
         ok = ok && mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
         if (ok) {
             tc_fence_after();
             if (lane == 0) {
-                for (int t = 0; t < 2; ++t)
-                    if (n_j[t] > 0) issue_qk(t, make_qk(t, 0));
+                if (n_j[0] > 0) issue_qk(I0{}, I0{});
+                if (n_j[1] > 0) issue_qk(I1{}, I0{});
                 umma_commit(smem_u32(&bars.k_empty[0]));
             }
             __syncwarp();
         }
-        for (int j = 0; j < n_max && ok; ++j) {
-            const int stage = j % KV_STAGES;
+        // one KV tile j held in stage S: PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1)
+        auto kv_step = [&](auto S, int j) -> bool {
+            constexpr int st = decltype(S)::value, st1 = st ^ 1;
+            using S1 = std::integral_constant<int, st1>;
             const int np = min(8, total_pages - 8 * j);
-            ok = mbar_wait(smem_u32(&bars.v_full[stage]), (j / KV_STAGES) & 1, abort_flag);
-            if (!ok) break;
+            if (!mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag)) return false;
             if (j == n_max - 1 && Lc < (8 * j + np) * 16) {
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
                 // that a zero probability never multiplies a NaN
                 const int r0 = Lc - j * KT, r1 = np * 16;
                 for (int idx = lane; idx < (r1 - r0) * 16; idx += 32) {
                     const int r = r0 + (idx >> 4), c = idx & 15;
-                    uint8_t* dst = smem_raw + ((smem + SMEM_V + stage * TILE_BYTES) - smem_u32(smem_raw)) +
+                    uint8_t* dst = smem_raw + ((smem + SMEM_V + st * TILE_BYTES) - smem_u32(smem_raw)) +
                                    (c >> 3) * HALF_BYTES + r * 128 + (c & 7) * 16;
                     *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
                 }
                 fence_proxy_async();
                 __syncwarp();
             }
-            for (int t = 0; t < 2 && ok; ++t) {
-                if (j >= n_j[t]) continue;
+            const uint32_t acc0 = j > 0 ? 1u : 0u;
+            auto tile = [&](auto T) -> bool {
+                constexpr int t = decltype(T)::value;
+                if (j >= n_j[t]) return true;
                 const bool more = j + 1 < n_j[t];
-                const PvOps pv = make_pv(t, stage);
-                const QkOps qk = make_qk(t, (j + 1) % KV_STAGES);
-                const uint32_t acc0 = j > 0 ? 1u : 0u;
-                if (more)
-                    ok = mbar_wait(smem_u32(&bars.k_full[(j + 1) % KV_STAGES]), ((j + 1) / KV_STAGES) & 1, abort_flag);
-                if (!ok) break;
-                ok = mbar_wait(smem_u32(&bars.p_full[t]), j & 1, abort_flag);
-                if (!ok) break;
+                if (more && !mbar_wait(smem_u32(&bars.k_full[st1]), ((j + 1) >> 1) & 1, abort_flag)) return false;
+                if (!mbar_wait(bar_p[t], j & 1, abort_flag)) return false;
                 tc_fence_after();
                 if (lane == 0) {
-                    issue_pv(t, pv, np, acc0);
-                    if (more) issue_qk(t, qk);
+                    issue_pv(T, S, np, acc0);
+                    if (more) issue_qk(T, S1{});
                 }
                 __syncwarp();
-            }
-            if (ok && lane == 0) {
-                umma_commit(smem_u32(&bars.v_empty[stage]));
-                if (j + 1 < n_max) umma_commit(smem_u32(&bars.k_empty[(j + 1) % KV_STAGES]));
+                return true;
+            };
+            if (!tile(I0{})) return false;
+            if (!tile(I1{})) return false;
+            if (lane == 0) {
+                umma_commit(smem_u32(&bars.v_empty[st]));
+                if (j + 1 < n_max) umma_commit(smem_u32(&bars.k_empty[st1]));
             }
             __syncwarp();
+            return true;
+        };
+        static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
+        for (int j = 0; j < n_max && ok; j += 2) {
+            ok = kv_step(I0{}, j);
+            if (ok && j + 1 < n_max) ok = kv_step(I1{}, j + 1);
         }
       }
     } else {
@@ -351,14 +349,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     ok = mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
-#pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        float ov[32];
-                        tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
+#pragma unroll 1
+                    for (int c = 0; c < 8; ++c) {
+                        float ov[16];
+                        tmem_ld16(tO + c * 16, reinterpret_cast<uint32_t*>(ov));
                         tmem_wait_ld();
 #pragma unroll
-                        for (int i = 0; i < 32; ++i) ov[i] *= f;
-                        tmem_st32(tO + c * 32, reinterpret_cast<const uint32_t*>(ov));
+                        for (int i = 0; i < 16; ++i) ov[i] *= f;
+                        tmem_st16(tO + c * 16, reinterpret_cast<const uint32_t*>(ov));
                     }
                 }
                 tmem_wait_st();
