@@ -37,6 +37,10 @@ UNIT = "query-tokens/s"
 WORKLOAD = ("configs[2] chat-like mixed batch: 48 decode seqs (lognormal ctx, median 4096, sigma 0.8, clip [128,16384]) "
             "+ 2 prefills of 2048 new tokens over 6144 cached, 512-token chunks; Hq 32, Hkv 8, D 128, block 16, bf16; "
             "one step = kv_append + mixed attention of one chunk iteration (t cycles 0..3)")
+# DRAM traffic per algorithmic byte of the split-K decode kernel, from the ncu capture summarised in
+# profiles/decode_splitk_decode_small.md (560.9 MB moved for 555.2 MB algorithmic); traffic grows in
+# proportion to the K/V bytes, so a full launch is scaled by its algorithmic bytes.
+DECODE_TRAFFIC_RATIO = 1.010
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -189,7 +193,7 @@ def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks):
     if ms_dec > 0:
         gbs = dec_bytes / ((ms_dec + ms_comb) * 1e-3) / 1e9
         out["decode"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                         "frac": gbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_RATIO * dec_bytes / steps,
                          "bytes_per_launch": dec_bytes / steps, "ms": (ms_dec + ms_comb) / steps}
     if ms_pre > 0:
         tf = pre_flops / (ms_pre * 1e-3) / 1e12
