@@ -115,6 +115,12 @@ cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
  * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
 cf_status cf_get_async_status(cf_ctx* ctx);
 
+/* Self-test of the bounded-wait machinery (no counterpart in the paper): enqueues one tiny kernel whose
+ * wait on a barrier that nothing signals expires after a few milliseconds; the kernel then sets the
+ * context's error word and returns normally.  After synchronising, cf_get_async_status must report
+ * CF_ERR_TIMEOUT once and CF_OK afterwards; the context stays usable. */
+cf_status cf_selftest_bounded_wait(cf_ctx* ctx, void* cuda_stream);
+
 /* Per-kernel timing for benchmarks.  After cf_set_timing(ctx, 1) every cf_mixed_attention records
  * CUDA events around its kernels on the caller's stream (no host synchronisation).
  * cf_get_timing_sums waits for the last timed call, returns the summed milliseconds of each

@@ -438,6 +438,14 @@ cf_status cf_get_async_status(cf_ctx* c)
     return CF_ERR_TIMEOUT;
 }
 
+cf_status cf_selftest_bounded_wait(cf_ctx* c, void* cuda_stream)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    return launch_wait_selftest(c->err_dev, (cudaStream_t)cuda_stream) == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
+
 cf_status cf_set_timing(cf_ctx* c, int enabled)
 {
     if (!c) return CF_ERR_INVALID_ARG;

@@ -33,4 +33,7 @@ bool prefill_tc_supported(const cf_cache_desc* desc);
 cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items,
                               cudaStream_t stream);
 
+// one CTA whose bounded wait must expire: sets *err and returns normally (status-path self-test)
+cudaError_t launch_wait_selftest(uint32_t* err, cudaStream_t stream);
+
 }  // namespace cf

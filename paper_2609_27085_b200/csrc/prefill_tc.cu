@@ -409,6 +409,29 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 }
 
 // ---------------------------------------------------------------------------------------------
+// Self-test of the bounded-wait path: one CTA waits, with a limit of a few milliseconds, on an
+// mbarrier that nothing ever arrives at, gives up, raises the error word and returns normally.
+__global__ void __launch_bounds__(32) wait_selftest_kernel(uint32_t* err)
+{
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ uint32_t abort_s;
+    if (threadIdx.x == 0) {
+        abort_s = 0;
+        mbar_init(smem_u32(&bar), 1);
+        fence_mbar_init();
+    }
+    __syncwarp();
+    const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_s, 1ll << 23);
+    __syncwarp();
+    if (!ok && threadIdx.x == 0 && err) atomicExch(err, 1u);
+}
+
+cudaError_t launch_wait_selftest(uint32_t* err, cudaStream_t stream)
+{
+    wait_selftest_kernel<<<1, 32, 0, stream>>>(err);
+    return cudaGetLastError();
+}
+
 namespace {
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,

@@ -34,7 +34,8 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
 // Bounded wait: gives up after about kWaitCycles SM cycles (a second or so), or as soon as another
 // thread of the CTA has raised *abort_flag.  Returns false then.
 constexpr long long kWaitCycles = 1ll << 31;
-__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag)
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile uint32_t* abort_flag,
+                                          long long limit_cycles = kWaitCycles)
 {
     if (mbar_try_wait(bar, parity)) return true;
     const long long t0 = clock64();
@@ -42,7 +43,7 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
         if (mbar_try_wait(bar, parity)) return true;
         if ((i & 15) == 0) {
             if (*abort_flag) return false;
-            if (clock64() - t0 > kWaitCycles) break;
+            if (clock64() - t0 > limit_cycles) break;
         }
     }
     *abort_flag = 1u;

@@ -201,3 +201,38 @@ def test_host_step_matches_device_step():
     ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
     compare(o_dev, None, ref_o, ref_lse)
     g.close()
+
+
+def test_bounded_wait_reports_timeout_and_context_survives():
+    """A wait that nothing satisfies gives up by itself; the host reads CF_ERR_TIMEOUT and the same
+    context then still computes correct attention."""
+    sc = small(27, 32, 8, 128, [300, 40], [[130, 1]])
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    cf.cf_selftest_bounded_wait(g.ctx)
+    torch.cuda.synchronize()
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_ERR_TIMEOUT
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    g.append(b)
+    o_bits, lse = g.attend(b)
+    k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
+    compare(o_bits, lse, ref_o, ref_lse)
+    g.close()
+
+
+def test_property_random_batches():
+    """Random small batches: sequence counts, chunk lengths, prefixes, group sizes, head dims."""
+    rng = np.random.default_rng(2024)
+    for trial in range(24):
+        Hkv = int(rng.choice([1, 2, 4]))
+        G = int(rng.choice([1, 2, 4, 8]))
+        D = int(rng.choice([64, 128]))
+        S = int(rng.integers(1, 9))
+        qlen = [int(x) for x in rng.choice([0, 1, 1, 1, 2, 7, 31, 64, 127, 128, 129, 200, 300], size=S)]
+        prefix = [int(x) for x in rng.integers(0, 601, size=S)]
+        prefix = [p if q > 0 else max(p, 0) for p, q in zip(prefix, qlen)]
+        if sum(qlen) == 0:
+            qlen[0] = 1
+        run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True))
