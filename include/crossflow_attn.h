@@ -115,6 +115,16 @@ cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
  * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
 cf_status cf_get_async_status(cf_ctx* ctx);
 
+/* Section 5 names two executor backends: the chunked mixed-batch path (time-multiplexed, the default
+ * here: one launch sequence on the caller's stream) and a spatial partition of the node between prefill
+ * and decode.  cf_set_overlap(ctx, 1) selects a spatial variant for later cf_mixed_attention calls that
+ * hold both kinds of work: the prefill kernel is enqueued first on a context-owned side stream and the
+ * decode + combine kernels on the caller's stream, so that decode (memory-bound) fills the SMs the
+ * prefill CTAs leave free; the side stream is joined back before the call returns, so the caller still
+ * sees one stream.  Results are bit-identical to the default.  The environment variable CF_OVERLAP=1
+ * sets the initial value.  Per-kernel timing (cf_set_timing) forces the serial sequence. */
+cf_status cf_set_overlap(cf_ctx* ctx, int enabled);
+
 /* Self-test of the bounded-wait machinery (no counterpart in the paper): enqueues one tiny kernel whose
  * wait on a barrier that nothing signals expires after a few milliseconds; the kernel then sets the
  * context's error word and returns normally.  After synchronising, cf_get_async_status must report

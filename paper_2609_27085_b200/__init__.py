@@ -33,7 +33,7 @@ CF_ERR_ARCH = 7
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
-           "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_status_string")
+           "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -76,6 +76,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
+    lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.cf_status_string.argtypes = [ctypes.c_int]
     lib.cf_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -178,6 +179,11 @@ def cf_get_async_status(ctx) -> int:
 def cf_selftest_bounded_wait(ctx, stream=None) -> None:
     """Enqueues the kernel whose bounded wait must expire (see cf_get_async_status)."""
     _check(load_library().cf_selftest_bounded_wait(ctx, _stream(stream)), "cf_selftest_bounded_wait")
+
+
+def cf_set_overlap(ctx, enabled: bool) -> None:
+    """Run the prefill kernel beside decode + combine (side stream, joined before return)."""
+    _check(load_library().cf_set_overlap(ctx, int(bool(enabled))), "cf_set_overlap")
 
 
 def cf_set_timing(ctx, enabled: bool) -> None:

@@ -43,6 +43,10 @@ struct cf_ctx {
     bool workspace_fixed = false;
     uint32_t* err_dev = nullptr;
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
+    // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
+    bool overlap = false;
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // host-staged step
     uint8_t* stage_dev = nullptr;
     size_t stage_bytes = 0;
@@ -216,6 +220,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", c->cfg.decode_min_chunk_pages);
     c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
     c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
+    c->overlap = env_int("CF_OVERLAP", 0) != 0;
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
@@ -223,6 +228,9 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->workspace_fixed = false;
     ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
     c->workspace_fixed = workspace_bytes != 0;
+    ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->err_dev, sizeof(uint32_t)) == cudaSuccess;
     ok = ok && cudaMemset(c->err_dev, 0, sizeof(uint32_t)) == cudaSuccess;
     if (!ok) {
@@ -248,6 +256,9 @@ cf_status cf_destroy(cf_ctx* c)
             if (tc.ev[i]) cudaEventDestroy(tc.ev[i]);
     if (c->workspace) cudaFree(c->workspace);
     if (c->err_dev) cudaFree(c->err_dev);
+    if (c->ev_fork) cudaEventDestroy(c->ev_fork);
+    if (c->ev_join) cudaEventDestroy(c->ev_join);
+    if (c->side) cudaStreamDestroy(c->side);
     if (c->stage_dev) cudaFree(c->stage_dev);
     delete c;
     return CF_OK;
@@ -365,14 +376,28 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
         tc->ran[1] = !pl.combine.empty();
         tc->ran[2] = !pl.prefill.empty() || !pl.prefill_tc.empty();
     }
-    if (tc) cudaEventRecord(tc->ev[0], stream);
-    if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
-    if (tc) cudaEventRecord(tc->ev[1], stream);
-    if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
-    if (tc) cudaEventRecord(tc->ev[2], stream);
-    if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
-    if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), stream);
-    if (tc) cudaEventRecord(tc->ev[3], stream);
+    const bool has_prefill = !pl.prefill.empty() || !pl.prefill_tc.empty();
+    if (c->overlap && !tc && has_prefill && !pl.decode.empty()) {
+        // prefill on the side stream, launched first so that its CTAs take their SMs; decode + combine
+        // on the caller's stream fill the rest of the machine; joined before returning to the caller
+        if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
+            e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), c->side);
+        if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
+        if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
+    } else {
+        if (tc) cudaEventRecord(tc->ev[0], stream);
+        if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
+        if (tc) cudaEventRecord(tc->ev[1], stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
+        if (tc) cudaEventRecord(tc->ev[2], stream);
+        if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), stream);
+        if (tc) cudaEventRecord(tc->ev[3], stream);
+    }
     c->launches = (int)!pl.decode.empty() + (int)!pl.combine.empty() + (int)!pl.prefill.empty() + (int)!pl.prefill_tc.empty();
     const cf_status fs = finish_slot(slot, stream);
     if (e != cudaSuccess) return CF_ERR_CUDA;
@@ -436,6 +461,13 @@ cf_status cf_get_async_status(cf_ctx* c)
     if (w == 0) return CF_OK;
     cudaMemset(c->err_dev, 0, sizeof w);
     return CF_ERR_TIMEOUT;
+}
+
+cf_status cf_set_overlap(cf_ctx* c, int enabled)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    c->overlap = enabled != 0;
+    return CF_OK;
 }
 
 cf_status cf_selftest_bounded_wait(cf_ctx* c, void* cuda_stream)

@@ -236,3 +236,21 @@ def test_property_random_batches():
         if sum(qlen) == 0:
             qlen[0] = 1
         run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True))
+
+
+def test_overlap_mode_is_bit_identical_to_the_serial_sequence():
+    sc = small(29, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    serial, lse0 = g.attend(b)
+    cf.cf_set_overlap(g.ctx, True)
+    for _ in range(3):
+        o, lse = g.attend(b)
+        assert np.array_equal(o, serial) and np.array_equal(lse, lse0)
+    cf.cf_set_overlap(g.ctx, False)
+    k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
+    compare(serial, lse0, ref_o, ref_lse)
+    g.close()
