@@ -100,16 +100,23 @@ cf_status cf_mixed_attention(cf_ctx* ctx, const cf_cache_desc* desc, const void*
                              const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
                              void* out, float* lse, void* cuda_stream);
 
-/* One whole unit from HOST buffers: copies q, k_new, v_new (HOST, pinned memory recommended) to
- * context-owned device staging, runs cf_kv_append + cf_mixed_attention, copies `out` back to
- * out_host, all on cuda_stream.  The caches and the block table stay DEVICE pointers (they are the
- * node's resident state).  Asynchronous; out_host is valid after the stream is synchronised. */
+/* One whole unit from HOST buffers (how a serving loop that keeps activations on the host would
+ * drive the library): copies q, k_new, v_new (HOST, pinned memory recommended) to context-owned
+ * device staging, runs cf_kv_append + cf_mixed_attention on cuda_stream, and copies `out` back to
+ * out_host.  The caches and the block table stay DEVICE pointers (they are the node's resident
+ * state).  The input copy and the read-back run on two context-owned copy streams, ordered against
+ * the kernels by events and triple-buffered, so that consecutive calls overlap step i+1's input copy
+ * and step i-1's read-back with step i's kernels.  Asynchronous.  out_host of every call issued so far
+ * is valid once cf_host_steps_flush(ctx, stream) has been called and `stream` synchronised; the host
+ * input buffers of a call must stay unchanged until then as well. */
 cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
                              const void* q_host, const void* k_new_host, const void* v_new_host,
                              void* k_cache, void* v_cache,
                              const int32_t* block_table, int32_t max_blocks_per_seq,
                              const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
                              void* out_host, void* cuda_stream);
+/* Makes cuda_stream wait for the read-backs of all cf_mixed_step_host calls issued so far. */
+cf_status cf_host_steps_flush(cf_ctx* ctx, void* cuda_stream);
 
 /* After the caller has synchronised the stream: CF_OK, or the first device-side finding
  * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */

@@ -31,7 +31,7 @@ CF_ERR_CUDA = 5
 CF_ERR_TIMEOUT = 6
 CF_ERR_ARCH = 7
 
-EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host",
+EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_status_string")
 
@@ -69,6 +69,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_kv_append.argtypes = [vp, dp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp]
     lib.cf_mixed_attention.argtypes = [vp, dp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
     lib.cf_mixed_step_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp]
+    lib.cf_host_steps_flush.argtypes = [vp, vp]
     lib.cf_get_async_status.argtypes = [vp]
     lib.cf_set_timing.argtypes = [vp, ctypes.c_int]
     lib.cf_get_timing_sums.argtypes = [vp, fp, fp, fp, i32p]
@@ -170,6 +171,11 @@ def cf_mixed_step_host(ctx, desc: CacheDesc, q_host, k_new_host, v_new_host, k_c
     if check:
         _check(st, "cf_mixed_step_host")
     return st
+
+
+def cf_host_steps_flush(ctx, stream=None) -> None:
+    """Makes `stream` wait for the read-backs of every cf_mixed_step_host call issued so far."""
+    _check(load_library().cf_host_steps_flush(ctx, _stream(stream)), "cf_host_steps_flush")
 
 
 def cf_get_async_status(ctx) -> int:

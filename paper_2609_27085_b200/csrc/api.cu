@@ -22,6 +22,16 @@ struct TimedCall {
     bool ran[3] = {false, false, false};
 };
 
+// Device staging of one host-buffer step (cf_mixed_step_host): inputs copied in on one copy stream,
+// result copied out on another, so that the copies of neighbouring steps overlap the kernels.
+static constexpr int kHostStages = 3;
+struct HostStage {
+    uint8_t* dev = nullptr;
+    size_t bytes = 0;
+    cudaEvent_t h2d_done = nullptr, compute_done = nullptr, d2h_done = nullptr;
+    bool used = false;
+};
+
 struct PlanSlot {
     uint8_t* host = nullptr;   // pinned
     uint8_t* dev = nullptr;
@@ -48,8 +58,9 @@ struct cf_ctx {
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // host-staged step
-    uint8_t* stage_dev = nullptr;
-    size_t stage_bytes = 0;
+    cf::HostStage stage[cf::kHostStages];
+    int next_stage = 0;
+    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
     // timing: one quad of events per timed call since the last cf_get_timing_sums
     bool timing = false;
     std::vector<cf::TimedCall> timed;
@@ -229,6 +240,13 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
     c->workspace_fixed = workspace_bytes != 0;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
+    for (int i = 0; i < kHostStages && ok; ++i) {
+        ok = cudaEventCreateWithFlags(&c->stage[i].h2d_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->stage[i].compute_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->stage[i].d2h_done, cudaEventDisableTiming) == cudaSuccess;
+    }
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaMalloc((void**)&c->err_dev, sizeof(uint32_t)) == cudaSuccess;
@@ -259,7 +277,15 @@ cf_status cf_destroy(cf_ctx* c)
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
-    if (c->stage_dev) cudaFree(c->stage_dev);
+    for (int i = 0; i < kHostStages; ++i) {
+        HostStage& hs = c->stage[i];
+        if (hs.dev) cudaFree(hs.dev);
+        if (hs.h2d_done) cudaEventDestroy(hs.h2d_done);
+        if (hs.compute_done) cudaEventDestroy(hs.compute_done);
+        if (hs.d2h_done) cudaEventDestroy(hs.d2h_done);
+    }
+    if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+    if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
     delete c;
     return CF_OK;
 }
@@ -426,29 +452,56 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
     const size_t q_bytes = align_up(T * desc->num_q_heads * desc->head_dim * 2, 256);
     const size_t kv_bytes = align_up(T * desc->num_kv_heads * desc->head_dim * 2, 256);
     const size_t need = 2 * q_bytes + 2 * kv_bytes;
-    if (need > c->stage_bytes) {
+    HostStage& hs = c->stage[c->next_stage];
+    c->next_stage = (c->next_stage + 1) % kHostStages;
+    if (need > hs.bytes) {
         if (cudaDeviceSynchronize() != cudaSuccess) return CF_ERR_CUDA;
-        if (c->stage_dev) cudaFree(c->stage_dev);
-        c->stage_dev = nullptr;
-        c->stage_bytes = 0;
-        if (cudaMalloc((void**)&c->stage_dev, need) != cudaSuccess) return CF_ERR_CUDA;
-        c->stage_bytes = need;
+        if (hs.dev) cudaFree(hs.dev);
+        hs.dev = nullptr;
+        hs.bytes = 0;
+        if (cudaMalloc((void**)&hs.dev, need) != cudaSuccess) return CF_ERR_CUDA;
+        hs.bytes = need;
+        hs.used = false;
     }
-    uint8_t* dq = c->stage_dev;
+    uint8_t* dq = hs.dev;
     uint8_t* dk = dq + q_bytes;
     uint8_t* dv = dk + kv_bytes;
     uint8_t* dout = dv + kv_bytes;
     const size_t qb = T * desc->num_q_heads * desc->head_dim * 2, kb = T * desc->num_kv_heads * desc->head_dim * 2;
-    if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
-    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
-    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    // inputs: copy stream, after the kernels and the read-back that last used this staging set
+    if (hs.used) {
+        if (cudaStreamWaitEvent(c->h2d_stream, hs.compute_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+        if (cudaStreamWaitEvent(c->h2d_stream, hs.d2h_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+    }
+    if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaEventRecord(hs.h2d_done, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
+    // kernels: the caller's stream
+    if (cudaStreamWaitEvent(stream, hs.h2d_done, 0) != cudaSuccess) return CF_ERR_CUDA;
     st = cf_kv_append(c, desc, k_cache, v_cache, dk, dv, block_table, max_blocks_per_seq, context_len, query_len,
                       num_seqs, cuda_stream);
     if (st != CF_OK) return st;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);
     if (st != CF_OK) return st;
-    if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaEventRecord(hs.compute_done, stream) != cudaSuccess) return CF_ERR_CUDA;
+    // result: second copy stream
+    if (cudaStreamWaitEvent(c->d2h_stream, hs.compute_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(out_host, dout, qb, cudaMemcpyDeviceToHost, c->d2h_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaEventRecord(hs.d2h_done, c->d2h_stream) != cudaSuccess) return CF_ERR_CUDA;
+    hs.used = true;
+    return CF_OK;
+}
+
+cf_status cf_host_steps_flush(cf_ctx* c, void* cuda_stream)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    for (int i = 0; i < kHostStages; ++i)
+        if (c->stage[i].used && cudaStreamWaitEvent((cudaStream_t)cuda_stream, c->stage[i].d2h_done, 0) != cudaSuccess)
+            return CF_ERR_CUDA;
     return CF_OK;
 }
 

@@ -193,6 +193,7 @@ def test_host_step_matches_device_step():
     vh = torch.from_numpy(b.v_new.view(np.int16)).pin_memory()
     oh = torch.zeros_like(qh).pin_memory()
     cf.cf_mixed_step_host(g.ctx, g.desc, qh, kh, vh, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len, oh)
+    cf.cf_host_steps_flush(g.ctx)
     torch.cuda.synchronize()
     o_dev, _ = g.attend(b, want_lse=False)          # caches were appended by the host step
     assert np.array_equal(oh.numpy().view(np.uint16), o_dev)
@@ -254,3 +255,30 @@ def test_overlap_mode_is_bit_identical_to_the_serial_sequence():
     ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
     compare(serial, lse0, ref_o, ref_lse)
     g.close()
+
+
+def test_pipelined_host_steps_keep_their_order():
+    """Six host-buffer steps back to back (copies of neighbouring steps overlap the kernels): every
+    step's read-back equals the device-buffer path run step by step on a second copy of the caches."""
+    prefix = [300, 40, 999, 0]
+    qlens = [[100, 1, 1, 64], [37, 1, 1, 64], [200, 1, 1, 1], [1, 1, 1, 1], [64, 1, 1, 130], [5, 1, 1, 1]]
+    sc = small(31, 32, 8, 128, prefix, qlens, NB=1024)
+    ga, gb = GpuScenario(sc), GpuScenario(sc)
+    outs, keep = [], []
+    for b in sc.batches:
+        bt = torch.from_numpy(b.block_table).cuda()
+        qh = torch.from_numpy(b.q.view(np.int16)).pin_memory()
+        kh = torch.from_numpy(b.k_new.view(np.int16)).pin_memory()
+        vh = torch.from_numpy(b.v_new.view(np.int16)).pin_memory()
+        oh = torch.zeros_like(qh).pin_memory()
+        cf.cf_mixed_step_host(ga.ctx, ga.desc, qh, kh, vh, ga.k, ga.v, bt, b.max_blocks, b.context_len, b.query_len, oh)
+        outs.append(oh)
+        keep.append((bt, qh, kh, vh))
+    cf.cf_host_steps_flush(ga.ctx)
+    torch.cuda.synchronize()
+    for b, oh in zip(sc.batches, outs):
+        gb.append(b)
+        ref, _ = gb.attend(b, want_lse=False)
+        assert np.array_equal(oh.numpy().view(np.uint16), ref), b.label
+    ga.close()
+    gb.close()
