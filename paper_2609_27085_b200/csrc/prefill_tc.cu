@@ -207,64 +207,88 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         };
         using I0 = std::integral_constant<int, 0>;
         using I1 = std::integral_constant<int, 1>;
+        // One lane runs the whole role (the others go straight to the teardown barrier).  This lane is
+        // the critical resource of the kernel: it is a single dependent instruction stream that is also
+        // blocked while its MMAs queue up, so the work between two batches is kept to a handful of
+        // instructions, with a lean loop for interior tiles and the general step for the rest.
+        if (lane == 0) {
+        const uint32_t bar_kf[2] = {smem_u32(&bars.k_full[0]), smem_u32(&bars.k_full[1])};
+        const uint32_t bar_vf[2] = {smem_u32(&bars.v_full[0]), smem_u32(&bars.v_full[1])};
+        const uint32_t bar_ke[2] = {smem_u32(&bars.k_empty[0]), smem_u32(&bars.k_empty[1])};
+        const uint32_t bar_ve[2] = {smem_u32(&bars.v_empty[0]), smem_u32(&bars.v_empty[1])};
         bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
-        ok = ok && mbar_wait(smem_u32(&bars.k_full[0]), 0, abort_flag);
+        ok = ok && mbar_wait(bar_kf[0], 0, abort_flag);
         if (ok) {
             tc_fence_after();
-            if (lane == 0) {
-                if (n_j[0] > 0) issue_qk(I0{}, I0{});
-                if (n_j[1] > 0) issue_qk(I1{}, I0{});
-                umma_commit(smem_u32(&bars.k_empty[0]));
-            }
-            __syncwarp();
+            if (n_j[0] > 0) issue_qk(I0{}, I0{});
+            if (n_j[1] > 0) issue_qk(I1{}, I0{});
+            umma_commit(bar_ke[0]);
         }
-        // one KV tile j held in stage S: PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1)
+        // ---- interior tiles: both q tiles present and continuing, all 8 pages loaded, not the last tile
+        const int n_int = (n_j[0] > 0 && n_j[1] > 0) ? min(n_j[0], n_j[1]) - 1 : 0;
+        auto lean_step = [&](auto S, uint32_t par_v, uint32_t par_k1, uint32_t par_p, uint32_t acc0) -> bool {
+            constexpr int st = decltype(S)::value, st1 = st ^ 1;
+            using S1 = std::integral_constant<int, st1>;
+            if (!mbar_wait(bar_vf[st], par_v, abort_flag)) return false;
+            if (!mbar_wait(bar_kf[st1], par_k1, abort_flag)) return false;
+            if (!mbar_wait(bar_p[0], par_p, abort_flag)) return false;
+            tc_fence_after();
+            issue_pv(I0{}, S, 8, acc0);
+            issue_qk(I0{}, S1{});
+            if (!mbar_wait(bar_p[1], par_p, abort_flag)) return false;
+            tc_fence_after();
+            issue_pv(I1{}, S, 8, acc0);
+            issue_qk(I1{}, S1{});
+            umma_commit(bar_ve[st]);
+            umma_commit(bar_ke[st1]);
+            return true;
+        };
+        int j = 0;
+        {
+            uint32_t h = 0;                                   // (j >> 1) & 1 for the even tile of the pair
+            for (; ok && j + 1 < n_int; j += 2, h ^= 1u) {
+                ok = lean_step(I0{}, h, h, 0u, j > 0 ? 1u : 0u);
+                if (ok) ok = lean_step(I1{}, h, h ^ 1u, 1u, 1u);
+            }
+        }
+        // ---- general step: PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) with every edge case
         auto kv_step = [&](auto S, int j) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
             const int np = min(8, total_pages - 8 * j);
-            if (!mbar_wait(smem_u32(&bars.v_full[st]), (j >> 1) & 1, abort_flag)) return false;
+            if (!mbar_wait(bar_vf[st], (uint32_t)(j >> 1) & 1u, abort_flag)) return false;
             if (j == n_max - 1 && Lc < (8 * j + np) * 16) {
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
                 // that a zero probability never multiplies a NaN
                 const int r0 = Lc - j * KT, r1 = np * 16;
-                for (int idx = lane; idx < (r1 - r0) * 16; idx += 32) {
+                for (int idx = 0; idx < (r1 - r0) * 16; ++idx) {
                     const int r = r0 + (idx >> 4), c = idx & 15;
                     uint8_t* dst = smem_raw + ((smem + SMEM_V + st * TILE_BYTES) - smem_u32(smem_raw)) +
                                    (c >> 3) * HALF_BYTES + r * 128 + (c & 7) * 16;
                     *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
                 }
                 fence_proxy_async();
-                __syncwarp();
             }
             const uint32_t acc0 = j > 0 ? 1u : 0u;
             auto tile = [&](auto T) -> bool {
                 constexpr int t = decltype(T)::value;
                 if (j >= n_j[t]) return true;
                 const bool more = j + 1 < n_j[t];
-                if (more && !mbar_wait(smem_u32(&bars.k_full[st1]), ((j + 1) >> 1) & 1, abort_flag)) return false;
-                if (!mbar_wait(bar_p[t], j & 1, abort_flag)) return false;
+                if (more && !mbar_wait(bar_kf[st1], (uint32_t)((j + 1) >> 1) & 1u, abort_flag)) return false;
+                if (!mbar_wait(bar_p[t], (uint32_t)j & 1u, abort_flag)) return false;
                 tc_fence_after();
-                if (lane == 0) {
-                    issue_pv(T, S, np, acc0);
-                    if (more) issue_qk(T, S1{});
-                }
-                __syncwarp();
+                issue_pv(T, S, np, acc0);
+                if (more) issue_qk(T, S1{});
                 return true;
             };
             if (!tile(I0{})) return false;
             if (!tile(I1{})) return false;
-            if (lane == 0) {
-                umma_commit(smem_u32(&bars.v_empty[st]));
-                if (j + 1 < n_max) umma_commit(smem_u32(&bars.k_empty[st1]));
-            }
-            __syncwarp();
+            umma_commit(bar_ve[st]);
+            if (j + 1 < n_max) umma_commit(bar_ke[st1]);
             return true;
         };
         static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
-        for (int j = 0; j < n_max && ok; j += 2) {
-            ok = kv_step(I0{}, j);
-            if (ok && j + 1 < n_max) ok = kv_step(I1{}, j + 1);
+        for (; j < n_max && ok; ++j) ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
         }
       }
     } else {
