@@ -41,6 +41,7 @@ extern "C" {
 #endif
 
 typedef struct cf_ctx cf_ctx; /* opaque; one per device; owns plan staging and split-K workspace */
+typedef struct cf_plan cf_plan; /* opaque; a device-resident plan for one set of sequence lengths */
 
 typedef enum {
     CF_OK = 0,
@@ -99,6 +100,24 @@ cf_status cf_mixed_attention(cf_ctx* ctx, const cf_cache_desc* desc, const void*
                              const int32_t* block_table, int32_t max_blocks_per_seq,
                              const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
                              void* out, float* lse, void* cuda_stream);
+
+/* Plan once, launch many times.  The lengths of a scheduler iteration are the same for every layer
+ * of the model (Section 5: one mixed batch per iteration), so the host planning and the plan upload can
+ * be done once: cf_plan_create validates, plans and uploads (it allocates the plan's own device buffers
+ * and split-K partials, and enqueues one copy on cuda_stream); cf_kv_append_planned and
+ * cf_mixed_attention_planned then only enqueue kernels - no allocation, no host synchronisation, no
+ * host-side copy - with the same results as cf_kv_append / cf_mixed_attention.  That also makes the
+ * two planned calls legal inside a CUDA stream capture (the pointers passed are baked into the graph;
+ * the overlap variant and per-kernel timing do not apply to them when captured).  A plan must outlive
+ * every launch and every graph that uses it; cf_plan_destroy synchronises the device.  Planned calls
+ * on one context share its error word and must be ordered like all other calls. */
+cf_status cf_plan_create(cf_ctx* ctx, const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t max_blocks_per_seq, void* cuda_stream, cf_plan** out);
+cf_status cf_plan_destroy(cf_plan* plan);
+cf_status cf_kv_append_planned(cf_plan* plan, void* k_cache, void* v_cache, const void* k_new, const void* v_new,
+                               const int32_t* block_table, void* cuda_stream);
+cf_status cf_mixed_attention_planned(cf_plan* plan, const void* q, const void* k_cache, const void* v_cache,
+                                     const int32_t* block_table, void* out, float* lse, void* cuda_stream);
 
 /* One whole unit from HOST buffers (how a serving loop that keeps activations on the host would
  * drive the library): copies q, k_new, v_new (HOST, pinned memory recommended) to context-owned

@@ -33,7 +33,8 @@ CF_ERR_ARCH = 7
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
-           "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_status_string")
+           "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -78,6 +79,10 @@ def load_library() -> ctypes.CDLL:
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
+    lib.cf_plan_create.argtypes = [vp, dp, vp, vp, i32, i32, vp, ctypes.POINTER(vp)]
+    lib.cf_plan_destroy.argtypes = [vp]
+    lib.cf_kv_append_planned.argtypes = [vp, vp, vp, vp, vp, vp, vp]
+    lib.cf_mixed_attention_planned.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     lib.cf_status_string.argtypes = [ctypes.c_int]
     lib.cf_status_string.restype = ctypes.c_char_p
     for name in EXPORTS:
@@ -240,3 +245,26 @@ def cf_decode_attention_static(desc: CacheDesc, q, k_cache, v_cache, block_table
     if check:
         _check(st, "cf_decode_attention_static")
     return st
+
+
+def cf_plan_create(ctx, desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, stream=None) -> ctypes.c_void_p:
+    """Plans one set of lengths once; the returned handle serves every layer's planned calls."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    plan = ctypes.c_void_p()
+    _check(load_library().cf_plan_create(ctx, ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
+                                         int(max_blocks_per_seq), _stream(stream), ctypes.byref(plan)), "cf_plan_create")
+    return plan
+
+
+def cf_plan_destroy(plan) -> None:
+    _check(load_library().cf_plan_destroy(plan), "cf_plan_destroy")
+
+
+def cf_kv_append_planned(plan, k_cache, v_cache, k_new, v_new, block_table, stream=None) -> None:
+    _check(load_library().cf_kv_append_planned(plan, _dev(k_cache), _dev(v_cache), _dev(k_new), _dev(v_new),
+                                               _dev(block_table), _stream(stream)), "cf_kv_append_planned")
+
+
+def cf_mixed_attention_planned(plan, q, k_cache, v_cache, block_table, out, lse=None, stream=None) -> None:
+    _check(load_library().cf_mixed_attention_planned(plan, _dev(q), _dev(k_cache), _dev(v_cache), _dev(block_table),
+                                                     _dev(out), _dev(lse), _stream(stream)), "cf_mixed_attention_planned")

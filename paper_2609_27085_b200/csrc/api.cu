@@ -68,6 +68,20 @@ struct cf_ctx {
     int launches = 0;
 };
 
+// A plan that lives on the device for as long as the caller wants: built once per scheduler iteration
+// and used by every layer's append + attention calls (the lengths are the same for all layers).
+struct cf_plan {
+    cf_ctx* ctx = nullptr;
+    cf_cache_desc desc;
+    int32_t num_seqs = 0, max_blocks = 0;
+    uint8_t* host = nullptr;       // pinned copy (source of the one upload)
+    uint8_t* dev = nullptr;
+    float* part = nullptr;         // this plan's own split-K partials
+    size_t part_o_bytes = 0;
+    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, total = 0;
+    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, total_q = 0;
+};
+
 namespace cf {
 
 static int env_int(const char* name, int fallback)
@@ -185,6 +199,85 @@ static float scale_log2_of(const cf_cache_desc* d)
 {
     const float sc = d->softmax_scale > 0.f ? d->softmax_scale : 1.0f / std::sqrt((float)d->head_dim);
     return sc * 1.4426950408889634f;
+}
+
+}  // namespace cf
+
+namespace cf {
+
+struct PlanCounts {
+    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, total_q = 0;
+};
+
+// Enqueues decode -> combine -> prefill for a plan that already sits in device memory at `base`.
+static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const PlanCounts& n, const PlanLayout& L,
+                                  uint8_t* base, float* part_o, float* part_ml, const void* q, const void* k_cache,
+                                  const void* v_cache, const int32_t* block_table, int32_t max_blocks_per_seq, void* out,
+                                  float* lse, cudaStream_t stream, bool allow_timing)
+{
+    const int Hq = desc->num_q_heads, D = desc->head_dim;
+    AttnParams p;
+    p.q = (const __nv_bfloat16*)q;
+    p.k_cache = (const __nv_bfloat16*)k_cache;
+    p.v_cache = (const __nv_bfloat16*)v_cache;
+    p.out = (__nv_bfloat16*)out;
+    p.lse = lse;
+    p.block_table = block_table;
+    p.max_blocks = max_blocks_per_seq;
+    p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
+    p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
+    p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
+    p.scale_log2 = scale_log2_of(desc);
+    p.q_start = (const int32_t*)(base + L.off_qstart);
+    p.context_len = (const int32_t*)(base + L.off_ctx);
+    p.query_len = (const int32_t*)(base + L.off_qlen);
+    p.dec_items = (const DecodeItem*)(base + L.off_dec);
+    p.comb_items = (const CombineItem*)(base + L.off_comb);
+    p.pre_items = (const PrefillItem*)(base + L.off_pre);
+    p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
+    p.part_o = part_o;
+    p.part_ml = part_ml;
+    p.err = c->err_dev;
+
+    cudaError_t e = cudaSuccess;
+    TimedCall* tc = nullptr;
+    if (c->timing && allow_timing) {
+        if (c->timed_used == c->timed.size()) {
+            TimedCall fresh;
+            bool ok = true;
+            for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&fresh.ev[i]) == cudaSuccess;
+            if (!ok) return CF_ERR_CUDA;
+            c->timed.push_back(fresh);
+        }
+        tc = &c->timed[c->timed_used++];
+        tc->ran[0] = (n.n_dec > 0);
+        tc->ran[1] = (n.n_comb > 0);
+        tc->ran[2] = (n.n_pre > 0) || (n.n_pre_tc > 0);
+    }
+    const bool has_prefill = (n.n_pre > 0) || (n.n_pre_tc > 0);
+    if (c->overlap && !tc && has_prefill && (n.n_dec > 0)) {
+        // prefill on the side stream, launched first so that its CTAs take their SMs; decode + combine
+        // on the caller's stream fill the rest of the machine; joined before returning to the caller
+        if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
+            e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, c->side);
+        if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
+        if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
+    } else {
+        if (tc) cudaEventRecord(tc->ev[0], stream);
+        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
+        if (tc) cudaEventRecord(tc->ev[1], stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
+        if (tc) cudaEventRecord(tc->ev[2], stream);
+        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, stream);
+        if (tc) cudaEventRecord(tc->ev[3], stream);
+    }
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0);
+    return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
 }  // namespace cf
@@ -364,70 +457,117 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
     if (st != CF_OK) return st;
 
-    AttnParams p;
-    p.q = (const __nv_bfloat16*)q;
-    p.k_cache = (const __nv_bfloat16*)k_cache;
-    p.v_cache = (const __nv_bfloat16*)v_cache;
-    p.out = (__nv_bfloat16*)out;
-    p.lse = lse;
+    PlanCounts n;
+    n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_pre = (int)pl.prefill.size();
+    n.n_pre_tc = (int)pl.prefill_tc.size(); n.total_q = pl.total_q;
+    const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, (float*)((uint8_t*)c->workspace + part_o_bytes),
+                                          q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
+    const cf_status fs = finish_slot(slot, stream);
+    return ls != CF_OK ? ls : fs;
+}
+
+cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t max_blocks_per_seq, void* cuda_stream, cf_plan** out)
+{
+    if (!c || !desc || !out) return CF_ERR_INVALID_ARG;
+    *out = nullptr;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    Plan pl;
+    PlanConfig cfg = c->cfg;
+    cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
+    if (st != CF_OK) return st;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cf_plan* P = new (std::nothrow) cf_plan();
+    if (!P) return CF_ERR_CUDA;
+    P->ctx = c;
+    P->desc = *desc;
+    P->num_seqs = num_seqs;
+    P->max_blocks = max_blocks_per_seq;
+    const PlanLayout L = layout_of(num_seqs, pl);
+    P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
+    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->total = L.total;
+    P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size(); P->n_pre = (int)pl.prefill.size();
+    P->n_pre_tc = (int)pl.prefill_tc.size(); P->total_q = pl.total_q;
+    P->part_o_bytes = align_up((size_t)pl.n_part_slots * desc->num_q_heads * desc->head_dim * sizeof(float), 256);
+    const size_t part_bytes = P->part_o_bytes + align_up((size_t)pl.n_part_slots * desc->num_q_heads * 2 * sizeof(float), 256);
+    bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
+    if (ok && part_bytes) ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess;
+    if (ok) {
+        std::memcpy(P->host + L.off_qstart, pl.q_start.data(), sizeof(int32_t) * ((size_t)num_seqs + 1));
+        if (num_seqs > 0) {
+            std::memcpy(P->host + L.off_ctx, context_len, sizeof(int32_t) * (size_t)num_seqs);
+            std::memcpy(P->host + L.off_qlen, query_len, sizeof(int32_t) * (size_t)num_seqs);
+        }
+        if (P->n_dec) std::memcpy(P->host + L.off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
+        if (P->n_comb) std::memcpy(P->host + L.off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
+        if (P->n_pre) std::memcpy(P->host + L.off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
+        if (P->n_pre_tc) std::memcpy(P->host + L.off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
+        ok = cudaMemcpyAsync(P->dev, P->host, L.total, cudaMemcpyHostToDevice, (cudaStream_t)cuda_stream) == cudaSuccess;
+    }
+    if (!ok) {
+        cf_plan_destroy(P);
+        return CF_ERR_CUDA;
+    }
+    *out = P;
+    return CF_OK;
+}
+
+cf_status cf_plan_destroy(cf_plan* P)
+{
+    if (!P) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(P->ctx->device);
+    cudaDeviceSynchronize();
+    if (P->host) cudaFreeHost(P->host);
+    if (P->dev) cudaFree(P->dev);
+    if (P->part) cudaFree(P->part);
+    delete P;
+    return CF_OK;
+}
+
+cf_status cf_kv_append_planned(cf_plan* P, void* k_cache, void* v_cache, const void* k_new, const void* v_new,
+                               const int32_t* block_table, void* cuda_stream)
+{
+    if (!P) return CF_ERR_INVALID_ARG;
+    if (P->total_q == 0) return CF_OK;
+    if (!k_cache || !v_cache || !k_new || !v_new || !block_table) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(P->ctx->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    const cf_cache_desc* desc = &P->desc;
+    AppendParams p;
+    p.k_cache = (__nv_bfloat16*)k_cache;
+    p.v_cache = (__nv_bfloat16*)v_cache;
+    p.k_new = (const __nv_bfloat16*)k_new;
+    p.v_new = (const __nv_bfloat16*)v_new;
     p.block_table = block_table;
-    p.max_blocks = max_blocks_per_seq;
+    p.max_blocks = P->max_blocks;
     p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
-    p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
-    p.scale_log2 = scale_log2_of(desc);
-    p.q_start = (const int32_t*)(base + L.off_qstart);
-    p.context_len = (const int32_t*)(base + L.off_ctx);
-    p.query_len = (const int32_t*)(base + L.off_qlen);
-    p.dec_items = (const DecodeItem*)(base + L.off_dec);
-    p.comb_items = (const CombineItem*)(base + L.off_comb);
-    p.pre_items = (const PrefillItem*)(base + L.off_pre);
-    p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
-    p.part_o = c->workspace;
-    p.part_ml = (float*)((uint8_t*)c->workspace + part_o_bytes);
-    p.err = c->err_dev;
+    p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = P->num_seqs; p.total_rows = P->total_q;
+    p.q_start = (const int32_t*)(P->dev + P->off_qstart);
+    p.context_len = (const int32_t*)(P->dev + P->off_ctx);
+    p.query_len = (const int32_t*)(P->dev + P->off_qlen);
+    return launch_kv_append(p, (cudaStream_t)cuda_stream) == cudaSuccess ? CF_OK : CF_ERR_CUDA;
+}
 
-    cudaError_t e = cudaSuccess;
-    TimedCall* tc = nullptr;
-    if (c->timing) {
-        if (c->timed_used == c->timed.size()) {
-            TimedCall fresh;
-            bool ok = true;
-            for (int i = 0; i < 4 && ok; ++i) ok = cudaEventCreate(&fresh.ev[i]) == cudaSuccess;
-            if (!ok) return CF_ERR_CUDA;
-            c->timed.push_back(fresh);
-        }
-        tc = &c->timed[c->timed_used++];
-        tc->ran[0] = !pl.decode.empty();
-        tc->ran[1] = !pl.combine.empty();
-        tc->ran[2] = !pl.prefill.empty() || !pl.prefill_tc.empty();
-    }
-    const bool has_prefill = !pl.prefill.empty() || !pl.prefill_tc.empty();
-    if (c->overlap && !tc && has_prefill && !pl.decode.empty()) {
-        // prefill on the side stream, launched first so that its CTAs take their SMs; decode + combine
-        // on the caller's stream fill the rest of the machine; joined before returning to the caller
-        if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
-            e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), c->side);
-        if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
-        if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
-        if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
-    } else {
-        if (tc) cudaEventRecord(tc->ev[0], stream);
-        if (e == cudaSuccess) e = launch_decode(p, D, (int)pl.decode.size(), stream);
-        if (tc) cudaEventRecord(tc->ev[1], stream);
-        if (e == cudaSuccess) e = launch_combine(p, D, (int)pl.combine.size(), stream);
-        if (tc) cudaEventRecord(tc->ev[2], stream);
-        if (e == cudaSuccess) e = launch_prefill_mma(p, D, (int)pl.prefill.size(), stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, pl.total_q, (int)pl.prefill_tc.size(), stream);
-        if (tc) cudaEventRecord(tc->ev[3], stream);
-    }
-    c->launches = (int)!pl.decode.empty() + (int)!pl.combine.empty() + (int)!pl.prefill.empty() + (int)!pl.prefill_tc.empty();
-    const cf_status fs = finish_slot(slot, stream);
-    if (e != cudaSuccess) return CF_ERR_CUDA;
-    return fs;
+cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_cache, const void* v_cache,
+                                     const int32_t* block_table, void* out, float* lse, void* cuda_stream)
+{
+    if (!P) return CF_ERR_INVALID_ARG;
+    P->ctx->launches = 0;
+    if (P->total_q == 0) return CF_OK;
+    if (!q || !k_cache || !v_cache || !block_table || !out) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(P->ctx->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    PlanLayout L;
+    L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
+    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.total = P->total;
+    PlanCounts n;
+    n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.total_q = P->total_q;
+    return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, (float*)((uint8_t*)P->part + P->part_o_bytes), q, k_cache,
+                            v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);
 }
 
 cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,

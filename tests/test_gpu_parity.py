@@ -282,3 +282,43 @@ def test_pipelined_host_steps_keep_their_order():
         assert np.array_equal(oh.numpy().view(np.uint16), ref), b.label
     ga.close()
     gb.close()
+
+
+def test_planned_calls_match_and_replay_from_a_cuda_graph():
+    """Plan once, launch per layer: the planned calls give the bits of the unplanned ones, and a CUDA
+    graph captured around them replays with the same result."""
+    sc = small(33, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
+    b = sc.batches[0]
+    ga, gb = GpuScenario(sc), GpuScenario(sc)
+    ga.append(b)
+    ref, ref_lse = ga.attend(b)
+    bt = torch.from_numpy(b.block_table).cuda()
+    q, kn, vn = to_dev_bf16(b.q), to_dev_bf16(b.k_new), to_dev_bf16(b.v_new)
+    out = torch.zeros_like(q)
+    lse = torch.zeros((b.total_q, 32), dtype=torch.float32, device="cuda")
+    plan = cf.cf_plan_create(gb.ctx, gb.desc, b.context_len, b.query_len, b.max_blocks)
+    cf.cf_kv_append_planned(plan, gb.k, gb.v, kn, vn, bt)
+    cf.cf_mixed_attention_planned(plan, q, gb.k, gb.v, bt, out, lse)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(gb.k), to_host_bits(ga.k)) and np.array_equal(to_host_bits(gb.v), to_host_bits(ga.v))
+    assert np.array_equal(to_host_bits(out), ref) and np.array_equal(lse.cpu().numpy(), ref_lse)
+    # capture the two planned calls of one layer and replay them
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        out.zero_()
+        side.synchronize()
+        with torch.cuda.graph(graph, stream=side):
+            cf.cf_kv_append_planned(plan, gb.k, gb.v, kn, vn, bt, stream=side)
+            cf.cf_mixed_attention_planned(plan, q, gb.k, gb.v, bt, out, lse, stream=side)
+    out.zero_()
+    lse.zero_()
+    graph.replay()
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(out), ref) and np.array_equal(lse.cpu().numpy(), ref_lse)
+    assert cf.cf_get_async_status(gb.ctx) == cf.CF_OK
+    del graph
+    cf.cf_plan_destroy(plan)
+    ga.close()
+    gb.close()
