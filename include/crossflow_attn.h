@@ -193,6 +193,16 @@ cf_status cf_decode_attention_static(const cf_cache_desc* desc, const void* q,
                                      const int32_t* context_len, int32_t num_seqs,
                                      void* out, float* lse, void* cuda_stream);
 
+/* Section 4.2: a decode node publishes a lease whose compute credit is counted in token chunks, derived
+ * from its latency headroom.  cf_estimate_us predicts, on the host and without a GPU, the device time
+ * (microseconds) of the decode, combine and prefill kernels that cf_mixed_attention would launch for
+ * these lengths on a B200 with num_sms SMs (0 = 148), from a model fitted to this library's measured
+ * times: a scheduler can size the next prefill chunk so that the iteration stays inside its ITL budget.
+ * Accuracy on the five workload configurations: within about 15 %.  Any output pointer may be NULL. */
+cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                         float* us_decode, float* us_combine, float* us_prefill);
+
 /* Host planner, exposed for inspection and tests (no GPU needed).  Builds the plan that
  * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.
  *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}

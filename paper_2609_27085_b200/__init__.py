@@ -34,7 +34,7 @@ CF_ERR_ARCH = 7
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_status_string")
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
+    lib.cf_estimate_us.argtypes = [dp, vp, vp, i32, i32, i32, fp, fp, fp]
     lib.cf_plan_create.argtypes = [vp, dp, vp, vp, i32, i32, vp, ctypes.POINTER(vp)]
     lib.cf_plan_destroy.argtypes = [vp]
     lib.cf_kv_append_planned.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -268,3 +269,13 @@ def cf_kv_append_planned(plan, k_cache, v_cache, k_new, v_new, block_table, stre
 def cf_mixed_attention_planned(plan, q, k_cache, v_cache, block_table, out, lse=None, stream=None) -> None:
     _check(load_library().cf_mixed_attention_planned(plan, _dev(q), _dev(k_cache), _dev(v_cache), _dev(block_table),
                                                      _dev(out), _dev(lse), _stream(stream)), "cf_mixed_attention_planned")
+
+
+def cf_estimate_us(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148) -> Tuple[float, float, float]:
+    """Predicted (us_decode, us_combine, us_prefill) of one cf_mixed_attention call on a B200 (host only)."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    a, b, c = ctypes.c_float(), ctypes.c_float(), ctypes.c_float()
+    _check(load_library().cf_estimate_us(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
+                                         int(max_blocks_per_seq), int(num_sms), ctypes.byref(a), ctypes.byref(b),
+                                         ctypes.byref(c)), "cf_estimate_us")
+    return a.value, b.value, c.value

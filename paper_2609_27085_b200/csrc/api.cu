@@ -710,6 +710,28 @@ cf_status cf_get_last_launch_count(cf_ctx* c, int32_t* num_launches)
     return CF_OK;
 }
 
+cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                         float* us_decode, float* us_combine, float* us_prefill)
+{
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    PlanConfig cfg;
+    cfg.num_sms = num_sms > 0 ? num_sms : 148;
+    cfg.decode_waves = env_int("CF_DECODE_WAVES", cfg.decode_waves);
+    cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
+    cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
+    Plan pl;
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
+    if (st != CF_OK) return st;
+    const Estimate e = estimate_us(desc, context_len, query_len, pl, cfg.num_sms);
+    if (us_decode) *us_decode = e.us_decode;
+    if (us_combine) *us_combine = e.us_combine;
+    if (us_prefill) *us_prefill = e.us_prefill;
+    return CF_OK;
+}
+
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
                           int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
                           int32_t* decode_items, int32_t* combine_items, int32_t* prefill_items,

@@ -166,4 +166,44 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     return CF_OK;
 }
 
+Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
+                     int32_t num_sms)
+{
+    // Constants fitted on B200 (see the measured table in the design notes): split-K decode sustains
+    // ~7.1 TB/s on top of ~17 us of launch, ramp and tail; the combine launch is ~10 us; one tcgen05
+    // prefill item costs ~8 us plus ~1.9 us per 128-token KV tile; the mma.sync path runs ~220 TFLOP/s.
+    constexpr double kDecodeFixedUs = 17.0, kDecodeBytesPerUs = 7.1e6, kCombineUs = 10.0;
+    constexpr double kTcItemFixedUs = 8.0, kTcTileUs = 1.9, kMmaFlopsPerUs = 220e6, kLaunchUs = 4.0;
+    Estimate e;
+    const int32_t S = (int32_t)plan.q_start.size() - 1;
+    double dec_bytes = 0.0;
+    for (int32_t s = 0; s < S; ++s)
+        if (query_len[s] == 1)
+            dec_bytes += (double)context_len[s] * 2.0 * d->num_kv_heads * d->head_dim * 2.0 + 4.0 * d->num_q_heads * d->head_dim;
+    if (!plan.decode.empty()) e.us_decode = (float)(kDecodeFixedUs + dec_bytes / kDecodeBytesPerUs);
+    if (!plan.combine.empty()) e.us_combine = (float)kCombineUs;
+    if (!plan.prefill_tc.empty()) {
+        // items are already longest-first: greedy list scheduling onto num_sms machines
+        std::vector<double> load((size_t)std::max(1, num_sms), 0.0);
+        for (const PrefillTcItem& it : plan.prefill_tc) {
+            const int32_t prefix = context_len[it.seq] - query_len[it.seq];
+            int32_t hi = 0;
+            for (int t = 0; t < 2; ++t)
+                if (it.n_rows[t] > 0) hi = std::max(hi, prefix + it.row0[t] + it.n_rows[t]);
+            const double cost = kTcItemFixedUs + kTcTileUs * ((hi + 127) / 128);
+            *std::min_element(load.begin(), load.end()) += cost;
+        }
+        e.us_prefill = (float)(kLaunchUs + *std::max_element(load.begin(), load.end()));
+    } else if (!plan.prefill.empty()) {
+        double flops = 0.0;
+        for (int32_t s = 0; s < S; ++s)
+            if (query_len[s] > 1) {
+                const double lq = query_len[s], pre = context_len[s] - query_len[s];
+                flops += 4.0 * d->head_dim * d->num_q_heads * (lq * pre + lq * (lq + 1) / 2);
+            }
+        e.us_prefill = (float)(kLaunchUs + flops / kMmaFlopsPerUs);
+    }
+    return e;
+}
+
 }  // namespace cf

@@ -73,4 +73,14 @@ cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, c
 cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
                      int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan);
 
+// Predicted device time of one cf_mixed_attention call, in microseconds, from a model fitted to this
+// library's measured kernel times on B200 (decode: fixed cost + bytes at the sustained split-K rate;
+// prefill: work items scheduled longest-first onto the SMs, each costing a fixed part plus a time per
+// 128-token KV tile).  Meant for deriving a lease's compute credit from a latency headroom (Section 4.2).
+struct Estimate {
+    float us_decode = 0.f, us_combine = 0.f, us_prefill = 0.f;
+};
+Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
+                     int32_t num_sms);
+
 }  // namespace cf

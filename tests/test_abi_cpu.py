@@ -137,3 +137,17 @@ def test_calls_without_a_device_fail_with_a_status():
     assert st in (cf.CF_ERR_CUDA, cf.CF_ERR_INVALID_ARG) and not ctx.value
     with pytest.raises(cf.CfError):
         cf.cf_create(0)
+
+
+def test_cost_model_is_sane_on_the_host():
+    d = cf.make_desc(32, 8, 128, 16, 65536)
+    dec, comb, pre = cf.cf_estimate_us(d, [4096] * 64, [1] * 64, 4096)
+    assert pre == 0 and dec > 0
+    dec2, _, _ = cf.cf_estimate_us(d, [8192] * 64, [1] * 64, 4096)
+    assert dec2 > dec * 1.5                                       # decode time follows the K/V bytes
+    _, _, p1 = cf.cf_estimate_us(d, [6144 + 512], [512], 4096)
+    _, _, p2 = cf.cf_estimate_us(d, [24576 + 2048], [2048], 4096)
+    assert 0 < p1 < p2
+    _, _, p3 = cf.cf_estimate_us(d, [24576 + 2048], [2048], 4096, num_sms=74)
+    assert p3 > 1.5 * p2                                          # half the SMs, about twice the waves
+    assert cf.cf_estimate_us(d, [7], [0], 4096) == (0.0, 0.0, 0.0)

@@ -322,3 +322,27 @@ def test_planned_calls_match_and_replay_from_a_cuda_graph():
     cf.cf_plan_destroy(plan)
     ga.close()
     gb.close()
+
+
+def test_cost_model_tracks_measured_kernel_times():
+    """cf_estimate_us (host model, Section 4.2's compute credit) against CUDA-event times of the
+    kernels on two reduced workloads: within 30 %."""
+    import bench
+    for case in ("decode_small", "prefill_small"):
+        sc = bench.small_case(case)
+        b = sc.batches[0]
+        g = GpuScenario(sc)
+        g.append(b)
+        for _ in range(3):
+            g.attend(b, want_lse=False, poison=False)
+        cf.cf_set_timing(g.ctx, True)
+        for _ in range(5):
+            g.attend(b, want_lse=False, poison=False)
+        ms_dec, ms_comb, ms_pre, n = cf.cf_get_timing_sums(g.ctx)
+        cf.cf_set_timing(g.ctx, False)
+        est_dec, est_comb, est_pre = cf.cf_estimate_us(g.desc, b.context_len, b.query_len, b.max_blocks, 148)
+        if case == "decode_small":
+            assert abs(est_dec / (1e3 * ms_dec / n) - 1.0) < 0.3, (est_dec, ms_dec / n)
+        else:
+            assert abs(est_pre / (1e3 * ms_pre / n) - 1.0) < 0.3, (est_pre, ms_pre / n)
+        g.close()
