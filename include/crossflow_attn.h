@@ -151,6 +151,15 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  * sets the initial value.  Per-kernel timing (cf_set_timing) forces the serial sequence. */
 cf_status cf_set_overlap(cf_ctx* ctx, int enabled);
 
+/* Debug aid (synchronous): checks every block-table entry that cf_kv_append / cf_mixed_attention would
+ * dereference for these lengths (entries [0, ceil(context_len/B)) of each row) against [0, num_blocks).
+ * The kernels themselves trust the table - an entry outside the pool is an out-of-bounds access on the
+ * device - so a serving engine runs this in its debug builds or after a scheduler change.  Reads the
+ * table only.  Returns CF_OK, or CF_ERR_OUT_OF_RANGE with the number of bad entries in *num_bad. */
+cf_status cf_validate_block_table(cf_ctx* ctx, const cf_cache_desc* desc, const int32_t* block_table,
+                                  int32_t max_blocks_per_seq, const int32_t* context_len, const int32_t* query_len,
+                                  int32_t num_seqs, void* cuda_stream, int32_t* num_bad);
+
 /* Self-test of the bounded-wait machinery (no counterpart in the paper): enqueues one tiny kernel whose
  * wait on a barrier that nothing signals expires after a few milliseconds; the kernel then sets the
  * context's error word and returns normally.  After synchronising, cf_get_async_status must report

@@ -34,7 +34,7 @@ CF_ERR_ARCH = 7
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_status_string")
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -79,6 +79,7 @@ def load_library() -> ctypes.CDLL:
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
+    lib.cf_validate_block_table.argtypes = [vp, dp, vp, i32, vp, vp, i32, vp, i32p]
     lib.cf_estimate_us.argtypes = [dp, vp, vp, i32, i32, i32, fp, fp, fp]
     lib.cf_plan_create.argtypes = [vp, dp, vp, vp, i32, i32, vp, ctypes.POINTER(vp)]
     lib.cf_plan_destroy.argtypes = [vp]
@@ -279,3 +280,16 @@ def cf_estimate_us(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: 
                                          int(max_blocks_per_seq), int(num_sms), ctypes.byref(a), ctypes.byref(b),
                                          ctypes.byref(c)), "cf_estimate_us")
     return a.value, b.value, c.value
+
+
+def cf_validate_block_table(ctx, desc: CacheDesc, block_table, max_blocks_per_seq: int, context_len, query_len,
+                            stream=None) -> int:
+    """Number of block-table entries in use that fall outside the pool (0 = table is safe to use)."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    bad = ctypes.c_int32()
+    st = load_library().cf_validate_block_table(ctx, ctypes.byref(desc), _dev(block_table), int(max_blocks_per_seq),
+                                                lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]), _stream(stream),
+                                                ctypes.byref(bad))
+    if st not in (CF_OK, CF_ERR_OUT_OF_RANGE):
+        raise CfError(st, "cf_validate_block_table")
+    return bad.value

@@ -656,6 +656,43 @@ cf_status cf_get_async_status(cf_ctx* c)
     return CF_ERR_TIMEOUT;
 }
 
+cf_status cf_validate_block_table(cf_ctx* c, const cf_cache_desc* desc, const int32_t* block_table,
+                                  int32_t max_blocks_per_seq, const int32_t* context_len, const int32_t* query_len,
+                                  int32_t num_seqs, void* cuda_stream, int32_t* num_bad)
+{
+    if (!c || !desc || !num_bad) return CF_ERR_INVALID_ARG;
+    *num_bad = 0;
+    cf_status st = validate_desc(desc);
+    if (st != CF_OK) return st;
+    Plan pl;
+    st = validate_lengths(desc, context_len, query_len, num_seqs, max_blocks_per_seq, &pl);
+    if (st != CF_OK) return st;
+    if (num_seqs == 0) return CF_OK;
+    if (!block_table) return CF_ERR_INVALID_ARG;
+    DeviceGuard guard(c->device);
+    if (!guard.ok) return CF_ERR_CUDA;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    PlanLayout L;
+    uint8_t* base = nullptr;
+    PlanSlot* slot = nullptr;
+    st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
+    if (st != CF_OK) return st;
+    // the counter lives in the slot's device buffer, after the plan
+    uint32_t* counter = nullptr;
+    if (cudaMalloc((void**)&counter, sizeof(uint32_t)) != cudaSuccess) return CF_ERR_CUDA;
+    bool ok = cudaMemsetAsync(counter, 0, sizeof(uint32_t), stream) == cudaSuccess;
+    ok = ok && launch_validate_table(block_table, max_blocks_per_seq, (const int32_t*)(base + L.off_ctx), num_seqs,
+                                     desc->num_blocks, counter, stream) == cudaSuccess;
+    finish_slot(slot, stream);
+    uint32_t host = 0;
+    ok = ok && cudaMemcpyAsync(&host, counter, sizeof host, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
+    ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
+    cudaFree(counter);
+    if (!ok) return CF_ERR_CUDA;
+    *num_bad = (int32_t)host;
+    return host ? CF_ERR_OUT_OF_RANGE : CF_OK;
+}
+
 cf_status cf_set_overlap(cf_ctx* c, int enabled)
 {
     if (!c) return CF_ERR_INVALID_ARG;

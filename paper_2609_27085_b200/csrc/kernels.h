@@ -22,6 +22,8 @@ struct AppendParams {
 };
 
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream);
+cudaError_t launch_validate_table(const int32_t* block_table, int32_t max_blocks, const int32_t* context_len_dev,
+                                  int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 // mma.sync chunked prefill; tile height must equal kPrefillMmaTileRows

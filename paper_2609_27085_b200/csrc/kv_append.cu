@@ -37,6 +37,30 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p)
     }
 }
 
+// Debug aid: counts the block-table entries that a call with these lengths would dereference and that
+// fall outside [0, num_blocks).  Reads the table only; never touches the caches.
+__global__ void validate_table_kernel(const int32_t* block_table, int32_t max_blocks, const int32_t* context_len,
+                                      int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count)
+{
+    const int s = blockIdx.x;
+    if (s >= num_seqs) return;
+    const int used = (context_len[s] + 15) >> 4;
+    uint32_t bad = 0;
+    for (int i = threadIdx.x; i < used && i < max_blocks; i += blockDim.x) {
+        const int32_t b = block_table[(int64_t)s * max_blocks + i];
+        bad += (b < 0 || b >= num_blocks) ? 1u : 0u;
+    }
+    if (bad) atomicAdd(bad_count, bad);
+}
+
+cudaError_t launch_validate_table(const int32_t* block_table, int32_t max_blocks, const int32_t* context_len_dev,
+                                  int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count, cudaStream_t stream)
+{
+    if (num_seqs <= 0) return cudaSuccess;
+    validate_table_kernel<<<num_seqs, 128, 0, stream>>>(block_table, max_blocks, context_len_dev, num_seqs, num_blocks, bad_count);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_kv_append(const AppendParams& p, cudaStream_t stream)
 {
     if (p.total_rows <= 0) return cudaSuccess;

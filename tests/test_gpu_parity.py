@@ -346,3 +346,45 @@ def test_cost_model_tracks_measured_kernel_times():
         else:
             assert abs(est_pre / (1e3 * ms_pre / n) - 1.0) < 0.3, (est_pre, ms_pre / n)
         g.close()
+
+
+def test_validate_block_table_finds_entries_outside_the_pool():
+    sc = small(35, 8, 2, 64, [100, 40, 0], [[1, 20, 5]], NB=64)
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    bt = torch.from_numpy(b.block_table).cuda()
+    assert cf.cf_validate_block_table(g.ctx, g.desc, bt, b.max_blocks, b.context_len, b.query_len) == 0
+    bad = b.block_table.copy()
+    bad[0, 3] = 64            # one past the pool
+    bad[1, 0] = -5
+    bad[2, 3] = 9999          # beyond this sequence's used entries: not dereferenced, not counted
+    assert cf.cf_validate_block_table(g.ctx, g.desc, torch.from_numpy(bad).cuda(), b.max_blocks, b.context_len, b.query_len) == 2
+    g.close()
+
+
+def test_sequences_sharing_prefix_pages():
+    """Radix-cache reuse: several sequences whose block tables point at the same prefix pages
+    (Section 4.4: a lookup determines how much of the prompt is reusable)."""
+    geom = syn.Geometry(32, 8, 128, 16, 512)
+    rng = np.random.default_rng(37)
+    k_pool, v_pool = syn.empty_pools(geom)
+    shared = np.arange(100, 100 + 40, dtype=np.int32)            # 640 shared prefix tokens
+    syn.fill_prefix(rng, geom, k_pool, shared, 640)
+    syn.fill_prefix(rng, geom, v_pool, shared, 640)
+    prefix = [640 + 35, 640 + 300, 640]                          # own suffixes beyond the shared pages
+    qlen = [1, 150, 1]
+    table = np.full((3, 80), -1, dtype=np.int32)
+    nxt = 200
+    for s in range(3):
+        table[s, :40] = shared
+        own = (prefix[s] + qlen[s] + 15) // 16 - 40
+        table[s, 40:40 + own] = np.arange(nxt, nxt + own)
+        nxt += own
+        n_own = prefix[s] - 640
+        if n_own:
+            syn.fill_prefix(rng, geom, k_pool, table[s, 40:], n_own)
+            syn.fill_prefix(rng, geom, v_pool, table[s, 40:], n_own)
+    # sequence 2 appends its new token into a fresh page; the shared pages are never written
+    b = syn.make_batch(rng, geom, np.array(prefix) + np.array(qlen), qlen, table, label="shared-prefix")
+    sc = syn.Scenario("shared", geom, k_pool, v_pool, [b])
+    run_and_check(sc)
