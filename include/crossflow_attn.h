@@ -218,7 +218,9 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
  *   combine_items : int32 [cap, 3] = {q_row, first_partial_slot, num_chunks}
  *   prefill_items : int32 [cap, 6] = {seq, q_row_of_tile, first_row_in_chunk, num_rows, query_head, kv_head},
  *                   one entry per (q tile, query head) in launch order
- *   counts        : int32 [4]      = {n_decode_items, n_combine_items, n_prefill_entries, n_partial_slots}
+ *                   (a KV-split item is listed once)
+ *   counts        : int32 [6]      = {n_decode_items, n_combine_items, n_prefill_entries, n_partial_slots,
+ *                                     n_prefill_ctas (KV ranges of split items counted), n_kv_split_prefill_items}
  * Any output pointer may be NULL. */
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
                           int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,

@@ -224,7 +224,7 @@ def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq:
     dec = np.zeros((cap, 6), dtype=np.int32)
     comb = np.zeros((cap, 3), dtype=np.int32)
     pre = np.zeros((cap, 6), dtype=np.int32)
-    counts = np.zeros(4, dtype=np.int32)
+    counts = np.zeros(6, dtype=np.int32)
     st = load_library().cf_plan_inspect(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
                                         int(max_blocks_per_seq), int(num_sms), dec.ctypes.data, comb.ctypes.data,
                                         pre.ctypes.data, cap, counts.ctypes.data)

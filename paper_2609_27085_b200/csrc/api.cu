@@ -77,9 +77,9 @@ struct cf_plan {
     uint8_t* host = nullptr;       // pinned copy (source of the one upload)
     uint8_t* dev = nullptr;
     float* part = nullptr;         // this plan's own split-K partials
-    size_t part_o_bytes = 0;
-    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, total = 0;
-    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, total_q = 0;
+    int n_part_slots = 0, n_pre_slots = 0;
+    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, off_pre_comb = 0, total = 0;
+    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
 };
 
 namespace cf {
@@ -144,7 +144,7 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, off_pre_comb, total;
 };
 
 static PlanLayout layout_of(int32_t S, const Plan& pl)
@@ -158,6 +158,7 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_comb = at;   at = align_up(at + sizeof(CombineItem) * pl.combine.size(), 16);
     L.off_pre = at;    at = align_up(at + sizeof(PrefillItem) * pl.prefill.size(), 16);
     L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
+    L.off_pre_comb = at; at = align_up(at + sizeof(PrefillCombineItem) * pl.prefill_combine.size(), 16);
     L.total = at ? at : 16;
     return L;
 }
@@ -182,6 +183,8 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     if (!pl.prefill.empty()) std::memcpy(s.host + L->off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
     if (!pl.prefill_tc.empty())
         std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
+    if (!pl.prefill_combine.empty())
+        std::memcpy(s.host + L->off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
     if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
     *dev_base = s.dev;
     *slot_out = &s;
@@ -206,12 +209,28 @@ static float scale_log2_of(const cf_cache_desc* d)
 namespace cf {
 
 struct PlanCounts {
-    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, total_q = 0;
+    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
 };
+
+// Split-K workspace: decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact partial rows of
+// KV-split prefill items [row slot, D] + [row slot, 2].
+struct WsLayout {
+    size_t dec_o = 0, dec_ml = 0, pre_o = 0, pre_ml = 0, total = 0;
+};
+static WsLayout ws_layout(int n_part_slots, int n_pre_slots, int Hq, int D)
+{
+    WsLayout w;
+    w.dec_o = 0;
+    w.dec_ml = align_up((size_t)n_part_slots * Hq * D * sizeof(float), 256);
+    w.pre_o = w.dec_ml + align_up((size_t)n_part_slots * Hq * 2 * sizeof(float), 256);
+    w.pre_ml = w.pre_o + align_up((size_t)n_pre_slots * D * sizeof(float), 256);
+    w.total = w.pre_ml + align_up((size_t)n_pre_slots * 2 * sizeof(float), 256);
+    return w;
+}
 
 // Enqueues decode -> combine -> prefill for a plan that already sits in device memory at `base`.
 static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const PlanCounts& n, const PlanLayout& L,
-                                  uint8_t* base, float* part_o, float* part_ml, const void* q, const void* k_cache,
+                                  uint8_t* base, float* ws, const WsLayout& W, const void* q, const void* k_cache,
                                   const void* v_cache, const int32_t* block_table, int32_t max_blocks_per_seq, void* out,
                                   float* lse, cudaStream_t stream, bool allow_timing)
 {
@@ -235,8 +254,11 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.comb_items = (const CombineItem*)(base + L.off_comb);
     p.pre_items = (const PrefillItem*)(base + L.off_pre);
     p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
-    p.part_o = part_o;
-    p.part_ml = part_ml;
+    p.part_o = ws;
+    p.part_ml = (float*)((uint8_t*)ws + W.dec_ml);
+    p.pre_part_o = (float*)((uint8_t*)ws + W.pre_o);
+    p.pre_part_ml = (float*)((uint8_t*)ws + W.pre_ml);
+    p.pre_comb_items = (const PrefillCombineItem*)(base + L.off_pre_comb);
     p.err = c->err_dev;
 
     cudaError_t e = cudaSuccess;
@@ -262,6 +284,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, c->side);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, c->side);
+        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, c->side);
         if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
         if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
@@ -274,9 +297,10 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[2], stream);
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, stream);
+        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0);
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0);
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -323,6 +347,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.decode_waves = env_int("CF_DECODE_WAVES", c->cfg.decode_waves);
     c->cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", c->cfg.decode_min_chunk_pages);
     c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
+    c->cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
     c->overlap = env_int("CF_OVERLAP", 0) != 0;
     bool ok = true;
@@ -446,9 +471,8 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     cudaStream_t stream = (cudaStream_t)cuda_stream;
 
     const int Hq = desc->num_q_heads, D = desc->head_dim;
-    const size_t part_o_bytes = align_up((size_t)pl.n_part_slots * Hq * D * sizeof(float), 256);
-    const size_t part_ml_bytes = align_up((size_t)pl.n_part_slots * Hq * 2 * sizeof(float), 256);
-    st = ensure_workspace(c, part_o_bytes + part_ml_bytes);
+    const WsLayout W = ws_layout(pl.n_part_slots, pl.n_pre_slots, Hq, D);
+    st = ensure_workspace(c, W.total);
     if (st != CF_OK) return st;
 
     PlanLayout L;
@@ -459,8 +483,8 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
 
     PlanCounts n;
     n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_pre = (int)pl.prefill.size();
-    n.n_pre_tc = (int)pl.prefill_tc.size(); n.total_q = pl.total_q;
-    const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, (float*)((uint8_t*)c->workspace + part_o_bytes),
+    n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
+    const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
     const cf_status fs = finish_slot(slot, stream);
     return ls != CF_OK ? ls : fs;
@@ -488,11 +512,12 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->max_blocks = max_blocks_per_seq;
     const PlanLayout L = layout_of(num_seqs, pl);
     P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
-    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->total = L.total;
+    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb;
+    P->total = L.total;
     P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size(); P->n_pre = (int)pl.prefill.size();
-    P->n_pre_tc = (int)pl.prefill_tc.size(); P->total_q = pl.total_q;
-    P->part_o_bytes = align_up((size_t)pl.n_part_slots * desc->num_q_heads * desc->head_dim * sizeof(float), 256);
-    const size_t part_bytes = P->part_o_bytes + align_up((size_t)pl.n_part_slots * desc->num_q_heads * 2 * sizeof(float), 256);
+    P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
+    P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
+    const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
     if (ok && part_bytes) ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess;
     if (ok) {
@@ -505,6 +530,8 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
         if (P->n_comb) std::memcpy(P->host + L.off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
         if (P->n_pre) std::memcpy(P->host + L.off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
         if (P->n_pre_tc) std::memcpy(P->host + L.off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
+        if (P->n_pre_comb)
+            std::memcpy(P->host + L.off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
         ok = cudaMemcpyAsync(P->dev, P->host, L.total, cudaMemcpyHostToDevice, (cudaStream_t)cuda_stream) == cudaSuccess;
     }
     if (!ok) {
@@ -563,10 +590,13 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     if (!guard.ok) return CF_ERR_CUDA;
     PlanLayout L;
     L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
-    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.total = P->total;
+    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb;
+    L.total = P->total;
     PlanCounts n;
-    n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.total_q = P->total_q;
-    return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, (float*)((uint8_t*)P->part + P->part_o_bytes), q, k_cache,
+    n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
+    n.total_q = P->total_q;
+    const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim);
+    return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, W, q, k_cache,
                             v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);
 }
 
@@ -759,6 +789,7 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
     cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
     cfg.prefill_tile_rows = kPrefillMmaTileRows;
     cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
+    cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -782,6 +813,7 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
     cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
     cfg.prefill_tile_rows = kPrefillMmaTileRows;
     cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
+    cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -810,12 +842,14 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
         for (int32_t h = 0; h < desc->num_q_heads; ++h) emit(it.seq, it.q_row0, it.row0, it.n_rows, h, h / G);
     for (const PrefillTcItem& it : pl.prefill_tc)
         for (int t = 0; t < 2; ++t)
-            if (it.n_rows[t] > 0) emit(it.seq, it.q_row0[t], it.row0[t], it.n_rows[t], it.head[t], it.kvh);
+            if (it.n_rows[t] > 0 && it.part_c == 0) emit(it.seq, it.q_row0[t], it.row0[t], it.n_rows[t], it.head[t], it.kvh);
     if (counts) {
         counts[0] = (int32_t)pl.decode.size();
         counts[1] = (int32_t)pl.combine.size();
         counts[2] = (int32_t)n_pre;
         counts[3] = pl.n_part_slots;
+        counts[4] = (int32_t)pl.prefill_tc.size();          // prefill CTAs, KV ranges of split items included
+        counts[5] = (int32_t)pl.prefill_combine.size();     // KV-split prefill items
     }
     return CF_OK;
 }

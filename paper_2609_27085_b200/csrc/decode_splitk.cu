@@ -434,6 +434,7 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     p.comb_items = reinterpret_cast<const CombineItem*>(su.base + comb_off);
     p.pre_items = nullptr;
     p.pre_tc_items = nullptr;
+    p.pre_part_o = nullptr; p.pre_part_ml = nullptr; p.pre_comb_items = nullptr;
     // Partials need no clearing: every slot the combine kernel reads is fully written by its decode CTA
     // in the same call.
     p.part_o = reinterpret_cast<float*>(su.base + kStaticPlanBytes);

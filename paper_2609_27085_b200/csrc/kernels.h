@@ -35,6 +35,8 @@ bool prefill_tc_supported(const cf_cache_desc* desc);
 cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items,
                               cudaStream_t stream);
 
+// merges the fp32 partials of KV-split prefill items into `out` (one CTA per split item)
+cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream);
 // one CTA whose bounded wait must expire: sets *err and returns normally (status-path self-test)
 cudaError_t launch_wait_selftest(uint32_t* err, cudaStream_t stream);
 

@@ -1,6 +1,8 @@
 #include "plan.h"
 
 #include <algorithm>
+#include <climits>
+#include <cstdint>
 
 namespace cf {
 
@@ -104,6 +106,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         const int32_t G = d->num_q_heads / d->num_kv_heads;
         struct KeyedTc { int64_t extent; PrefillTcItem it; };
         std::vector<KeyedTc> items;
+        auto prefix_of = [&](int32_t s) { return context_len[s] - query_len[s]; };
         for (int32_t s = 0; s < num_seqs; ++s) {
             const int32_t lq = query_len[s];
             if (lq <= 1) continue;
@@ -116,6 +119,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                         for (int32_t i = 0; i < G; i += 2) {
                             PrefillTcItem it;
                             it.seq = s; it.kvh = kvh;
+                            it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
                             for (int t = 0; t < 2; ++t) {
                                 it.q_row0[t] = plan->q_start[s] + tile * TR;
                                 it.row0[t] = tile * TR;
@@ -129,6 +133,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     for (int32_t h = 0; h < d->num_q_heads; ++h) {
                         PrefillTcItem it;
                         it.seq = s; it.kvh = h;
+                        it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
                         int32_t last = tile;
                         for (int t = 0; t < 2; ++t) {
                             const int32_t tt = tile + t;
@@ -143,9 +148,90 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     }
             }
         }
+        // Few items (short chunks, few heads per GPU under tensor parallelism): a CTA's time is set by the
+        // per-tile softmax -> MMA chain, not by how many q tiles it carries, so pairs are split into
+        // single-tile items while that still leaves SMs idle.  Sharing K/V tiles matters only when the
+        // machine is full.
+        if (items.size() * 2 <= (size_t)std::max(1, cfg.num_sms)) {
+            std::vector<KeyedTc> singles;
+            singles.reserve(items.size() * 2);
+            for (const KeyedTc& k : items)
+                for (int t = 0; t < 2; ++t) {
+                    if (k.it.n_rows[t] == 0) continue;
+                    PrefillTcItem one = k.it;
+                    one.q_row0[0] = k.it.q_row0[t]; one.row0[0] = k.it.row0[t]; one.n_rows[0] = k.it.n_rows[t];
+                    one.head[0] = k.it.head[t];
+                    one.q_row0[1] = 0; one.row0[1] = 0; one.n_rows[1] = 0; one.head[1] = k.it.head[t];
+                    singles.push_back(KeyedTc{(int64_t)prefix_of(k.it.seq) + one.row0[0] + one.n_rows[0], one});
+                }
+            items.swap(singles);
+        }
         std::stable_sort(items.begin(), items.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
-        plan->prefill_tc.reserve(items.size());
-        for (const KeyedTc& k : items) plan->prefill_tc.push_back(k.it);
+        // ---- KV split of the last, incomplete wave.  Items run one per SM; after the full waves the
+        // remaining r items would occupy r SMs for a whole item time.  Cutting each of them into k KV
+        // ranges lets them fill the machine; the ranges write fp32 partials that a combine pass merges.
+        // k minimises (rounds x range time) + partial traffic + the extra launch, by the same constants as
+        // the cost model; a range never starts inside the diagonal band and has at least 4 tiles.
+        const size_t M = (size_t)std::max(1, cfg.num_sms);
+        const size_t n_items = items.size();
+        const size_t r = n_items % M, first_tail = n_items - r;
+        int32_t k_best = 1;
+        if (cfg.prefill_force_split >= 2) {
+            k_best = std::min(cfg.prefill_force_split, 8);
+        } else if (cfg.prefill_force_split == 1) {
+            k_best = 1;                                   // splitting switched off
+        } else if (r > 0) {
+            double tiles = 0.0;
+            for (size_t i = first_tail; i < n_items; ++i) tiles += (double)((items[i].extent + 127) / 128);
+            tiles /= (double)r;
+            double best = 1e30;
+            for (int32_t k = 1; k <= 8; ++k) {
+                if (k > 1 && tiles / k < 4.0) break;
+                const double rounds = (double)((r * (size_t)k + M - 1) / M);
+                // a whole item costs ~8 us + 1.9 us per tile; a KV range pays ~13 us (fp32 partial epilogue)
+                double t = rounds * ((k > 1 ? 13.0 : 8.0) + 1.9 * tiles / k);
+                if (k > 1) t += 8.0 + 0.05 * (double)(r * (size_t)k);     // combine launch + partial write/read
+                if (t < best * 0.97) { best = t; k_best = k; }             // split only for a clear gain
+            }
+        }
+        plan->prefill_tc.reserve(items.size() + (k_best > 1 ? r * (size_t)(k_best - 1) : 0));
+        const size_t split_from = cfg.prefill_force_split >= 2 ? 0 : first_tail;
+        for (size_t i = 0; i < n_items; ++i) {
+            PrefillTcItem it = items[i].it;
+            if (k_best <= 1 || i < split_from) {
+                plan->prefill_tc.push_back(it);
+                continue;
+            }
+            // tiles every present q tile takes part in, and the last tile boundary outside the diagonal band
+            const int32_t prefix = prefix_of(it.seq);
+            int32_t n_min = INT32_MAX, safe = INT32_MAX;
+            for (int t = 0; t < 2; ++t)
+                if (it.n_rows[t] > 0) {
+                    n_min = std::min(n_min, (prefix + it.row0[t] + it.n_rows[t] + 127) / 128);
+                    safe = std::min(safe, (prefix + it.row0[t]) / 128);
+                }
+            const int32_t k = std::min(k_best, std::max(1, std::min(n_min, safe + 1) / 4));
+            if (k <= 1) {
+                plan->prefill_tc.push_back(it);
+                continue;
+            }
+            PrefillCombineItem ci;
+            ci.part_k = k;
+            for (int t = 0; t < 2; ++t) {
+                ci.q_row0[t] = it.q_row0[t]; ci.n_rows[t] = it.n_rows[t]; ci.head[t] = it.head[t];
+                ci.part_slot[t] = it.n_rows[t] > 0 ? plan->n_pre_slots : -1;
+                plan->n_pre_slots += it.n_rows[t] * k;
+            }
+            plan->prefill_combine.push_back(ci);
+            for (int32_t c = 0; c < k; ++c) {
+                PrefillTcItem f = it;
+                f.j_begin = std::min((int32_t)((int64_t)c * n_min / k), safe);
+                f.j_end = c + 1 < k ? std::min((int32_t)((int64_t)(c + 1) * n_min / k), safe) : INT32_MAX;
+                f.part_slot[0] = ci.part_slot[0]; f.part_slot[1] = ci.part_slot[1];
+                f.part_k = k; f.part_c = c;
+                plan->prefill_tc.push_back(f);
+            }
+        }
         return CF_OK;
     }
     const int32_t tr = std::max(1, cfg.prefill_tile_rows);
@@ -190,10 +276,12 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
             int32_t hi = 0;
             for (int t = 0; t < 2; ++t)
                 if (it.n_rows[t] > 0) hi = std::max(hi, prefix + it.row0[t] + it.n_rows[t]);
-            const double cost = kTcItemFixedUs + kTcTileUs * ((hi + 127) / 128);
+            const int32_t tiles = std::max(0, std::min((hi + 127) / 128, it.j_end) - it.j_begin);
+            const double cost = kTcItemFixedUs + kTcTileUs * tiles;
             *std::min_element(load.begin(), load.end()) += cost;
         }
         e.us_prefill = (float)(kLaunchUs + *std::max_element(load.begin(), load.end()));
+        if (!plan.prefill_combine.empty()) e.us_prefill += (float)(6.0 + 0.05 * (double)plan.prefill_tc.size());
     } else if (!plan.prefill.empty()) {
         double flops = 0.0;
         for (int32_t s = 0; s < S; ++s)

@@ -40,6 +40,20 @@ struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one
     int32_t row0[2];       // index of that row inside the chunk
     int32_t n_rows[2];     // 0 = tile absent
     int32_t head[2];       // query head of each tile
+    // KV split: this item covers KV tiles [j_begin, j_end) (128-token tiles; j_end clamps to the item's
+    // own extent).  part_slot[t] >= 0: tile t writes an fp32 partial for row r into slot
+    // part_slot[t] + r * part_k + part_c instead of the final output.
+    int32_t j_begin, j_end;
+    int32_t part_slot[2];
+    int32_t part_k, part_c;
+};
+
+struct PrefillCombineItem { // one KV-split tcgen05 item: merges its part_k partials per row
+    int32_t q_row0[2];
+    int32_t n_rows[2];
+    int32_t head[2];
+    int32_t part_slot[2];
+    int32_t part_k;
 };
 
 struct PlanConfig {
@@ -50,6 +64,7 @@ struct PlanConfig {
     int32_t decode_page_quantum = 4;  // chunk lengths are multiples of this many pages (warps per CTA)
     int32_t prefill_tile_rows = 64;   // tile height of the mma.sync prefill kernel
     bool prefill_tc = false;          // true: plan items for the tcgen05 kernel (128-row tile pairs)
+    int32_t prefill_force_split = 0;  // >= 2: split every tcgen05 item that many ways (tests); 0: cost model decides
 };
 
 struct Plan {
@@ -57,7 +72,9 @@ struct Plan {
     std::vector<DecodeItem> decode;   // longest chunk first
     std::vector<CombineItem> combine;
     std::vector<PrefillItem> prefill; // longest KV extent first (mma.sync kernel)
-    std::vector<PrefillTcItem> prefill_tc;   // longest KV extent first (tcgen05 kernel)
+    std::vector<PrefillTcItem> prefill_tc;   // longest KV extent first (tcgen05 kernel); KV-split items appear part_k times
+    std::vector<PrefillCombineItem> prefill_combine;   // one per KV-split item
+    int32_t n_pre_slots = 0;          // fp32 partial rows of KV-split prefill items (compact, D floats each)
     int32_t n_part_slots = 0;
     int32_t total_q = 0;
     int32_t n_decode_seqs = 0;

@@ -115,11 +115,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
         kv_hi_t[t] = it.n_rows[t] > 0 ? prefix + it.row0[t] + it.n_rows[t] : 0;
-        n_j[t] = (kv_hi_t[t] + KT - 1) / KT;
+        // number of KV tiles of this item's range [j_begin, j_end) that tile t takes part in
+        n_j[t] = max(0, min((kv_hi_t[t] + KT - 1) / KT, it.j_end) - it.j_begin);
     }
     const int kv_hi = max(kv_hi_t[0], kv_hi_t[1]);
     const int n_max = max(n_j[0], n_j[1]);
     const int total_pages = (kv_hi + 15) >> 4;
+    const int jb = it.j_begin;                // loop indices below are relative to it; jb + j is the absolute tile
     volatile uint32_t* abort_flag = &abort_s;
 
     if (threadIdx.x == 0) {
@@ -167,8 +169,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         bool ok = true;
         for (int j = 0; j < n_max && ok; ++j) {
             const int stage = j % KV_STAGES, use = j / KV_STAGES;
-            const int np = min(8, total_pages - 8 * j);
-            const int32_t pid = lane < np ? __ldg(bt + 8 * j + lane) : 0;
+            const int np = min(8, total_pages - 8 * (jb + j));
+            const int32_t pid = lane < np ? __ldg(bt + 8 * (jb + j) + lane) : 0;
             const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
             const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
             // K tile
@@ -282,12 +284,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         auto kv_step = [&](auto S, int j) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
-            const int np = min(8, total_pages - 8 * j);
+            const int np = min(8, total_pages - 8 * (jb + j));
             if (!mbar_wait(bar_vf[st], (uint32_t)(j >> 1) & 1u, abort_flag)) return false;
-            if (j == n_max - 1 && Lc < (8 * j + np) * 16) {
+            if (j == n_max - 1 && Lc < (8 * (jb + j) + np) * 16) {
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
                 // that a zero probability never multiplies a NaN
-                const int r0 = Lc - j * KT, r1 = np * 16;
+                const int r0 = Lc - (jb + j) * KT, r1 = np * 16;
                 for (int idx = 0; idx < (r1 - r0) * 16; ++idx) {
                     const int r = r0 + (idx >> 4), c = idx & 15;
                     uint8_t* dst = smem_raw + ((smem + SMEM_V + st * TILE_BYTES) - smem_u32(smem_raw)) +
@@ -338,13 +340,14 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(&sv[c * 32]));
             tmem_wait_ld();
-            const int col_limit = limit - j * KT;            // columns <= col_limit are visible
+            const int col_limit = limit - (jb + j) * KT;     // columns <= col_limit are visible
             if (__any_sync(0xffffffffu, col_limit < KT - 1)) {
 #pragma unroll
                 for (int c = 0; c < 128; ++c) sv[c] = (c <= col_limit) ? sv[c] : -INFINITY;
             }
             if (j == 0) {
-                // first tile: exact row maximum (key 0 is visible to every row, so it is finite)
+                // first tile: exact row maximum.  It is finite: every row sees a key of the item's first
+                // tile (key 0 for a whole item; the planner never starts a split inside the diagonal band)
                 float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
                 for (int c = 4; c < 128; c += 8) {
@@ -424,13 +427,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tc_fence_after();
             const float inv = 1.f / l_sum;
             const bool live = row < it.n_rows[t];
+            const bool partial = it.part_slot[t] >= 0;
             __nv_bfloat16* orow = p.out + ((int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]) * D;
+            // KV-split item: un-normalised fp32 row plus (reference maximum, sum) for the combine pass
+            const int64_t pslot = (int64_t)it.part_slot[t] + (int64_t)row * it.part_k + it.part_c;
+            float* prow = p.pre_part_o + pslot * D;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
                 float ov[32];
                 tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
                 tmem_wait_ld();
-                if (live) {
+                if (live && partial) {
+#pragma unroll
+                    for (int i = 0; i < 8; ++i)
+                        *reinterpret_cast<float4*>(prow + c * 32 + i * 4) = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
+                } else if (live) {
 #pragma unroll
                     for (int i = 0; i < 4; ++i) {
                         uint4 w;
@@ -442,7 +453,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                 }
             }
-            if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
+            if (live && partial) *reinterpret_cast<float2*>(p.pre_part_ml + pslot * 2) = make_float2(m_used, l_sum);
+            else if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
         }
       }
     }
@@ -457,6 +469,58 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         __syncthreads();
     }
     if (warp == 0) tmem_dealloc<512>(tmem);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Merges the partials of KV-split prefill items: for every row of the item's q tiles,
+//   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
+// in fixed range order.  One warp per row (8 rows per CTA, 32 CTAs per split item), one float4 of the
+// row per lane; the partials of a row are fetched with independent loads (part_k <= 8).
+constexpr int kMaxSplit = 8;
+__global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p)
+{
+    const PrefillCombineItem it = p.pre_comb_items[blockIdx.x >> 5];
+    const int lane = threadIdx.x & 31;
+    const int rb = blockIdx.x & 31;                  // 32 blocks of 8 rows = 2 tiles x 128 rows
+    const int t = rb >> 4, r = (rb & 15) * 8 + (threadIdx.x >> 5);
+    if (r >= it.n_rows[t]) return;
+    const int k = it.part_k;
+    const int64_t s0 = (int64_t)it.part_slot[t] + (int64_t)r * k;
+    float2 ml[kMaxSplit];
+    float4 v[kMaxSplit];
+#pragma unroll
+    for (int c = 0; c < kMaxSplit; ++c)
+        if (c < k) {
+            ml[c] = __ldg(reinterpret_cast<const float2*>(p.pre_part_ml + (s0 + c) * 2));
+            v[c] = __ldg(reinterpret_cast<const float4*>(p.pre_part_o + (s0 + c) * D + lane * 4));
+        }
+    float M = -INFINITY;
+#pragma unroll
+    for (int c = 0; c < kMaxSplit; ++c)
+        if (c < k) M = fmaxf(M, ml[c].x);
+    float L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+    for (int c = 0; c < kMaxSplit; ++c)
+        if (c < k) {
+            const float f = fast_exp2(ml[c].x - M);
+            L += ml[c].y * f;
+            acc.x += v[c].x * f; acc.y += v[c].y * f; acc.z += v[c].z * f; acc.w += v[c].w * f;
+        }
+    const float inv = 1.f / L;
+    uint2 w;
+    w.x = pack_bf16(acc.x * inv, acc.y * inv);
+    w.y = pack_bf16(acc.z * inv, acc.w * inv);
+    const int64_t orow = (int64_t)(it.q_row0[t] + r) * p.Hq + it.head[t];
+    *reinterpret_cast<uint2*>(p.out + orow * D + lane * 4) = w;
+    if (p.lse && lane == 0) p.lse[orow] = (M + log2f(L)) * kLn2;
+}
+
+cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    prefill_combine_kernel<<<n_items * 32, 256, 0, stream>>>(p);
+    return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------------------------------------

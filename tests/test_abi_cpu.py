@@ -151,3 +151,29 @@ def test_cost_model_is_sane_on_the_host():
     _, _, p3 = cf.cf_estimate_us(d, [24576 + 2048], [2048], 4096, num_sms=74)
     assert p3 > 1.5 * p2                                          # half the SMs, about twice the waves
     assert cf.cf_estimate_us(d, [7], [0], 4096) == (0.0, 0.0, 0.0)
+
+
+def test_kv_split_of_the_last_prefill_wave():
+    """256 equal items on 148 SMs leave a last wave of 108: the planner cuts those into KV ranges that
+    tile each item's extent, never start inside the diagonal band, and fill the machine."""
+    import ctypes
+    d = cf.make_desc(32, 8, 128, 16, 65536)
+    lc, lq = [24576 + 2048], [2048]
+    st, dec, comb, pre, parts = cf.cf_plan_inspect(d, lc, lq, 4096, 148)
+    counts = np.zeros(6, dtype=np.int32)
+    lcn, lqn = np.array(lc, np.int32), np.array(lq, np.int32)
+    cf.load_library().cf_plan_inspect(ctypes.byref(d), lcn.ctypes.data, lqn.ctypes.data, 1, 4096, 148, None, None, None, 0,
+                                      counts.ctypes.data)
+    n_items = 16 * 16                                   # 16 q tiles x 16 head pairs
+    assert counts[5] == n_items % 148                   # the 108 items of the last wave are split
+    k = (counts[4] - (n_items - counts[5])) // counts[5]
+    assert k >= 2 and counts[4] == (n_items - counts[5]) + counts[5] * k
+    cover = np.zeros((2048, 32), dtype=np.int32)        # listed once per (row, head) all the same
+    for _, q_row0, row0, n_rows, head, kvh in pre:
+        cover[row0:row0 + n_rows, head] += 1
+    assert (cover == 1).all()
+    # 128 equal items on 148 SMs: splitting would not pay for its partial traffic
+    cf.load_library().cf_plan_inspect(ctypes.byref(d), np.array([6656, 6656], np.int32).ctypes.data,
+                                      np.array([512, 512], np.int32).ctypes.data, 2, 4096, 148, None, None, None, 0,
+                                      counts.ctypes.data)
+    assert counts[5] == 0 and counts[4] == 128

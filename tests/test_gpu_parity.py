@@ -388,3 +388,22 @@ def test_sequences_sharing_prefix_pages():
     b = syn.make_batch(rng, geom, np.array(prefix) + np.array(qlen), qlen, table, label="shared-prefix")
     sc = syn.Scenario("shared", geom, k_pool, v_pool, [b])
     run_and_check(sc)
+
+
+@pytest.mark.parametrize("k", [2, 3])
+def test_kv_split_prefill_items_match_the_oracle(k, monkeypatch):
+    """Every tcgen05 prefill item cut into k KV ranges (fp32 partials + the prefill combine kernel):
+    group sizes 1, 4 and 8, ragged chunks, a chunk with no prefix."""
+    monkeypatch.setenv("CF_PREFILL_SPLIT", str(k))           # read when the context is created
+    prefix = [2000, 0, 700, 4097, 300]
+    qlen = [300, 700, 129, 64, 1]
+    for Hq, Hkv in ((4, 4), (32, 8), (16, 2)):
+        sc = small(41 + Hq, Hq, Hkv, 128, prefix, [qlen], NB=2048)
+        d = cf.make_desc(Hq, Hkv, 128, 16, 2048)
+        import ctypes
+        counts = np.zeros(6, dtype=np.int32)
+        b = sc.batches[0]
+        cf.load_library().cf_plan_inspect(ctypes.byref(d), b.context_len.ctypes.data, b.query_len.ctypes.data, b.num_seqs,
+                                          b.max_blocks, 148, None, None, None, 0, counts.ctypes.data)
+        assert counts[5] > 0                                  # some items really were split
+        run_and_check(sc)
