@@ -26,3 +26,12 @@ def test_config4_agentic_first_and_last_iteration():
 @pytest.mark.parametrize("budget,n", [(0, 0), (512, 4), (2048, 3), (8192, 1)])
 def test_config5_sweep_points(budget, n):
     print(run_and_check(syn.config5_sweep_point(budget, n), max_prefill_rows=8, check_append=False))
+
+
+def test_paper_context_limit_128k():
+    """The paper's workers run a 128K-token context with 512 reserved (Section 6.1): one decode sequence
+    at that limit, one at a page boundary below it, and a 300-token prefill chunk that ends at the limit."""
+    geom = syn.Geometry(32, 8, 128, 16, 32768)
+    limit = 131072 - 512
+    sc = syn.scenario_from_lengths("ctx128k", geom, 4242, [limit - 1, 65536 - 1, limit - 300], [[1, 1, 300]])
+    print(run_and_check(sc, max_prefill_rows=16, check_append=False))
