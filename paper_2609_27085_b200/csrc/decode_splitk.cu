@@ -215,6 +215,7 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
 // ---------------------------------------------------------------------------------------------
 // Combine: merges the partials of a split sequence in fixed chunk order (deterministic).
 //   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
+// (evaluated as a running merge over groups of eight chunks)
 // grid (n_combine_items, Hq), D/4 threads, one float4 of the head each.
 template <int D>
 __global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
@@ -222,18 +223,36 @@ __global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
     const CombineItem it = p.comb_items[blockIdx.x];
     const int hq = blockIdx.y;
     const int d = threadIdx.x * 4;
-    float M = -INFINITY;
-    for (int c = 0; c < it.n_chunks; ++c)
-        M = fmaxf(M, __ldg(p.part_ml + ((int64_t)(it.part_first + c) * p.Hq + hq) * 2));
-    float L = 0.f;
+    // Partials are fetched eight chunks at a time with independent loads (a dependent load per chunk
+    // would cost a memory round trip each) and folded into a running (M, L, acc) in chunk order.
+    constexpr int GROUP = 8;
+    float M = -INFINITY, L = 0.f;
     float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c = 0; c < it.n_chunks; ++c) {
-        const int64_t pr = (int64_t)(it.part_first + c) * p.Hq + hq;
-        const float2 ml = __ldg(reinterpret_cast<const float2*>(p.part_ml + pr * 2));
-        const float f = fast_exp2(ml.x - M);
-        const float4 v = __ldg(reinterpret_cast<const float4*>(p.part_o + pr * D + d));
-        L += ml.y * f;
-        acc.x += v.x * f; acc.y += v.y * f; acc.z += v.z * f; acc.w += v.w * f;
+    for (int c0 = 0; c0 < it.n_chunks; c0 += GROUP) {
+        float2 ml[GROUP];
+        float4 v[GROUP];
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < it.n_chunks) {
+                const int64_t pr = (int64_t)(it.part_first + c0 + i) * p.Hq + hq;
+                ml[i] = __ldg(reinterpret_cast<const float2*>(p.part_ml + pr * 2));
+                v[i] = __ldg(reinterpret_cast<const float4*>(p.part_o + pr * D + d));
+            }
+        float Mg = M;
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < it.n_chunks) Mg = fmaxf(Mg, ml[i].x);
+        const float fold = fast_exp2(M - Mg);               // 0 on the first group (M = -inf)
+        L *= fold;
+        acc.x *= fold; acc.y *= fold; acc.z *= fold; acc.w *= fold;
+        M = Mg;
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < it.n_chunks) {
+                const float f = fast_exp2(ml[i].x - M);
+                L += ml[i].y * f;
+                acc.x += v[i].x * f; acc.y += v[i].y * f; acc.z += v[i].z * f; acc.w += v[i].w * f;
+            }
     }
     const float inv = 1.f / L;
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
