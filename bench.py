@@ -13,7 +13,7 @@ data-path collective; the only collective is the max-over-ranks of the device ti
 
 `--impl reference` times the fp64 CPU oracle (as it stands) on the host cores instead.
 `--report` additionally writes a per-configuration table (all five workload configurations) to
-gpurun_out/bench_report.json.
+bench_report.json under $CF_REPORT_DIR (default: ./bench_out).
 """
 from __future__ import annotations
 
@@ -37,8 +37,8 @@ UNIT = "query-tokens/s"
 WORKLOAD = ("configs[2] chat-like mixed batch: 48 decode seqs (lognormal ctx, median 4096, sigma 0.8, clip [128,16384]) "
             "+ 2 prefills of 2048 new tokens over 6144 cached, 512-token chunks; Hq 32, Hkv 8, D 128, block 16, bf16; "
             "one step = kv_append + mixed attention of one chunk iteration (t cycles 0..3)")
-# DRAM traffic per algorithmic byte of the split-K decode kernel, from the ncu capture summarised in
-# profiles/decode_splitk_decode_small.md (560.9 MB moved for 555.2 MB algorithmic); traffic grows in
+# DRAM traffic per algorithmic byte of the split-K decode kernel, from an ncu capture on the reduced
+# decode case (dram bytes read + written: 560.9 MB for 555.2 MB algorithmic); traffic grows in
 # proportion to the K/V bytes, so a full launch is scaled by its algorithmic bytes.
 DECODE_TRAFFIC_RATIO = 1.010
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
@@ -412,8 +412,9 @@ def write_report(torch, cf, ctx, stream, peaks):
         rows.append({"config": name, "ms_per_step": ms / steps, "query_tokens_per_s": toks / (ms * 1e-3), **kern})
         del wl
         torch.cuda.empty_cache()
-    os.makedirs(os.path.join(ROOT, "gpurun_out"), exist_ok=True)
-    with open(os.path.join(ROOT, "gpurun_out", "bench_report.json"), "w") as f:
+    out_dir = os.environ.get("CF_REPORT_DIR", os.path.join(ROOT, "bench_out"))
+    os.makedirs(out_dir, exist_ok=True)
+    with open(os.path.join(out_dir, "bench_report.json"), "w") as f:
         json.dump({"peaks": peaks, "rows": rows}, f, indent=1)
     for r in rows:
         d, p = r.get("decode"), r.get("prefill")

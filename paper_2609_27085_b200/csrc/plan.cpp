@@ -255,7 +255,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
                      int32_t num_sms)
 {
-    // Constants fitted on B200 (see the measured table in the design notes): split-K decode sustains
+    // Constants fitted to CUDA-event times of the kernels on a B200: split-K decode sustains
     // ~7.1 TB/s on top of ~17 us of launch, ramp and tail; the combine launch is ~10 us; one tcgen05
     // prefill item costs ~8 us plus ~1.9 us per 128-token KV tile; the mma.sync path runs ~220 TFLOP/s.
     constexpr double kDecodeFixedUs = 17.0, kDecodeBytesPerUs = 7.1e6, kCombineUs = 10.0;
