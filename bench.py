@@ -396,7 +396,7 @@ def write_report(torch, cf, ctx, stream, peaks):
     """Per-configuration table over the workload configurations (device times only)."""
     rows = []
     scenarios = [("cfg2_decode", lambda: syn.config2_decode_only()), ("cfg3_chat", lambda: syn.config3_chat()),
-                 ("cfg4_agentic", lambda: syn.config4_agentic())]
+                 ("cfg3_tp4_shard", lambda: syn.config3_chat_tp4_shard()), ("cfg4_agentic", lambda: syn.config4_agentic())]
     scenarios += [(f"cfg5_b{b}_n{n}", (lambda b=b, n=n: syn.config5_sweep_point(b, n))) for b, n in
                   [(0, 0), (512, 4), (2048, 1), (8192, 1), (8192, 4)]]
     for name, make in scenarios:

@@ -249,6 +249,17 @@ def config3_chat(k: int = 0, iterations: Sequence[int] = (0, 1, 2, 3)) -> Scenar
     return sc
 
 
+def config3_chat_tp4_shard(k: int = 0, iterations: Sequence[int] = (0, 1, 2, 3)) -> Scenario:
+    """One tensor-parallel rank's share of the chat-like batch under the paper's TP4 deployment
+    (Section 6.1): the same sequences, a quarter of the heads (8 query heads, 2 KV heads)."""
+    lc = config3_lengths(k)
+    n_it = max(iterations) + 1
+    prefix = [6144, 6144] + list(lc - 1)
+    qlen = [[512, 512] + [1] * 48 for _ in range(n_it)]
+    geom = Geometry(num_q_heads=8, num_kv_heads=2, head_dim=128, block_size=16, num_blocks=65536)
+    return scenario_from_lengths("cfg3_chat_tp4", geom, _seed(3, k) + 40, prefix, qlen)
+
+
 def config4_lengths(k: int = 0) -> np.ndarray:
     rng = np.random.default_rng(_seed(4, k) + 500)
     return uniform_int(rng, 16, 8192, 32768)

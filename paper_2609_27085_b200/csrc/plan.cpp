@@ -2,6 +2,8 @@
 
 #include <algorithm>
 #include <climits>
+#include <cmath>
+#include <functional>
 #include <cstdint>
 
 namespace cf {
@@ -149,11 +151,11 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             }
         }
         // Few items (short chunks, few heads per GPU under tensor parallelism): a CTA's time is set by the
-        // per-tile softmax -> MMA chain, not by how many q tiles it carries, so pairs are split into
-        // single-tile items while that still leaves SMs idle.  Sharing K/V tiles matters only when the
-        // machine is full.
+        // per-tile softmax -> MMA chain, not by how many q tiles it carries, so single-tile items are an
+        // alternative while pairs would leave SMs idle (sharing K/V tiles matters only when the machine is
+        // full).  Whether pairs or singles are used is decided below, together with the KV split.
+        std::vector<KeyedTc> singles;
         if (items.size() * 2 <= (size_t)std::max(1, cfg.num_sms)) {
-            std::vector<KeyedTc> singles;
             singles.reserve(items.size() * 2);
             for (const KeyedTc& k : items)
                 for (int t = 0; t < 2; ++t) {
@@ -164,41 +166,97 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     one.q_row0[1] = 0; one.row0[1] = 0; one.n_rows[1] = 0; one.head[1] = k.it.head[t];
                     singles.push_back(KeyedTc{(int64_t)prefix_of(k.it.seq) + one.row0[0] + one.n_rows[0], one});
                 }
-            items.swap(singles);
+            std::stable_sort(singles.begin(), singles.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
         }
         std::stable_sort(items.begin(), items.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
-        // ---- KV split of the last, incomplete wave.  Items run one per SM; after the full waves the
-        // remaining r items would occupy r SMs for a whole item time.  Cutting each of them into k KV
-        // ranges lets them fill the machine; the ranges write fp32 partials that a combine pass merges.
-        // k minimises (rounds x range time) + partial traffic + the extra launch, by the same constants as
-        // the cost model; a range never starts inside the diagonal band and has at least 4 tiles.
+        // ---- KV split.  Items run one per SM, so a long item or an incomplete last wave leaves SMs idle.
+        // An item may be cut into k <= 8 KV ranges that write fp32 partials, merged by a combine pass; k
+        // comes from the cost model's constants; a range never starts inside the diagonal band and has at
+        // least 4 tiles.
         const size_t M = (size_t)std::max(1, cfg.num_sms);
-        const size_t n_items = items.size();
-        const size_t r = n_items % M, first_tail = n_items - r;
-        int32_t k_best = 1;
+        // decides the KV ranges per item for one candidate item list; returns the predicted time (us)
+        auto decide = [&](const std::vector<KeyedTc>& its, const double tile_us, std::vector<int32_t>& k_of) -> double {
+        const size_t n_items = its.size();
+        k_of.assign(n_items, 1);
+        double predicted = 0.0;
+        auto tiles_of = [&](size_t i) { return (double)((its[i].extent + 127) / 128); };
+        // a whole item costs ~8 us + 1.9 us per tile; a KV range pays ~13 us (fp32 partial epilogue);
+        // splitting adds the combine launch and the partial write/read
+        auto split_extra = [](size_t n_ranges) { return 8.0 + 0.05 * (double)n_ranges; };
         if (cfg.prefill_force_split >= 2) {
-            k_best = std::min(cfg.prefill_force_split, 8);
-        } else if (cfg.prefill_force_split == 1) {
-            k_best = 1;                                   // splitting switched off
-        } else if (r > 0) {
+            std::fill(k_of.begin(), k_of.end(), std::min(cfg.prefill_force_split, 8));
+        } else if (cfg.prefill_force_split == 1 || n_items == 0) {
+            // splitting switched off / nothing to do
+        } else if (n_items <= M) {
+            // One wave of unequal items (a few prompts with different prefixes): the longest item sets the
+            // time.  Try a few target times T; an item is cut into ceil(time / T) ranges; the candidate
+            // whose list-scheduled makespan (plus the split overhead) is smallest wins.
+            double total = 0.0, longest = 0.0;
+            for (size_t i = 0; i < n_items; ++i) {
+                total += tile_us * tiles_of(i);
+                longest = std::max(longest, tile_us * tiles_of(i));
+            }
+            double best = 8.0 + longest;                  // no split
+            predicted = best;
+            std::vector<int32_t> cand(n_items);
+            std::vector<double> load(M);
+            for (double f : {1.0, 1.2, 1.5, 2.0, 3.0}) {
+                const double T = std::max(f * total / (double)M, 8.0);
+                size_t n_ranges = 0;
+                bool any = false;
+                std::vector<double> jobs;
+                for (size_t i = 0; i < n_items; ++i) {
+                    const double tl = tiles_of(i);
+                    int32_t k = (int32_t)std::min(8.0, std::ceil(tile_us * tl / T));
+                    k = std::max(1, std::min(k, (int32_t)(tl / 4.0)));
+                    cand[i] = k;
+                    any = any || k > 1;
+                    n_ranges += (size_t)k;
+                    for (int32_t c = 0; c < k; ++c) jobs.push_back((k > 1 ? 13.0 : 8.0) + tile_us * tl / k);
+                }
+                if (!any) continue;
+                std::sort(jobs.begin(), jobs.end(), std::greater<double>());
+                std::fill(load.begin(), load.end(), 0.0);
+                for (double j : jobs) *std::min_element(load.begin(), load.end()) += j;
+                const double t = *std::max_element(load.begin(), load.end()) + split_extra(n_ranges);
+                if (t < best * 0.95) { best = t; k_of = cand; predicted = t; }
+            }
+        } else if (n_items % M != 0) {
+            // Several waves of similar items: after the full waves the remaining r items would hold r SMs
+            // for a whole item time; cutting each into k ranges lets them fill the machine.
+            const size_t r = n_items % M, first_tail = n_items - r;
             double tiles = 0.0;
-            for (size_t i = first_tail; i < n_items; ++i) tiles += (double)((items[i].extent + 127) / 128);
+            for (size_t i = first_tail; i < n_items; ++i) tiles += tiles_of(i);
             tiles /= (double)r;
             double best = 1e30;
+            int32_t k_best = 1;
             for (int32_t k = 1; k <= 8; ++k) {
                 if (k > 1 && tiles / k < 4.0) break;
                 const double rounds = (double)((r * (size_t)k + M - 1) / M);
-                // a whole item costs ~8 us + 1.9 us per tile; a KV range pays ~13 us (fp32 partial epilogue)
-                double t = rounds * ((k > 1 ? 13.0 : 8.0) + 1.9 * tiles / k);
-                if (k > 1) t += 8.0 + 0.05 * (double)(r * (size_t)k);     // combine launch + partial write/read
+                double t = rounds * ((k > 1 ? 13.0 : 8.0) + tile_us * tiles / k);
+                if (k > 1) t += split_extra(r * (size_t)k);
                 if (t < best * 0.97) { best = t; k_best = k; }             // split only for a clear gain
             }
+            for (size_t i = first_tail; i < n_items; ++i) k_of[i] = k_best;
         }
-        plan->prefill_tc.reserve(items.size() + (k_best > 1 ? r * (size_t)(k_best - 1) : 0));
-        const size_t split_from = cfg.prefill_force_split >= 2 ? 0 : first_tail;
+        return predicted;
+        };
+        std::vector<int32_t> k_of;
+        double t_pairs = decide(items, 1.9, k_of);
+        if (!singles.empty() && cfg.prefill_force_split == 0) {
+            std::vector<int32_t> k_single;
+            const double t_single = decide(singles, 1.8, k_single);
+            if (t_single < t_pairs) {
+                items.swap(singles);
+                k_of.swap(k_single);
+                t_pairs = t_single;
+            }
+        }
+        const size_t n_items = items.size();
         for (size_t i = 0; i < n_items; ++i) {
             PrefillTcItem it = items[i].it;
-            if (k_best <= 1 || i < split_from) {
+            const int32_t k_want = k_of[i];
+            if (k_want <= 1) {
                 plan->prefill_tc.push_back(it);
                 continue;
             }
@@ -210,7 +268,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     n_min = std::min(n_min, (prefix + it.row0[t] + it.n_rows[t] + 127) / 128);
                     safe = std::min(safe, (prefix + it.row0[t]) / 128);
                 }
-            const int32_t k = std::min(k_best, std::max(1, std::min(n_min, safe + 1) / 4));
+            const int32_t k = std::min(k_want, std::max(1, std::min(n_min, safe + 1) / 4));
             if (k <= 1) {
                 plan->prefill_tc.push_back(it);
                 continue;

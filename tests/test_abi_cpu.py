@@ -177,3 +177,17 @@ def test_kv_split_of_the_last_prefill_wave():
                                       np.array([512, 512], np.int32).ctypes.data, 2, 4096, 148, None, None, None, 0,
                                       counts.ctypes.data)
     assert counts[5] == 0 and counts[4] == 128
+
+
+def test_few_items_are_cut_into_kv_ranges():
+    """A 512-token chunk over an 8K prefix on one TP4 rank (16 query heads, 2 KV heads) is only 32 tile
+    pairs for 148 SMs: the planner cuts them into KV ranges until the machine is about full."""
+    import ctypes
+    d = cf.make_desc(16, 2, 128, 16, 65536)
+    lc, lq = np.array([8192 + 512], np.int32), np.array([512], np.int32)
+    counts = np.zeros(6, dtype=np.int32)
+    cf.load_library().cf_plan_inspect(ctypes.byref(d), lc.ctypes.data, lq.ctypes.data, 1, 8192, 148, None, None, None, 0,
+                                      counts.ctypes.data)
+    assert counts[5] > 0 and 96 <= counts[4] <= 148
+    _, _, whole = cf.cf_estimate_us(d, lc, lq, 8192, num_sms=148)
+    assert whole < 0.6 * (8 + 1.9 * 68)                 # well under the time of one unsplit item
