@@ -4,9 +4,27 @@
 #include <climits>
 #include <cmath>
 #include <functional>
+#include <queue>
 #include <cstdint>
 
 namespace cf {
+
+// Makespan of jobs taken in the given order by whichever of m machines is free first (what the GPU's
+// block scheduler does with a grid of one-CTA-per-SM work items).
+static double list_schedule(const std::vector<double>& jobs, size_t m)
+{
+    if (jobs.size() <= m) return jobs.empty() ? 0.0 : *std::max_element(jobs.begin(), jobs.end());
+    std::priority_queue<double, std::vector<double>, std::greater<double>> free_at;
+    for (size_t i = 0; i < m; ++i) free_at.push(0.0);
+    double end = 0.0;
+    for (double j : jobs) {
+        const double t = free_at.top() + j;
+        free_at.pop();
+        free_at.push(t);
+        end = std::max(end, t);
+    }
+    return end;
+}
 
 cf_status validate_desc(const cf_cache_desc* d)
 {
@@ -199,7 +217,6 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             double best = 8.0 + longest;                  // no split
             predicted = best;
             std::vector<int32_t> cand(n_items);
-            std::vector<double> load(M);
             for (double f : {1.0, 1.2, 1.5, 2.0, 3.0}) {
                 const double T = std::max(f * total / (double)M, 8.0);
                 size_t n_ranges = 0;
@@ -216,9 +233,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 }
                 if (!any) continue;
                 std::sort(jobs.begin(), jobs.end(), std::greater<double>());
-                std::fill(load.begin(), load.end(), 0.0);
-                for (double j : jobs) *std::min_element(load.begin(), load.end()) += j;
-                const double t = *std::max_element(load.begin(), load.end()) + split_extra(n_ranges);
+                const double t = list_schedule(jobs, M) + split_extra(n_ranges);
                 if (t < best * 0.95) { best = t; k_of = cand; predicted = t; }
             }
         } else if (n_items % M != 0) {
@@ -328,7 +343,8 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
     if (!plan.combine.empty()) e.us_combine = (float)kCombineUs;
     if (!plan.prefill_tc.empty()) {
         // items are already longest-first: greedy list scheduling onto num_sms machines
-        std::vector<double> load((size_t)std::max(1, num_sms), 0.0);
+        std::vector<double> jobs;
+        jobs.reserve(plan.prefill_tc.size());
         for (const PrefillTcItem& it : plan.prefill_tc) {
             const int32_t prefix = context_len[it.seq] - query_len[it.seq];
             int32_t hi = 0;
@@ -336,9 +352,9 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
                 if (it.n_rows[t] > 0) hi = std::max(hi, prefix + it.row0[t] + it.n_rows[t]);
             const int32_t tiles = std::max(0, std::min((hi + 127) / 128, it.j_end) - it.j_begin);
             const double cost = kTcItemFixedUs + kTcTileUs * tiles;
-            *std::min_element(load.begin(), load.end()) += cost;
+            jobs.push_back(cost);
         }
-        e.us_prefill = (float)(kLaunchUs + *std::max_element(load.begin(), load.end()));
+        e.us_prefill = (float)(kLaunchUs + list_schedule(jobs, (size_t)std::max(1, num_sms)));
         if (!plan.prefill_combine.empty()) e.us_prefill += (float)(6.0 + 0.05 * (double)plan.prefill_tc.size());
     } else if (!plan.prefill.empty()) {
         double flops = 0.0;
