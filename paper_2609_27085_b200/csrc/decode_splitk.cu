@@ -35,6 +35,9 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
     const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
     const DecodeItem it = p.dec_items[item_id];
     const int G = p.G;
+    // lets the combine kernel (launched with programmatic stream serialisation) become resident while
+    // this grid drains; it still waits for this grid's completion before it reads a partial
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
 
     // ---- Q^T fragments (B operand): thread holds Q[head = lane/4][d = 16*ks + 2*(lane%4) + {0,1} (+8)]
     uint32_t qf[KSTEPS][2];
@@ -222,6 +225,7 @@ __global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
 {
     const CombineItem it = p.comb_items[blockIdx.x];
     const int hq = blockIdx.y;
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the decode grid has completed and its partials are visible
     const int d = threadIdx.x * 4;
     // Partials are fetched eight chunks at a time with independent loads (a dependent load per chunk
     // would cost a memory round trip each) and folded into a running (M, L, acc) in chunk order.
@@ -303,9 +307,19 @@ cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaS
 {
     if (n_items <= 0) return cudaSuccess;
     dim3 grid(n_items, p.Hq);
-    if (head_dim == 128) combine_kernel<128><<<grid, 32, 0, stream>>>(p);
-    else combine_kernel<64><<<grid, 16, 0, stream>>>(p);
-    return cudaGetLastError();
+    // programmatic dependent launch: the grid may be scheduled while the decode kernel drains; every CTA
+    // executes griddepcontrol.wait before touching the partials
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(head_dim == 128 ? 32 : 16);
+    cfg.dynamicSmemBytes = 0;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return head_dim == 128 ? cudaLaunchKernelEx(&cfg, combine_kernel<128>, p) : cudaLaunchKernelEx(&cfg, combine_kernel<64>, p);
 }
 
 }  // namespace cf

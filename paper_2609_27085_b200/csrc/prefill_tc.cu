@@ -109,6 +109,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const PrefillTcItem it = p.pre_tc_items[blockIdx.x];
+    // lets a following prefill_combine grid become resident while this grid drains (it waits for this
+    // grid's completion before reading a partial)
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const int Lq = __ldg(p.query_len + it.seq), Lc = __ldg(p.context_len + it.seq);
     const int prefix = Lc - Lq;
     int kv_hi_t[2], n_j[2];
@@ -145,6 +148,10 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem = tmem_base_s;
+    // Launched with programmatic stream serialisation: everything above overlaps the tail of the kernel
+    // before this one in the stream; from here on that kernel has completed and its writes are visible
+    // (the K/V rows of cf_kv_append when the batch has no decode part).
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 
     const bool live_cta = abort_s == 0;       // otherwise nothing is issued: fall through to the teardown
     if (warp < 4) {
@@ -480,6 +487,7 @@ constexpr int kMaxSplit = 8;
 __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p)
 {
     const PrefillCombineItem it = p.pre_comb_items[blockIdx.x >> 5];
+    asm volatile("griddepcontrol.wait;" ::: "memory");     // the prefill grid has completed and its partials are visible
     const int lane = threadIdx.x & 31;
     const int rb = blockIdx.x & 31;                  // 32 blocks of 8 rows = 2 tiles x 128 rows
     const int t = rb >> 4, r = (rb & 15) * 8 + (threadIdx.x >> 5);
@@ -519,8 +527,16 @@ __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p
 cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream)
 {
     if (n_items <= 0) return cudaSuccess;
-    prefill_combine_kernel<<<n_items * 32, 256, 0, stream>>>(p);
-    return cudaGetLastError();
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_items * 32);
+    cfg.blockDim = dim3(256);
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_combine_kernel, p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -625,8 +641,19 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
-    prefill_tc_kernel<<<n_items, NTHREADS, smem, stream>>>(mq, mk, mv, p);
-    return cudaGetLastError();
+    // Programmatic dependent launch: barrier set-up and tensor-memory allocation run while the kernel
+    // before this one in the stream drains; the kernel waits (griddepcontrol.wait) before its first read.
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = dim3(n_items);
+    cfg.blockDim = dim3(NTHREADS);
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p);
 }
 
 }  // namespace cf
