@@ -143,13 +143,16 @@ cf_status cf_get_async_status(cf_ctx* ctx);
 
 /* Section 5 names two executor backends: the chunked mixed-batch path (time-multiplexed, the default
  * here: one launch sequence on the caller's stream) and a spatial partition of the node between prefill
- * and decode.  cf_set_overlap(ctx, 1) selects a spatial variant for later cf_mixed_attention calls that
- * hold both kinds of work: the prefill kernel is enqueued first on a context-owned side stream and the
- * decode + combine kernels on the caller's stream, so that decode (memory-bound) fills the SMs the
- * prefill CTAs leave free; the side stream is joined back before the call returns, so the caller still
- * sees one stream.  Results are bit-identical to the default.  The environment variable CF_OVERLAP=1
- * sets the initial value.  Per-kernel timing (cf_set_timing) forces the serial sequence. */
-cf_status cf_set_overlap(cf_ctx* ctx, int enabled);
+ * and decode.  cf_set_overlap(ctx, n) with n > 0 selects the spatial variant for later cf_mixed_attention
+ * calls that hold both kinds of work: n persistent prefill CTAs (one per SM; n = 1 means the library's
+ * default share of the SMs) are enqueued first on a context-owned side stream; the caller's stream waits,
+ * with a stream memory operation, until they hold their SMs, then runs decode + combine on the SMs left
+ * over, and behind them a second prefill grid that draws from the same work queue, so the SMs decode
+ * frees join the prefill.  The side stream is joined back before the call returns, so the caller still
+ * sees one stream.  Results are bit-identical to the default.  n = 0 switches back.  The environment
+ * variables CF_OVERLAP=1 and CF_SPATIAL_SMS=n set the initial values.  Per-kernel timing (cf_set_timing)
+ * forces the serial sequence. */
+cf_status cf_set_overlap(cf_ctx* ctx, int n);
 
 /* Debug aid (synchronous): checks every block-table entry that cf_kv_append / cf_mixed_attention would
  * dereference for these lengths (entries [0, ceil(context_len/B)) of each row) against [0, num_blocks).

@@ -194,9 +194,10 @@ def cf_selftest_bounded_wait(ctx, stream=None) -> None:
     _check(load_library().cf_selftest_bounded_wait(ctx, _stream(stream)), "cf_selftest_bounded_wait")
 
 
-def cf_set_overlap(ctx, enabled: bool) -> None:
-    """Run the prefill kernel beside decode + combine (side stream, joined before return)."""
-    _check(load_library().cf_set_overlap(ctx, int(bool(enabled))), "cf_set_overlap")
+def cf_set_overlap(ctx, n) -> None:
+    """Spatial launch sequence: n > 0 persistent prefill CTAs take their SMs first (1 or True = the
+    library's default share), decode + combine run beside them; 0 = the serial sequence."""
+    _check(load_library().cf_set_overlap(ctx, int(n)), "cf_set_overlap")
 
 
 def cf_set_timing(ctx, enabled: bool) -> None:

@@ -1,5 +1,7 @@
 // C ABI of the library: context, plan upload and the launch sequence.
 // See include/crossflow_attn.h for the contract of every entry point.
+#include <cuda.h>
+
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -55,6 +57,7 @@ struct cf_ctx {
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = false;
+    int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // host-staged step
@@ -78,7 +81,7 @@ struct cf_plan {
     uint8_t* dev = nullptr;
     float* part = nullptr;         // this plan's own split-K partials
     int n_part_slots = 0, n_pre_slots = 0;
-    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, off_pre_comb = 0, total = 0;
+    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
 };
 
@@ -144,7 +147,7 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, off_pre_comb, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, off_pre_comb, off_queue, total;
 };
 
 static PlanLayout layout_of(int32_t S, const Plan& pl)
@@ -159,7 +162,8 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_pre = at;    at = align_up(at + sizeof(PrefillItem) * pl.prefill.size(), 16);
     L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
     L.off_pre_comb = at; at = align_up(at + sizeof(PrefillCombineItem) * pl.prefill_combine.size(), 16);
-    L.total = at ? at : 16;
+    L.off_queue = at;  at += 16;   // ticket counter + exit counter of the persistent prefill CTAs; uploaded as zeros
+    L.total = at;
     return L;
 }
 
@@ -185,6 +189,7 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
         std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
     if (!pl.prefill_combine.empty())
         std::memcpy(s.host + L->off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
+    std::memset(s.host + L->off_queue, 0, 16);
     if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
     *dev_base = s.dev;
     *slot_out = &s;
@@ -196,6 +201,31 @@ static cf_status finish_slot(PlanSlot* s, cudaStream_t stream)
     if (cudaEventRecord(s->done, stream) != cudaSuccess) return CF_ERR_CUDA;
     s->used = true;
     return CF_OK;
+}
+
+// Stream memory operations of the driver API (the runtime has no counterpart), looked up once.
+struct StreamMemOps {
+    typedef CUresult (*Fn)(CUstream, CUdeviceptr, cuuint32_t, unsigned int);
+    Fn wait = nullptr, write = nullptr;
+    bool ok = false;
+};
+static const StreamMemOps& stream_mem_ops()
+{
+    static StreamMemOps ops;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void *w = nullptr, *r = nullptr;
+        cudaDriverEntryPointQueryResult q1, q2;
+        if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &w, cudaEnableDefault, &q1) == cudaSuccess &&
+            cudaGetDriverEntryPoint("cuStreamWriteValue32", &r, cudaEnableDefault, &q2) == cudaSuccess &&
+            q1 == cudaDriverEntryPointSuccess && q2 == cudaDriverEntryPointSuccess && w && r) {
+            ops.wait = reinterpret_cast<StreamMemOps::Fn>(w);
+            ops.write = reinterpret_cast<StreamMemOps::Fn>(r);
+            ops.ok = true;
+        }
+    }
+    return ops;
 }
 
 static float scale_log2_of(const cf_cache_desc* d)
@@ -259,6 +289,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.pre_part_o = (float*)((uint8_t*)ws + W.pre_o);
     p.pre_part_ml = (float*)((uint8_t*)ws + W.pre_ml);
     p.pre_comb_items = (const PrefillCombineItem*)(base + L.off_pre_comb);
+    p.pre_queue = (uint32_t*)(base + L.off_queue);
     p.err = c->err_dev;
 
     cudaError_t e = cudaSuccess;
@@ -277,18 +308,45 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         tc->ran[2] = (n.n_pre > 0) || (n.n_pre_tc > 0);
     }
     const bool has_prefill = (n.n_pre > 0) || (n.n_pre_tc > 0);
+    int second_grid = 0;
+    const int sms = c->num_sms > 0 ? c->num_sms : 148;
+    const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
     if (c->overlap && !tc && has_prefill && (n.n_dec > 0)) {
-        // prefill on the side stream, launched first so that its CTAs take their SMs; decode + combine
-        // on the caller's stream fill the rest of the machine; joined before returning to the caller
+        // Spatial partition.  `front` persistent prefill CTAs (one per SM: a CTA takes an SM's whole shared
+        // memory) go first, on the side stream; decode + combine on the caller's stream run on the SMs left
+        // over; a second prefill grid behind them on the caller's stream draws from the same ticket counter,
+        // so the SMs that decode frees join the prefill as soon as decode is done.
+        int front = c->spatial_sms > 0 ? c->spatial_sms : (sms * 3) / 5;
+        if (front > sms) front = sms;
+        if (front > n.n_pre_tc) front = n.n_pre_tc;
+        int tail = n.n_pre_tc - front;
+        if (tail > sms) tail = sms;
+        second_grid = tail > 0;
+        // Decode must not start before the front CTAs hold their SMs (its grid would otherwise fill the
+        // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end):
+        // the front CTAs count themselves in, and the caller's stream waits for that count with a stream
+        // memory operation.  Not used while the stream is being captured.
+        uint32_t* resident = nullptr;
+        const StreamMemOps& mo = stream_mem_ops();
+        cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+        if (front > 0 && mo.ok && cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+            resident = p.pre_queue + 2;
+            if (mo.write(stream, (CUdeviceptr)(uintptr_t)resident, 0u, 0u) != CUDA_SUCCESS) e = cudaErrorUnknown;
+        }
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, c->side);
-        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, resident, c->side);
         if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
+        // only after the front grid has been enqueued without an error, so that the count is certain to arrive
+        if (e == cudaSuccess && resident &&
+            mo.wait(stream, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+            e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
         if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, nullptr, stream);
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
     } else {
         if (tc) cudaEventRecord(tc->ev[0], stream);
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
@@ -296,11 +354,11 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0);
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -350,6 +408,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
     c->overlap = env_int("CF_OVERLAP", 0) != 0;
+    c->spatial_sms = env_int("CF_SPATIAL_SMS", 0);
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
@@ -512,7 +571,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->max_blocks = max_blocks_per_seq;
     const PlanLayout L = layout_of(num_seqs, pl);
     P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
-    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb;
+    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
     P->total = L.total;
     P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size(); P->n_pre = (int)pl.prefill.size();
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
@@ -532,6 +591,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
         if (P->n_pre_tc) std::memcpy(P->host + L.off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
         if (P->n_pre_comb)
             std::memcpy(P->host + L.off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
+        std::memset(P->host + L.off_queue, 0, 16);
         ok = cudaMemcpyAsync(P->dev, P->host, L.total, cudaMemcpyHostToDevice, (cudaStream_t)cuda_stream) == cudaSuccess;
     }
     if (!ok) {
@@ -590,7 +650,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     if (!guard.ok) return CF_ERR_CUDA;
     PlanLayout L;
     L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
-    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb;
+    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
     L.total = P->total;
     PlanCounts n;
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
@@ -726,7 +786,9 @@ cf_status cf_validate_block_table(cf_ctx* c, const cf_cache_desc* desc, const in
 cf_status cf_set_overlap(cf_ctx* c, int enabled)
 {
     if (!c) return CF_ERR_INVALID_ARG;
+    if (enabled < 0) return CF_ERR_INVALID_ARG;
     c->overlap = enabled != 0;
+    if (enabled > 1) c->spatial_sms = enabled;
     return CF_OK;
 }
 

@@ -32,6 +32,7 @@ struct AttnParams {
     float* pre_part_o;                // [row slot, D] fp32 partial rows of KV-split prefill items
     float* pre_part_ml;               // [row slot, 2]
     const PrefillCombineItem* pre_comb_items;
+    uint32_t* pre_queue;              // [2] ticket counter of the persistent prefill CTAs, and how many of them have left
     uint32_t* err;                    // device error word
 };
 

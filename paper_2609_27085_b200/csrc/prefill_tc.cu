@@ -56,6 +56,7 @@ struct Bars {
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
     uint64_t s_full[2], p_full[2], o_done[2];
+    uint64_t mma_done;        // the issuer's last commit of an item: all of its MMAs have completed
 };
 
 __device__ __forceinline__ uint32_t lane_field(int warp) { return (uint32_t)((warp & 3) * 32) << 16; }
@@ -97,51 +98,58 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 
 }  // namespace
 
+// What a role needs to know about the work item it is on.
+struct ItemCtx {
+    PrefillTcItem it;
+    int Lc, prefix;
+    int kv_hi_t[2], n_j[2];   // per q tile: end of its visible keys; number of KV tiles of [j_begin, j_end) it takes part in
+    int n_max, total_pages, jb;
+};
+__device__ __forceinline__ ItemCtx load_item(const AttnParams& p, int idx)
+{
+    ItemCtx c;
+    c.it = p.pre_tc_items[idx];
+    const int Lq = __ldg(p.query_len + c.it.seq);
+    c.Lc = __ldg(p.context_len + c.it.seq);
+    c.prefix = c.Lc - Lq;
+#pragma unroll
+    for (int t = 0; t < 2; ++t) {
+        c.kv_hi_t[t] = c.it.n_rows[t] > 0 ? c.prefix + c.it.row0[t] + c.it.n_rows[t] : 0;
+        c.n_j[t] = max(0, min((c.kv_hi_t[t] + KT - 1) / KT, c.it.j_end) - c.it.j_begin);
+    }
+    c.n_max = max(c.n_j[0], c.n_j[1]);
+    c.total_pages = (max(c.kv_hi_t[0], c.kv_hi_t[1]) + 15) >> 4;
+    c.jb = c.it.j_begin;       // loop indices are relative to it; jb + j is the absolute tile
+    return c;
+}
+
+// Persistent CTAs: every CTA of the launch sequence draws work items (longest first) from one ticket
+// counter in global memory, p.pre_queue[0], until the tickets run out.  `queue_ctas` is the number of CTAs
+// that draw from the counter (over all grids that share it); the last of them to leave puts the two
+// counter words back to zero, so that a replay of the same launches needs no host-side reset.
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
-                  const __grid_constant__ CUtensorMap map_v, const AttnParams p)
+                  const __grid_constant__ CUtensorMap map_v, const AttnParams p, const int n_items, const int queue_ctas,
+                  uint32_t* const resident)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(8) Bars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ uint32_t abort_s;
+    __shared__ int item_s;
 
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const PrefillTcItem it = p.pre_tc_items[blockIdx.x];
-    // lets a following prefill_combine grid become resident while this grid drains (it waits for this
-    // grid's completion before reading a partial)
+    // lets the next grid of the stream become resident while this grid drains (it waits for this grid's
+    // completion before it reads anything this grid wrote)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
-    const int Lq = __ldg(p.query_len + it.seq), Lc = __ldg(p.context_len + it.seq);
-    const int prefix = Lc - Lq;
-    int kv_hi_t[2], n_j[2];
-#pragma unroll
-    for (int t = 0; t < 2; ++t) {
-        kv_hi_t[t] = it.n_rows[t] > 0 ? prefix + it.row0[t] + it.n_rows[t] : 0;
-        // number of KV tiles of this item's range [j_begin, j_end) that tile t takes part in
-        n_j[t] = max(0, min((kv_hi_t[t] + KT - 1) / KT, it.j_end) - it.j_begin);
-    }
-    const int kv_hi = max(kv_hi_t[0], kv_hi_t[1]);
-    const int n_max = max(n_j[0], n_j[1]);
-    const int total_pages = (kv_hi + 15) >> 4;
-    const int jb = it.j_begin;                // loop indices below are relative to it; jb + j is the absolute tile
     volatile uint32_t* abort_flag = &abort_s;
 
     if (threadIdx.x == 0) {
         abort_s = (p.err != nullptr && *reinterpret_cast<volatile uint32_t*>(p.err) != 0u) ? 2u : 0u;   // an earlier CTA gave up
-        mbar_init(smem_u32(&bars.q_full), 1);
-        for (int s = 0; s < KV_STAGES; ++s) {
-            mbar_init(smem_u32(&bars.k_full[s]), 1);
-            mbar_init(smem_u32(&bars.k_empty[s]), 1);
-            mbar_init(smem_u32(&bars.v_full[s]), 1);
-            mbar_init(smem_u32(&bars.v_empty[s]), 1);
-        }
-        for (int t = 0; t < 2; ++t) {
-            mbar_init(smem_u32(&bars.s_full[t]), 1);
-            mbar_init(smem_u32(&bars.p_full[t]), 4);      // one arrival per softmax warp
-            mbar_init(smem_u32(&bars.o_done[t]), 1);
-        }
-        fence_mbar_init();
+        // spatial launch sequence: the stream that carries the decode kernel waits (a stream memory
+        // operation, not a kernel) until every CTA of this grid holds its SM
+        if (resident != nullptr) atomicAdd(resident, 1u);
     }
     if (warp == 0) tmem_alloc<512>(smem_u32(&tmem_base_s));
     tc_fence_before();
@@ -153,12 +161,57 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     // (the K/V rows of cf_kv_append when the batch has no decode part).
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    const bool live_cta = abort_s == 0;       // otherwise nothing is issued: fall through to the teardown
+    // Called by the ten working warps between items (named barrier 1; the two spare warps wait at the
+    // teardown barrier).  After the first barrier every role has left the previous item - its MMAs have
+    // completed, tensor memory has been read out - so thread 0 may draw a ticket and re-arm the barriers.
+    auto next_item = [&]() -> int {
+        __syncwarp();
+        tc_fence_before();
+        asm volatile("bar.sync 1, 320;" ::: "memory");
+        if (threadIdx.x == 0) {
+            int idx = n_items;
+            if (abort_s == 0u) idx = (int)atomicAdd(p.pre_queue, 1u);
+            if (idx < n_items) {
+                mbar_init(smem_u32(&bars.q_full), 1);
+                for (int s = 0; s < KV_STAGES; ++s) {
+                    mbar_init(smem_u32(&bars.k_full[s]), 1);
+                    mbar_init(smem_u32(&bars.k_empty[s]), 1);
+                    mbar_init(smem_u32(&bars.v_full[s]), 1);
+                    mbar_init(smem_u32(&bars.v_empty[s]), 1);
+                }
+                for (int t = 0; t < 2; ++t) {
+                    mbar_init(smem_u32(&bars.s_full[t]), 1);
+                    mbar_init(smem_u32(&bars.p_full[t]), 4);      // one arrival per softmax warp
+                    mbar_init(smem_u32(&bars.o_done[t]), 1);
+                }
+                mbar_init(smem_u32(&bars.mma_done), 1);
+                fence_mbar_init();
+            } else {
+                idx = n_items;
+                if (atomicAdd(p.pre_queue + 1, 1u) == (uint32_t)(queue_ctas - 1)) {   // every other CTA has drawn its last ticket
+                    p.pre_queue[0] = 0u;
+                    p.pre_queue[1] = 0u;
+                    __threadfence();
+                }
+            }
+            item_s = idx;
+        }
+        asm volatile("bar.sync 1, 320;" ::: "memory");
+        tc_fence_after();
+        return item_s;
+    };
+
     if (warp < 4) {
       reg_dec<REGS_ROLE>();
-      if (!live_cta || warp >= 2) {
+      if (warp >= 2) {
         // spare warps of the first warpgroup
       } else if (warp == 0) {
+       for (;;) {
+        const int item = next_item();
+        if (item >= n_items) break;
+        const ItemCtx cx = load_item(p, item);
+        const PrefillTcItem& it = cx.it;
+        const int n_max = cx.n_max, total_pages = cx.total_pages, jb = cx.jb;
         // =========================================================== TMA producer
         if (lane == 0) {
             prefetch_tensormap(&map_q);
@@ -197,7 +250,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane & 1) * 64, 0, it.kvh, my_pid,
                             smem_u32(&bars.v_full[stage]));
         }
-    } else if (warp == 1) {
+       }
+      } else {
         // =========================================================== MMA issuer
         constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
         constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, true);
@@ -247,11 +301,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // the critical resource of the kernel: it is a single dependent instruction stream that is also
         // blocked while its MMAs queue up, so the work between two batches is kept to a handful of
         // instructions, with a lean loop for interior tiles and the general step for the rest.
-        if (lane == 0) {
         const uint32_t bar_kf[2] = {smem_u32(&bars.k_full[0]), smem_u32(&bars.k_full[1])};
         const uint32_t bar_vf[2] = {smem_u32(&bars.v_full[0]), smem_u32(&bars.v_full[1])};
         const uint32_t bar_ke[2] = {smem_u32(&bars.k_empty[0]), smem_u32(&bars.k_empty[1])};
         const uint32_t bar_ve[2] = {smem_u32(&bars.v_empty[0]), smem_u32(&bars.v_empty[1])};
+       for (;;) {
+        const int item = next_item();
+        if (item >= n_items) break;
+        if (lane == 0) {
+        const ItemCtx cx = load_item(p, item);
+        const int Lc = cx.Lc, n_max = cx.n_max, total_pages = cx.total_pages, jb = cx.jb;
+        const int n_j[2] = {cx.n_j[0], cx.n_j[1]};
         bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
         ok = ok && mbar_wait(bar_kf[0], 0, abort_flag);
         if (ok) {
@@ -325,18 +385,31 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         };
         static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
         for (; j < n_max && ok; ++j) ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
+        // every MMA of the item has completed (and every commit above has arrived) before the barriers are re-armed
+        if (ok) {
+            umma_commit(smem_u32(&bars.mma_done));
+            mbar_wait(smem_u32(&bars.mma_done), 0, abort_flag);
         }
+        }
+       }
       }
     } else {
       reg_inc<REGS_SOFTMAX>();
-      if (live_cta) {
-        // =========================================================== softmax + epilogue, one thread per q row
-        const int t = (warp - 4) >> 2;
-        const int row = (warp & 3) * 32 + lane;
-        const uint32_t lanes = lane_field(warp);
-        const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
-        const int limit = min(prefix + it.row0[t] + row, kv_hi_t[t] - 1);   // last visible key of this row
-        const float sc = p.scale_log2;
+      // =========================================================== softmax + epilogue, one thread per q row
+      const int t = (warp - 4) >> 2;
+      const int row = (warp & 3) * 32 + lane;
+      const uint32_t lanes = lane_field(warp);
+      const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
+      const float sc = p.scale_log2;
+      for (;;) {
+        const int item = next_item();
+        if (item >= n_items) break;
+        {
+        const ItemCtx cx = load_item(p, item);
+        const PrefillTcItem& it = cx.it;
+        const int jb = cx.jb;
+        const int n_j[2] = {cx.n_j[0], cx.n_j[1]};
+        const int limit = min(cx.prefix + it.row0[t] + row, cx.kv_hi_t[t] - 1);   // last visible key of this row
         float m_used = -INFINITY, l_sum = 0.f;
         bool ok = true;
         for (int j = 0; j < n_j[t]; ++j) {
@@ -463,10 +536,11 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (live && partial) *reinterpret_cast<float2*>(p.pre_part_ml + pslot * 2) = make_float2(m_used, l_sum);
             else if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
         }
+        }
       }
     }
 
-    // ---- teardown: every role has left its loop (normally, or because the abort flag went up)
+    // ---- teardown: every role has left its loop (the tickets ran out, or the abort flag went up)
     tc_fence_before();
     __syncthreads();
     if (abort_s == 1u) {
@@ -618,9 +692,10 @@ bool prefill_tc_supported(const cf_cache_desc* d)
     return d->head_dim == D && d->block_size == 16;
 }
 
-cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, cudaStream_t stream)
+cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
+                              int queue_ctas, uint32_t* resident, cudaStream_t stream)
 {
-    if (n_items <= 0) return cudaSuccess;
+    if (n_items <= 0 || n_ctas <= 0) return cudaSuccess;
     CUtensorMap mq, mk, mv;
     if (!encode_q(&mq, p.q, total_q_rows, p.Hq) ||
         !encode_pool(&mk, p.k_cache, desc->num_blocks, p.Hkv, p.ks_block, p.ks_head, p.ks_token) ||
@@ -644,7 +719,7 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
     // Programmatic dependent launch: barrier set-up and tensor-memory allocation run while the kernel
     // before this one in the stream drains; the kernel waits (griddepcontrol.wait) before its first read.
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(n_items);
+    cfg.gridDim = dim3(n_ctas);
     cfg.blockDim = dim3(NTHREADS);
     cfg.dynamicSmemBytes = smem;
     cfg.stream = stream;
@@ -653,7 +728,7 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p);
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p, n_items, queue_ctas, resident);
 }
 
 }  // namespace cf

@@ -245,11 +245,14 @@ def test_overlap_mode_is_bit_identical_to_the_serial_sequence():
     g = GpuScenario(sc)
     g.append(b)
     serial, lse0 = g.attend(b)
-    cf.cf_set_overlap(g.ctx, True)
-    for _ in range(3):
+    # default share of the SMs; then 8 and 3 front CTAs, so that every CTA works through several items and
+    # the second grid (behind decode, same queue) takes part
+    for n in (1, 1, 8, 3, 8):
+        cf.cf_set_overlap(g.ctx, n)
         o, lse = g.attend(b)
         assert np.array_equal(o, serial) and np.array_equal(lse, lse0)
-    cf.cf_set_overlap(g.ctx, False)
+    cf.cf_set_overlap(g.ctx, 0)
+    assert cf.cf_get_async_status(g.ctx) == 0
     k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
     oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
     ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
