@@ -56,7 +56,8 @@ struct cf_ctx {
     uint32_t* err_dev = nullptr;
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
-    bool overlap = false;
+    bool overlap = true;
+    bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -83,6 +84,7 @@ struct cf_plan {
     int n_part_slots = 0, n_pre_slots = 0;
     size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    float pre_over_dec = 0.f;
 };
 
 namespace cf {
@@ -240,6 +242,7 @@ namespace cf {
 
 struct PlanCounts {
     int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
 };
 
 // Split-K workspace: decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact partial rows of
@@ -311,12 +314,15 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     int second_grid = 0;
     const int sms = c->num_sms > 0 ? c->num_sms : 148;
     const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
-    if (c->overlap && !tc && has_prefill && (n.n_dec > 0)) {
+    if (c->overlap && !c->in_host_step && !tc && has_prefill && (n.n_dec > 0)) {
         // Spatial partition.  `front` persistent prefill CTAs (one per SM: a CTA takes an SM's whole shared
         // memory) go first, on the side stream; decode + combine on the caller's stream run on the SMs left
         // over; a second prefill grid behind them on the caller's stream draws from the same ticket counter,
         // so the SMs that decode frees join the prefill as soon as decode is done.
-        int front = c->spatial_sms > 0 ? c->spatial_sms : (sms * 3) / 5;
+        // Default share: three fifths of the SMs.  When the prefill work dwarfs the decode kernel, sharing the
+        // machine no longer pays (the tensor-bound kernel already runs at the power limit): prefill takes
+        // every SM first and decode + combine fill in as its CTAs retire.
+        int front = c->spatial_sms > 0 ? c->spatial_sms : (n.pre_over_dec > 3.9f ? sms : (sms * 3) / 5);
         if (front > sms) front = sms;
         if (front > n.n_pre_tc) front = n.n_pre_tc;
         int tail = n.n_pre_tc - front;
@@ -407,7 +413,10 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
     c->cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
-    c->overlap = env_int("CF_OVERLAP", 0) != 0;
+    {
+        const char* v = std::getenv("CF_OVERLAP");          // spatial sequence unless CF_OVERLAP=0
+        c->overlap = !(v && v[0] == '0' && v[1] == 0);
+    }
     c->spatial_sms = env_int("CF_SPATIAL_SMS", 0);
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
@@ -543,6 +552,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     PlanCounts n;
     n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_pre = (int)pl.prefill.size();
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
+    n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
     const cf_status fs = finish_slot(slot, stream);
@@ -575,6 +585,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->total = L.total;
     P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size(); P->n_pre = (int)pl.prefill.size();
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
+    P->pre_over_dec = prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms);
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
     const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
@@ -655,6 +666,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     PlanCounts n;
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
     n.total_q = P->total_q;
+    n.pre_over_dec = P->pre_over_dec;
     const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim);
     return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, W, q, k_cache,
                             v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);
@@ -712,8 +724,12 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
     st = cf_kv_append(c, desc, k_cache, v_cache, dk, dv, block_table, max_blocks_per_seq, context_len, query_len,
                       num_seqs, cuda_stream);
     if (st != CF_OK) return st;
+    // The step is bound by the copies over PCIe, not by the kernels; measured on the chat-like workload the
+    // spatial sequence (side stream, stream memory operations) made it slower (0.49 ms against 0.41 ms).
+    c->in_host_step = true;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);
+    c->in_host_step = false;
     if (st != CF_OK) return st;
     if (cudaEventRecord(hs.compute_done, stream) != cudaSuccess) return CF_ERR_CUDA;
     // result: second copy stream

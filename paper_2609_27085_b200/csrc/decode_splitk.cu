@@ -62,6 +62,7 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
 
     int cache_base = 0;
     int32_t pid_cache = (lane < my_n) ? __ldg(bt + lane * NWARPS) : 0;
+    const uint64_t stream_once = l2_policy_evict_first();
 
     auto issue = [&](int i) {
         if (i - cache_base == 32) {             // refill the per-lane page-id cache
@@ -79,8 +80,8 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
             const int t = id / CPR, c = id % CPR;
             const bool ok = tok0 + t < it.kv_end;     // slack slots of the last page are zero-filled
             const int tt = ok ? t : 0;
-            cp_async16(sbase + tile_off<16>(t, c), kp + tt * p.ks_token + c * 8, ok ? 16 : 0);
-            cp_async16(sbase + PAGE_BYTES + tile_off<16>(t, c), vp + tt * p.vs_token + c * 8, ok ? 16 : 0);
+            cp_async16_hint(sbase + tile_off<16>(t, c), kp + tt * p.ks_token + c * 8, ok ? 16 : 0, stream_once);
+            cp_async16_hint(sbase + PAGE_BYTES + tile_off<16>(t, c), vp + tt * p.vs_token + c * 8, ok ? 16 : 0, stream_once);
         }
     };
 

@@ -138,7 +138,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     for (int32_t kvh = 0; kvh < d->num_kv_heads; ++kvh)
                         for (int32_t i = 0; i < G; i += 2) {
                             PrefillTcItem it;
-                            it.seq = s; it.kvh = kvh;
+                            it.seq = s; it.kvh = kvh; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
                             it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
                             for (int t = 0; t < 2; ++t) {
                                 it.q_row0[t] = plan->q_start[s] + tile * TR;
@@ -152,7 +152,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 for (int32_t tile = 0; tile < n_tiles; tile += 2)
                     for (int32_t h = 0; h < d->num_q_heads; ++h) {
                         PrefillTcItem it;
-                        it.seq = s; it.kvh = h;
+                        it.seq = s; it.kvh = h; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
                         it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
                         int32_t last = tile;
                         for (int t = 0; t < 2; ++t) {
@@ -323,6 +323,24 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     plan->prefill.reserve(tiles.size());
     for (const Keyed& k : tiles) plan->prefill.push_back(k.it);
     return CF_OK;
+}
+
+float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
+                              int32_t num_sms)
+{
+    if (plan.decode.empty() || plan.prefill_tc.empty()) return 0.f;
+    const int32_t S = (int32_t)plan.q_start.size() - 1;
+    double dec_bytes = 0.0;
+    for (int32_t s = 0; s < S; ++s)
+        if (query_len[s] == 1) dec_bytes += (double)context_len[s] * 2.0 * d->num_kv_heads * d->head_dim * 2.0;
+    double work = 0.0;
+    for (const PrefillTcItem& it : plan.prefill_tc) {
+        int32_t hi = 0;
+        for (int t = 0; t < 2; ++t)
+            if (it.n_rows[t] > 0) hi = std::max(hi, it.prefix + it.row0[t] + it.n_rows[t]);
+        work += 8.0 + 1.9 * (double)std::max(0, std::min((hi + 127) / 128, it.j_end) - it.j_begin);
+    }
+    return (float)((work / (double)std::max(1, num_sms)) / (17.0 + dec_bytes / 7.1e6));
 }
 
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,

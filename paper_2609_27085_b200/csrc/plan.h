@@ -46,7 +46,10 @@ struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one
     int32_t j_begin, j_end;
     int32_t part_slot[2];
     int32_t part_k, part_c;
+    int32_t prefix, ctx_len;   // of the sequence (copied here so that a role needs one load per item)
+    int32_t pad[2];            // 80 bytes: five 16-byte words
 };
+static_assert(sizeof(PrefillTcItem) == 80, "PrefillTcItem is copied as five 16-byte words");
 
 struct PrefillCombineItem { // one KV-split tcgen05 item: merges its part_k partials per row
     int32_t q_row0[2];
@@ -97,6 +100,10 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
 struct Estimate {
     float us_decode = 0.f, us_combine = 0.f, us_prefill = 0.f;
 };
+// Time the tcgen05 prefill items would take spread evenly over num_sms SMs, divided by the time of the
+// decode kernel (same constants as estimate_us; no scheduling, O(items)).  0 when either part is absent.
+float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
+                              int32_t num_sms);
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
                      int32_t num_sms);
 

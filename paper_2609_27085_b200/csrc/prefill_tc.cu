@@ -52,11 +52,11 @@ constexpr uint32_t SMEM_TOTAL = SMEM_V + KV_STAGES * TILE_BYTES;   // 192 KB
 constexpr uint32_t TM_S = 0, TM_O = 256;   // column offsets; tile t adds 128 * t
 
 struct Bars {
-    uint64_t q_full;
+    uint64_t q_full, q_empty;
     uint64_t k_full[KV_STAGES], k_empty[KV_STAGES];
     uint64_t v_full[KV_STAGES], v_empty[KV_STAGES];
     uint64_t s_full[2], p_full[2], o_done[2];
-    uint64_t mma_done;        // the issuer's last commit of an item: all of its MMAs have completed
+    uint64_t item_full[2];    // the producer has put an item context into slot s
 };
 
 __device__ __forceinline__ uint32_t lane_field(int warp) { return (uint32_t)((warp & 3) * 32) << 16; }
@@ -98,45 +98,75 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 
 }  // namespace
 
-// What a role needs to know about the work item it is on.
+// Development aid, compiled only with -DCF_TRACE: one CTA stamps clock64 at the marked points of every role
+// (rows: 0 producer, 1 issuer, 2/3 first softmax thread of q tile 0/1); cf_trace_read copies the stamps out.
+#ifdef CF_TRACE
+#ifndef CF_TRACE_CTA
+#define CF_TRACE_CTA 0
+#endif
+__device__ unsigned long long cf_trace_buf[4][256][2];
+#define TR_DECL unsigned tr_n = 0u
+#define TR(role, id)                                                                      \
+    do {                                                                                  \
+        if (blockIdx.x == CF_TRACE_CTA && tr_n < 256u) {                                  \
+            cf_trace_buf[role][tr_n][0] = (unsigned long long)(id);                       \
+            cf_trace_buf[role][tr_n][1] = (unsigned long long)clock64();                  \
+            ++tr_n;                                                                       \
+        }                                                                                 \
+    } while (0)
+#ifdef CF_TRACE_FINE
+#define TRF(role, id) TR(role, id)
+#else
+#define TRF(role, id)
+#endif
+#else
+#define TR_DECL
+#define TR(role, id)
+#define TRF(role, id)
+#endif
+
+// What a role needs to know about the work item it is on.  The producer warp builds it and hands it
+// to the other roles through a two-slot ring in shared memory.
 struct ItemCtx {
     PrefillTcItem it;
-    int Lc, prefix;
     int kv_hi_t[2], n_j[2];   // per q tile: end of its visible keys; number of KV tiles of [j_begin, j_end) it takes part in
-    int n_max, total_pages, jb;
+    int n_max, total_pages;
+    int live, pad;            // live = 0: no more work, every role leaves
 };
-__device__ __forceinline__ ItemCtx load_item(const AttnParams& p, int idx)
+static_assert(sizeof(ItemCtx) % 16 == 0, "copied as 16-byte words");
+__device__ __forceinline__ void derive_item(ItemCtx& c)
 {
-    ItemCtx c;
-    c.it = p.pre_tc_items[idx];
-    const int Lq = __ldg(p.query_len + c.it.seq);
-    c.Lc = __ldg(p.context_len + c.it.seq);
-    c.prefix = c.Lc - Lq;
 #pragma unroll
     for (int t = 0; t < 2; ++t) {
-        c.kv_hi_t[t] = c.it.n_rows[t] > 0 ? c.prefix + c.it.row0[t] + c.it.n_rows[t] : 0;
+        c.kv_hi_t[t] = c.it.n_rows[t] > 0 ? c.it.prefix + c.it.row0[t] + c.it.n_rows[t] : 0;
         c.n_j[t] = max(0, min((c.kv_hi_t[t] + KT - 1) / KT, c.it.j_end) - c.it.j_begin);
     }
     c.n_max = max(c.n_j[0], c.n_j[1]);
     c.total_pages = (max(c.kv_hi_t[0], c.kv_hi_t[1]) + 15) >> 4;
-    c.jb = c.it.j_begin;       // loop indices are relative to it; jb + j is the absolute tile
-    return c;
+    c.live = 1;
+    c.pad = 0;
 }
 
 // Persistent CTAs: every CTA of the launch sequence draws work items (longest first) from one ticket
 // counter in global memory, p.pre_queue[0], until the tickets run out.  `queue_ctas` is the number of CTAs
 // that draw from the counter (over all grids that share it); the last of them to leave puts the two
 // counter words back to zero, so that a replay of the same launches needs no host-side reset.
+// The roles run through the items without a CTA-wide barrier in between: every mbarrier keeps counting
+// phases across items (each role carries the running phase of the barriers it uses), the producer is up
+// to two K/V tiles and one item context ahead, the issuer puts the first S = Q K^T of the next item
+// right behind the last P V of the current one, and a softmax thread goes from the epilogue of one item
+// straight to the first tile of the next.
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const AttnParams p, const int n_items, const int queue_ctas,
                   uint32_t* const resident)
 {
     extern __shared__ uint8_t smem_raw[];
+    __shared__ __align__(16) ItemCtx ctx_s[2];
     __shared__ __align__(8) Bars bars;
     __shared__ uint32_t tmem_base_s;
     __shared__ uint32_t abort_s;
-    __shared__ int item_s;
+    __shared__ uint32_t issuer_state[4];
 
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -150,6 +180,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // spatial launch sequence: the stream that carries the decode kernel waits (a stream memory
         // operation, not a kernel) until every CTA of this grid holds its SM
         if (resident != nullptr) atomicAdd(resident, 1u);
+        mbar_init(smem_u32(&bars.q_full), 1);
+        mbar_init(smem_u32(&bars.q_empty), 1);
+        for (int s = 0; s < KV_STAGES; ++s) {
+            mbar_init(smem_u32(&bars.k_full[s]), 1);
+            mbar_init(smem_u32(&bars.k_empty[s]), 1);
+            mbar_init(smem_u32(&bars.v_full[s]), 1);
+            mbar_init(smem_u32(&bars.v_empty[s]), 1);
+        }
+        for (int t = 0; t < 2; ++t) {
+            mbar_init(smem_u32(&bars.s_full[t]), 1);
+            mbar_init(smem_u32(&bars.p_full[t]), 4);      // one arrival per softmax warp
+            mbar_init(smem_u32(&bars.o_done[t]), 1);
+            mbar_init(smem_u32(&bars.item_full[t]), 1);
+        }
+        fence_mbar_init();
     }
     if (warp == 0) tmem_alloc<512>(smem_u32(&tmem_base_s));
     tc_fence_before();
@@ -161,96 +206,141 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     // (the K/V rows of cf_kv_append when the batch has no decode part).
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
-    // Called by the ten working warps between items (named barrier 1; the two spare warps wait at the
-    // teardown barrier).  After the first barrier every role has left the previous item - its MMAs have
-    // completed, tensor memory has been read out - so thread 0 may draw a ticket and re-arm the barriers.
-    auto next_item = [&]() -> int {
-        __syncwarp();
-        tc_fence_before();
-        asm volatile("bar.sync 1, 320;" ::: "memory");
-        if (threadIdx.x == 0) {
-            int idx = n_items;
-            if (abort_s == 0u) idx = (int)atomicAdd(p.pre_queue, 1u);
-            if (idx < n_items) {
-                mbar_init(smem_u32(&bars.q_full), 1);
-                for (int s = 0; s < KV_STAGES; ++s) {
-                    mbar_init(smem_u32(&bars.k_full[s]), 1);
-                    mbar_init(smem_u32(&bars.k_empty[s]), 1);
-                    mbar_init(smem_u32(&bars.v_full[s]), 1);
-                    mbar_init(smem_u32(&bars.v_empty[s]), 1);
-                }
-                for (int t = 0; t < 2; ++t) {
-                    mbar_init(smem_u32(&bars.s_full[t]), 1);
-                    mbar_init(smem_u32(&bars.p_full[t]), 4);      // one arrival per softmax warp
-                    mbar_init(smem_u32(&bars.o_done[t]), 1);
-                }
-                mbar_init(smem_u32(&bars.mma_done), 1);
-                fence_mbar_init();
-            } else {
-                idx = n_items;
-                if (atomicAdd(p.pre_queue + 1, 1u) == (uint32_t)(queue_ctas - 1)) {   // every other CTA has drawn its last ticket
-                    p.pre_queue[0] = 0u;
-                    p.pre_queue[1] = 0u;
-                    __threadfence();
-                }
-            }
-            item_s = idx;
-        }
-        asm volatile("bar.sync 1, 320;" ::: "memory");
-        tc_fence_after();
-        return item_s;
+    // the context of a role's k-th item (slot k & 1, filled for the (k >> 1)-th time); null on an abort.
+    // A role copies the fields it needs at once: the slot is rewritten two items later.
+    auto wait_item = [&](int k) -> const ItemCtx* {
+        if (!mbar_wait(smem_u32(&bars.item_full[k & 1]), (uint32_t)(k >> 1) & 1u, abort_flag)) return nullptr;
+        return &ctx_s[k & 1];
     };
 
     if (warp < 4) {
       reg_dec<REGS_ROLE>();
-      if (warp >= 2) {
-        // spare warps of the first warpgroup
+      if (warp == 3) {
+        // spare warp of the first warpgroup
+      } else if (warp == 2) {
+        // =========================================================== TMA producer of the V tiles
+        // (a warp issues the 16 boxes of a tile one after the other; K and V from one warp would make the
+        // producer as slow as the tensor pipe)
+        uint32_t ub[2] = {0u, 0u};
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+            const ItemCtx* cs = wait_item(k);
+            if (cs == nullptr || cs->live == 0) break;
+            const int n_max = cs->n_max, total_pages = cs->total_pages, jb = cs->it.j_begin, kvh = cs->it.kvh;
+            const int32_t* bt = p.block_table + (int64_t)cs->it.seq * p.max_blocks;
+            int32_t pid = lane < min(8, total_pages - 8 * jb) ? __ldg(bt + 8 * jb + lane) : 0;
+            for (int j = 0; j < n_max && ok; ++j) {
+                const int stage = j & 1;
+                const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
+                const int np = min(8, total_pages - 8 * (jb + j));
+                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
+                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
+                const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
+                if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1u, abort_flag));
+                if (!ok) break;
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 4096);
+                __syncwarp();
+                if (lane < 2 * np)
+                    tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane & 1) * 64, 0, kvh, my_pid,
+                                smem_u32(&bars.v_full[stage]));
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            ub[0] += (uint32_t)(n_max + 1) >> 1;
+            ub[1] += (uint32_t)n_max >> 1;
+        }
       } else if (warp == 0) {
-       for (;;) {
-        const int item = next_item();
-        if (item >= n_items) break;
-        const ItemCtx cx = load_item(p, item);
-        const PrefillTcItem& it = cx.it;
-        const int n_max = cx.n_max, total_pages = cx.total_pages, jb = cx.jb;
-        // =========================================================== TMA producer
+        // =========================================================== TMA producer of Q and the K tiles, keeper of the work queue
         if (lane == 0) {
             prefetch_tensormap(&map_q);
             prefetch_tensormap(&map_k);
             prefetch_tensormap(&map_v);
-            const int nq = (it.n_rows[0] > 0) + (it.n_rows[1] > 0);
-            mbar_arrive_expect_tx(smem_u32(&bars.q_full), nq * TILE_BYTES);
-            for (int t = 0; t < 2; ++t)
-                if (it.n_rows[t] > 0)
-                    for (int h = 0; h < 2; ++h)
-                        tma_load_3d(smem + SMEM_Q + t * TILE_BYTES + h * HALF_BYTES, &map_q, h * 64, it.head[t],
-                                    it.q_row0[t], smem_u32(&bars.q_full));
         }
-        const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks;
+        bool counted_out = false;
+        TR_DECL;
+        if (lane == 0) TR(0, 100);
+        // draws the next ticket; on the first empty draw the CTA is counted out and the last CTA resets the counters
+        auto draw = [&](ItemCtx& cx) {
+            int idx = n_items;
+            if (lane == 0 && *abort_flag == 0u && !counted_out) idx = (int)atomicAdd(p.pre_queue, 1u);
+            idx = __shfl_sync(0xffffffffu, idx, 0);
+            if (idx < n_items) {
+                const uint4* src = reinterpret_cast<const uint4*>(p.pre_tc_items + idx);
+                uint4* dst = reinterpret_cast<uint4*>(&cx.it);
+#pragma unroll
+                for (int i = 0; i < (int)(sizeof(PrefillTcItem) / 16); ++i) dst[i] = __ldg(src + i);
+                derive_item(cx);
+            } else {
+                cx.live = 0;
+                if (!counted_out && lane == 0 && atomicAdd(p.pre_queue + 1, 1u) == (uint32_t)(queue_ctas - 1)) {
+                    p.pre_queue[0] = 0u;      // every other CTA has made its last draw
+                    p.pre_queue[1] = 0u;
+                    __threadfence();
+                }
+                counted_out = true;
+            }
+        };
+        ItemCtx cx, nx;
+        draw(cx);
+        if (lane == 0) TR(0, 101);
+        uint32_t ub[2] = {0u, 0u};              // how often each K/V ring stage has been filled before this item
         bool ok = true;
-        for (int j = 0; j < n_max && ok; ++j) {
-            const int stage = j % KV_STAGES, use = j / KV_STAGES;
-            const int np = min(8, total_pages - 8 * (jb + j));
-            const int32_t pid = lane < np ? __ldg(bt + 8 * (jb + j) + lane) : 0;
-            const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
-            const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
-            // K tile
-            if (use > 0) ok = mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1, abort_flag);
+        for (int k = 0; ok; ++k) {
+            // Q tiles and the context slot are free once every S = Q K^T of the previous item has completed
+            if (k > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.q_empty), (uint32_t)(k - 1) & 1u, abort_flag));
             if (!ok) break;
-            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 4096);
-            __syncwarp();
-            if (lane < 2 * np)
-                tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane & 1) * 64, 0, it.kvh, my_pid,
-                            smem_u32(&bars.k_full[stage]));
-            // V tile
-            if (use > 0) ok = mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1, abort_flag);
-            if (!ok) break;
-            if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 4096);
-            __syncwarp();
-            if (lane < 2 * np)
-                tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane & 1) * 64, 0, it.kvh, my_pid,
-                            smem_u32(&bars.v_full[stage]));
+            if (lane == 0) {
+                const uint4* src = reinterpret_cast<const uint4*>(&cx);
+                uint4* dst = reinterpret_cast<uint4*>(&ctx_s[k & 1]);
+#pragma unroll
+                for (int i = 0; i < (int)(sizeof(ItemCtx) / 16); ++i) dst[i] = src[i];
+                mbar_arrive(smem_u32(&bars.item_full[k & 1]));
+                TR(0, 102);
+            }
+            if (!cx.live) break;
+            const PrefillTcItem& it = cx.it;
+            if (lane == 0) {
+                const int nq = (it.n_rows[0] > 0) + (it.n_rows[1] > 0);
+                mbar_arrive_expect_tx(smem_u32(&bars.q_full), nq * TILE_BYTES);
+                for (int t = 0; t < 2; ++t)
+                    if (it.n_rows[t] > 0)
+                        for (int h = 0; h < 2; ++h)
+                            tma_load_3d(smem + SMEM_Q + t * TILE_BYTES + h * HALF_BYTES, &map_q, h * 64, it.head[t],
+                                        it.q_row0[t], smem_u32(&bars.q_full));
+            }
+            const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks;
+            const int n_max = cx.n_max, total_pages = cx.total_pages, jb = it.j_begin;
+            const int j_draw = min(2, n_max - 1);       // the next ticket is drawn once the first tiles are on their way
+            bool drawn = false;
+            // page ids of a tile are fetched while the tile before it is being issued
+            int32_t pid = lane < min(8, total_pages - 8 * jb) ? __ldg(bt + 8 * jb + lane) : 0;
+            for (int j = 0; j < n_max && ok; ++j) {
+                const int stage = j & 1;
+                const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
+                const int np = min(8, total_pages - 8 * (jb + j));
+                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
+                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
+                const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
+                if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1u, abort_flag));
+                if (!ok) break;
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 4096);
+                __syncwarp();
+                if (lane < 2 * np)
+                    tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane & 1) * 64, 0, it.kvh, my_pid,
+                                smem_u32(&bars.k_full[stage]));
+                if (lane == 0 && (j < 5 || j >= n_max - 2)) TR(0, 200 + j);
+                if (j == j_draw) {
+                    draw(nx);
+                    drawn = true;
+                    if (lane == 0) TR(0, 104);
+                }
+            }
+            ok = __all_sync(0xffffffffu, ok);
+            if (ok && !drawn) draw(nx);
+            ub[0] += (uint32_t)(n_max + 1) >> 1;
+            ub[1] += (uint32_t)n_max >> 1;
+            cx = nx;
         }
-       }
+        if (!counted_out) draw(nx);               // left on an abort (the flag is up, so no ticket is taken): still count this CTA out
       } else {
         // =========================================================== MMA issuer
         constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
@@ -301,58 +391,87 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // the critical resource of the kernel: it is a single dependent instruction stream that is also
         // blocked while its MMAs queue up, so the work between two batches is kept to a handful of
         // instructions, with a lean loop for interior tiles and the general step for the rest.
+        if (lane == 0) {
         const uint32_t bar_kf[2] = {smem_u32(&bars.k_full[0]), smem_u32(&bars.k_full[1])};
         const uint32_t bar_vf[2] = {smem_u32(&bars.v_full[0]), smem_u32(&bars.v_full[1])};
         const uint32_t bar_ke[2] = {smem_u32(&bars.k_empty[0]), smem_u32(&bars.k_empty[1])};
         const uint32_t bar_ve[2] = {smem_u32(&bars.v_empty[0]), smem_u32(&bars.v_empty[1])};
-       for (;;) {
-        const int item = next_item();
-        if (item >= n_items) break;
-        if (lane == 0) {
-        const ItemCtx cx = load_item(p, item);
-        const int Lc = cx.Lc, n_max = cx.n_max, total_pages = cx.total_pages, jb = cx.jb;
-        const int n_j[2] = {cx.n_j[0], cx.n_j[1]};
-        bool ok = mbar_wait(smem_u32(&bars.q_full), 0, abort_flag);
-        ok = ok && mbar_wait(bar_kf[0], 0, abort_flag);
-        if (ok) {
-            tc_fence_after();
-            if (n_j[0] > 0) issue_qk(I0{}, I0{});
-            if (n_j[1] > 0) issue_qk(I1{}, I0{});
-            umma_commit(bar_ke[0]);
-        }
+        const uint32_t bar_qe = smem_u32(&bars.q_empty);
+        // Running phases: ub[s] = fills of K/V ring stage s before this item (tile j of an item sits in
+        // stage j & 1 and is that stage's fill number ub[j & 1] + (j >> 1)); sb[t] = tiles of q tile t
+        // before this item (s_full / p_full / o_done complete one phase per tile).
+        // Only this lane touches issuer_state (= ub[0], ub[1], sb[0], sb[1]).  The lane has no registers to
+        // spare beside its 48 descriptors, so the running phases live in shared memory, the item's fields are
+        // read from the context slot where they are needed (the slot is not rewritten before this lane has
+        // left the next item's last S = Q K^T behind), and only the interior loop keeps its parities in registers.
+        volatile uint32_t* const ist = issuer_state;
+        TR_DECL;
+        TR(1, 100);
+        ist[0] = ist[1] = ist[2] = ist[3] = 0u;
+        bool ok = true;
+        for (int k = 0; ok; ++k) {
+        const ItemCtx* cs = wait_item(k);
+        if (cs == nullptr || cs->live == 0) break;
+        const volatile ItemCtx* const vs = cs;
+        TR(1, 1);
+        const int n_max = cs->n_max;
+        const int n_j[2] = {cs->n_j[0], cs->n_j[1]};
+        ok = mbar_wait(smem_u32(&bars.q_full), (uint32_t)k & 1u, abort_flag);
+        ok = ok && mbar_wait(bar_kf[0], ist[0] & 1u, abort_flag);
+        if (!ok) break;
+        tc_fence_after();
+        if (n_j[0] > 0) issue_qk(I0{}, I0{});
+        if (n_j[1] > 0) issue_qk(I1{}, I0{});
+        umma_commit(bar_ke[0]);
+        TR(1, 3);
+        // q_empty: arrives when every S = Q K^T of the item has completed (the last one is issued in step n_max - 2)
+        if (n_max <= 1) umma_commit(bar_qe);
         // ---- interior tiles: both q tiles present and continuing, all 8 pages loaded, not the last tile
         const int n_int = (n_j[0] > 0 && n_j[1] > 0) ? min(n_j[0], n_j[1]) - 1 : 0;
-        auto lean_step = [&](auto S, uint32_t par_v, uint32_t par_k1, uint32_t par_p, uint32_t acc0) -> bool {
+        auto lean_step = [&](auto S, uint32_t par_v, uint32_t par_k1, uint32_t par_p0, uint32_t par_p1, uint32_t acc0) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
+            TRF(1, 10);
             if (!mbar_wait(bar_vf[st], par_v, abort_flag)) return false;
+            TRF(1, 11);
             if (!mbar_wait(bar_kf[st1], par_k1, abort_flag)) return false;
-            if (!mbar_wait(bar_p[0], par_p, abort_flag)) return false;
+            TRF(1, 12);
+            if (!mbar_wait(bar_p[0], par_p0, abort_flag)) return false;
+            TRF(1, 13);
             tc_fence_after();
             issue_pv(I0{}, S, 8, acc0);
             issue_qk(I0{}, S1{});
-            if (!mbar_wait(bar_p[1], par_p, abort_flag)) return false;
+            TRF(1, 14);
+            if (!mbar_wait(bar_p[1], par_p1, abort_flag)) return false;
+            TRF(1, 15);
             tc_fence_after();
             issue_pv(I1{}, S, 8, acc0);
             issue_qk(I1{}, S1{});
             umma_commit(bar_ve[st]);
             umma_commit(bar_ke[st1]);
+            TRF(1, 16);
             return true;
         };
         int j = 0;
         {
-            uint32_t h = 0;                                   // (j >> 1) & 1 for the even tile of the pair
-            for (; ok && j + 1 < n_int; j += 2, h ^= 1u) {
-                ok = lean_step(I0{}, h, h, 0u, j > 0 ? 1u : 0u);
-                if (ok) ok = lean_step(I1{}, h, h ^ 1u, 1u, 1u);
+            // parities of the even tile j of a pair: stage 0 fill ub[0] + j/2 (V now), stage 1 fill ub[1] + j/2
+            // (K of tile j + 1), softmax phases sb[t] + j; the odd tile j + 1 flips all but the stage-0 K
+            // fill of tile j + 2, which is ub[0] + j/2 + 1
+            uint32_t h0 = ist[0] & 1u, h1 = ist[1] & 1u;
+            const uint32_t p0 = ist[2] & 1u, p1 = ist[3] & 1u;
+            for (; ok && j + 1 < n_int; j += 2, h0 ^= 1u, h1 ^= 1u) {
+                ok = lean_step(I0{}, h0, h1, p0, p1, j > 0 ? 1u : 0u);
+                if (ok) ok = lean_step(I1{}, h1, h0 ^ 1u, p0 ^ 1u, p1 ^ 1u, 1u);
             }
+            if (ok && j > 0 && j >= n_max - 1) umma_commit(bar_qe);     // the pair loop issued the item's last S = Q K^T
         }
         // ---- general step: PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) with every edge case
         auto kv_step = [&](auto S, int j) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
-            const int np = min(8, total_pages - 8 * (jb + j));
-            if (!mbar_wait(bar_vf[st], (uint32_t)(j >> 1) & 1u, abort_flag)) return false;
+            const int jb = vs->it.j_begin, Lc = vs->it.ctx_len;
+            const int np = min(8, vs->total_pages - 8 * (jb + j));
+            if (!mbar_wait(bar_vf[st], (ist[st] + (uint32_t)(j >> 1)) & 1u, abort_flag)) return false;
             if (j == n_max - 1 && Lc < (8 * (jb + j) + np) * 16) {
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
                 // that a zero probability never multiplies a NaN
@@ -370,8 +489,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 constexpr int t = decltype(T)::value;
                 if (j >= n_j[t]) return true;
                 const bool more = j + 1 < n_j[t];
-                if (more && !mbar_wait(bar_kf[st1], (uint32_t)((j + 1) >> 1) & 1u, abort_flag)) return false;
-                if (!mbar_wait(bar_p[t], (uint32_t)j & 1u, abort_flag)) return false;
+                if (more && !mbar_wait(bar_kf[st1], (ist[st1] + (uint32_t)((j + 1) >> 1)) & 1u, abort_flag)) return false;
+                if (!mbar_wait(bar_p[t], (ist[2 + t] + (uint32_t)j) & 1u, abort_flag)) return false;
                 tc_fence_after();
                 issue_pv(T, S, np, acc0);
                 if (more) issue_qk(T, S1{});
@@ -381,17 +500,21 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!tile(I1{})) return false;
             umma_commit(bar_ve[st]);
             if (j + 1 < n_max) umma_commit(bar_ke[st1]);
+            if (j + 1 == n_max - 1) umma_commit(bar_qe);
             return true;
         };
         static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
-        for (; j < n_max && ok; ++j) ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
-        // every MMA of the item has completed (and every commit above has arrived) before the barriers are re-armed
-        if (ok) {
-            umma_commit(smem_u32(&bars.mma_done));
-            mbar_wait(smem_u32(&bars.mma_done), 0, abort_flag);
+        for (; j < n_max && ok; ++j) {
+            ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
+            TR(1, 300 + j);
+        }
+        TR(1, 4);
+        ist[0] += (uint32_t)(n_max + 1) >> 1;
+        ist[1] += (uint32_t)n_max >> 1;
+        ist[2] += (uint32_t)n_j[0];
+        ist[3] += (uint32_t)n_j[1];
         }
         }
-       }
       }
     } else {
       reg_inc<REGS_SOFTMAX>();
@@ -401,20 +524,24 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const uint32_t lanes = lane_field(warp);
       const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
       const float sc = p.scale_log2;
-      for (;;) {
-        const int item = next_item();
-        if (item >= n_items) break;
+      TR_DECL;
+      if ((warp & 3) == 0 && lane == 0) TR(2 + t, 100);
+      uint32_t sbt = 0u;                       // tiles of this q tile in earlier items: running phase of s_full / p_full / o_done
+      bool ok = true;
+      for (int k = 0; ok; ++k) {
+        const ItemCtx* cs = wait_item(k);
+        if (cs == nullptr || cs->live == 0) break;
         {
-        const ItemCtx cx = load_item(p, item);
-        const PrefillTcItem& it = cx.it;
-        const int jb = cx.jb;
-        const int n_j[2] = {cx.n_j[0], cx.n_j[1]};
-        const int limit = min(cx.prefix + it.row0[t] + row, cx.kv_hi_t[t] - 1);   // last visible key of this row
+        // this q tile's fields of the item
+        const int jb = cs->it.j_begin, n_jt = cs->n_j[t], kv_hi = cs->kv_hi_t[t];
+        const int it_row0 = cs->it.row0[t], it_n_rows = cs->it.n_rows[t], it_q_row0 = cs->it.q_row0[t], it_head = cs->it.head[t];
+        const int it_part_slot = cs->it.part_slot[t], it_part_k = cs->it.part_k, it_part_c = cs->it.part_c;
+        const int limit = min(cs->it.prefix + it_row0 + row, kv_hi - 1);   // last visible key of this row
         float m_used = -INFINITY, l_sum = 0.f;
-        bool ok = true;
-        for (int j = 0; j < n_j[t]; ++j) {
-            ok = mbar_wait(smem_u32(&bars.s_full[t]), j & 1, abort_flag);
+        for (int j = 0; j < n_jt; ++j) {
+            ok = mbar_wait(smem_u32(&bars.s_full[t]), (sbt + (uint32_t)j) & 1u, abort_flag);
             if (!ok) break;
+            if ((warp & 3) == 0 && lane == 0 && (j < 5 || j >= n_jt - 2)) TR(2 + t, 400 + j);
             tc_fence_after();
             float sv[128];
 #pragma unroll
@@ -480,7 +607,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 m_used += d;
                 l_sum *= f;
                 if (j > 0) {
-                    ok = mbar_wait(smem_u32(&bars.o_done[t]), (j - 1) & 1, abort_flag);
+                    ok = mbar_wait(smem_u32(&bars.o_done[t]), (sbt + (uint32_t)(j - 1)) & 1u, abort_flag);
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll 1
@@ -501,16 +628,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
+            if ((warp & 3) == 0 && lane == 0 && (j < 5 || j >= n_jt - 2)) TR(2 + t, 500 + j);
         }
-        if (ok && n_j[t] > 0) ok = mbar_wait(smem_u32(&bars.o_done[t]), (n_j[t] - 1) & 1, abort_flag);
-        if (ok && n_j[t] > 0) {
+        if (ok && n_jt > 0) ok = mbar_wait(smem_u32(&bars.o_done[t]), (sbt + (uint32_t)(n_jt - 1)) & 1u, abort_flag);
+        if ((warp & 3) == 0 && lane == 0) TR(2 + t, 6);
+        if (ok && n_jt > 0) {
             tc_fence_after();
             const float inv = 1.f / l_sum;
-            const bool live = row < it.n_rows[t];
-            const bool partial = it.part_slot[t] >= 0;
-            __nv_bfloat16* orow = p.out + ((int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]) * D;
+            const bool live = row < it_n_rows;
+            const bool partial = it_part_slot >= 0;
+            __nv_bfloat16* orow = p.out + ((int64_t)(it_q_row0 + row) * p.Hq + it_head) * D;
             // KV-split item: un-normalised fp32 row plus (reference maximum, sum) for the combine pass
-            const int64_t pslot = (int64_t)it.part_slot[t] + (int64_t)row * it.part_k + it.part_c;
+            const int64_t pslot = (int64_t)it_part_slot + (int64_t)row * it_part_k + it_part_c;
             float* prow = p.pre_part_o + pslot * D;
 #pragma unroll
             for (int c = 0; c < 4; ++c) {
@@ -534,8 +663,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
             }
             if (live && partial) *reinterpret_cast<float2*>(p.pre_part_ml + pslot * 2) = make_float2(m_used, l_sum);
-            else if (live && p.lse) p.lse[(int64_t)(it.q_row0[t] + row) * p.Hq + it.head[t]] = (m_used + log2f(l_sum)) * kLn2;
+            else if (live && p.lse) p.lse[(int64_t)(it_q_row0 + row) * p.Hq + it_head] = (m_used + log2f(l_sum)) * kLn2;
+            // O_t has been read out: the p_full arrival of the next item's first tile, later in this thread's
+            // program order, is what allows the issuer to overwrite it
+            tc_fence_before();
         }
+        if ((warp & 3) == 0 && lane == 0) TR(2 + t, 7);
+        sbt += (uint32_t)n_jt;
         }
       }
     }
@@ -550,6 +684,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         __syncthreads();
     }
     if (warp == 0) tmem_dealloc<512>(tmem);
+#ifdef CF_TRACE
+    if (threadIdx.x == 0 && blockIdx.x == CF_TRACE_CTA) {
+        cf_trace_buf[0][255][0] = 999ull;
+        cf_trace_buf[0][255][1] = (unsigned long long)clock64();
+    }
+#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -732,3 +872,10 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
 }
 
 }  // namespace cf
+
+#ifdef CF_TRACE
+extern "C" int cf_trace_read(void* dst)
+{
+    return (int)cudaMemcpyFromSymbol(dst, cf::cf_trace_buf, sizeof(cf::cf_trace_buf));
+}
+#endif

@@ -239,11 +239,12 @@ def test_property_random_batches():
         run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True))
 
 
-def test_overlap_mode_is_bit_identical_to_the_serial_sequence():
+def test_spatial_sequence_is_bit_identical_to_the_serial_sequence():
     sc = small(29, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
     b = sc.batches[0]
     g = GpuScenario(sc)
     g.append(b)
+    cf.cf_set_overlap(g.ctx, 0)
     serial, lse0 = g.attend(b)
     # default share of the SMs; then 8 and 3 front CTAs, so that every CTA works through several items and
     # the second grid (behind decode, same queue) takes part
@@ -251,7 +252,7 @@ def test_overlap_mode_is_bit_identical_to_the_serial_sequence():
         cf.cf_set_overlap(g.ctx, n)
         o, lse = g.attend(b)
         assert np.array_equal(o, serial) and np.array_equal(lse, lse0)
-    cf.cf_set_overlap(g.ctx, 0)
+    cf.cf_set_overlap(g.ctx, 1)
     assert cf.cf_get_async_status(g.ctx) == 0
     k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
     oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
