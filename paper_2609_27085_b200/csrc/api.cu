@@ -528,6 +528,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
+    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
     cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -568,6 +569,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
+    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
     cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;

@@ -191,7 +191,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // An item may be cut into k <= 8 KV ranges that write fp32 partials, merged by a combine pass; k
         // comes from the cost model's constants; a range never starts inside the diagonal band and has at
         // least 4 tiles.
-        const size_t M = (size_t)std::max(1, cfg.num_sms);
+        const size_t M = (size_t)std::max(1, (cfg.prefill_sms_mixed > 0 && !plan->decode.empty()) ? cfg.prefill_sms_mixed : cfg.num_sms);
         // decides the KV ranges per item for one candidate item list; returns the predicted time (us)
         auto decide = [&](const std::vector<KeyedTc>& its, const double tile_us, std::vector<int32_t>& k_of) -> double {
         const size_t n_items = its.size();

@@ -67,6 +67,8 @@ struct PlanConfig {
     int32_t decode_page_quantum = 4;  // chunk lengths are multiples of this many pages (warps per CTA)
     int32_t prefill_tile_rows = 64;   // tile height of the mma.sync prefill kernel
     bool prefill_tc = false;          // true: plan items for the tcgen05 kernel (128-row tile pairs)
+    int32_t prefill_sms_mixed = 0;    // > 0: SMs the prefill items are balanced over when the batch also holds decode
+                                      // work (spatial launch sequence: the first prefill grid's share); 0: num_sms
     int32_t prefill_force_split = 0;  // >= 2: split every tcgen05 item that many ways (tests); 0: cost model decides
 };
 
