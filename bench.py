@@ -401,7 +401,10 @@ def write_report(torch, cf, ctx, stream, peaks):
                  ("cfg3_tp4_shard", lambda: syn.config3_chat_tp4_shard()), ("cfg4_agentic", lambda: syn.config4_agentic())]
     scenarios += [(f"cfg5_b{b}_n{n}", (lambda b=b, n=n: syn.config5_sweep_point(b, n))) for b, n in
                   [(0, 0), (512, 4), (2048, 1), (8192, 1), (8192, 4)]]
+    only = [x for x in os.environ.get("CF_REPORT_ONLY", "").split(",") if x]
     for name, make in scenarios:
+        if only and name not in only:
+            continue
         sc = make()
         wl = DeviceWorkload(sc, torch, cf, ctx)
         n_it = len(sc.batches)

@@ -342,7 +342,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, resident, c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, 1, front, resident, c->side);
         if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
         // only after the front grid has been enqueued without an error, so that the count is certain to arrive
         if (e == cudaSuccess && resident &&
@@ -350,7 +350,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
         if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, nullptr, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, stream);
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
     } else {
@@ -360,7 +360,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, nullptr, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
@@ -528,7 +528,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
-    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
+    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
     cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;

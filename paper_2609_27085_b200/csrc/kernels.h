@@ -32,11 +32,13 @@ cudaError_t launch_prefill_mma(const AttnParams& p, int head_dim, int n_items, c
 
 // tcgen05 / tensor-memory chunked prefill (head_dim 128): `n_ctas` persistent CTAs draw the `n_items`
 // PrefillTcItems from the ticket counter p.pre_queue, which `queue_ctas` CTAs share in total (several
-// launches may draw from one counter; the last CTA to leave resets it).  `resident`, when not null, is a
-// device word that every CTA increments as it starts.
+// launches may draw from one counter; the last CTA to leave resets it).  Ticket t stands for item
+// ticket_base + t; with first_static set, CTA b starts on item b without a draw (then ticket_base = n_ctas of
+// that grid, also for a second grid that shares the counter).  `resident`, when not null, is a device word that
+// every CTA increments as it starts.
 bool prefill_tc_supported(const cf_cache_desc* desc);
 cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
-                              int queue_ctas, uint32_t* resident, cudaStream_t stream);
+                              int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
 
 // merges the fp32 partials of KV-split prefill items into `out` (one CTA per split item)
 cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream);

@@ -89,6 +89,13 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x)
 #ifndef CF_POLY_MASK
 #define CF_POLY_MASK 0x8080u
 #endif
+// 32-byte store (address 32-byte aligned)
+__device__ __forceinline__ void st_global_256(void* p, const uint32_t* v)
+{
+    asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(p), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3]), "r"(v[4]),
+                 "r"(v[5]), "r"(v[6]), "r"(v[7])
+                 : "memory");
+}
 __device__ __forceinline__ float max3(float a, float b, float c)
 {
     float d;
@@ -151,6 +158,8 @@ __device__ __forceinline__ void derive_item(ItemCtx& c)
 // counter in global memory, p.pre_queue[0], until the tickets run out.  `queue_ctas` is the number of CTAs
 // that draw from the counter (over all grids that share it); the last of them to leave puts the two
 // counter words back to zero, so that a replay of the same launches needs no host-side reset.
+// Ticket t stands for item ticket_base + t; with first_static set, CTA b starts on item b without a draw
+// (the grid that is launched first takes items 0 .. gridDim.x - 1 this way, so ticket_base is its size).
 // The roles run through the items without a CTA-wide barrier in between: every mbarrier keeps counting
 // phases across items (each role carries the running phase of the barriers it uses), the producer is up
 // to two K/V tiles and one item context ahead, the issuer puts the first S = Q K^T of the next item
@@ -159,7 +168,7 @@ __device__ __forceinline__ void derive_item(ItemCtx& c)
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const AttnParams p, const int n_items, const int queue_ctas,
-                  uint32_t* const resident)
+                  const int first_static, const int ticket_base, uint32_t* const resident)
 {
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(16) ItemCtx ctx_s[2];
@@ -170,6 +179,16 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     const uint32_t smem = (smem_u32(smem_raw) + 1023u) & ~1023u;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    // the first item of a CTA that starts on a fixed item: fetched now, in use after the set-up below (the plan
+    // was uploaded before the kernel that precedes this one in the stream, so it may be read this early)
+    const bool has_static = first_static != 0 && (int)blockIdx.x < n_items;
+    PrefillTcItem first_it;
+    if (warp == 0 && has_static) {
+        const uint4* src = reinterpret_cast<const uint4*>(p.pre_tc_items + blockIdx.x);
+        uint4* dst = reinterpret_cast<uint4*>(&first_it);
+#pragma unroll
+        for (int i = 0; i < (int)(sizeof(PrefillTcItem) / 16); ++i) dst[i] = __ldg(src + i);
+    }
     // lets the next grid of the stream become resident while this grid drains (it waits for this grid's
     // completion before it reads anything this grid wrote)
     asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
@@ -261,7 +280,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // draws the next ticket; on the first empty draw the CTA is counted out and the last CTA resets the counters
         auto draw = [&](ItemCtx& cx) {
             int idx = n_items;
-            if (lane == 0 && *abort_flag == 0u && !counted_out) idx = (int)atomicAdd(p.pre_queue, 1u);
+            if (lane == 0 && *abort_flag == 0u && !counted_out) idx = ticket_base + (int)atomicAdd(p.pre_queue, 1u);
             idx = __shfl_sync(0xffffffffu, idx, 0);
             if (idx < n_items) {
                 const uint4* src = reinterpret_cast<const uint4*>(p.pre_tc_items + idx);
@@ -280,7 +299,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             }
         };
         ItemCtx cx, nx;
-        draw(cx);
+        if (has_static && *abort_flag == 0u) {
+            cx.it = first_it;
+            derive_item(cx);
+        } else {
+            draw(cx);
+        }
         if (lane == 0) TR(0, 101);
         uint32_t ub[2] = {0u, 0u};              // how often each K/V ring stage has been filled before this item
         bool ok = true;
@@ -646,19 +670,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 float ov[32];
                 tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
                 tmem_wait_ld();
+                // a thread owns a row, so a warp's store touches 32 rows: 32-byte stores halve the number of
+                // memory transactions of the 16-byte ones
                 if (live && partial) {
 #pragma unroll
-                    for (int i = 0; i < 8; ++i)
-                        *reinterpret_cast<float4*>(prow + c * 32 + i * 4) = make_float4(ov[4 * i], ov[4 * i + 1], ov[4 * i + 2], ov[4 * i + 3]);
+                    for (int i = 0; i < 4; ++i) st_global_256(prow + c * 32 + i * 8, reinterpret_cast<const uint32_t*>(ov + 8 * i));
                 } else if (live) {
 #pragma unroll
-                    for (int i = 0; i < 4; ++i) {
-                        uint4 w;
-                        w.x = pack_bf16(ov[8 * i + 0] * inv, ov[8 * i + 1] * inv);
-                        w.y = pack_bf16(ov[8 * i + 2] * inv, ov[8 * i + 3] * inv);
-                        w.z = pack_bf16(ov[8 * i + 4] * inv, ov[8 * i + 5] * inv);
-                        w.w = pack_bf16(ov[8 * i + 6] * inv, ov[8 * i + 7] * inv);
-                        *reinterpret_cast<uint4*>(orow + c * 32 + i * 8) = w;
+                    for (int i = 0; i < 2; ++i) {
+                        uint32_t w[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) w[e] = pack_bf16(ov[16 * i + 2 * e] * inv, ov[16 * i + 2 * e + 1] * inv);
+                        st_global_256(orow + c * 32 + i * 16, w);
                     }
                 }
             }
@@ -833,7 +856,7 @@ bool prefill_tc_supported(const cf_cache_desc* d)
 }
 
 cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
-                              int queue_ctas, uint32_t* resident, cudaStream_t stream)
+                              int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream)
 {
     if (n_items <= 0 || n_ctas <= 0) return cudaSuccess;
     CUtensorMap mq, mk, mv;
@@ -868,7 +891,7 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p, n_items, queue_ctas, resident);
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p, n_items, queue_ctas, first_static, ticket_base, resident);
 }
 
 }  // namespace cf
