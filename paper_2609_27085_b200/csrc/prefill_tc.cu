@@ -1,12 +1,15 @@
 // Chunked-prefill attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
 // tensor memory), head_dim 128.
 //
-// One CTA = one work item = two 128-row q tiles that share a KV head (two query heads of one group
-// over the same rows; for G = 1 two consecutive row tiles of one head), so every K/V tile fetched
-// into shared memory feeds two S = Q K^T and two O += P V products.  384 threads, warp-specialised
-// (the first warpgroup hands most of its registers to the two softmax warpgroups with setmaxnreg):
-//   warp 0      TMA producer: Q tiles once, then 128-token K and V tiles, one 16-token page-half per
-//               TMA box, gathered through the block table into 128B-swizzled shared memory rings.
+// A work item = two 128-row q tiles that share a KV head (two query heads of one group over the same
+// rows; for G = 1 two consecutive row tiles of one head), so every K/V tile fetched into shared memory
+// feeds two S = Q K^T and two O += P V products.  CTAs are persistent (one per SM): CTA b starts on
+// item b and then draws items from a ticket counter; the roles run from item to item without a
+// CTA-wide barrier.  384 threads, warp-specialised (the first warpgroup hands most of its registers to
+// the two softmax warpgroups with setmaxnreg):
+//   warp 0      work queue; TMA producer of the Q tiles and of the 128-token K tiles, one 16-token
+//               page-half per TMA box, gathered through the block table into a 128B-swizzled ring.
+//   warp 2      TMA producer of the V tiles (same box shape, its own ring).
 //   warp 1      MMA issuer (one elected lane): S_t = Q_t K^T, O_t += P_t V, in the order
 //               PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) so that the tensor pipe works on one tile while
 //               the other tile's softmax runs.
