@@ -38,6 +38,7 @@ struct PlanSlot {
     uint8_t* host = nullptr;   // pinned
     uint8_t* dev = nullptr;
     cudaEvent_t done = nullptr;
+    cudaEvent_t uploaded = nullptr;   // host-staged steps: the plan copy runs on the input copy stream
     bool used = false;
 };
 
@@ -57,6 +58,7 @@ struct cf_ctx {
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
+    cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
     bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
     cudaStream_t side = nullptr;
@@ -192,7 +194,14 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     if (!pl.prefill_combine.empty())
         std::memcpy(s.host + L->off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
     std::memset(s.host + L->off_queue, 0, 16);
-    if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
+    // A host-staged step sends its plans down the input copy stream: a small copy enqueued on the caller's
+    // stream would sit in the copy engine's queue until that stream's kernels are done, and hold back the
+    // next step's input copies behind it.
+    cudaStream_t copy_stream = c->plan_copy_stream ? c->plan_copy_stream : stream;
+    if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, copy_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (c->plan_copy_stream &&
+        (cudaEventRecord(s.uploaded, copy_stream) != cudaSuccess || cudaStreamWaitEvent(stream, s.uploaded, 0) != cudaSuccess))
+        return CF_ERR_CUDA;
     *dev_base = s.dev;
     *slot_out = &s;
     return CF_OK;
@@ -420,7 +429,8 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->spatial_sms = env_int("CF_SPATIAL_SMS", 0);
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
-        ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess;
+        ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->slots[i].uploaded, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && ensure_plan_capacity(c, kDefaultPlanBytes) == CF_OK;
     c->workspace_fixed = false;
     ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
@@ -454,6 +464,7 @@ cf_status cf_destroy(cf_ctx* c)
         if (c->slots[i].host) cudaFreeHost(c->slots[i].host);
         if (c->slots[i].dev) cudaFree(c->slots[i].dev);
         if (c->slots[i].done) cudaEventDestroy(c->slots[i].done);
+        if (c->slots[i].uploaded) cudaEventDestroy(c->slots[i].uploaded);
     }
     for (cf::TimedCall& tc : c->timed)
         for (int i = 0; i < 4; ++i)
@@ -723,15 +734,20 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
     if (cudaEventRecord(hs.h2d_done, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
     // kernels: the caller's stream
     if (cudaStreamWaitEvent(stream, hs.h2d_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+    c->plan_copy_stream = c->h2d_stream;
     st = cf_kv_append(c, desc, k_cache, v_cache, dk, dv, block_table, max_blocks_per_seq, context_len, query_len,
                       num_seqs, cuda_stream);
-    if (st != CF_OK) return st;
+    if (st != CF_OK) {
+        c->plan_copy_stream = nullptr;
+        return st;
+    }
     // The step is bound by the copies over PCIe, not by the kernels; measured on the chat-like workload the
-    // spatial sequence (side stream, stream memory operations) made it slower (0.49 ms against 0.41 ms).
+    // spatial sequence (side stream, stream memory operations) made it slower (0.38 ms against 0.365 ms).
     c->in_host_step = true;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);
     c->in_host_step = false;
+    c->plan_copy_stream = nullptr;
     if (st != CF_OK) return st;
     if (cudaEventRecord(hs.compute_done, stream) != cudaSuccess) return CF_ERR_CUDA;
     // result: second copy stream
