@@ -58,6 +58,7 @@ struct cf_ctx {
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
+    cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
     cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
     bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
@@ -194,13 +195,14 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     if (!pl.prefill_combine.empty())
         std::memcpy(s.host + L->off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
     std::memset(s.host + L->off_queue, 0, 16);
-    // A host-staged step sends its plans down the input copy stream: a small copy enqueued on the caller's
-    // stream would sit in the copy engine's queue until that stream's kernels are done, and hold back the
-    // next step's input copies behind it.
-    cudaStream_t copy_stream = c->plan_copy_stream ? c->plan_copy_stream : stream;
+    // The copy does not go on the caller's stream: there it would start only when that stream's earlier
+    // kernels are done (a few microseconds of copy-engine latency between kernels, every call) and, queued in
+    // the copy engine meanwhile, hold back copies enqueued after it.  It runs on a context-owned stream (a
+    // host-staged step: on its input copy stream) and the caller's stream waits for it through an event; the
+    // slot's device buffer is free by then (the host waited for the slot's last use above).
+    cudaStream_t copy_stream = c->plan_copy_stream ? c->plan_copy_stream : c->upload_stream;
     if (cudaMemcpyAsync(s.dev, s.host, L->total, cudaMemcpyHostToDevice, copy_stream) != cudaSuccess) return CF_ERR_CUDA;
-    if (c->plan_copy_stream &&
-        (cudaEventRecord(s.uploaded, copy_stream) != cudaSuccess || cudaStreamWaitEvent(stream, s.uploaded, 0) != cudaSuccess))
+    if (cudaEventRecord(s.uploaded, copy_stream) != cudaSuccess || cudaStreamWaitEvent(stream, s.uploaded, 0) != cudaSuccess)
         return CF_ERR_CUDA;
     *dev_base = s.dev;
     *slot_out = &s;
@@ -436,6 +438,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     ok = ok && ensure_workspace(c, workspace_bytes ? workspace_bytes : kDefaultWorkspace) == CF_OK;
     c->workspace_fixed = workspace_bytes != 0;
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->upload_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; i < kHostStages && ok; ++i) {
@@ -474,6 +477,7 @@ cf_status cf_destroy(cf_ctx* c)
     if (c->ev_fork) cudaEventDestroy(c->ev_fork);
     if (c->ev_join) cudaEventDestroy(c->ev_join);
     if (c->side) cudaStreamDestroy(c->side);
+    if (c->upload_stream) cudaStreamDestroy(c->upload_stream);
     for (int i = 0; i < kHostStages; ++i) {
         HostStage& hs = c->stage[i];
         if (hs.dev) cudaFree(hs.dev);
