@@ -146,6 +146,7 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
     c->workspace_bytes = 0;
     size_t nb = align_up(need + need / 4, 1u << 20);
     if (cudaMalloc((void**)&c->workspace, nb) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemset(c->workspace, 0, nb) != cudaSuccess) return CF_ERR_CUDA;       // the ticket counters at its front start at zero
     c->workspace_bytes = nb;
     return CF_OK;
 }
@@ -254,18 +255,23 @@ namespace cf {
 struct PlanCounts {
     int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
+    int n_part_slots = 0;
 };
 
 // Split-K workspace: decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact partial rows of
 // KV-split prefill items [row slot, D] + [row slot, 2].
+// The first kCounterBytes hold the fused-combine ticket counters of the decode kernel (one per first partial
+// slot of a split sequence and KV head): zeroed when the buffer is allocated, put back to zero by the kernel.
+// A batch with more counters than fit uses the separate combine kernel.
+static constexpr size_t kCounterBytes = 256u << 10;
 struct WsLayout {
     size_t dec_o = 0, dec_ml = 0, pre_o = 0, pre_ml = 0, total = 0;
 };
 static WsLayout ws_layout(int n_part_slots, int n_pre_slots, int Hq, int D)
 {
     WsLayout w;
-    w.dec_o = 0;
-    w.dec_ml = align_up((size_t)n_part_slots * Hq * D * sizeof(float), 256);
+    w.dec_o = kCounterBytes;
+    w.dec_ml = w.dec_o + align_up((size_t)n_part_slots * Hq * D * sizeof(float), 256);
     w.pre_o = w.dec_ml + align_up((size_t)n_part_slots * Hq * 2 * sizeof(float), 256);
     w.pre_ml = w.pre_o + align_up((size_t)n_pre_slots * D * sizeof(float), 256);
     w.total = w.pre_ml + align_up((size_t)n_pre_slots * 2 * sizeof(float), 256);
@@ -298,8 +304,10 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.comb_items = (const CombineItem*)(base + L.off_comb);
     p.pre_items = (const PrefillItem*)(base + L.off_pre);
     p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
-    p.part_o = ws;
+    p.part_o = (float*)((uint8_t*)ws + W.dec_o);
     p.part_ml = (float*)((uint8_t*)ws + W.dec_ml);
+    const bool fused_combine = (size_t)n.n_part_slots * desc->num_kv_heads * sizeof(uint32_t) <= kCounterBytes;
+    p.dec_counters = fused_combine ? (uint32_t*)ws : nullptr;
     p.pre_part_o = (float*)((uint8_t*)ws + W.pre_o);
     p.pre_part_ml = (float*)((uint8_t*)ws + W.pre_ml);
     p.pre_comb_items = (const PrefillCombineItem*)(base + L.off_pre_comb);
@@ -318,7 +326,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         }
         tc = &c->timed[c->timed_used++];
         tc->ran[0] = (n.n_dec > 0);
-        tc->ran[1] = (n.n_comb > 0);
+        tc->ran[1] = (n.n_comb > 0) && !fused_combine;
         tc->ran[2] = (n.n_pre > 0) || (n.n_pre_tc > 0);
     }
     const bool has_prefill = (n.n_pre > 0) || (n.n_pre_tc > 0);
@@ -360,7 +368,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
             mo.wait(stream, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
-        if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, stream);
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
@@ -368,14 +376,14 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[0], stream);
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
         if (tc) cudaEventRecord(tc->ev[1], stream);
-        if (e == cudaSuccess) e = launch_combine(p, D, n.n_comb, stream);
+        if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -568,6 +576,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     PlanCounts n;
     n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_pre = (int)pl.prefill.size();
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
+    n.n_part_slots = pl.n_part_slots;
     n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
@@ -606,7 +615,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
     const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
-    if (ok && part_bytes) ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess;
+    if (ok && part_bytes) ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess && cudaMemset(P->part, 0, kCounterBytes) == cudaSuccess;
     if (ok) {
         std::memcpy(P->host + L.off_qstart, pl.q_start.data(), sizeof(int32_t) * ((size_t)num_seqs + 1));
         if (num_seqs > 0) {
@@ -684,6 +693,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
     n.total_q = P->total_q;
     n.pre_over_dec = P->pre_over_dec;
+    n.n_part_slots = P->n_part_slots;
     const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim);
     return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, W, q, k_cache,
                             v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);

@@ -20,6 +20,56 @@
 
 namespace cf {
 
+// ---------------------------------------------------------------------------------------------
+// Merge of the partials of one (split sequence, query head) in fixed chunk order (deterministic), one float4
+// of the head per calling thread:
+//   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
+// evaluated as a running merge over groups of eight chunks.  Partials are fetched eight chunks at a time
+// with independent L2 loads (a dependent load per chunk would cost a memory round trip each; L2 loads,
+// because in the fused path other CTAs of the same grid wrote them).
+template <int D>
+__device__ __forceinline__ void merge_partials(const AttnParams& p, int q_row, int part_first, int n_chunks, int hq, int d,
+                                               bool write_lse)
+{
+    constexpr int GROUP = 8;
+    float M = -INFINITY, L = 0.f;
+    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
+    for (int c0 = 0; c0 < n_chunks; c0 += GROUP) {
+        float2 ml[GROUP];
+        float4 v[GROUP];
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < n_chunks) {
+                const int64_t pr = (int64_t)(part_first + c0 + i) * p.Hq + hq;
+                ml[i] = __ldcg(reinterpret_cast<const float2*>(p.part_ml + pr * 2));
+                v[i] = __ldcg(reinterpret_cast<const float4*>(p.part_o + pr * D + d));
+            }
+        float Mg = M;
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < n_chunks) Mg = fmaxf(Mg, ml[i].x);
+        const float fold = fast_exp2(M - Mg);               // 0 on the first group (M = -inf)
+        L *= fold;
+        acc.x *= fold; acc.y *= fold; acc.z *= fold; acc.w *= fold;
+        M = Mg;
+#pragma unroll
+        for (int i = 0; i < GROUP; ++i)
+            if (c0 + i < n_chunks) {
+                const float f = fast_exp2(ml[i].x - M);
+                L += ml[i].y * f;
+                acc.x += v[i].x * f; acc.y += v[i].y * f; acc.z += v[i].z * f; acc.w += v[i].w * f;
+            }
+    }
+    const float inv = 1.f / L;
+    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
+    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
+    uint2 packed;
+    packed.x = *reinterpret_cast<uint32_t*>(&lo);
+    packed.y = *reinterpret_cast<uint32_t*>(&hi);
+    *reinterpret_cast<uint2*>(p.out + ((int64_t)q_row * p.Hq + hq) * D + d) = packed;
+    if (p.lse && write_lse) p.lse[(int64_t)q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
+}
+
 template <int D, int NWARPS, int NSTAGE>
 __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const AttnParams p)
 {
@@ -214,6 +264,27 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
             if (d == 0) *reinterpret_cast<float2*>(p.part_ml + pr * 2) = make_float2(M, L);
         }
     }
+
+    // ---- Fused combine: the CTA that finishes a (sequence, KV head) last merges that head group's partials.
+    // Every CTA publishes its partial (fence), then takes a ticket; the one that draws the last ticket sees
+    // all of them (fence again, L2 loads).  The merge walks the chunks in index order, so the result does
+    // not depend on which CTA performs it; that CTA also puts the counter back to zero for the next launch.
+    if (it.part_slot >= 0 && p.dec_counters != nullptr) {
+        __shared__ int last_s;
+        __threadfence();
+        __syncthreads();
+        uint32_t* counter = p.dec_counters + (int64_t)(it.part_slot - it.chunk) * p.Hkv + kvh;
+        if (threadIdx.x == 0) last_s = (atomicAdd(counter, 1u) == (uint32_t)(it.n_chunks - 1)) ? 1 : 0;
+        __syncthreads();
+        if (last_s) {
+            __threadfence();
+            for (int idx = threadIdx.x; idx < G * (D / 4); idx += NWARPS * 32) {
+                const int head = idx / (D / 4), d = (idx % (D / 4)) * 4;
+                merge_partials<D>(p, it.q_row, it.part_slot - it.chunk, it.n_chunks, kvh * G + head, d, d == 0);
+            }
+            if (threadIdx.x == 0) *counter = 0u;
+        }
+    }
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -227,46 +298,7 @@ __global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
     const CombineItem it = p.comb_items[blockIdx.x];
     const int hq = blockIdx.y;
     asm volatile("griddepcontrol.wait;" ::: "memory");     // the decode grid has completed and its partials are visible
-    const int d = threadIdx.x * 4;
-    // Partials are fetched eight chunks at a time with independent loads (a dependent load per chunk
-    // would cost a memory round trip each) and folded into a running (M, L, acc) in chunk order.
-    constexpr int GROUP = 8;
-    float M = -INFINITY, L = 0.f;
-    float4 acc = make_float4(0.f, 0.f, 0.f, 0.f);
-    for (int c0 = 0; c0 < it.n_chunks; c0 += GROUP) {
-        float2 ml[GROUP];
-        float4 v[GROUP];
-#pragma unroll
-        for (int i = 0; i < GROUP; ++i)
-            if (c0 + i < it.n_chunks) {
-                const int64_t pr = (int64_t)(it.part_first + c0 + i) * p.Hq + hq;
-                ml[i] = __ldg(reinterpret_cast<const float2*>(p.part_ml + pr * 2));
-                v[i] = __ldg(reinterpret_cast<const float4*>(p.part_o + pr * D + d));
-            }
-        float Mg = M;
-#pragma unroll
-        for (int i = 0; i < GROUP; ++i)
-            if (c0 + i < it.n_chunks) Mg = fmaxf(Mg, ml[i].x);
-        const float fold = fast_exp2(M - Mg);               // 0 on the first group (M = -inf)
-        L *= fold;
-        acc.x *= fold; acc.y *= fold; acc.z *= fold; acc.w *= fold;
-        M = Mg;
-#pragma unroll
-        for (int i = 0; i < GROUP; ++i)
-            if (c0 + i < it.n_chunks) {
-                const float f = fast_exp2(ml[i].x - M);
-                L += ml[i].y * f;
-                acc.x += v[i].x * f; acc.y += v[i].y * f; acc.z += v[i].z * f; acc.w += v[i].w * f;
-            }
-    }
-    const float inv = 1.f / L;
-    __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
-    __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
-    uint2 packed;
-    packed.x = *reinterpret_cast<uint32_t*>(&lo);
-    packed.y = *reinterpret_cast<uint32_t*>(&hi);
-    *reinterpret_cast<uint2*>(p.out + ((int64_t)it.q_row * p.Hq + hq) * D + d) = packed;
-    if (p.lse && threadIdx.x == 0) p.lse[(int64_t)it.q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
+    merge_partials<D>(p, it.q_row, it.part_first, it.n_chunks, hq, threadIdx.x * 4, threadIdx.x == 0);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -429,6 +461,8 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
             DecodeItem& it = pl.items[pl.n_items++];
             it.seq = s;
             it.q_row = s;
+            it.n_chunks = (int32_t)n;
+            it.pad = 0;
             it.kv_begin = (int32_t)(c * per * B);
             it.kv_end = (int32_t)(((c + 1) * per * B < lc) ? (c + 1) * per * B : lc);
             it.part_slot = n > 1 ? first + (int32_t)c : -1;
@@ -473,6 +507,8 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     // in the same call.
     p.part_o = reinterpret_cast<float*>(su.base + kStaticPlanBytes);
     p.part_ml = reinterpret_cast<float*>(su.base + kStaticPlanBytes + part_o_bytes);
+    p.dec_counters = nullptr;     // this entry point keeps the separate combine kernel: nothing in the array has to start at zero
+    p.pre_queue = nullptr;
     p.err = nullptr;
     if (launch_decode(p, D, pl.n_items, stream) != cudaSuccess) return CF_ERR_CUDA;
     if (launch_combine(p, D, pl.n_comb, stream) != cudaSuccess) return CF_ERR_CUDA;

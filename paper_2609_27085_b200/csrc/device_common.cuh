@@ -29,6 +29,7 @@ struct AttnParams {
     const PrefillTcItem* pre_tc_items;
     float* part_o;                    // [slot, Hq, D] fp32 un-normalised partial outputs
     float* part_ml;                   // [slot, Hq, 2] running max (log2 domain) and sum
+    uint32_t* dec_counters;           // [first slot of a split sequence, Hkv] chunks finished; null: the combine kernel merges
     float* pre_part_o;                // [row slot, D] fp32 partial rows of KV-split prefill items
     float* pre_part_ml;               // [row slot, 2]
     const PrefillCombineItem* pre_comb_items;

@@ -111,6 +111,8 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             it.kv_end = (int32_t)std::min<int64_t>((c + 1) * per * B, lc);
             it.part_slot = n > 1 ? first + (int32_t)c : -1;
             it.chunk = (int32_t)c;
+            it.n_chunks = (int32_t)n;
+            it.pad = 0;
             plan->decode.push_back(it);
         }
     }

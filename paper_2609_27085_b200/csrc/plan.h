@@ -18,6 +18,8 @@ struct DecodeItem {        // one (decode sequence, KV chunk); the kernel adds t
     int32_t kv_end;        // one past the last token (== context_len for the last chunk)
     int32_t part_slot;     // partial slot to write, or -1: the only chunk, write `out` directly
     int32_t chunk;         // index of this chunk within its sequence
+    int32_t n_chunks;      // chunks of the sequence (its partial slots are part_slot - chunk + [0, n_chunks))
+    int32_t pad;
 };
 
 struct CombineItem {       // one decode sequence that was split
