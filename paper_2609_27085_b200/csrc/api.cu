@@ -55,6 +55,7 @@ struct cf_ctx {
     size_t workspace_bytes = 0;
     bool workspace_fixed = false;
     uint32_t* err_dev = nullptr;
+    bool fused_combine = true; // split-K merge inside the decode kernel (CF_FUSED_COMBINE=0: the separate combine kernel)
     bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
@@ -306,7 +307,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
     p.part_o = (float*)((uint8_t*)ws + W.dec_o);
     p.part_ml = (float*)((uint8_t*)ws + W.dec_ml);
-    const bool fused_combine = (size_t)n.n_part_slots * desc->num_kv_heads * sizeof(uint32_t) <= kCounterBytes;
+    const bool fused_combine = c->fused_combine && (size_t)n.n_part_slots * desc->num_kv_heads * sizeof(uint32_t) <= kCounterBytes;
     p.dec_counters = fused_combine ? (uint32_t*)ws : nullptr;
     p.pre_part_o = (float*)((uint8_t*)ws + W.pre_o);
     p.pre_part_ml = (float*)((uint8_t*)ws + W.pre_ml);
@@ -432,6 +433,10 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
     c->cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
+    {
+        const char* v = std::getenv("CF_FUSED_COMBINE");
+        c->fused_combine = !(v && v[0] == '0' && v[1] == 0);
+    }
     {
         const char* v = std::getenv("CF_OVERLAP");          // spatial sequence unless CF_OVERLAP=0
         c->overlap = !(v && v[0] == '0' && v[1] == 0);

@@ -239,6 +239,29 @@ def test_property_random_batches():
         run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True))
 
 
+def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge(monkeypatch):
+    """The split-K merge runs inside the decode kernel by default; CF_FUSED_COMBINE=0 (read when the context is
+    created) keeps the separate combine kernel.  Same merge routine, same chunk order: identical bits."""
+    sc = small(47, 32, 8, 128, [9000, 5000, 300, 16000, 2047], [[1, 1, 1, 1, 1]], NB=4096)
+    b = sc.batches[0]
+    fused = GpuScenario(sc)
+    fused.append(b)
+    o1, l1 = fused.attend(b)
+    assert cf.cf_get_last_launch_count(fused.ctx) == 1
+    monkeypatch.setenv("CF_FUSED_COMBINE", "0")
+    sep = GpuScenario(sc)
+    monkeypatch.delenv("CF_FUSED_COMBINE")
+    sep.append(b)
+    o2, l2 = sep.attend(b)
+    assert cf.cf_get_last_launch_count(sep.ctx) == 2
+    assert np.array_equal(o1, o2) and np.array_equal(l1, l2)
+    for _ in range(3):                       # the ticket counters are back at zero after every launch
+        o3, l3 = fused.attend(b)
+        assert np.array_equal(o1, o3) and np.array_equal(l1, l3)
+    fused.close()
+    sep.close()
+
+
 def test_more_prefill_items_than_sms():
     """A chunk whose q tiles x head pairs exceed the SM count (11 tiles x 16 pairs + 2 x 16 = 208 items, ragged
     last tiles): every persistent CTA works through several items, in the serial and in the spatial sequence,
