@@ -348,10 +348,11 @@ float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
                      int32_t num_sms)
 {
-    // Constants fitted to CUDA-event times of the kernels on a B200: split-K decode sustains
-    // ~7.1 TB/s on top of ~17 us of launch, ramp and tail; the combine launch is ~10 us; one tcgen05
+    // Constants fitted to CUDA-event times of the kernels on a B200: split-K decode (with the merge of the
+    // partials fused in) sustains ~7.56 TB/s on top of ~22 us of launch, ramp and tail; the separate combine
+    // launch, when it is used, ~8 us, reported as 0 here because the default path has none; one tcgen05
     // prefill item costs ~8 us plus ~1.9 us per 128-token KV tile; the mma.sync path runs ~220 TFLOP/s.
-    constexpr double kDecodeFixedUs = 17.0, kDecodeBytesPerUs = 7.1e6, kCombineUs = 10.0;
+    constexpr double kDecodeFixedUs = 22.0, kDecodeBytesPerUs = 7.56e6, kCombineUs = 0.0;
     constexpr double kTcItemFixedUs = 8.0, kTcTileUs = 1.9, kMmaFlopsPerUs = 220e6, kLaunchUs = 4.0;
     Estimate e;
     const int32_t S = (int32_t)plan.q_start.size() - 1;
