@@ -141,17 +141,24 @@ cf_status cf_host_steps_flush(cf_ctx* ctx, void* cuda_stream);
  * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
 cf_status cf_get_async_status(cf_ctx* ctx);
 
-/* Section 5 names two executor backends: the chunked mixed-batch path (time-multiplexed, the default
- * here: one launch sequence on the caller's stream) and a spatial partition of the node between prefill
- * and decode.  cf_set_overlap(ctx, n) with n > 0 selects the spatial variant for later cf_mixed_attention
- * calls that hold both kinds of work: n persistent prefill CTAs (one per SM; n = 1 means the library's
- * default share of the SMs) are enqueued first on a context-owned side stream; the caller's stream waits,
- * with a stream memory operation, until they hold their SMs, then runs decode + combine on the SMs left
- * over, and behind them a second prefill grid that draws from the same work queue, so the SMs decode
- * frees join the prefill.  The side stream is joined back before the call returns, so the caller still
- * sees one stream.  Results are bit-identical to the default.  n = 0 switches back.  The environment
- * variables CF_OVERLAP=1 and CF_SPATIAL_SMS=n set the initial values.  Per-kernel timing (cf_set_timing)
- * forces the serial sequence. */
+/* Section 5 names two executor backends: the chunked mixed-batch path (time-multiplexed) and a spatial
+ * partition of the node between prefill and decode.  Both are launch sequences of cf_mixed_attention; a
+ * batch that holds both kinds of work runs the spatial one unless it is switched off.  The same plan gives the
+ * same bits in either sequence (planned calls); an unplanned call plans for the sequence it will run (the
+ * spatial one balances the prefill items over its first grid's SMs and may cut other items into KV ranges), so
+ * across sequences unplanned results agree to rounding.
+ *   cf_set_overlap(ctx, 0): serial sequence, decode -> (combine) -> prefill -> (prefill combine) on the
+ *     caller's stream alone.
+ *   cf_set_overlap(ctx, n), n > 0 (the initial state is n = 1): n persistent prefill CTAs, one per SM (n = 1:
+ *     the library's default share of the SMs), are enqueued first on a context-owned side stream; the caller's
+ *     stream waits, with a stream memory operation, until they hold their SMs, then runs decode on the SMs
+ *     left over, and behind it a second prefill grid that draws from the same work queue, so the SMs decode
+ *     frees join the prefill.  The side stream is forked from and joined back into the caller's stream inside
+ *     the call, so the caller still sees one stream.
+ * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n.  cf_set_timing and cf_mixed_step_host
+ * use the serial sequence.  Other switches read at cf_create (debugging aids): CF_FUSED_COMBINE=0 (separate
+ * combine kernel), CF_PREFILL_MMA=1 (mma.sync prefill kernel), CF_PREFILL_SPLIT=k, CF_DECODE_WAVES,
+ * CF_DECODE_MIN_CHUNK_PAGES. */
 cf_status cf_set_overlap(cf_ctx* ctx, int n);
 
 /* Debug aid (synchronous): checks every block-table entry that cf_kv_append / cf_mixed_attention would

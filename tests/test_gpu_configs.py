@@ -28,6 +28,41 @@ def test_config5_sweep_points(budget, n):
     print(run_and_check(syn.config5_sweep_point(budget, n), max_prefill_rows=8, check_append=False))
 
 
+@pytest.mark.parametrize("make", [lambda: syn.config3_chat(iterations=(3,)), lambda: syn.config5_sweep_point(2048, 3)])
+def test_launch_sequences_agree_bit_for_bit_on_one_plan_at_full_size(make):
+    """One plan of a full-size mixed batch run as the serial sequence, the default spatial sequence and with a
+    20-CTA front grid (every CTA works through many items, the second grid takes part): identical output
+    and lse bits.  (Unplanned calls plan per launch sequence - the spatial one balances the prefill items
+    over the front grid's SMs and may cut other items into KV ranges - so across sequences they agree to
+    rounding, not to the bit; each of them is held to the oracle by the tests above.)"""
+    import numpy as np
+    import torch
+    import paper_2609_27085_b200 as cf
+    from harness import GpuScenario, to_dev_bf16, to_host_bits
+    sc = make()
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    bt = torch.from_numpy(b.block_table).cuda()
+    q = to_dev_bf16(b.q)
+    plan = cf.cf_plan_create(g.ctx, g.desc, b.context_len, b.query_len, b.max_blocks)
+    outs = []
+    for mode in (0, 1, 20):
+        cf.cf_set_overlap(g.ctx, mode)
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((b.total_q, sc.geom.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+        cf.cf_mixed_attention_planned(plan, q, g.k, g.v, bt, out, lse)
+        torch.cuda.synchronize()
+        outs.append((to_host_bits(out), lse.cpu().numpy()))
+    cf.cf_set_overlap(g.ctx, 1)
+    assert np.isfinite(outs[0][1]).all()
+    for o, l in outs[1:]:
+        assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    cf.cf_plan_destroy(plan)
+    g.close()
+
+
 def test_paper_context_limit_128k():
     """The paper's workers run a 128K-token context with 512 reserved (Section 6.1): one decode sequence
     at that limit, one at a page boundary below it, and a 300-token prefill chunk that ends at the limit."""
