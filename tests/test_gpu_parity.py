@@ -262,15 +262,17 @@ def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge(monkeypatch):
     sep.close()
 
 
-def test_more_prefill_items_than_sms():
+def test_more_prefill_items_than_sms(monkeypatch):
     """A chunk whose q tiles x head pairs exceed the SM count (11 tiles x 16 pairs + 2 x 16 = 208 items, ragged
     last tiles): every persistent CTA works through several items, in the serial and in the spatial sequence,
-    with and without decode sequences beside it."""
+    with and without decode sequences beside it (KV split off, so that all sequences run one plan)."""
     for qlen in ([[1300, 130]], [[1300, 130, 1, 1, 1]]):
         prefix = [700, 40, 5000, 300, 17][:len(qlen[0])]
         sc = small(41, 32, 8, 128, prefix, qlen, NB=2048)
         b = sc.batches[0]
+        monkeypatch.setenv("CF_PREFILL_SPLIT", "1")
         g = GpuScenario(sc)
+        monkeypatch.delenv("CF_PREFILL_SPLIT")
         g.append(b)
         outs = []
         for mode in (0, 1, 5):
@@ -288,10 +290,14 @@ def test_more_prefill_items_than_sms():
         g.close()
 
 
-def test_spatial_sequence_is_bit_identical_to_the_serial_sequence():
+def test_spatial_sequence_is_bit_identical_to_the_serial_sequence(monkeypatch):
+    """With the planner's KV split switched off the plan does not depend on the launch sequence, and then
+    neither does any bit of the result: which CTA runs an item, and when, never matters."""
     sc = small(29, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
     b = sc.batches[0]
+    monkeypatch.setenv("CF_PREFILL_SPLIT", "1")
     g = GpuScenario(sc)
+    monkeypatch.delenv("CF_PREFILL_SPLIT")
     g.append(b)
     cf.cf_set_overlap(g.ctx, 0)
     serial, lse0 = g.attend(b)
