@@ -62,6 +62,18 @@ def test_long_split_decode_uses_partials_and_combine():
     run_and_check(sc)
 
 
+@pytest.mark.parametrize("Hq,Hkv,D", [(16, 2, 64), (8, 1, 128), (64, 8, 128)])
+def test_many_chunk_merge_other_geometries(Hq, Hkv, D):
+    """Sequences cut into up to ~40 chunks (the fused merge folds its partials eight at a time) beside
+    one- and two-chunk sequences, for head_dim 64, a single KV head and group size 8."""
+    sc = small(17, Hq, Hkv, D, [20000 - 1, 9000 - 1, 511, 513, 4100], [[1, 1, 1, 1, 1]], NB=4096)
+    d = cf.make_desc(Hq, Hkv, D, 16, 4096)
+    b = sc.batches[0]
+    _, dec, comb, _, parts = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks)
+    assert max(c[2] for c in comb) > 8
+    run_and_check(sc)
+
+
 def test_chunking_invariance_on_gpu():
     """One 300-token unit vs. three ragged units (Section 4.4): same rows within tolerance, and both match the oracle."""
     one = small(15, 8, 2, 64, [77], [[300]])
