@@ -56,7 +56,7 @@ struct cf_ctx {
     bool workspace_fixed = false;
     uint32_t* err_dev = nullptr;
     bool fused_combine = true; // split-K merge inside the decode kernel (CF_FUSED_COMBINE=0: the separate combine kernel)
-    bool use_tc = true;        // chunked prefill on tcgen05 when the geometry allows (CF_PREFILL_MMA=1 forces mma.sync)
+    bool use_tc = true;        // chunked prefill on tcgen05 (CF_PREFILL_MMA=1 forces the mma.sync kernel)
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
     cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
@@ -372,7 +372,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, stream);
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
+        if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
     } else {
         if (tc) cudaEventRecord(tc->ev[0], stream);
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
@@ -381,7 +381,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[2], stream);
         if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
-        if (e == cudaSuccess) e = launch_prefill_combine(p, n.n_pre_comb, stream);
+        if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
     c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;

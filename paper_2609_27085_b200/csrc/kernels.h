@@ -30,7 +30,7 @@ cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaS
 constexpr int kPrefillMmaTileRows = 64;
 cudaError_t launch_prefill_mma(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 
-// tcgen05 / tensor-memory chunked prefill (head_dim 128): `n_ctas` persistent CTAs draw the `n_items`
+// tcgen05 / tensor-memory chunked prefill (head_dim 64 or 128): `n_ctas` persistent CTAs draw the `n_items`
 // PrefillTcItems from the ticket counter p.pre_queue, which `queue_ctas` CTAs share in total (several
 // launches may draw from one counter; the last CTA to leave resets it).  Ticket t stands for item
 // ticket_base + t; with first_static set, CTA b starts on item b without a draw (then ticket_base = n_ctas of
@@ -41,7 +41,7 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
                               int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
 
 // merges the fp32 partials of KV-split prefill items into `out` (one CTA per split item)
-cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream);
+cudaError_t launch_prefill_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 // one CTA whose bounded wait must expire: sets *err and returns normally (status-path self-test)
 cudaError_t launch_wait_selftest(uint32_t* err, cudaStream_t stream);
 

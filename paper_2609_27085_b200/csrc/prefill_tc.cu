@@ -1,5 +1,5 @@
 // Chunked-prefill attention on the 5th-generation tensor cores (tcgen05.mma, accumulators in
-// tensor memory), head_dim 128.
+// tensor memory), head_dim 128 or 64 (template parameter D; the sizes quoted below are those of D = 128).
 //
 // A work item = two 128-row q tiles that share a KV head (two query heads of one group over the same
 // rows; for G = 1 two consecutive row tiles of one head), so every K/V tile fetched into shared memory
@@ -35,11 +35,9 @@ using namespace tc;
 
 namespace {
 
-constexpr int D = 128;
 constexpr int QT = 128;                    // rows per q tile
 constexpr int KT = 128;                    // tokens per K/V tile
 constexpr int HALF_BYTES = 128 * 128;      // [128 rows][64 elements] bf16
-constexpr int TILE_BYTES = 2 * HALF_BYTES; // 32 KB
 constexpr int KV_STAGES = 2;
 constexpr int NTHREADS = 384;
 // Register hand-over (setmaxnreg).  The kernel launches with LAUNCH_REGS registers per thread; the
@@ -48,11 +46,20 @@ constexpr int NTHREADS = 384;
 // cover the growth or the kernel never returns; the launcher also checks the compiled register count.
 constexpr int LAUNCH_REGS = 168, REGS_ROLE = 136, REGS_SOFTMAX = 184;
 static_assert(4 * (LAUNCH_REGS - REGS_ROLE) >= 8 * (REGS_SOFTMAX - LAUNCH_REGS), "setmaxnreg.inc would block forever");
-constexpr uint32_t SMEM_Q = 0;
-constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
-constexpr uint32_t SMEM_V = SMEM_K + KV_STAGES * TILE_BYTES;
-constexpr uint32_t SMEM_TOTAL = SMEM_V + KV_STAGES * TILE_BYTES;   // 192 KB
-constexpr uint32_t TM_S = 0, TM_O = 256;   // column offsets; tile t adds 128 * t
+// Per head dimension (128 or 64): a Q, K or V tile is 128 rows x D elements, stored as D / 64 halves of
+// [128 rows][64 elements]; the O accumulator of a q tile takes D fp32 columns of tensor memory.
+template <int D>
+struct Geo {
+    static_assert(D == 64 || D == 128, "head_dim 64 or 128");
+    static constexpr int HALVES = D / 64;
+    static constexpr int TILE_BYTES = HALVES * HALF_BYTES;                 // 32 KB / 16 KB
+    static constexpr uint32_t SMEM_Q = 0;
+    static constexpr uint32_t SMEM_K = 2 * TILE_BYTES;
+    static constexpr uint32_t SMEM_V = SMEM_K + KV_STAGES * TILE_BYTES;
+    static constexpr uint32_t SMEM_TOTAL = SMEM_V + KV_STAGES * TILE_BYTES;   // 192 KB / 96 KB
+    static constexpr int KS = D / 16;                                      // K = 16 steps of S = Q K^T
+};
+constexpr uint32_t TM_S = 0, TM_O = 256;   // column offsets: S_t at TM_S + 128 t, O_t at TM_O + D t
 
 struct Bars {
     uint64_t q_full, q_empty;
@@ -168,11 +175,14 @@ __device__ __forceinline__ void derive_item(ItemCtx& c)
 // to two K/V tiles and one item context ahead, the issuer puts the first S = Q K^T of the next item
 // right behind the last P V of the current one, and a softmax thread goes from the epilogue of one item
 // straight to the first tile of the next.
+template <int D>
 __global__ void __launch_bounds__(NTHREADS, 1)
 prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_k,
                   const __grid_constant__ CUtensorMap map_v, const AttnParams p, const int n_items, const int queue_ctas,
                   const int first_static, const int ticket_base, uint32_t* const resident)
 {
+    constexpr int HALVES = Geo<D>::HALVES, TILE_BYTES = Geo<D>::TILE_BYTES, KS = Geo<D>::KS;
+    constexpr uint32_t SMEM_Q = Geo<D>::SMEM_Q, SMEM_K = Geo<D>::SMEM_K, SMEM_V = Geo<D>::SMEM_V;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(16) ItemCtx ctx_s[2];
     __shared__ __align__(8) Bars bars;
@@ -255,15 +265,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
-                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
+                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
                 if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
-                const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
+                const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
-                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 4096);
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 16 * D * 2);
                 __syncwarp();
-                if (lane < 2 * np)
-                    tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane & 1) * 64, 0, kvh, my_pid,
+                if (lane < HALVES * np)
+                    tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane % HALVES) * 64, 0, kvh, my_pid,
                                 smem_u32(&bars.v_full[stage]));
             }
             ok = __all_sync(0xffffffffu, ok);
@@ -330,7 +340,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 mbar_arrive_expect_tx(smem_u32(&bars.q_full), nq * TILE_BYTES);
                 for (int t = 0; t < 2; ++t)
                     if (it.n_rows[t] > 0)
-                        for (int h = 0; h < 2; ++h)
+                        for (int h = 0; h < HALVES; ++h)
                             tma_load_3d(smem + SMEM_Q + t * TILE_BYTES + h * HALF_BYTES, &map_q, h * 64, it.head[t],
                                         it.q_row0[t], smem_u32(&bars.q_full));
             }
@@ -344,15 +354,15 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
-                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane >> 1);
+                const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
                 if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
-                const uint32_t dst_off = (lane & 1) * HALF_BYTES + (lane >> 1) * 2048;
+                const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
-                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 4096);
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 16 * D * 2);
                 __syncwarp();
-                if (lane < 2 * np)
-                    tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane & 1) * 64, 0, it.kvh, my_pid,
+                if (lane < HALVES * np)
+                    tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane % HALVES) * 64, 0, it.kvh, my_pid,
                                 smem_u32(&bars.k_full[stage]));
                 if (lane == 0 && (j < 5 || j >= n_max - 2)) TR(0, 200 + j);
                 if (j == j_draw) {
@@ -371,36 +381,39 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       } else {
         // =========================================================== MMA issuer
         constexpr uint32_t IDESC_QK = idesc_bf16(128, 128, false);
-        constexpr uint32_t IDESC_PV = idesc_bf16(128, 128, true);
+        constexpr uint32_t IDESC_PV = idesc_bf16(128, D, true);
         constexpr uint64_t HI64 = (uint64_t)desc_hi_sw128(1024) << 32;
         // The issuing lane shares its scheduler with two softmax warps and gets roughly one issue
         // slot in ten, while a 128x128x16 MMA lasts only 64 cycles.  Every shared-memory descriptor
         // (q tile x k-step, K/V stage x k-step) is therefore built once and kept in registers, and the
         // tile / stage indices are compile-time, so that a batch is MMAs back to back.
-        uint64_t qd[2][8], kd[KV_STAGES][8], vd[KV_STAGES][8];
+        uint64_t qd[2][KS], kd[KV_STAGES][KS], vd[KV_STAGES][8];
 #pragma unroll
-        for (int i = 0; i < 2; ++i)
+        for (int i = 0; i < 2; ++i) {
 #pragma unroll
-            for (int ks = 0; ks < 8; ++ks) {
+            for (int ks = 0; ks < KS; ++ks) {
                 const uint32_t off = (uint32_t)(((ks >> 2) * HALF_BYTES + (ks & 3) * 32) >> 4);
                 qd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_Q + i * TILE_BYTES, 16) + off);
                 kd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_K + i * TILE_BYTES, 16) + off);
-                vd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_V + i * TILE_BYTES, HALF_BYTES) + ks * (2048 >> 4));
             }
+#pragma unroll
+            for (int ks = 0; ks < 8; ++ks)
+                vd[i][ks] = HI64 | (desc_lo_sw128(smem + SMEM_V + i * TILE_BYTES, HALF_BYTES) + ks * (2048 >> 4));
+        }
         const uint32_t bar_s[2] = {smem_u32(&bars.s_full[0]), smem_u32(&bars.s_full[1])};
         const uint32_t bar_o[2] = {smem_u32(&bars.o_done[0]), smem_u32(&bars.o_done[1])};
         const uint32_t bar_p[2] = {smem_u32(&bars.p_full[0]), smem_u32(&bars.p_full[1])};
-        auto issue_qk = [&](auto T, auto S) {             // S_t = Q_t K^T over D = 128 (8 steps of K = 16)
+        auto issue_qk = [&](auto T, auto S) {             // S_t = Q_t K^T over the head dimension (D / 16 steps of K = 16)
             constexpr int t = decltype(T)::value, st = decltype(S)::value;
             const uint32_t dS = tmem + TM_S + t * 128;
             umma_ss(dS, qd[t][0], kd[st][0], IDESC_QK, 0u);
 #pragma unroll
-            for (int ks = 1; ks < 8; ++ks) umma_ss(dS, qd[t][ks], kd[st][ks], IDESC_QK, 1u);
+            for (int ks = 1; ks < KS; ++ks) umma_ss(dS, qd[t][ks], kd[st][ks], IDESC_QK, 1u);
             umma_commit(bar_s[t]);
         };
         auto issue_pv = [&](auto T, auto S, int n_steps, uint32_t acc0) {   // O_t (+)= P_t V, one step per loaded page
             constexpr int t = decltype(T)::value, st = decltype(S)::value;
-            const uint32_t dO = tmem + TM_O + t * 128, aP = tmem + TM_S + t * 128;
+            const uint32_t dO = tmem + TM_O + t * D, aP = tmem + TM_S + t * 128;
             umma_ts(dO, aP, vd[st][0], IDESC_PV, acc0);
             if (n_steps == 8) {
 #pragma unroll
@@ -503,8 +516,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
                 // that a zero probability never multiplies a NaN
                 const int r0 = Lc - (jb + j) * KT, r1 = np * 16;
-                for (int idx = 0; idx < (r1 - r0) * 16; ++idx) {
-                    const int r = r0 + (idx >> 4), c = idx & 15;
+                for (int idx = 0; idx < (r1 - r0) * (D / 8); ++idx) {
+                    const int r = r0 + idx / (D / 8), c = idx % (D / 8);
                     uint8_t* dst = smem_raw + ((smem + SMEM_V + st * TILE_BYTES) - smem_u32(smem_raw)) +
                                    (c >> 3) * HALF_BYTES + r * 128 + (c & 7) * 16;
                     *reinterpret_cast<uint4*>(dst) = make_uint4(0u, 0u, 0u, 0u);
@@ -549,7 +562,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const int t = (warp - 4) >> 2;
       const int row = (warp & 3) * 32 + lane;
       const uint32_t lanes = lane_field(warp);
-      const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * 128 + lanes;
+      const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * D + lanes;
       const float sc = p.scale_log2;
       TR_DECL;
       if ((warp & 3) == 0 && lane == 0) TR(2 + t, 100);
@@ -638,7 +651,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     if (!ok) break;
                     tc_fence_after();
 #pragma unroll 1
-                    for (int c = 0; c < 8; ++c) {
+                    for (int c = 0; c < D / 16; ++c) {
                         float ov[16];
                         tmem_ld16(tO + c * 16, reinterpret_cast<uint32_t*>(ov));
                         tmem_wait_ld();
@@ -669,7 +682,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int64_t pslot = (int64_t)it_part_slot + (int64_t)row * it_part_k + it_part_c;
             float* prow = p.pre_part_o + pslot * D;
 #pragma unroll
-            for (int c = 0; c < 4; ++c) {
+            for (int c = 0; c < D / 32; ++c) {
                 float ov[32];
                 tmem_ld32(tO + c * 32, reinterpret_cast<uint32_t*>(ov));
                 tmem_wait_ld();
@@ -722,8 +735,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 // Merges the partials of KV-split prefill items: for every row of the item's q tiles,
 //   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
 // in fixed range order.  One warp per row (8 rows per CTA, 32 CTAs per split item), one float4 of the
-// row per lane; the partials of a row are fetched with independent loads (part_k <= 8).
+// row per lane (D / 4 lanes take part); the partials of a row are fetched with independent loads (part_k <= 8).
 constexpr int kMaxSplit = 8;
+template <int D>
 __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p)
 {
     const PrefillCombineItem it = p.pre_comb_items[blockIdx.x >> 5];
@@ -734,13 +748,14 @@ __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p
     if (r >= it.n_rows[t]) return;
     const int k = it.part_k;
     const int64_t s0 = (int64_t)it.part_slot[t] + (int64_t)r * k;
+    const bool holds = lane < D / 4;                 // head_dim 64: half of the lanes hold a float4 of the row
     float2 ml[kMaxSplit];
     float4 v[kMaxSplit];
 #pragma unroll
     for (int c = 0; c < kMaxSplit; ++c)
         if (c < k) {
             ml[c] = __ldg(reinterpret_cast<const float2*>(p.pre_part_ml + (s0 + c) * 2));
-            v[c] = __ldg(reinterpret_cast<const float4*>(p.pre_part_o + (s0 + c) * D + lane * 4));
+            v[c] = holds ? __ldg(reinterpret_cast<const float4*>(p.pre_part_o + (s0 + c) * D + lane * 4)) : make_float4(0.f, 0.f, 0.f, 0.f);
         }
     float M = -INFINITY;
 #pragma unroll
@@ -760,11 +775,11 @@ __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p
     w.x = pack_bf16(acc.x * inv, acc.y * inv);
     w.y = pack_bf16(acc.z * inv, acc.w * inv);
     const int64_t orow = (int64_t)(it.q_row0[t] + r) * p.Hq + it.head[t];
-    *reinterpret_cast<uint2*>(p.out + orow * D + lane * 4) = w;
+    if (holds) *reinterpret_cast<uint2*>(p.out + orow * D + lane * 4) = w;
     if (p.lse && lane == 0) p.lse[orow] = (M + log2f(L)) * kLn2;
 }
 
-cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_t stream)
+cudaError_t launch_prefill_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
 {
     if (n_items <= 0) return cudaSuccess;
     cudaLaunchConfig_t cfg = {};
@@ -776,7 +791,7 @@ cudaError_t launch_prefill_combine(const AttnParams& p, int n_items, cudaStream_
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_combine_kernel, p);
+    return head_dim == 128 ? cudaLaunchKernelEx(&cfg, prefill_combine_kernel<128>, p) : cudaLaunchKernelEx(&cfg, prefill_combine_kernel<64>, p);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -825,7 +840,7 @@ EncodeTiledFn get_encode()
 }
 
 // pool viewed as (d, token-in-page, head, block); one box = 64 elements x 16 tokens of one head of one page
-bool encode_pool(CUtensorMap* m, const void* base, int num_blocks, int Hkv, int64_t s_block, int64_t s_head, int64_t s_token)
+bool encode_pool(CUtensorMap* m, const void* base, int D, int num_blocks, int Hkv, int64_t s_block, int64_t s_head, int64_t s_token)
 {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -838,7 +853,7 @@ bool encode_pool(CUtensorMap* m, const void* base, int num_blocks, int Hkv, int6
 }
 
 // q viewed as (d, head, row); one box = 64 elements x 1 head x 128 rows; rows past the end read as zero
-bool encode_q(CUtensorMap* m, const void* base, int total_rows, int Hq)
+bool encode_q(CUtensorMap* m, const void* base, int D, int total_rows, int Hq)
 {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -854,31 +869,31 @@ bool encode_q(CUtensorMap* m, const void* base, int total_rows, int Hq)
 
 bool prefill_tc_supported(const cf_cache_desc* d)
 {
-    // TMA needs 16-byte aligned strides (checked for every descriptor) and a 128-element head
-    return d->head_dim == D && d->block_size == 16;
+    // TMA needs 16-byte aligned strides (checked for every descriptor); rows of 64 or 128 elements
+    return (d->head_dim == 128 || d->head_dim == 64) && d->block_size == 16;
 }
 
-cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
-                              int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream)
+namespace {
+
+template <int D>
+cudaError_t launch_prefill_tc_t(const CUtensorMap& mq, const CUtensorMap& mk, const CUtensorMap& mv, const AttnParams& p,
+                                int n_items, int n_ctas, int queue_ctas, int first_static, int ticket_base, uint32_t* resident,
+                                cudaStream_t stream)
 {
-    if (n_items <= 0 || n_ctas <= 0) return cudaSuccess;
-    CUtensorMap mq, mk, mv;
-    if (!encode_q(&mq, p.q, total_q_rows, p.Hq) ||
-        !encode_pool(&mk, p.k_cache, desc->num_blocks, p.Hkv, p.ks_block, p.ks_head, p.ks_token) ||
-        !encode_pool(&mv, p.v_cache, desc->num_blocks, p.Hkv, p.vs_block, p.vs_head, p.vs_token))
-        return cudaErrorInvalidValue;
-    const size_t smem = SMEM_TOTAL + 1024;
+    const size_t smem = Geo<D>::SMEM_TOTAL + 1024;
+    // The register hand-over inside the kernel (setmaxnreg) is sized for LAUNCH_REGS registers per thread at
+    // launch; with any other count a grow request could block forever, so such a build is never launched.
     static int regs_ok = -1;
     if (regs_ok < 0) {
         cudaFuncAttributes fa;
-        regs_ok = (cudaFuncGetAttributes(&fa, prefill_tc_kernel) == cudaSuccess && fa.numRegs == LAUNCH_REGS) ? 1 : 0;
+        regs_ok = (cudaFuncGetAttributes(&fa, prefill_tc_kernel<D>) == cudaSuccess && fa.numRegs == LAUNCH_REGS) ? 1 : 0;
     }
-    if (!regs_ok) return cudaErrorLaunchOutOfResources;   // the register hand-over arithmetic would not hold
+    if (!regs_ok) return cudaErrorLaunchOutOfResources;
     static bool configured[64] = {};
     int dev = 0;
     cudaGetDevice(&dev);
     if (dev >= 0 && dev < 64 && !configured[dev]) {
-        cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
         configured[dev] = true;
     }
@@ -894,7 +909,23 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
     attr[0].val.programmaticStreamSerializationAllowed = 1;
     cfg.attrs = attr;
     cfg.numAttrs = 1;
-    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel, mq, mk, mv, p, n_items, queue_ctas, first_static, ticket_base, resident);
+    return cudaLaunchKernelEx(&cfg, prefill_tc_kernel<D>, mq, mk, mv, p, n_items, queue_ctas, first_static, ticket_base, resident);
+}
+
+}  // namespace
+
+cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
+                              int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream)
+{
+    if (n_items <= 0 || n_ctas <= 0) return cudaSuccess;
+    const int D = desc->head_dim;
+    CUtensorMap mq, mk, mv;
+    if (!encode_q(&mq, p.q, D, total_q_rows, p.Hq) ||
+        !encode_pool(&mk, p.k_cache, D, desc->num_blocks, p.Hkv, p.ks_block, p.ks_head, p.ks_token) ||
+        !encode_pool(&mv, p.v_cache, D, desc->num_blocks, p.Hkv, p.vs_block, p.vs_head, p.vs_token))
+        return cudaErrorInvalidValue;
+    return D == 128 ? launch_prefill_tc_t<128>(mq, mk, mv, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream)
+                    : launch_prefill_tc_t<64>(mq, mk, mv, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream);
 }
 
 }  // namespace cf
