@@ -34,6 +34,18 @@ def test_prefill_only_ragged(Hq, Hkv, D):
     run_and_check(small(5, Hq, Hkv, D, prefix, [qlen]))
 
 
+@pytest.mark.parametrize("D", [64, 128])
+def test_mma_sync_prefill_kernel_behind_its_switch(D, monkeypatch):
+    """CF_PREFILL_MMA=1 (read when the context is created) selects the warp-level mma.sync prefill kernel."""
+    monkeypatch.setenv("CF_PREFILL_MMA", "1")
+    ctx = cf.cf_create(0)
+    monkeypatch.delenv("CF_PREFILL_MMA")
+    try:
+        run_and_check(small(5, 8, 2, D, [0, 100, 700, 33], [[129, 64, 200, 1]]), ctx=ctx)
+    finally:
+        cf.cf_destroy(ctx)
+
+
 def test_mixed_shuffled_order_with_empty_sequences():
     prefix = [10, 0, 500, 77, 0, 2000, 31, 640, 5, 1]
     qlen = [1, 90, 1, 0, 1, 1, 130, 1, 0, 64]
