@@ -248,9 +248,11 @@ def test_bounded_wait_reports_timeout_and_context_survives():
 
 
 def test_property_random_batches():
-    """Random small batches: sequence counts, chunk lengths, prefixes, group sizes, head dims."""
+    """Random small batches: sequence counts, chunk lengths, prefixes, group sizes, head dims, and the launch
+    sequence (serial, default spatial share, a 7-CTA front grid)."""
     rng = np.random.default_rng(2024)
-    for trial in range(24):
+    ctx = cf.cf_create(0)
+    for trial in range(36):
         Hkv = int(rng.choice([1, 2, 4]))
         G = int(rng.choice([1, 2, 4, 8]))
         D = int(rng.choice([64, 128]))
@@ -260,7 +262,9 @@ def test_property_random_batches():
         prefix = [p if q > 0 else max(p, 0) for p, q in zip(prefix, qlen)]
         if sum(qlen) == 0:
             qlen[0] = 1
-        run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True))
+        cf.cf_set_overlap(ctx, int(rng.choice([0, 1, 7])))
+        run_and_check(small(3000 + trial, Hkv * G, Hkv, D, prefix, [qlen], NB=1024, shuffle=True), ctx=ctx)
+    cf.cf_destroy(ctx)
 
 
 def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge(monkeypatch):
