@@ -4,12 +4,15 @@
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--report]
 
 One *step* = one unit of one layer of the chat-like mixed batch: cf_kv_append followed by
-cf_mixed_attention (split-K decode -> combine -> chunked prefill) over 48 decode sequences
+cf_mixed_attention (split-K decode with its merge, chunked prefill) over 48 decode sequences
 (lognormal contexts, median 4096) plus two 512-token prefill chunks that sit on 6144 + 512*t
 cached tokens; steps cycle through the four chunks t = 0..3 of the 2048-token prompts.
 Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank runs
 an independent replica of the batch on its own GPU: the path has no exchange step, so there is no
 data-path collective; the only collective is the max-over-ranks of the device time.
+`value` is measured in the library's default launch sequence (for this batch: a first grid of
+prefill CTAs beside decode); the `serial` key repeats the steps with one kernel after the other,
+which is also the sequence the per-kernel times under `kernels` / `roofline` are taken in.
 
 `--impl reference` times the fp64 CPU oracle (as it stands) on the host cores instead.
 `--report` additionally writes a per-configuration table (all five workload configurations) to
@@ -365,7 +368,7 @@ def run_ours(args):
     if rank == 0:
         dominant = "prefill" if kern.get("prefill", {}).get("ms", 0) >= kern.get("decode", {}).get("ms", 0) else "decode"
         roof = {k: kern[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
-        roof["kernel"] = "prefill_tc_kernel" if dominant == "prefill" else "decode_splitk_kernel+combine_kernel"
+        roof["kernel"] = "prefill_tc_kernel" if dominant == "prefill" else "decode_splitk_kernel (merge of the partials fused in)"
         roof["peak_source"] = peaks["source"] + (" burst bf16" if dominant == "prefill" else " copy")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
                 "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
@@ -378,7 +381,7 @@ def run_ours(args):
                 "e2e": {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps},
                 "serial": {"value": world * tokens / (ms_serial * 1e-3), "unit": UNIT, "ms_per_step": ms_serial / steps,
-                           "note": "cf_set_overlap(0): decode -> combine -> prefill one after the other; `value` is the "
+                           "note": "cf_set_overlap(0): decode -> prefill one after the other; `value` is the "
                                    "library's default sequence (prefill CTAs beside decode, joined per call); the per-kernel "
                                    "times under `kernels` are taken in the serial sequence"},
                 "gpu_launches": launches, "clocks": clk.summary()}
