@@ -336,12 +336,13 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
     if (c->overlap && !c->in_host_step && !tc && has_prefill && (n.n_dec > 0)) {
         // Spatial partition.  `front` persistent prefill CTAs (one per SM: a CTA takes an SM's whole shared
-        // memory) go first, on the side stream; decode + combine on the caller's stream run on the SMs left
-        // over; a second prefill grid behind them on the caller's stream draws from the same ticket counter,
-        // so the SMs that decode frees join the prefill as soon as decode is done.
+        // memory) go first, on the caller's stream; decode runs on the SMs left over, on a context-owned side
+        // stream forked from the caller's; a second prefill grid behind decode on that stream draws from the
+        // same ticket counter, so the SMs that decode frees join the prefill as soon as decode is done; the
+        // side stream is joined back before the prefill combine.
         // Default share: three fifths of the SMs.  When the prefill work dwarfs the decode kernel, sharing the
         // machine no longer pays (the tensor-bound kernel already runs at the power limit): prefill takes
-        // every SM first and decode + combine fill in as its CTAs retire.
+        // every SM first and decode fills in as its CTAs retire.
         int front = c->spatial_sms > 0 ? c->spatial_sms : (n.pre_over_dec > 3.9f ? sms : (sms * 3) / 5);
         if (front > sms) front = sms;
         if (front > n.n_pre_tc) front = n.n_pre_tc;
@@ -349,9 +350,11 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tail > sms) tail = sms;
         second_grid = tail > 0;
         // Decode must not start before the front CTAs hold their SMs (its grid would otherwise fill the
-        // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end):
-        // the front CTAs count themselves in, and the caller's stream waits for that count with a stream
-        // memory operation.  Not used while the stream is being captured.
+        // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end).  The
+        // front grid is enqueued first and on the stream that needs no cross-stream event; on top of that the
+        // front CTAs count themselves in and the side stream waits for that count with a stream memory
+        // operation before decode.  The wait is left out while the stream is being captured (in a graph the
+        // two branches start together and the memory-operation nodes cost more than they return).
         uint32_t* resident = nullptr;
         const StreamMemOps& mo = stream_mem_ops();
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -361,16 +364,16 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         }
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, 1, front, resident, c->side);
-        if (e == cudaSuccess && cudaEventRecord(c->ev_join, c->side) != cudaSuccess) e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, 1, front, resident, stream);
         // only after the front grid has been enqueued without an error, so that the count is certain to arrive
         if (e == cudaSuccess && resident &&
-            mo.wait(stream, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+            mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
-        if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, stream);
+        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, c->side);
+        if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
+        if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
     } else {
