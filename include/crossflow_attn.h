@@ -151,11 +151,12 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  *     caller's stream alone.
  *   cf_set_overlap(ctx, n), n > 0 (the initial state is n = 1): n persistent prefill CTAs, one per SM (n = 1:
  *     the library's default share of the SMs), are enqueued first, on the caller's stream; a context-owned
- *     side stream, forked from the caller's, waits with a stream memory operation until they hold their SMs,
- *     then runs decode on the SMs left over, and behind it a second prefill grid that draws from the same work
- *     queue, so the SMs decode frees join the prefill.  The side stream is joined back into the caller's
- *     stream inside the call, so the caller still sees one stream.
- * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n.  cf_set_timing and cf_mixed_step_host
+ *     side stream, forked from the caller's, runs decode on the SMs left over, and behind it a second prefill
+ *     grid that draws from the same work queue, so the SMs decode frees join the prefill.  The side stream is
+ *     joined back into the caller's stream inside the call, so the caller still sees one stream.
+ * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n, CF_SPATIAL_WAIT=1 (decode waits, with a
+ * stream memory operation, until the first prefill grid's CTAs hold their SMs, instead of relying on the order
+ * of the launches).  cf_set_timing and cf_mixed_step_host
  * use the serial sequence.  Other switches read at cf_create (debugging aids): CF_FUSED_COMBINE=0 (separate
  * combine kernel), CF_PREFILL_MMA=1 (mma.sync prefill kernel), CF_PREFILL_SPLIT=k, CF_DECODE_WAVES,
  * CF_DECODE_MIN_CHUNK_PAGES. */

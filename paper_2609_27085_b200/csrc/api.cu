@@ -62,6 +62,7 @@ struct cf_ctx {
     cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
     cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
     bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
+    bool spatial_wait = false; // CF_SPATIAL_WAIT=1: decode waits (stream memory operation) for the front prefill CTAs to be resident
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
@@ -351,14 +352,15 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         second_grid = tail > 0;
         // Decode must not start before the front CTAs hold their SMs (its grid would otherwise fill the
         // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end).  The
-        // front grid is enqueued first and on the stream that needs no cross-stream event; on top of that the
-        // front CTAs count themselves in and the side stream waits for that count with a stream memory
-        // operation before decode.  The wait is left out while the stream is being captured (in a graph the
-        // two branches start together and the memory-operation nodes cost more than they return).
+        // front grid is therefore enqueued first and on the stream that needs no cross-stream event, which in
+        // every measurement so far is enough.  CF_SPATIAL_WAIT=1 adds a guarantee: the front CTAs count
+        // themselves in and the side stream waits for that count with a stream memory operation before decode
+        // (3-9 us per step; never while the stream is being captured: in a graph the two branches start
+        // together and the memory-operation nodes cost more than they return).
         uint32_t* resident = nullptr;
         const StreamMemOps& mo = stream_mem_ops();
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
-        if (front > 0 && mo.ok && cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
+        if (front > 0 && c->spatial_wait && mo.ok && cudaStreamIsCapturing(stream, &cap) == cudaSuccess && cap == cudaStreamCaptureStatusNone) {
             resident = p.pre_queue + 2;
             if (mo.write(stream, (CUdeviceptr)(uintptr_t)resident, 0u, 0u) != CUDA_SUCCESS) e = cudaErrorUnknown;
         }
@@ -445,6 +447,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
         c->overlap = !(v && v[0] == '0' && v[1] == 0);
     }
     c->spatial_sms = env_int("CF_SPATIAL_SMS", 0);
+    c->spatial_wait = env_int("CF_SPATIAL_WAIT", 0) != 0;
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess &&
@@ -764,7 +767,7 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
         return st;
     }
     // The step is bound by the copies over PCIe, not by the kernels; measured on the chat-like workload the
-    // spatial sequence (side stream, stream memory operations) made it slower (0.38 ms against 0.365 ms).
+    // spatial sequence made it slower (0.40 ms against 0.355 ms).
     c->in_host_step = true;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);

@@ -344,6 +344,28 @@ def test_spatial_sequence_is_bit_identical_to_the_serial_sequence(monkeypatch):
     g.close()
 
 
+def test_spatial_sequence_with_the_resident_wait(monkeypatch):
+    """CF_SPATIAL_WAIT=1 (read when the context is created): decode waits, through a stream memory operation, for
+    the front prefill CTAs; same plan, same bits as without the wait, over repeated calls."""
+    sc = small(31, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
+    b = sc.batches[0]
+    plain = GpuScenario(sc)
+    plain.append(b)
+    o0, l0 = plain.attend(b)
+    monkeypatch.setenv("CF_SPATIAL_WAIT", "1")
+    waited = GpuScenario(sc)
+    monkeypatch.delenv("CF_SPATIAL_WAIT")
+    waited.append(b)
+    for n in (1, 1, 5, 1):
+        cf.cf_set_overlap(waited.ctx, n)
+        o1, l1 = waited.attend(b)
+        if n == 1:
+            assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+    assert cf.cf_get_async_status(waited.ctx) == 0
+    plain.close()
+    waited.close()
+
+
 def test_pipelined_host_steps_keep_their_order():
     """Six host-buffer steps back to back (copies of neighbouring steps overlap the kernels): every
     step's read-back equals the device-buffer path run step by step on a second copy of the caches."""
