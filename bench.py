@@ -487,6 +487,9 @@ def small_case(name: str) -> syn.Scenario:
     if name == "prefill_small":
         geom = syn.Geometry(32, 8, 128, 16, 4096)
         return syn.scenario_from_lengths(name, geom, 44, [3072], [[1024]])
+    if name == "prefill_multi":      # 32 q tiles x 16 head pairs = 512 items: every persistent CTA works through 3-4 of them
+        geom = syn.Geometry(32, 8, 128, 16, 16384)
+        return syn.scenario_from_lengths(name, geom, 45, [8192], [[4096]])
     raise SystemExit(f"unknown case {name}")
 
 
@@ -510,7 +513,7 @@ def run_case(args):
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run a reduced workload (decode_small | prefill_small) and exit")
+    ap.add_argument("--case", default=None, help="run a reduced workload (decode_small | prefill_small | prefill_multi) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
