@@ -30,7 +30,7 @@ static constexpr int kHostStages = 3;
 struct HostStage {
     uint8_t* dev = nullptr;
     size_t bytes = 0;
-    cudaEvent_t h2d_done = nullptr, compute_done = nullptr, d2h_done = nullptr;
+    cudaEvent_t h2d_done = nullptr, h2d_kv_done = nullptr, compute_done = nullptr, d2h_done = nullptr;
     bool used = false;
 };
 
@@ -69,7 +69,7 @@ struct cf_ctx {
     // host-staged step
     cf::HostStage stage[cf::kHostStages];
     int next_stage = 0;
-    cudaStream_t h2d_stream = nullptr, d2h_stream = nullptr;
+    cudaStream_t h2d_stream = nullptr, h2d_kv_stream = nullptr, d2h_stream = nullptr;
     // timing: one quad of events per timed call since the last cf_get_timing_sums
     bool timing = false;
     std::vector<cf::TimedCall> timed;
@@ -459,9 +459,11 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     ok = ok && cudaStreamCreateWithFlags(&c->side, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->upload_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->h2d_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaStreamCreateWithFlags(&c->h2d_kv_stream, cudaStreamNonBlocking) == cudaSuccess;
     ok = ok && cudaStreamCreateWithFlags(&c->d2h_stream, cudaStreamNonBlocking) == cudaSuccess;
     for (int i = 0; i < kHostStages && ok; ++i) {
         ok = cudaEventCreateWithFlags(&c->stage[i].h2d_done, cudaEventDisableTiming) == cudaSuccess &&
+             cudaEventCreateWithFlags(&c->stage[i].h2d_kv_done, cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->stage[i].compute_done, cudaEventDisableTiming) == cudaSuccess &&
              cudaEventCreateWithFlags(&c->stage[i].d2h_done, cudaEventDisableTiming) == cudaSuccess;
     }
@@ -501,10 +503,12 @@ cf_status cf_destroy(cf_ctx* c)
         HostStage& hs = c->stage[i];
         if (hs.dev) cudaFree(hs.dev);
         if (hs.h2d_done) cudaEventDestroy(hs.h2d_done);
+        if (hs.h2d_kv_done) cudaEventDestroy(hs.h2d_kv_done);
         if (hs.compute_done) cudaEventDestroy(hs.compute_done);
         if (hs.d2h_done) cudaEventDestroy(hs.d2h_done);
     }
     if (c->h2d_stream) cudaStreamDestroy(c->h2d_stream);
+    if (c->h2d_kv_stream) cudaStreamDestroy(c->h2d_kv_stream);
     if (c->d2h_stream) cudaStreamDestroy(c->d2h_stream);
     delete c;
     return CF_OK;
@@ -749,16 +753,20 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
     uint8_t* dout = dv + kv_bytes;
     const size_t qb = T * desc->num_q_heads * desc->head_dim * 2, kb = T * desc->num_kv_heads * desc->head_dim * 2;
     // inputs: copy stream, after the kernels and the read-back that last used this staging set
+    // (q on one copy stream, k_new and v_new on a second: the small copies run at two thirds of the link rate
+    // on their own and fill in beside the large one)
     if (hs.used) {
         if (cudaStreamWaitEvent(c->h2d_stream, hs.compute_done, 0) != cudaSuccess) return CF_ERR_CUDA;
         if (cudaStreamWaitEvent(c->h2d_stream, hs.d2h_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+        if (cudaStreamWaitEvent(c->h2d_kv_stream, hs.compute_done, 0) != cudaSuccess) return CF_ERR_CUDA;
     }
+    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, c->h2d_kv_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, c->h2d_kv_stream) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaEventRecord(hs.h2d_kv_done, c->h2d_kv_stream) != cudaSuccess) return CF_ERR_CUDA;
     if (cudaMemcpyAsync(dq, q_host, qb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
-    if (cudaMemcpyAsync(dk, k_new_host, kb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
-    if (cudaMemcpyAsync(dv, v_new_host, kb, cudaMemcpyHostToDevice, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
     if (cudaEventRecord(hs.h2d_done, c->h2d_stream) != cudaSuccess) return CF_ERR_CUDA;
     // kernels: the caller's stream
-    if (cudaStreamWaitEvent(stream, hs.h2d_done, 0) != cudaSuccess) return CF_ERR_CUDA;
+    if (cudaStreamWaitEvent(stream, hs.h2d_kv_done, 0) != cudaSuccess) return CF_ERR_CUDA;
     c->plan_copy_stream = c->h2d_stream;
     st = cf_kv_append(c, desc, k_cache, v_cache, dk, dv, block_table, max_blocks_per_seq, context_len, query_len,
                       num_seqs, cuda_stream);
@@ -768,6 +776,10 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
     }
     // The step is bound by the copies over PCIe, not by the kernels; measured on the chat-like workload the
     // spatial sequence made it slower (0.40 ms against 0.355 ms).
+    if (cudaStreamWaitEvent(stream, hs.h2d_done, 0) != cudaSuccess) {
+        c->plan_copy_stream = nullptr;
+        return CF_ERR_CUDA;
+    }
     c->in_host_step = true;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);
