@@ -86,6 +86,36 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                           * std::max(1, cfg.decode_waves);
     const int32_t quantum = std::max(1, cfg.decode_page_quantum);
     int64_t target = (total_pages * d->num_kv_heads + slots - 1) / slots;
+    const bool shares_sms = cfg.prefill_sms_mixed > 0 && plan->n_prefill_seqs > 0;   // spatial sequence: decode runs on part of the machine, beside prefill
+    if (target < cfg.decode_min_chunk_pages && total_pages > 0 && !shares_sms) {
+        // A small batch: chunks of the minimum length would not fill `decode_waves` waves, and how many waves
+        // of (num_sms x ctas_per_sm) CTAs they do fall into decides the time (a last wave that is a quarter
+        // full costs a whole CTA time).  Try chunk lengths from the minimum to four times it and keep the
+        // one with the smallest waves x (CTA start-up + chunk streaming time).  (Not when decode shares the SMs
+        // with a prefill grid: there the short chunks measured better, 81 against 90 us on the TP4 shard.)
+        const int64_t wave = (int64_t)std::max(1, cfg.num_sms) * std::max(1, cfg.decode_ctas_per_sm);
+        const double page_us = (2.0 * B * d->head_dim * 2.0) / (7.56e6 / (double)wave);   // one (page, head) of K and V at a CTA's share of HBM
+        const double cta_us = 2.5;
+        double best = 1e30;
+        int64_t best_c = cfg.decode_min_chunk_pages;
+        for (int64_t c = (cfg.decode_min_chunk_pages + quantum - 1) / quantum * quantum; c <= 4 * (int64_t)cfg.decode_min_chunk_pages;
+             c += quantum) {
+            int64_t ctas = 0, longest = 0;
+            for (int32_t s = 0; s < num_seqs; ++s) {
+                if (query_len[s] != 1) continue;
+                const int64_t pages = (context_len[s] + B - 1) / B;
+                int64_t n = (pages + c - 1) / c;
+                int64_t per = ((pages + n - 1) / n + quantum - 1) / quantum * quantum;
+                n = (pages + per - 1) / per;
+                ctas += n;
+                longest = std::max(longest, std::min(per, pages));
+            }
+            ctas *= d->num_kv_heads;
+            const double t = (double)((ctas + wave - 1) / wave) * (cta_us + page_us * (double)longest);
+            if (t < best * 0.999) { best = t; best_c = c; }
+        }
+        target = best_c;
+    }
     target = std::max<int64_t>(target, cfg.decode_min_chunk_pages);
     target = (target + quantum - 1) / quantum * quantum;
 

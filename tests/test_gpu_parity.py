@@ -195,7 +195,7 @@ def test_abi_rejects_bad_arguments_without_launching():
 
 
 def test_fixed_workspace_too_small_is_reported():
-    sc = small(23, 32, 8, 128, [60000], [[1]], NB=4096)
+    sc = small(23, 32, 8, 128, [60000, 60000, 60000], [[1, 1, 1]], NB=12288)     # ~90 partial slots x 16 KB: more than the 1 MB a tiny request is rounded up to
     b = sc.batches[0]
     ctx = cf.cf_create(0, workspace_bytes=4096)
     g = GpuScenario(sc, ctx=ctx)
