@@ -206,6 +206,11 @@ def batch_accounting(sc: syn.Scenario):
     return acc
 
 
+# nominal chip figures (HGX B200: 7.7 TB/s HBM3e, 2.25 PFLOP/s dense bf16), reported beside the measured peaks
+NOMINAL_HBM_GBS = 7700.0
+NOMINAL_BF16_TFLOPS = 2250.0
+
+
 def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks):
     """Per-kernel CUDA-event times (inside the library, on the launching stream) over `steps` steps."""
     acc = batch_accounting(wl.sc)
@@ -221,12 +226,13 @@ def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks):
     if ms_dec > 0:
         gbs = dec_bytes / ((ms_dec + ms_comb) * 1e-3) / 1e9
         out["decode"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
-                         "frac": gbs / peaks["hbm_gbs"], "traffic": DECODE_TRAFFIC_RATIO * dec_bytes / steps,
+                         "frac": gbs / peaks["hbm_gbs"], "frac_of_nominal": gbs / NOMINAL_HBM_GBS,
+                         "traffic": DECODE_TRAFFIC_RATIO * dec_bytes / steps,
                          "bytes_per_launch": dec_bytes / steps, "ms": (ms_dec + ms_comb) / steps}
     if ms_pre > 0:
         tf = pre_flops / (ms_pre * 1e-3) / 1e12
         out["prefill"] = {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                          "frac": tf / peaks["bf16_tflops"], "traffic": None,
+                          "frac": tf / peaks["bf16_tflops"], "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS, "traffic": None,
                           "flops_per_launch": pre_flops / steps, "ms": ms_pre / steps}
     return out, launches
 
@@ -401,7 +407,7 @@ def run_ours(args):
 
     if rank == 0:
         dominant = "prefill" if kern.get("prefill", {}).get("ms", 0) >= kern.get("decode", {}).get("ms", 0) else "decode"
-        roof = {k: kern[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic")}
+        roof = {k: kern[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "frac_of_nominal")}
         roof["kernel"] = "prefill_tc_kernel" if dominant == "prefill" else "decode_splitk_kernel (merge of the partials fused in)"
         roof["peak_source"] = peaks["source"] + (" burst bf16" if dominant == "prefill" else " copy")
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
