@@ -99,6 +99,9 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x)
 #ifndef CF_POLY_MASK
 #define CF_POLY_MASK 0x8080u
 #endif
+#ifndef CF_POLY_MASK_D64
+#define CF_POLY_MASK_D64 0x8080u
+#endif
 // 32-byte store (address 32-byte aligned)
 __device__ __forceinline__ void st_global_256(void* p, const uint32_t* v)
 {
@@ -182,6 +185,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                   const int first_static, const int ticket_base, uint32_t* const resident)
 {
     constexpr int HALVES = Geo<D>::HALVES, TILE_BYTES = Geo<D>::TILE_BYTES, KS = Geo<D>::KS;
+    constexpr uint32_t kPolyMask = D == 64 ? CF_POLY_MASK_D64 : CF_POLY_MASK;
     constexpr uint32_t SMEM_Q = Geo<D>::SMEM_Q, SMEM_K = Geo<D>::SMEM_K, SMEM_V = Geo<D>::SMEM_V;
     extern __shared__ uint8_t smem_raw[];
     __shared__ __align__(16) ItemCtx ctx_s[2];
@@ -622,7 +626,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                     for (int i = 0; i < 16; ++i) {
                         const float2 x = fma2(make_float2(sv[c * 32 + 2 * i], sv[c * 32 + 2 * i + 1]), sc2, nm2);
-                        const float2 pr = ((CF_POLY_MASK >> i) & 1u) ? exp2_poly2(x) : make_float2(fast_exp2(x.x), fast_exp2(x.y));
+                        const float2 pr = ((kPolyMask >> i) & 1u) ? exp2_poly2(x) : make_float2(fast_exp2(x.x), fast_exp2(x.y));
                         acc2[i & 3] = add2(acc2[i & 3], pr);
                         pk[i] = pack_bf16(pr.x, pr.y);
                     }
