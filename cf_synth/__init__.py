@@ -328,6 +328,23 @@ def decode_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray)
     return int(4 * geom.head_dim * geom.num_q_heads * lc.sum())
 
 
+def tile_edge_rows(batch: Batch, tile: int = 128, stride: int = 41) -> np.ndarray:
+    """Packed q-row indices to check at full size: every decode row; for a prefill sequence the first and
+    last row of every `tile`-row q tile (so that no q tile, and with all heads checked no work item, goes
+    unchecked), the chunk's last row, and every `stride`-th row."""
+    qs = batch.q_start()
+    rows: List[np.ndarray] = []
+    for s in range(batch.num_seqs):
+        n = int(batch.query_len[s])
+        if n == 0:
+            continue
+        idx = np.arange(n)
+        if n > 1:
+            idx = idx[(idx % tile == 0) | (idx % tile == tile - 1) | (idx % stride == 0) | (idx == n - 1)]
+        rows.append(qs[s] + idx)
+    return np.concatenate(rows).astype(np.int64) if rows else np.zeros(0, dtype=np.int64)
+
+
 def sample_rows(batch: Batch, max_prefill_rows_per_seq: int = 0) -> np.ndarray:
     """Packed q-row indices to check: every decode row; for prefill sequences either all rows or
     a deterministic subsample (first and last row of every 128-row tile plus every 7th row,

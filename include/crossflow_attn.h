@@ -21,7 +21,10 @@
  *     [sum_{t<s} query_len[t], ... + query_len[s]).  Decode (query_len 1) and prefill
  *     (query_len > 1) sequences may appear in any order; query_len 0 is legal (no rows).
  *   - Block-table entries past ceil(context_len/B), cache slots past context_len and unassigned
- *     pages are never read into the result (they may hold NaN).
+ *     pages are never read into the result (they may hold NaN).  An entry in use that lies outside
+ *     [0, num_blocks) is never dereferenced: a new row aimed at it is not written, attention reads page 0
+ *     in its place (the rows of that sequence are then meaningless) and cf_get_async_status reports
+ *     CF_ERR_OUT_OF_RANGE.
  *   - Pointers marked DEVICE must be device memory of the context's GPU and stay alive until the
  *     stream has finished the enqueued work.  Pointers marked HOST are read before the call returns.
  *   - All calls on one context must be issued on one stream (or be ordered by the caller): they
@@ -51,7 +54,8 @@ typedef enum {
     CF_ERR_WORKSPACE = 4,    /* fixed-size workspace too small for this batch */
     CF_ERR_CUDA = 5,         /* a CUDA runtime call or launch failed */
     CF_ERR_TIMEOUT = 6,      /* a bounded device-side wait expired (reported by cf_get_async_status) */
-    CF_ERR_ARCH = 7          /* device is not sm_100 */
+    CF_ERR_ARCH = 7,         /* device is not sm_100 */
+    CF_ERR_BUSY = 8          /* cf_destroy while plans of the context are still alive */
 } cf_status;
 
 /* Geometry of the paged cache.  Strides are in ELEMENTS (bf16); head_dim is contiguous.
@@ -70,6 +74,8 @@ typedef struct {
  * size and grows when a batch needs more (growth allocates and synchronises the device);
  * workspace_bytes > 0: fixed size, a batch that needs more gets CF_ERR_WORKSPACE. */
 cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes);
+/* Synchronises the device and frees everything the context owns.  A context that still has live plans
+ * (cf_plan_create without cf_plan_destroy) is not destroyed: CF_ERR_BUSY, nothing freed. */
 cf_status cf_destroy(cf_ctx* ctx);
 
 /* Section 2.1: prefill "materializes" the KV cache; decode appends one token per step.
@@ -137,8 +143,10 @@ cf_status cf_mixed_step_host(cf_ctx* ctx, const cf_cache_desc* desc,
 /* Makes cuda_stream wait for the read-backs of all cf_mixed_step_host calls issued so far. */
 cf_status cf_host_steps_flush(cf_ctx* ctx, void* cuda_stream);
 
-/* After the caller has synchronised the stream: CF_OK, or the first device-side finding
- * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up; the kernel returned normally). */
+/* After the caller has synchronised the stream: CF_OK, or what the kernels found since the last query
+ * (CF_ERR_TIMEOUT: a bounded wait inside a kernel gave up and the kernel returned normally;
+ * CF_ERR_OUT_OF_RANGE: a block-table entry in use was outside the pool and was not dereferenced;
+ * a timeout is reported first when both happened).  Reading clears the record. */
 cf_status cf_get_async_status(cf_ctx* ctx);
 
 /* Section 5 names two executor backends: the chunked mixed-batch path (time-multiplexed) and a spatial
@@ -154,12 +162,8 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  *     side stream, forked from the caller's, runs decode on the SMs left over, and behind it a second prefill
  *     grid that draws from the same work queue, so the SMs decode frees join the prefill.  The side stream is
  *     joined back into the caller's stream inside the call, so the caller still sees one stream.
- * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n, CF_SPATIAL_WAIT=1 (decode waits, with a
- * stream memory operation, until the first prefill grid's CTAs hold their SMs, instead of relying on the order
- * of the launches).  cf_set_timing and cf_mixed_step_host
- * use the serial sequence.  Other switches read at cf_create (debugging aids): CF_FUSED_COMBINE=0 (separate
- * combine kernel), CF_PREFILL_MMA=1 (mma.sync prefill kernel), CF_PREFILL_SPLIT=k, CF_DECODE_WAVES,
- * CF_DECODE_MIN_CHUNK_PAGES. */
+ * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n (the share that n = 1 stands for).
+ * cf_set_timing and cf_mixed_step_host use the serial sequence. */
 cf_status cf_set_overlap(cf_ctx* ctx, int n);
 
 /* Debug aid (synchronous): checks every block-table entry that cf_kv_append / cf_mixed_attention would
@@ -170,6 +174,23 @@ cf_status cf_set_overlap(cf_ctx* ctx, int n);
 cf_status cf_validate_block_table(cf_ctx* ctx, const cf_cache_desc* desc, const int32_t* block_table,
                                   int32_t max_blocks_per_seq, const int32_t* context_len, const int32_t* query_len,
                                   int32_t num_seqs, void* cuda_stream, int32_t* num_bad);
+
+/* TEST ONLY: planner and launch-sequence switches that the test-suite uses to force paths the cost model
+ * would not pick on small inputs.  Not part of the supported surface; values <= 0 restore the default.
+ *   CF_DEBUG_PREFILL_SPLIT          k >= 2: cut every prefill item into k KV ranges; 1: never split
+ *   CF_DEBUG_SEPARATE_COMBINE       1: merge split-K decode partials in the separate combine kernel
+ *   CF_DEBUG_DECODE_WAVES           target number of decode CTA waves
+ *   CF_DEBUG_DECODE_MIN_CHUNK_PAGES shortest decode chunk, in pages
+ *   CF_DEBUG_SPATIAL_WAIT           1: in the spatial sequence decode waits, through a stream memory operation,
+ *                                   until the first prefill grid's CTAs hold their SMs */
+typedef enum {
+    CF_DEBUG_PREFILL_SPLIT = 0,
+    CF_DEBUG_SEPARATE_COMBINE = 1,
+    CF_DEBUG_DECODE_WAVES = 2,
+    CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3,
+    CF_DEBUG_SPATIAL_WAIT = 4
+} cf_debug_option;
+cf_status cf_set_debug_option(cf_ctx* ctx, cf_debug_option option, int value);
 
 /* Self-test of the bounded-wait machinery (no counterpart in the paper): enqueues one tiny kernel whose
  * wait on a barrier that nothing signals expires after a few milliseconds; the kernel then sets the
@@ -195,18 +216,21 @@ cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
  * lock.  This entry point needs no cf_ctx: the split-K scratch (work items and fp32 partials) is a
  * fixed 16 MiB array inside the library's device image, resident on every GPU that loads the library
  * until the process exits.  It calls no cudaMalloc / cudaFree / cudaMallocHost and no allocating
- * library routine; the host plan lives on the stack (about 110 KB).
+ * library routine; the host plan lives on the caller's stack (about 124 KB: mind small thread stacks).
  *   Every sequence decodes exactly one token: q / out are bf16 [num_seqs, Hq, D], lse fp32
  *   [num_seqs, Hq] or NULL, context_len HOST int32 [num_seqs] (>= 1, includes the new token);
  *   caches, block_table and desc as in cf_mixed_attention.  Runs on the CURRENT device.
- *   Limits: num_seqs <= 1024, <= 4096 KV chunks, and partials (chunks of split sequences x Hq x
+ *   Limits: num_seqs <= 1024, <= 3584 KV chunks, and partials (chunks of split sequences x Hq x
  *   (D+2) x 4 bytes) + 128 KiB <= 16 MiB; anything larger returns CF_ERR_WORKSPACE and enqueues nothing.
- *   The first call on a device resolves the array's address and sets kernel attributes; make that
- *   call before any stream capture begins.  All calls share the one array and it keeps the previous
- *   call's contents (nothing in it has to start at zero: every partial that is read is written first
- *   by the same call), so two calls whose GPU work overlaps - different streams, or different host
- *   threads - race; keep them on one stream or order them yourself.  Results are identical to
- *   cf_mixed_attention on the same all-decode batch. */
+ *   The first call on a device resolves the array's address (host threads may race to it: it is
+ *   serialised inside).  The call must NOT be made while cuda_stream is being captured into a graph -
+ *   its plan is copied from the caller's stack, which a replay would read after it is gone - and
+ *   returns CF_ERR_UNSUPPORTED then.  All calls share the one array and it keeps the previous call's
+ *   contents (nothing in it has to start at zero: every partial that is read is written first by the
+ *   same call), so two calls whose GPU work overlaps - different streams, or different host threads -
+ *   race; keep them on one stream or order them yourself.  The sequences are cut into KV chunks by the
+ *   routine cf_mixed_attention uses and merged in the same order, so on an all-decode batch the two
+ *   give identical bits (for a context with default planner settings). */
 cf_status cf_decode_attention_static(const cf_cache_desc* desc, const void* q,
                                      const void* k_cache, const void* v_cache,
                                      const int32_t* block_table, int32_t max_blocks_per_seq,
@@ -224,17 +248,24 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
                          float* us_decode, float* us_combine, float* us_prefill);
 
 /* Host planner, exposed for inspection and tests (no GPU needed).  Builds the plan that
- * cf_mixed_attention would build for `num_sms` SMs and copies out up to `cap` items of each kind.
+ * cf_mixed_attention would build and copies out up to `cap` items of each kind.
+ *   opts          : planner settings, or NULL for the defaults of a 148-SM device.  Zero fields mean
+ *                   "default"; prefill_sms_mixed > 0 plans a mixed batch for the spatial sequence with
+ *                   that many SMs in the first prefill grid; prefill_force_split as CF_DEBUG_PREFILL_SPLIT.
  *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}
  *   combine_items : int32 [cap, 3] = {q_row, first_partial_slot, num_chunks}
- *   prefill_items : int32 [cap, 6] = {seq, q_row_of_tile, first_row_in_chunk, num_rows, query_head, kv_head},
- *                   one entry per (q tile, query head) in launch order
- *                   (a KV-split item is listed once)
+ *   prefill_items : int32 [cap, 8] = {seq, q_row_of_tile, first_row_in_chunk, num_rows, query_head, kv_head,
+ *                   first_kv_tile, end_kv_tile}, one entry per (q tile, query head, KV range) in launch
+ *                   order; KV tiles are 128 tokens, end_kv_tile is clamped to the tile's own extent; an item
+ *                   that is not KV-split has one entry covering all of its tiles
  *   counts        : int32 [6]      = {n_decode_items, n_combine_items, n_prefill_entries, n_partial_slots,
  *                                     n_prefill_ctas (KV ranges of split items counted), n_kv_split_prefill_items}
  * Any output pointer may be NULL. */
+typedef struct {
+    int32_t num_sms, prefill_sms_mixed, prefill_force_split, decode_waves, decode_min_chunk_pages;
+} cf_plan_options;
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
-                          int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                          int32_t num_seqs, int32_t max_blocks_per_seq, const cf_plan_options* opts,
                           int32_t* decode_items, int32_t* combine_items, int32_t* prefill_items,
                           int32_t cap, int32_t* counts);
 

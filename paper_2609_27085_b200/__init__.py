@@ -6,7 +6,7 @@ There is no CPU fallback: if the library is missing, loading raises.
 
 Names mirror the C ABI (``include/crossflow_attn.h``): ``cf_create``, ``cf_kv_append``,
 ``cf_mixed_attention``, ``cf_mixed_step_host``, ``cf_get_async_status``, ``cf_set_timing``,
-``cf_get_timing_sums``, ``cf_get_last_launch_count``, ``cf_plan_inspect``, ``cf_decode_attention_static``, ``cf_status_string``.
+``cf_get_timing_sums``, ``cf_get_last_launch_count``, ``cf_plan_inspect``, ``cf_decode_attention_static``, ``cf_status_string``, ...
 
 Device arguments may be torch tensors (their ``data_ptr()`` is used) or integer addresses; the
 length arrays are host ``int32`` numpy arrays (anything array-like is converted).
@@ -30,11 +30,20 @@ CF_ERR_WORKSPACE = 4
 CF_ERR_CUDA = 5
 CF_ERR_TIMEOUT = 6
 CF_ERR_ARCH = 7
+CF_ERR_BUSY = 8
+
+# cf_debug_option (test-only switches)
+CF_DEBUG_PREFILL_SPLIT = 0
+CF_DEBUG_SEPARATE_COMBINE = 1
+CF_DEBUG_DECODE_WAVES = 2
+CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3
+CF_DEBUG_SPATIAL_WAIT = 4
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_status_string")
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option",
+           "cf_status_string")
 
 
 class CacheDesc(ctypes.Structure):
@@ -44,6 +53,12 @@ class CacheDesc(ctypes.Structure):
                 ("k_stride_block", ctypes.c_int64), ("k_stride_head", ctypes.c_int64), ("k_stride_token", ctypes.c_int64),
                 ("v_stride_block", ctypes.c_int64), ("v_stride_head", ctypes.c_int64), ("v_stride_token", ctypes.c_int64),
                 ("softmax_scale", ctypes.c_float)]
+
+
+class PlanOptions(ctypes.Structure):
+    """Mirror of ``cf_plan_options`` (zero = default)."""
+    _fields_ = [("num_sms", ctypes.c_int32), ("prefill_sms_mixed", ctypes.c_int32), ("prefill_force_split", ctypes.c_int32),
+                ("decode_waves", ctypes.c_int32), ("decode_min_chunk_pages", ctypes.c_int32)]
 
 
 class CfError(RuntimeError):
@@ -75,7 +90,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_set_timing.argtypes = [vp, ctypes.c_int]
     lib.cf_get_timing_sums.argtypes = [vp, fp, fp, fp, i32p]
     lib.cf_get_last_launch_count.argtypes = [vp, i32p]
-    lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, i32, vp, vp, vp, i32, vp]
+    lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, ctypes.POINTER(PlanOptions), vp, vp, vp, i32, vp]
+    lib.cf_set_debug_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
@@ -200,6 +216,11 @@ def cf_set_overlap(ctx, n) -> None:
     _check(load_library().cf_set_overlap(ctx, int(n)), "cf_set_overlap")
 
 
+def cf_set_debug_option(ctx, option: int, value: int) -> None:
+    """Test-only planner / launch-sequence switches (CF_DEBUG_*); value <= 0 restores the default."""
+    _check(load_library().cf_set_debug_option(ctx, int(option), int(value)), "cf_set_debug_option")
+
+
 def cf_set_timing(ctx, enabled: bool) -> None:
     _check(load_library().cf_set_timing(ctx, int(bool(enabled))), "cf_set_timing")
 
@@ -219,19 +240,24 @@ def cf_get_last_launch_count(ctx) -> int:
 
 
 def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148,
-                    cap: int = 1 << 16, check: bool = True):
-    """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,6], n_partial_slots)."""
+                    cap: int = 1 << 16, check: bool = True, prefill_sms_mixed: int = 0, prefill_force_split: int = 0,
+                    decode_waves: int = 0, decode_min_chunk_pages: int = 0, want_counts: bool = False):
+    """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,8], n_partial_slots)
+    and, with want_counts, the six counters as a last element."""
     lc, lq = _host_i32(context_len), _host_i32(query_len)
     dec = np.zeros((cap, 6), dtype=np.int32)
     comb = np.zeros((cap, 3), dtype=np.int32)
-    pre = np.zeros((cap, 6), dtype=np.int32)
+    pre = np.zeros((cap, 8), dtype=np.int32)
     counts = np.zeros(6, dtype=np.int32)
+    opts = PlanOptions(int(num_sms), int(prefill_sms_mixed), int(prefill_force_split), int(decode_waves),
+                       int(decode_min_chunk_pages))
     st = load_library().cf_plan_inspect(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
-                                        int(max_blocks_per_seq), int(num_sms), dec.ctypes.data, comb.ctypes.data,
+                                        int(max_blocks_per_seq), ctypes.byref(opts), dec.ctypes.data, comb.ctypes.data,
                                         pre.ctypes.data, cap, counts.ctypes.data)
     if check:
         _check(st, "cf_plan_inspect")
-    return st, dec[:counts[0]], comb[:counts[1]], pre[:counts[2]], int(counts[3])
+    res = (st, dec[:counts[0]], comb[:counts[1]], pre[:counts[2]], int(counts[3]))
+    return res + (counts,) if want_counts else res
 
 
 def cf_decode_attention_static(desc: CacheDesc, q, k_cache, v_cache, block_table, max_blocks_per_seq: int,

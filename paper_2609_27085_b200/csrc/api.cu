@@ -2,6 +2,7 @@
 // See include/crossflow_attn.h for the contract of every entry point.
 #include <cuda.h>
 
+#include <atomic>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -18,6 +19,10 @@ namespace cf {
 static constexpr int kRing = 4;                         // plan slots in flight
 static constexpr size_t kDefaultWorkspace = 64u << 20;  // split-K partials
 static constexpr size_t kDefaultPlanBytes = 1u << 20;
+// The first kCounterBytes of a split-K workspace hold the fused-combine ticket counters of the decode kernel
+// (one per first partial slot of a split sequence and KV head): zeroed when the buffer is allocated, put back
+// to zero by the kernel.  A batch with more counters than fit uses the separate combine kernel.
+static constexpr size_t kCounterBytes = 256u << 10;
 
 struct TimedCall {
     cudaEvent_t ev[4] = {nullptr, nullptr, nullptr, nullptr};
@@ -54,16 +59,17 @@ struct cf_ctx {
     float* workspace = nullptr;
     size_t workspace_bytes = 0;
     bool workspace_fixed = false;
-    uint32_t* err_dev = nullptr;
-    bool fused_combine = true; // split-K merge inside the decode kernel (CF_FUSED_COMBINE=0: the separate combine kernel)
-    bool use_tc = true;        // chunked prefill on tcgen05 (CF_PREFILL_MMA=1 forces the mma.sync kernel)
+    uint32_t* err_dev = nullptr;      // [0] device-side findings (bit 0: a wait expired, bit 1: block id outside the pool); [1] scratch counter of cf_validate_block_table
+    bool fused_combine = true; // split-K merge inside the decode kernel (CF_DEBUG_SEPARATE_COMBINE: the separate combine kernel)
+    std::atomic<int> live_plans{0};
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
     cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
     cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
     bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
-    bool spatial_wait = false; // CF_SPATIAL_WAIT=1: decode waits (stream memory operation) for the front prefill CTAs to be resident
-    int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths; CF_SPATIAL_SMS)
+    bool spatial_wait = false; // CF_DEBUG_SPATIAL_WAIT: decode waits (stream memory operation) for the front prefill CTAs to be resident
+    int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths)
+    int spatial_sms_default = 0;   // CF_SPATIAL_SMS at cf_create: what cf_set_overlap(ctx, 1) goes back to
     cudaStream_t side = nullptr;
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     // host-staged step
@@ -87,8 +93,8 @@ struct cf_plan {
     uint8_t* dev = nullptr;
     float* part = nullptr;         // this plan's own split-K partials
     int n_part_slots = 0, n_pre_slots = 0;
-    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
-    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
+    int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     float pre_over_dec = 0.f;
 };
 
@@ -148,14 +154,17 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
     c->workspace_bytes = 0;
     size_t nb = align_up(need + need / 4, 1u << 20);
     if (cudaMalloc((void**)&c->workspace, nb) != cudaSuccess) return CF_ERR_CUDA;
-    if (cudaMemset(c->workspace, 0, nb) != cudaSuccess) return CF_ERR_CUDA;       // the ticket counters at its front start at zero
+    // The ticket counters at its front start at zero.  cudaMemset runs on the legacy default stream, which is not
+    // ordered against non-blocking streams: wait for it here, before any kernel of the caller's stream can count.
+    if (cudaMemset(c->workspace, 0, kCounterBytes < nb ? kCounterBytes : nb) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess)
+        return CF_ERR_CUDA;
     c->workspace_bytes = nb;
     return CF_OK;
 }
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre, off_pre_tc, off_pre_comb, off_queue, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre_tc, off_pre_comb, off_queue, total;
 };
 
 static PlanLayout layout_of(int32_t S, const Plan& pl)
@@ -167,7 +176,6 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_qlen = at;   at = align_up(at + sizeof(int32_t) * (size_t)S, 16);
     L.off_dec = at;    at = align_up(at + sizeof(DecodeItem) * pl.decode.size(), 16);
     L.off_comb = at;   at = align_up(at + sizeof(CombineItem) * pl.combine.size(), 16);
-    L.off_pre = at;    at = align_up(at + sizeof(PrefillItem) * pl.prefill.size(), 16);
     L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
     L.off_pre_comb = at; at = align_up(at + sizeof(PrefillCombineItem) * pl.prefill_combine.size(), 16);
     L.off_queue = at;  at += 16;   // ticket counter + exit counter of the persistent prefill CTAs; uploaded as zeros
@@ -192,7 +200,6 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     }
     if (!pl.decode.empty()) std::memcpy(s.host + L->off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
     if (!pl.combine.empty()) std::memcpy(s.host + L->off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
-    if (!pl.prefill.empty()) std::memcpy(s.host + L->off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
     if (!pl.prefill_tc.empty())
         std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
     if (!pl.prefill_combine.empty())
@@ -255,17 +262,13 @@ static float scale_log2_of(const cf_cache_desc* d)
 namespace cf {
 
 struct PlanCounts {
-    int n_dec = 0, n_comb = 0, n_pre = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
     int n_part_slots = 0;
 };
 
-// Split-K workspace: decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact partial rows of
-// KV-split prefill items [row slot, D] + [row slot, 2].
-// The first kCounterBytes hold the fused-combine ticket counters of the decode kernel (one per first partial
-// slot of a split sequence and KV head): zeroed when the buffer is allocated, put back to zero by the kernel.
-// A batch with more counters than fit uses the separate combine kernel.
-static constexpr size_t kCounterBytes = 256u << 10;
+// Split-K workspace: the ticket counters, decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact
+// partial rows of KV-split prefill items [row slot, D] + [row slot, 2].
 struct WsLayout {
     size_t dec_o = 0, dec_ml = 0, pre_o = 0, pre_ml = 0, total = 0;
 };
@@ -295,6 +298,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.lse = lse;
     p.block_table = block_table;
     p.max_blocks = max_blocks_per_seq;
+    p.num_blocks = desc->num_blocks;
     p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
@@ -304,7 +308,6 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.query_len = (const int32_t*)(base + L.off_qlen);
     p.dec_items = (const DecodeItem*)(base + L.off_dec);
     p.comb_items = (const CombineItem*)(base + L.off_comb);
-    p.pre_items = (const PrefillItem*)(base + L.off_pre);
     p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
     p.part_o = (float*)((uint8_t*)ws + W.dec_o);
     p.part_ml = (float*)((uint8_t*)ws + W.dec_ml);
@@ -329,9 +332,9 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         tc = &c->timed[c->timed_used++];
         tc->ran[0] = (n.n_dec > 0);
         tc->ran[1] = (n.n_comb > 0) && !fused_combine;
-        tc->ran[2] = (n.n_pre > 0) || (n.n_pre_tc > 0);
+        tc->ran[2] = n.n_pre_tc > 0;
     }
-    const bool has_prefill = (n.n_pre > 0) || (n.n_pre_tc > 0);
+    const bool has_prefill = n.n_pre_tc > 0;
     int second_grid = 0;
     const int sms = c->num_sms > 0 ? c->num_sms : 148;
     const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
@@ -366,7 +369,6 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         }
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, 1, front, resident, stream);
         // only after the front grid has been enqueued without an error, so that the count is certain to arrive
         if (e == cudaSuccess && resident &&
@@ -384,12 +386,11 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
-        if (e == cudaSuccess) e = launch_prefill_mma(p, D, n.n_pre, stream);
         if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre > 0) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -410,6 +411,7 @@ const char* cf_status_string(cf_status s)
         case CF_ERR_CUDA: return "CF_ERR_CUDA";
         case CF_ERR_TIMEOUT: return "CF_ERR_TIMEOUT";
         case CF_ERR_ARCH: return "CF_ERR_ARCH";
+        case CF_ERR_BUSY: return "CF_ERR_BUSY";
     }
     return "CF_ERR_UNKNOWN";
 }
@@ -433,21 +435,11 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     c->device = device;
     c->num_sms = prop.multiProcessorCount;
     c->cfg.num_sms = c->num_sms;
-    c->cfg.decode_waves = env_int("CF_DECODE_WAVES", c->cfg.decode_waves);
-    c->cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", c->cfg.decode_min_chunk_pages);
-    c->cfg.prefill_tile_rows = kPrefillMmaTileRows;
-    c->cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
-    c->use_tc = env_int("CF_PREFILL_MMA", 0) == 0;
-    {
-        const char* v = std::getenv("CF_FUSED_COMBINE");
-        c->fused_combine = !(v && v[0] == '0' && v[1] == 0);
-    }
     {
         const char* v = std::getenv("CF_OVERLAP");          // spatial sequence unless CF_OVERLAP=0
         c->overlap = !(v && v[0] == '0' && v[1] == 0);
     }
-    c->spatial_sms = env_int("CF_SPATIAL_SMS", 0);
-    c->spatial_wait = env_int("CF_SPATIAL_WAIT", 0) != 0;
+    c->spatial_sms = c->spatial_sms_default = env_int("CF_SPATIAL_SMS", 0);
     bool ok = true;
     for (int i = 0; i < kRing && ok; ++i)
         ok = cudaEventCreateWithFlags(&c->slots[i].done, cudaEventDisableTiming) == cudaSuccess &&
@@ -469,8 +461,8 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
     }
     ok = ok && cudaEventCreateWithFlags(&c->ev_fork, cudaEventDisableTiming) == cudaSuccess;
     ok = ok && cudaEventCreateWithFlags(&c->ev_join, cudaEventDisableTiming) == cudaSuccess;
-    ok = ok && cudaMalloc((void**)&c->err_dev, sizeof(uint32_t)) == cudaSuccess;
-    ok = ok && cudaMemset(c->err_dev, 0, sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMalloc((void**)&c->err_dev, 2 * sizeof(uint32_t)) == cudaSuccess;
+    ok = ok && cudaMemset(c->err_dev, 0, 2 * sizeof(uint32_t)) == cudaSuccess && cudaDeviceSynchronize() == cudaSuccess;
     if (!ok) {
         cf_destroy(c);
         return CF_ERR_CUDA;
@@ -482,6 +474,7 @@ cf_status cf_create(cf_ctx** out, int device, size_t workspace_bytes)
 cf_status cf_destroy(cf_ctx* c)
 {
     if (!c) return CF_ERR_INVALID_ARG;
+    if (c->live_plans.load() > 0) return CF_ERR_BUSY;      // a plan holds a pointer to its context
     DeviceGuard guard(c->device);
     cudaDeviceSynchronize();
     for (int i = 0; i < kRing; ++i) {
@@ -546,6 +539,7 @@ cf_status cf_kv_append(cf_ctx* c, const cf_cache_desc* desc, void* k_cache, void
     p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = num_seqs; p.total_rows = pl.total_q;
+    p.num_blocks = desc->num_blocks; p.err = c->err_dev;
     p.q_start = (const int32_t*)(base + L.off_qstart);
     p.context_len = (const int32_t*)(base + L.off_ctx);
     p.query_len = (const int32_t*)(base + L.off_qlen);
@@ -567,7 +561,6 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     Plan pl;
     PlanConfig cfg = c->cfg;
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
-    cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
     c->launches = 0;
@@ -589,7 +582,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     if (st != CF_OK) return st;
 
     PlanCounts n;
-    n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_pre = (int)pl.prefill.size();
+    n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size();
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
     n.n_part_slots = pl.n_part_slots;
     n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
@@ -609,7 +602,6 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     Plan pl;
     PlanConfig cfg = c->cfg;
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
-    cfg.prefill_tc = c->use_tc && prefill_tc_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
     DeviceGuard guard(c->device);
@@ -622,15 +614,19 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->max_blocks = max_blocks_per_seq;
     const PlanLayout L = layout_of(num_seqs, pl);
     P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
-    P->off_comb = L.off_comb; P->off_pre = L.off_pre; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
+    P->off_comb = L.off_comb; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
     P->total = L.total;
-    P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size(); P->n_pre = (int)pl.prefill.size();
+    P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size();
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
     P->pre_over_dec = prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms);
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
     const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
-    if (ok && part_bytes) ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess && cudaMemset(P->part, 0, kCounterBytes) == cudaSuccess;
+    // the ticket counters are zeroed on the caller's stream, like the plan copy: every launch that uses the plan
+    // is ordered behind this call on that stream (or by the caller)
+    if (ok && part_bytes)
+        ok = cudaMalloc((void**)&P->part, part_bytes) == cudaSuccess &&
+             cudaMemsetAsync(P->part, 0, kCounterBytes, (cudaStream_t)cuda_stream) == cudaSuccess;
     if (ok) {
         std::memcpy(P->host + L.off_qstart, pl.q_start.data(), sizeof(int32_t) * ((size_t)num_seqs + 1));
         if (num_seqs > 0) {
@@ -639,13 +635,13 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
         }
         if (P->n_dec) std::memcpy(P->host + L.off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
         if (P->n_comb) std::memcpy(P->host + L.off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
-        if (P->n_pre) std::memcpy(P->host + L.off_pre, pl.prefill.data(), sizeof(PrefillItem) * pl.prefill.size());
         if (P->n_pre_tc) std::memcpy(P->host + L.off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
         if (P->n_pre_comb)
             std::memcpy(P->host + L.off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
         std::memset(P->host + L.off_queue, 0, 16);
         ok = cudaMemcpyAsync(P->dev, P->host, L.total, cudaMemcpyHostToDevice, (cudaStream_t)cuda_stream) == cudaSuccess;
     }
+    c->live_plans.fetch_add(1);
     if (!ok) {
         cf_plan_destroy(P);
         return CF_ERR_CUDA;
@@ -662,6 +658,7 @@ cf_status cf_plan_destroy(cf_plan* P)
     if (P->host) cudaFreeHost(P->host);
     if (P->dev) cudaFree(P->dev);
     if (P->part) cudaFree(P->part);
+    P->ctx->live_plans.fetch_sub(1);
     delete P;
     return CF_OK;
 }
@@ -685,6 +682,7 @@ cf_status cf_kv_append_planned(cf_plan* P, void* k_cache, void* v_cache, const v
     p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = P->num_seqs; p.total_rows = P->total_q;
+    p.num_blocks = desc->num_blocks; p.err = P->ctx->err_dev;
     p.q_start = (const int32_t*)(P->dev + P->off_qstart);
     p.context_len = (const int32_t*)(P->dev + P->off_ctx);
     p.query_len = (const int32_t*)(P->dev + P->off_qlen);
@@ -702,10 +700,10 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     if (!guard.ok) return CF_ERR_CUDA;
     PlanLayout L;
     L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
-    L.off_comb = P->off_comb; L.off_pre = P->off_pre; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
+    L.off_comb = P->off_comb; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
     L.total = P->total;
     PlanCounts n;
-    n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre = P->n_pre; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
+    n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
     n.total_q = P->total_q;
     n.pre_over_dec = P->pre_over_dec;
     n.n_part_slots = P->n_part_slots;
@@ -813,8 +811,10 @@ cf_status cf_get_async_status(cf_ctx* c)
     uint32_t w = 0;
     if (cudaMemcpy(&w, c->err_dev, sizeof w, cudaMemcpyDeviceToHost) != cudaSuccess) return CF_ERR_CUDA;
     if (w == 0) return CF_OK;
-    cudaMemset(c->err_dev, 0, sizeof w);
-    return CF_ERR_TIMEOUT;
+    if (cudaMemset(c->err_dev, 0, sizeof w) != cudaSuccess || cudaDeviceSynchronize() != cudaSuccess) return CF_ERR_CUDA;
+    if (w & kErrTimeout) return CF_ERR_TIMEOUT;
+    if (w & kErrBlockId) return CF_ERR_OUT_OF_RANGE;
+    return CF_ERR_CUDA;
 }
 
 cf_status cf_validate_block_table(cf_ctx* c, const cf_cache_desc* desc, const int32_t* block_table,
@@ -838,9 +838,7 @@ cf_status cf_validate_block_table(cf_ctx* c, const cf_cache_desc* desc, const in
     PlanSlot* slot = nullptr;
     st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
     if (st != CF_OK) return st;
-    // the counter lives in the slot's device buffer, after the plan
-    uint32_t* counter = nullptr;
-    if (cudaMalloc((void**)&counter, sizeof(uint32_t)) != cudaSuccess) return CF_ERR_CUDA;
+    uint32_t* counter = c->err_dev + 1;      // context-owned scratch word
     bool ok = cudaMemsetAsync(counter, 0, sizeof(uint32_t), stream) == cudaSuccess;
     ok = ok && launch_validate_table(block_table, max_blocks_per_seq, (const int32_t*)(base + L.off_ctx), num_seqs,
                                      desc->num_blocks, counter, stream) == cudaSuccess;
@@ -848,7 +846,6 @@ cf_status cf_validate_block_table(cf_ctx* c, const cf_cache_desc* desc, const in
     uint32_t host = 0;
     ok = ok && cudaMemcpyAsync(&host, counter, sizeof host, cudaMemcpyDeviceToHost, stream) == cudaSuccess;
     ok = ok && cudaStreamSynchronize(stream) == cudaSuccess;
-    cudaFree(counter);
     if (!ok) return CF_ERR_CUDA;
     *num_bad = (int32_t)host;
     return host ? CF_ERR_OUT_OF_RANGE : CF_OK;
@@ -860,7 +857,24 @@ cf_status cf_set_overlap(cf_ctx* c, int enabled)
     if (enabled < 0) return CF_ERR_INVALID_ARG;
     c->overlap = enabled != 0;
     if (enabled > 1) c->spatial_sms = enabled;
+    if (enabled == 1) c->spatial_sms = c->spatial_sms_default;
     return CF_OK;
+}
+
+cf_status cf_set_debug_option(cf_ctx* c, cf_debug_option option, int value)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    const PlanConfig defaults;
+    switch (option) {
+        case CF_DEBUG_PREFILL_SPLIT: c->cfg.prefill_force_split = value > 0 ? value : 0; return CF_OK;
+        case CF_DEBUG_SEPARATE_COMBINE: c->fused_combine = value <= 0; return CF_OK;
+        case CF_DEBUG_DECODE_WAVES: c->cfg.decode_waves = value > 0 ? value : defaults.decode_waves; return CF_OK;
+        case CF_DEBUG_DECODE_MIN_CHUNK_PAGES:
+            c->cfg.decode_min_chunk_pages = value > 0 ? value : defaults.decode_min_chunk_pages;
+            return CF_OK;
+        case CF_DEBUG_SPATIAL_WAIT: c->spatial_wait = value > 0; return CF_OK;
+    }
+    return CF_ERR_INVALID_ARG;
 }
 
 cf_status cf_selftest_bounded_wait(cf_ctx* c, void* cuda_stream)
@@ -918,11 +932,6 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
     if (st != CF_OK) return st;
     PlanConfig cfg;
     cfg.num_sms = num_sms > 0 ? num_sms : 148;
-    cfg.decode_waves = env_int("CF_DECODE_WAVES", cfg.decode_waves);
-    cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
-    cfg.prefill_tile_rows = kPrefillMmaTileRows;
-    cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
-    cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -934,19 +943,20 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
 }
 
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
-                          int32_t num_seqs, int32_t max_blocks_per_seq, int32_t num_sms,
+                          int32_t num_seqs, int32_t max_blocks_per_seq, const cf_plan_options* opts,
                           int32_t* decode_items, int32_t* combine_items, int32_t* prefill_items,
                           int32_t cap, int32_t* counts)
 {
     cf_status st = validate_desc(desc);
     if (st != CF_OK) return st;
     PlanConfig cfg;
-    cfg.num_sms = num_sms > 0 ? num_sms : 148;
-    cfg.decode_waves = env_int("CF_DECODE_WAVES", cfg.decode_waves);
-    cfg.decode_min_chunk_pages = env_int("CF_DECODE_MIN_CHUNK_PAGES", cfg.decode_min_chunk_pages);
-    cfg.prefill_tile_rows = kPrefillMmaTileRows;
-    cfg.prefill_tc = env_int("CF_PREFILL_MMA", 0) == 0 && prefill_tc_supported(desc);
-    cfg.prefill_force_split = env_int("CF_PREFILL_SPLIT", 0);
+    if (opts) {
+        if (opts->num_sms > 0) cfg.num_sms = opts->num_sms;
+        if (opts->prefill_sms_mixed > 0) cfg.prefill_sms_mixed = opts->prefill_sms_mixed;
+        if (opts->prefill_force_split > 0) cfg.prefill_force_split = opts->prefill_force_split;
+        if (opts->decode_waves > 0) cfg.decode_waves = opts->decode_waves;
+        if (opts->decode_min_chunk_pages > 0) cfg.decode_min_chunk_pages = opts->decode_min_chunk_pages;
+    }
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -963,19 +973,18 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
             o[0] = pl.combine[i].q_row; o[1] = pl.combine[i].part_first; o[2] = pl.combine[i].n_chunks;
         }
     size_t n_pre = 0;
-    auto emit = [&](int32_t seq, int32_t q_row0, int32_t row0, int32_t n_rows, int32_t head, int32_t kvh) {
-        if (prefill_items && n_pre < (size_t)cap) {
-            int32_t* o = prefill_items + 6 * n_pre;
-            o[0] = seq; o[1] = q_row0; o[2] = row0; o[3] = n_rows; o[4] = head; o[5] = kvh;
-        }
-        ++n_pre;
-    };
-    const int32_t G = desc->num_q_heads / desc->num_kv_heads;
-    for (const PrefillItem& it : pl.prefill)
-        for (int32_t h = 0; h < desc->num_q_heads; ++h) emit(it.seq, it.q_row0, it.row0, it.n_rows, h, h / G);
     for (const PrefillTcItem& it : pl.prefill_tc)
-        for (int t = 0; t < 2; ++t)
-            if (it.n_rows[t] > 0 && it.part_c == 0) emit(it.seq, it.q_row0[t], it.row0[t], it.n_rows[t], it.head[t], it.kvh);
+        for (int t = 0; t < 2; ++t) {
+            if (it.n_rows[t] <= 0) continue;
+            const int32_t tiles = (it.prefix + it.row0[t] + it.n_rows[t] + 127) / 128;      // KV tiles this q tile can see
+            if (prefill_items && n_pre < (size_t)cap) {
+                int32_t* o = prefill_items + 8 * n_pre;
+                o[0] = it.seq; o[1] = it.q_row0[t]; o[2] = it.row0[t]; o[3] = it.n_rows[t]; o[4] = it.head[t]; o[5] = it.kvh;
+                o[6] = it.j_begin < tiles ? it.j_begin : tiles;
+                o[7] = it.j_end < tiles ? it.j_end : tiles;
+            }
+            ++n_pre;
+        }
     if (counts) {
         counts[0] = (int32_t)pl.decode.size();
         counts[1] = (int32_t)pl.combine.size();

@@ -15,6 +15,10 @@
 //
 // Output: a sequence with a single chunk writes bf16 `out` (and lse) directly; otherwise the CTA
 // writes an fp32 partial (o, m, l) that the combine kernel merges in fixed chunk order.
+#include <algorithm>
+#include <atomic>
+#include <mutex>
+
 #include "device_common.cuh"
 #include "kernels.h"
 
@@ -110,14 +114,21 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
     const __nv_bfloat16* kbase = p.k_cache + (int64_t)kvh * p.ks_head;
     const __nv_bfloat16* vbase = p.v_cache + (int64_t)kvh * p.vs_head;
 
+    // A block id outside the pool is never dereferenced: page 0 is read in its place and the error word is set
+    // (the result of that sequence is then meaningless, but nothing faults).
+    auto checked = [&](int32_t id) -> int32_t {
+        if ((uint32_t)id < (uint32_t)p.num_blocks) return id;
+        if (p.err) atomicOr(p.err, kErrBlockId);
+        return 0;
+    };
     int cache_base = 0;
-    int32_t pid_cache = (lane < my_n) ? __ldg(bt + lane * NWARPS) : 0;
+    int32_t pid_cache = (lane < my_n) ? checked(__ldg(bt + lane * NWARPS)) : 0;
     const uint64_t stream_once = l2_policy_evict_first();
 
     auto issue = [&](int i) {
         if (i - cache_base == 32) {             // refill the per-lane page-id cache
             cache_base = i;
-            pid_cache = (i + lane < my_n) ? __ldg(bt + (i + lane) * NWARPS) : 0;
+            pid_cache = (i + lane < my_n) ? checked(__ldg(bt + (i + lane) * NWARPS)) : 0;
         }
         const int32_t pid = __shfl_sync(0xffffffffu, pid_cache, i - cache_base);
         const int tok0 = it.kv_begin + (i * NWARPS + warp) * 16;
@@ -318,13 +329,14 @@ static cudaError_t launch_decode_t(const AttnParams& p, int n_items, cudaStream_
 {
     auto kern = decode_splitk_kernel<D, kDecWarps, kDecStages>;
     const size_t smem = decode_smem_bytes<D>();
-    static bool configured[64] = {};
+    // set once per device; two host threads racing here both set the same value
+    static std::atomic<bool> configured[64];
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (dev >= 0 && dev < 64 && !configured[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        configured[dev].store(true, std::memory_order_release);
     }
     kern<<<n_items * p.Hkv, kDecWarps * 32, smem, stream>>>(p);
     return cudaGetLastError();
@@ -375,7 +387,7 @@ namespace {
 constexpr size_t kStaticScratchBytes = (size_t)16 << 20;          // whole array
 constexpr size_t kStaticPlanBytes = (size_t)128 << 10;            // items + combine items
 constexpr int kStaticMaxSeqs = 1024;
-constexpr int kStaticMaxItems = 4096;
+constexpr int kStaticMaxItems = 3584;                             // 3584 x 32 B + 1024 x 12 B fits the plan region
 constexpr int kMaxDevices = 64;
 
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
@@ -386,12 +398,15 @@ struct StaticSetup {
     int num_sms = 0;
 };
 StaticSetup g_static_setup[kMaxDevices];
+std::mutex g_static_setup_mutex;     // two host threads may make a device's first call at the same time
 
-struct StaticPlan {                  // fixed capacity, lives on the caller's stack
+struct StaticPlan {                  // fixed capacity, lives on the caller's stack (about 124 KB)
     cf::DecodeItem items[kStaticMaxItems];
     cf::CombineItem comb[kStaticMaxSeqs];
     int n_items = 0, n_comb = 0, n_slots = 0;
 };
+static_assert(sizeof(cf::DecodeItem) * kStaticMaxItems + 256 + sizeof(cf::CombineItem) * kStaticMaxSeqs <= kStaticPlanBytes,
+              "the plan region of the scratch array holds the largest plan");
 
 }  // namespace
 
@@ -408,48 +423,53 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     if (num_seqs == 0) return CF_OK;
     if (!q || !k_cache || !v_cache || !block_table || !context_len || !out) return CF_ERR_INVALID_ARG;
     if (num_seqs > kStaticMaxSeqs) return CF_ERR_WORKSPACE;
+    cudaStream_t stream = (cudaStream_t)cuda_stream;
+    // The plan is copied from this function's stack frame: a captured copy node would read a dead frame on
+    // every replay, so the call is refused while the stream is being captured.
+    cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
+    if (cudaStreamIsCapturing(stream, &cap) != cudaSuccess) return CF_ERR_CUDA;
+    if (cap != cudaStreamCaptureStatusNone) return CF_ERR_UNSUPPORTED;
 
     // ---- once per device: resolve the scratch address, read the SM count (no allocation)
     int dev = -1;
     if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= kMaxDevices) return CF_ERR_CUDA;
-    StaticSetup& su = g_static_setup[dev];
-    if (!su.ready) {
-        int major = 0, sms = 0;
-        if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return CF_ERR_CUDA;
-        if (major != 10) return CF_ERR_ARCH;
-        if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CF_ERR_CUDA;
-        void* ptr = nullptr;
-        if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return CF_ERR_CUDA;
-        su.base = static_cast<unsigned char*>(ptr);
-        su.num_sms = sms;
-        su.ready = true;
+    StaticSetup su;
+    {
+        std::lock_guard<std::mutex> lock(g_static_setup_mutex);
+        StaticSetup& slot = g_static_setup[dev];
+        if (!slot.ready) {
+            int major = 0, sms = 0;
+            if (cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) return CF_ERR_CUDA;
+            if (major != 10) return CF_ERR_ARCH;
+            if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return CF_ERR_CUDA;
+            void* ptr = nullptr;
+            if (cudaGetSymbolAddress(&ptr, g_static_scratch) != cudaSuccess || !ptr) return CF_ERR_CUDA;
+            slot.base = static_cast<unsigned char*>(ptr);
+            slot.num_sms = sms;
+            slot.ready = true;
+        }
+        su = slot;
     }
 
-    // ---- plan: same chunking rule as the context path, into fixed-capacity arrays
+    // ---- plan: the chunking routine of the context path (decode_target_pages / decode_split with the default
+    // planner settings), into fixed-capacity arrays
     const int32_t B = desc->block_size, Hq = desc->num_q_heads, D = desc->head_dim;
     PlanConfig cfg;
     cfg.num_sms = su.num_sms;
-    int64_t total_pages = 0;
     for (int32_t s = 0; s < num_seqs; ++s) {
         const int32_t lc = context_len[s];
         if (lc < 1) return CF_ERR_INVALID_ARG;                       // every sequence decodes one token
         if ((int64_t)lc > (int64_t)max_blocks_per_seq * B) return CF_ERR_OUT_OF_RANGE;
-        total_pages += (lc + B - 1) / B;
     }
-    const int64_t slots = (int64_t)cfg.num_sms * cfg.decode_ctas_per_sm * cfg.decode_waves;
-    const int32_t quantum = cfg.decode_page_quantum;
-    int64_t target = (total_pages * desc->num_kv_heads + slots - 1) / slots;
-    if (target < cfg.decode_min_chunk_pages) target = cfg.decode_min_chunk_pages;
-    target = (target + quantum - 1) / quantum * quantum;
+    const int64_t target = decode_target_pages(num_seqs, [&](int32_t s) -> int64_t { return context_len[s]; }, B,
+                                               desc->num_kv_heads, D, cfg, false);
 
     StaticPlan pl;
     for (int32_t s = 0; s < num_seqs; ++s) {
         const int32_t lc = context_len[s];
         const int64_t pages = (lc + B - 1) / B;
-        int64_t n = (pages + target - 1) / target;
-        int64_t per = (pages + n - 1) / n;
-        per = (per + quantum - 1) / quantum * quantum;
-        n = (pages + per - 1) / per;
+        int64_t n = 1, per = pages;
+        decode_split(pages, target, cfg.decode_page_quantum, &n, &per);
         if (pl.n_items + n > kStaticMaxItems) return CF_ERR_WORKSPACE;
         int32_t first = -1;
         if (n > 1) {
@@ -469,6 +489,13 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
             it.chunk = (int32_t)c;
         }
     }
+    // longest chunk first, like the context path (std::sort works in place: no temporary buffer); the order of
+    // the items does not change any bit of the result
+    std::sort(pl.items, pl.items + pl.n_items, [](const DecodeItem& a, const DecodeItem& b) {
+        const int32_t la = a.kv_end - a.kv_begin, lb = b.kv_end - b.kv_begin;
+        if (la != lb) return la > lb;
+        return a.seq != b.seq ? a.seq < b.seq : a.chunk < b.chunk;
+    });
     const size_t items_bytes = sizeof(DecodeItem) * (size_t)pl.n_items;
     const size_t comb_off = (items_bytes + 255) / 256 * 256;
     const size_t comb_bytes = sizeof(CombineItem) * (size_t)pl.n_comb;
@@ -479,13 +506,12 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
 
     // Pageable-source copies: the runtime stages the bytes before returning, so the stack arrays
     // may go out of scope as soon as this function returns.
-    cudaStream_t stream = (cudaStream_t)cuda_stream;
     if (cudaMemcpyAsync(su.base, pl.items, items_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess) return CF_ERR_CUDA;
     if (comb_bytes &&
         cudaMemcpyAsync(su.base + comb_off, pl.comb, comb_bytes, cudaMemcpyHostToDevice, stream) != cudaSuccess)
         return CF_ERR_CUDA;
 
-    AttnParams p;
+    AttnParams p = {};
     p.q = (const __nv_bfloat16*)q;
     p.k_cache = (const __nv_bfloat16*)k_cache;
     p.v_cache = (const __nv_bfloat16*)v_cache;
@@ -493,23 +519,18 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     p.lse = lse;
     p.block_table = block_table;
     p.max_blocks = max_blocks_per_seq;
+    p.num_blocks = desc->num_blocks;
     p.ks_block = desc->k_stride_block; p.ks_head = desc->k_stride_head; p.ks_token = desc->k_stride_token;
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
     p.scale_log2 = (desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf((float)D)) * 1.4426950408889634f;
-    p.context_len = nullptr; p.query_len = nullptr; p.q_start = nullptr;   // not read by these two kernels
     p.dec_items = reinterpret_cast<const DecodeItem*>(su.base);
     p.comb_items = reinterpret_cast<const CombineItem*>(su.base + comb_off);
-    p.pre_items = nullptr;
-    p.pre_tc_items = nullptr;
-    p.pre_part_o = nullptr; p.pre_part_ml = nullptr; p.pre_comb_items = nullptr;
     // Partials need no clearing: every slot the combine kernel reads is fully written by its decode CTA
-    // in the same call.
+    // in the same call.  This entry point keeps the separate combine kernel (no ticket counters), so nothing
+    // in the array has to start at zero; the merge routine and its chunk order are those of the fused merge.
     p.part_o = reinterpret_cast<float*>(su.base + kStaticPlanBytes);
     p.part_ml = reinterpret_cast<float*>(su.base + kStaticPlanBytes + part_o_bytes);
-    p.dec_counters = nullptr;     // this entry point keeps the separate combine kernel: nothing in the array has to start at zero
-    p.pre_queue = nullptr;
-    p.err = nullptr;
     if (launch_decode(p, D, pl.n_items, stream) != cudaSuccess) return CF_ERR_CUDA;
     if (launch_combine(p, D, pl.n_comb, stream) != cudaSuccess) return CF_ERR_CUDA;
     return CF_OK;

@@ -16,6 +16,7 @@ struct AttnParams {
     float* lse;                       // may be null
     const int32_t* block_table;
     int32_t max_blocks;
+    int32_t num_blocks;               // pool size; block ids outside [0, num_blocks) are skipped and reported
     int64_t ks_block, ks_head, ks_token;
     int64_t vs_block, vs_head, vs_token;
     int32_t Hq, Hkv, G;
@@ -25,7 +26,6 @@ struct AttnParams {
     const int32_t* q_start;
     const DecodeItem* dec_items;
     const CombineItem* comb_items;
-    const PrefillItem* pre_items;
     const PrefillTcItem* pre_tc_items;
     float* part_o;                    // [slot, Hq, D] fp32 un-normalised partial outputs
     float* part_ml;                   // [slot, Hq, 2] running max (log2 domain) and sum
@@ -34,8 +34,12 @@ struct AttnParams {
     float* pre_part_ml;               // [row slot, 2]
     const PrefillCombineItem* pre_comb_items;
     uint32_t* pre_queue;              // [2] ticket counter of the persistent prefill CTAs, and how many of them have left
-    uint32_t* err;                    // device error word
+    uint32_t* err;                    // device error word (bits below); may be null
 };
+
+// Bits of the device error word
+constexpr uint32_t kErrTimeout = 1u;      // a bounded wait expired
+constexpr uint32_t kErrBlockId = 2u;      // a block-table entry in use lay outside the pool; its page was skipped
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p)
 {

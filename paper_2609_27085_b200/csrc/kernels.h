@@ -16,6 +16,8 @@ struct AppendParams {
     int64_t ks_block, ks_head, ks_token;
     int64_t vs_block, vs_head, vs_token;
     int32_t Hkv, D, num_seqs, total_rows;
+    int32_t num_blocks;               // pool size: a block id outside [0, num_blocks) is reported, its row not written
+    uint32_t* err;                    // device error word (may be null)
     const int32_t* context_len;
     const int32_t* query_len;
     const int32_t* q_start;
@@ -26,17 +28,12 @@ cudaError_t launch_validate_table(const int32_t* block_table, int32_t max_blocks
                                   int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
-// mma.sync chunked prefill; tile height must equal kPrefillMmaTileRows
-constexpr int kPrefillMmaTileRows = 64;
-cudaError_t launch_prefill_mma(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
-
 // tcgen05 / tensor-memory chunked prefill (head_dim 64 or 128): `n_ctas` persistent CTAs draw the `n_items`
 // PrefillTcItems from the ticket counter p.pre_queue, which `queue_ctas` CTAs share in total (several
 // launches may draw from one counter; the last CTA to leave resets it).  Ticket t stands for item
 // ticket_base + t; with first_static set, CTA b starts on item b without a draw (then ticket_base = n_ctas of
 // that grid, also for a second grid that shares the counter).  `resident`, when not null, is a device word that
 // every CTA increments as it starts.
-bool prefill_tc_supported(const cf_cache_desc* desc);
 cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
                               int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
 

@@ -19,6 +19,10 @@ __global__ void __launch_bounds__(256) kv_append_kernel(const AppendParams p)
     const int pos = __ldg(p.context_len + s) - __ldg(p.query_len + s) + i;
     const int64_t blk = __ldg(p.block_table + (int64_t)s * p.max_blocks + (pos >> 4));
     const int slot = pos & 15;
+    if (blk < 0 || blk >= p.num_blocks) {        // never write outside the pool
+        if (threadIdx.x == 0 && p.err) atomicOr(p.err, kErrBlockId);
+        return;
+    }
 
     const int chunks_per_head = p.D / 8;
     const int per_tensor = p.Hkv * chunks_per_head;

@@ -74,59 +74,21 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     const int32_t B = d->block_size;
 
     // ---- decode: near-equal KV chunks, sized so that (chunks x kv heads) fills the machine a few times
-    int64_t total_pages = 0;
     for (int32_t s = 0; s < num_seqs; ++s)
-        if (query_len[s] == 1) {
-            total_pages += (context_len[s] + B - 1) / B;
-            ++plan->n_decode_seqs;
-        } else if (query_len[s] > 1) {
-            ++plan->n_prefill_seqs;
-        }
-    const int64_t slots = (int64_t)std::max(1, cfg.num_sms) * std::max(1, cfg.decode_ctas_per_sm)
-                          * std::max(1, cfg.decode_waves);
+        if (query_len[s] == 1) ++plan->n_decode_seqs;
+        else if (query_len[s] > 1) ++plan->n_prefill_seqs;
     const int32_t quantum = std::max(1, cfg.decode_page_quantum);
-    int64_t target = (total_pages * d->num_kv_heads + slots - 1) / slots;
     const bool shares_sms = cfg.prefill_sms_mixed > 0 && plan->n_prefill_seqs > 0;   // spatial sequence: decode runs on part of the machine, beside prefill
-    if (target < cfg.decode_min_chunk_pages && total_pages > 0 && !shares_sms) {
-        // A small batch: chunks of the minimum length would not fill `decode_waves` waves, and how many waves
-        // of (num_sms x ctas_per_sm) CTAs they do fall into decides the time (a last wave that is a quarter
-        // full costs a whole CTA time).  Try chunk lengths from the minimum to four times it and keep the
-        // one with the smallest waves x (CTA start-up + chunk streaming time).  (Not when decode shares the SMs
-        // with a prefill grid: there the short chunks measured better, 81 against 90 us on the TP4 shard.)
-        const int64_t wave = (int64_t)std::max(1, cfg.num_sms) * std::max(1, cfg.decode_ctas_per_sm);
-        const double page_us = (2.0 * B * d->head_dim * 2.0) / (7.56e6 / (double)wave);   // one (page, head) of K and V at a CTA's share of HBM
-        const double cta_us = 2.5;
-        double best = 1e30;
-        int64_t best_c = cfg.decode_min_chunk_pages;
-        for (int64_t c = (cfg.decode_min_chunk_pages + quantum - 1) / quantum * quantum; c <= 4 * (int64_t)cfg.decode_min_chunk_pages;
-             c += quantum) {
-            int64_t ctas = 0, longest = 0;
-            for (int32_t s = 0; s < num_seqs; ++s) {
-                if (query_len[s] != 1) continue;
-                const int64_t pages = (context_len[s] + B - 1) / B;
-                int64_t n = (pages + c - 1) / c;
-                int64_t per = ((pages + n - 1) / n + quantum - 1) / quantum * quantum;
-                n = (pages + per - 1) / per;
-                ctas += n;
-                longest = std::max(longest, std::min(per, pages));
-            }
-            ctas *= d->num_kv_heads;
-            const double t = (double)((ctas + wave - 1) / wave) * (cta_us + page_us * (double)longest);
-            if (t < best * 0.999) { best = t; best_c = c; }
-        }
-        target = best_c;
-    }
-    target = std::max<int64_t>(target, cfg.decode_min_chunk_pages);
-    target = (target + quantum - 1) / quantum * quantum;
+    const int64_t target = decode_target_pages(
+        num_seqs, [&](int32_t s) -> int64_t { return query_len[s] == 1 ? (int64_t)context_len[s] : -1; }, B, d->num_kv_heads,
+        d->head_dim, cfg, shares_sms);
 
     for (int32_t s = 0; s < num_seqs; ++s) {
         if (query_len[s] != 1) continue;
         const int32_t lc = context_len[s];
         const int64_t pages = (lc + B - 1) / B;
-        int64_t n = (pages + target - 1) / target;
-        int64_t per = (pages + n - 1) / n;
-        per = (per + quantum - 1) / quantum * quantum;
-        n = (pages + per - 1) / per;
+        int64_t n = 1, per = pages;
+        decode_split(pages, target, quantum, &n, &per);
         int32_t first = -1;
         if (n > 1) {
             first = plan->n_part_slots;
@@ -151,7 +113,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     });
 
     // ---- prefill: q tiles of every chunk, the tile with the longest visible KV range first
-    if (cfg.prefill_tc) {
+    {
         // pairs of 128-row tiles that share a KV head: two heads of a group over the same rows, or
         // (group size 1) two consecutive row tiles of one head
         constexpr int32_t TR = 128;
@@ -337,23 +299,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 plan->prefill_tc.push_back(f);
             }
         }
-        return CF_OK;
     }
-    const int32_t tr = std::max(1, cfg.prefill_tile_rows);
-    struct Keyed { int64_t extent; PrefillItem it; };
-    std::vector<Keyed> tiles;
-    for (int32_t s = 0; s < num_seqs; ++s) {
-        const int32_t lq = query_len[s];
-        if (lq <= 1) continue;
-        const int32_t prefix = context_len[s] - lq;
-        for (int32_t r0 = 0; r0 < lq; r0 += tr) {
-            const int32_t n = std::min(tr, lq - r0);
-            tiles.push_back(Keyed{(int64_t)prefix + r0 + n, PrefillItem{s, plan->q_start[s] + r0, r0, n}});
-        }
-    }
-    std::stable_sort(tiles.begin(), tiles.end(), [](const Keyed& a, const Keyed& b) { return a.extent > b.extent; });
-    plan->prefill.reserve(tiles.size());
-    for (const Keyed& k : tiles) plan->prefill.push_back(k.it);
     return CF_OK;
 }
 
@@ -381,9 +327,9 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
     // Constants fitted to CUDA-event times of the kernels on a B200: split-K decode (with the merge of the
     // partials fused in) sustains ~7.56 TB/s on top of ~22 us of launch, ramp and tail; the separate combine
     // launch, when it is used, ~8 us, reported as 0 here because the default path has none; one tcgen05
-    // prefill item costs ~8 us plus ~1.9 us per 128-token KV tile; the mma.sync path runs ~220 TFLOP/s.
+    // prefill item costs ~8 us plus ~1.9 us per 128-token KV tile.
     constexpr double kDecodeFixedUs = 22.0, kDecodeBytesPerUs = 7.56e6, kCombineUs = 0.0;
-    constexpr double kTcItemFixedUs = 8.0, kTcTileUs = 1.9, kMmaFlopsPerUs = 220e6, kLaunchUs = 4.0;
+    constexpr double kTcItemFixedUs = 8.0, kTcTileUs = 1.9, kLaunchUs = 4.0;
     Estimate e;
     const int32_t S = (int32_t)plan.q_start.size() - 1;
     double dec_bytes = 0.0;
@@ -407,14 +353,6 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
         }
         e.us_prefill = (float)(kLaunchUs + list_schedule(jobs, (size_t)std::max(1, num_sms)));
         if (!plan.prefill_combine.empty()) e.us_prefill += (float)(6.0 + 0.05 * (double)plan.prefill_tc.size());
-    } else if (!plan.prefill.empty()) {
-        double flops = 0.0;
-        for (int32_t s = 0; s < S; ++s)
-            if (query_len[s] > 1) {
-                const double lq = query_len[s], pre = context_len[s] - query_len[s];
-                flops += 4.0 * d->head_dim * d->num_q_heads * (lq * pre + lq * (lq + 1) / 2);
-            }
-        e.us_prefill = (float)(kLaunchUs + flops / kMmaFlopsPerUs);
     }
     return e;
 }

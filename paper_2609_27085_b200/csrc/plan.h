@@ -28,13 +28,6 @@ struct CombineItem {       // one decode sequence that was split
     int32_t n_chunks;
 };
 
-struct PrefillItem {       // one q tile of one prefill chunk; the kernel adds the head index
-    int32_t seq;
-    int32_t q_row0;        // packed row of the tile's first row
-    int32_t row0;          // index of that row inside the chunk (0-based)
-    int32_t n_rows;        // rows in this tile (<= tile height)
-};
-
 struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one KV head (tile 1 may be absent)
     int32_t seq;
     int32_t kvh;
@@ -67,8 +60,6 @@ struct PlanConfig {
     int32_t decode_waves = 4;         // target number of CTA waves (load balance vs. partial traffic)
     int32_t decode_min_chunk_pages = 32;
     int32_t decode_page_quantum = 4;  // chunk lengths are multiples of this many pages (warps per CTA)
-    int32_t prefill_tile_rows = 64;   // tile height of the mma.sync prefill kernel
-    bool prefill_tc = false;          // true: plan items for the tcgen05 kernel (128-row tile pairs)
     int32_t prefill_sms_mixed = 0;    // > 0: SMs the prefill items are balanced over when the batch also holds decode
                                       // work (spatial launch sequence: the first prefill grid's share); 0: num_sms
     int32_t prefill_force_split = 0;  // >= 2: split every tcgen05 item that many ways (tests); 0: cost model decides
@@ -78,7 +69,6 @@ struct Plan {
     std::vector<int32_t> q_start;     // [S+1] exclusive prefix sum of query_len
     std::vector<DecodeItem> decode;   // longest chunk first
     std::vector<CombineItem> combine;
-    std::vector<PrefillItem> prefill; // longest KV extent first (mma.sync kernel)
     std::vector<PrefillTcItem> prefill_tc;   // longest KV extent first (tcgen05 kernel); KV-split items appear part_k times
     std::vector<PrefillCombineItem> prefill_combine;   // one per KV-split item
     int32_t n_pre_slots = 0;          // fp32 partial rows of KV-split prefill items (compact, D floats each)
@@ -93,6 +83,71 @@ cf_status validate_desc(const cf_cache_desc* d);
 // Validates lengths against the block-table width; fills q_start/total_q.
 cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
                            int32_t num_seqs, int32_t max_blocks_per_seq, Plan* plan);
+// Decode chunking, shared by build_plan and by the allocation-free entry point (plain loops over the
+// caller's arrays: nothing here allocates).  `lc_of(s)` returns the context length of sequence s if it is
+// a decode sequence and a negative number otherwise.
+//   decode_target_pages: the chunk length (in pages) that fills the machine `decode_waves` times, or, for a
+//     batch too small for that, the length from [min, 4 x min] with the smallest waves x CTA time.
+//   decode_split: near-equal chunks of at most `target` pages, each a multiple of the page quantum.
+template <class LcOf>
+inline int64_t decode_target_pages(int32_t num_seqs, LcOf lc_of, int32_t B, int32_t Hkv, int32_t D, const PlanConfig& cfg,
+                                   bool shares_sms)
+{
+    const int64_t wave = (int64_t)(cfg.num_sms > 1 ? cfg.num_sms : 1) * (cfg.decode_ctas_per_sm > 1 ? cfg.decode_ctas_per_sm : 1);
+    const int64_t slots = wave * (cfg.decode_waves > 1 ? cfg.decode_waves : 1);
+    const int64_t quantum = cfg.decode_page_quantum > 1 ? cfg.decode_page_quantum : 1;
+    const int64_t min_pages = cfg.decode_min_chunk_pages > 1 ? cfg.decode_min_chunk_pages : 1;
+    int64_t total_pages = 0;
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int64_t lc = lc_of(s);
+        if (lc >= 0) total_pages += (lc + B - 1) / B;
+    }
+    int64_t target = (total_pages * Hkv + slots - 1) / slots;
+    if (target < min_pages && total_pages > 0 && !shares_sms) {
+        // A small batch: chunks of the minimum length would not fill `decode_waves` waves, and how many waves
+        // of (num_sms x ctas_per_sm) CTAs they do fall into decides the time (a last wave that is a quarter
+        // full costs a whole CTA time).  Try chunk lengths from the minimum to four times it and keep the
+        // one with the smallest waves x (CTA start-up + chunk streaming time).  (Not when decode shares the SMs
+        // with a prefill grid: there the short chunks measured better.)
+        const double page_us = (2.0 * B * D * 2.0) / (7.56e6 / (double)wave);   // one (page, head) of K and V at a CTA's share of HBM
+        const double cta_us = 2.5;
+        double best = 1e30;
+        int64_t best_c = min_pages;
+        for (int64_t c = (min_pages + quantum - 1) / quantum * quantum; c <= 4 * min_pages; c += quantum) {
+            int64_t ctas = 0, longest = 0;
+            for (int32_t s = 0; s < num_seqs; ++s) {
+                const int64_t lc = lc_of(s);
+                if (lc < 0) continue;
+                const int64_t pages = (lc + B - 1) / B;
+                int64_t n = (pages + c - 1) / c;
+                if (n < 1) n = 1;
+                const int64_t per = ((pages + n - 1) / n + quantum - 1) / quantum * quantum;
+                n = per > 0 ? (pages + per - 1) / per : 1;
+                ctas += n;
+                const int64_t len = per < pages ? per : pages;
+                if (len > longest) longest = len;
+            }
+            ctas *= Hkv;
+            const double t = (double)((ctas + wave - 1) / wave) * (cta_us + page_us * (double)longest);
+            if (t < best * 0.999) { best = t; best_c = c; }
+        }
+        target = best_c;
+    }
+    if (target < min_pages) target = min_pages;
+    return (target + quantum - 1) / quantum * quantum;
+}
+inline void decode_split(int64_t pages, int64_t target, int32_t quantum, int64_t* n_chunks, int64_t* pages_per_chunk)
+{
+    const int64_t qn = quantum > 1 ? quantum : 1;
+    int64_t n = (pages + target - 1) / target;
+    if (n < 1) n = 1;
+    int64_t per = (pages + n - 1) / n;
+    per = (per + qn - 1) / qn * qn;
+    if (per < qn) per = qn;
+    *n_chunks = (pages + per - 1) / per > 0 ? (pages + per - 1) / per : 1;
+    *pages_per_chunk = per;
+}
+
 // Full plan (calls validate_lengths).
 cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
                      int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan);

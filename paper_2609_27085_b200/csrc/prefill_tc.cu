@@ -23,6 +23,7 @@
 // are never loaded.
 // Every wait is bounded: on expiry the CTA raises an abort flag, every role leaves its loop, the
 // error word is set and tensor memory is released.
+#include <atomic>
 #include <type_traits>
 
 #include "device_common.cuh"
@@ -74,13 +75,16 @@ template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setma
 template <int N> __device__ __forceinline__ void reg_inc() { asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(N)); }
 // 2^x for a packed pair on the FMA and integer pipes (no special-function unit): x = n + f with
 // n = round(x) taken from the low mantissa bits of x + 1.5*2^23, 2^f on [-1/2, 1/2] by a degree-4
-// polynomial (relative error 2.7e-6), and n added into the exponent field.  x is clamped at -126
-// (masked scores are -inf); x must stay below +127.
+// polynomial (relative error 2.7e-6), and n added into the exponent field.  x is clamped to
+// [-126, 127]: masked scores are -inf, and a score far above a stale reference maximum (tiles after
+// the first run against a reference that is only raised on demand) must come out as a huge finite
+// value, >= 2^127, so that the tile's row sum exceeds the rescale threshold; unclamped, the exponent
+// add would wrap into the sign bit and the key would silently vanish.
 __device__ __forceinline__ float2 exp2_poly2(float2 x)
 {
     const float kMagic = 12582912.f;
-    x.x = fmaxf(x.x, -126.f);
-    x.y = fmaxf(x.y, -126.f);
+    x.x = fminf(fmaxf(x.x, -126.f), 127.f);
+    x.y = fminf(fmaxf(x.y, -126.f), 127.f);
     const float2 t = add2(x, make_float2(kMagic, kMagic));
     const float2 n = add2(t, make_float2(-kMagic, -kMagic));
     const float2 f = fma2(n, make_float2(-1.f, -1.f), x);
@@ -117,33 +121,6 @@ __device__ __forceinline__ float max3(float a, float b, float c)
 }
 
 }  // namespace
-
-// Development aid, compiled only with -DCF_TRACE: one CTA stamps clock64 at the marked points of every role
-// (rows: 0 producer, 1 issuer, 2/3 first softmax thread of q tile 0/1); cf_trace_read copies the stamps out.
-#ifdef CF_TRACE
-#ifndef CF_TRACE_CTA
-#define CF_TRACE_CTA 0
-#endif
-__device__ unsigned long long cf_trace_buf[4][256][2];
-#define TR_DECL unsigned tr_n = 0u
-#define TR(role, id)                                                                      \
-    do {                                                                                  \
-        if (blockIdx.x == CF_TRACE_CTA && tr_n < 256u) {                                  \
-            cf_trace_buf[role][tr_n][0] = (unsigned long long)(id);                       \
-            cf_trace_buf[role][tr_n][1] = (unsigned long long)clock64();                  \
-            ++tr_n;                                                                       \
-        }                                                                                 \
-    } while (0)
-#ifdef CF_TRACE_FINE
-#define TRF(role, id) TR(role, id)
-#else
-#define TRF(role, id)
-#endif
-#else
-#define TR_DECL
-#define TR(role, id)
-#define TRF(role, id)
-#endif
 
 // What a role needs to know about the work item it is on.  The producer warp builds it and hands it
 // to the other roles through a two-slot ring in shared memory.
@@ -212,7 +189,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     volatile uint32_t* abort_flag = &abort_s;
 
     if (threadIdx.x == 0) {
-        abort_s = (p.err != nullptr && *reinterpret_cast<volatile uint32_t*>(p.err) != 0u) ? 2u : 0u;   // an earlier CTA gave up
+        abort_s = (p.err != nullptr && (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrTimeout) != 0u) ? 2u : 0u;   // an earlier CTA gave up
         // spatial launch sequence with CF_SPATIAL_WAIT=1: the stream that carries the decode kernel waits (a
         // stream memory operation, not a kernel) until every CTA of this grid holds its SM
         if (resident != nullptr) atomicAdd(resident, 1u);
@@ -242,6 +219,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     // (the K/V rows of cf_kv_append when the batch has no decode part).
     asm volatile("griddepcontrol.wait;" ::: "memory");
 
+    // A block id outside the pool is not used as a TMA coordinate: page 0 is fetched in its place and the error
+    // word is set (the rows of that sequence are then meaningless, but nothing is read outside the pool).
+    auto checked_pid = [&](int32_t id) -> int32_t {
+        if ((uint32_t)id < (uint32_t)p.num_blocks) return id;
+        if (p.err) atomicOr(p.err, kErrBlockId);
+        return 0;
+    };
     // the context of a role's k-th item (slot k & 1, filled for the (k >> 1)-th time); null on an abort.
     // A role copies the fields it needs at once: the slot is rewritten two items later.
     auto wait_item = [&](int k) -> const ItemCtx* {
@@ -264,13 +248,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (cs == nullptr || cs->live == 0) break;
             const int n_max = cs->n_max, total_pages = cs->total_pages, jb = cs->it.j_begin, kvh = cs->it.kvh;
             const int32_t* bt = p.block_table + (int64_t)cs->it.seq * p.max_blocks;
-            int32_t pid = lane < min(8, total_pages - 8 * jb) ? __ldg(bt + 8 * jb + lane) : 0;
+            int32_t pid = lane < min(8, total_pages - 8 * jb) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
             for (int j = 0; j < n_max && ok; ++j) {
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
                 const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
-                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
+                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? checked_pid(__ldg(bt + 8 * (jb + j + 1) + lane)) : 0;
                 const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
@@ -292,8 +276,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             prefetch_tensormap(&map_v);
         }
         bool counted_out = false;
-        TR_DECL;
-        if (lane == 0) TR(0, 100);
         // draws the next ticket; on the first empty draw the CTA is counted out and the last CTA resets the counters
         auto draw = [&](ItemCtx& cx) {
             int idx = n_items;
@@ -322,7 +304,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         } else {
             draw(cx);
         }
-        if (lane == 0) TR(0, 101);
         uint32_t ub[2] = {0u, 0u};              // how often each K/V ring stage has been filled before this item
         bool ok = true;
         for (int k = 0; ok; ++k) {
@@ -335,7 +316,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
                 for (int i = 0; i < (int)(sizeof(ItemCtx) / 16); ++i) dst[i] = src[i];
                 mbar_arrive(smem_u32(&bars.item_full[k & 1]));
-                TR(0, 102);
             }
             if (!cx.live) break;
             const PrefillTcItem& it = cx.it;
@@ -353,13 +333,13 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const int j_draw = min(2, n_max - 1);       // the next ticket is drawn once the first tiles are on their way
             bool drawn = false;
             // page ids of a tile are fetched while the tile before it is being issued
-            int32_t pid = lane < min(8, total_pages - 8 * jb) ? __ldg(bt + 8 * jb + lane) : 0;
+            int32_t pid = lane < min(8, total_pages - 8 * jb) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
             for (int j = 0; j < n_max && ok; ++j) {
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
                 const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
-                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? __ldg(bt + 8 * (jb + j + 1) + lane) : 0;
+                if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? checked_pid(__ldg(bt + 8 * (jb + j + 1) + lane)) : 0;
                 const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
@@ -368,11 +348,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (lane < HALVES * np)
                     tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane % HALVES) * 64, 0, it.kvh, my_pid,
                                 smem_u32(&bars.k_full[stage]));
-                if (lane == 0 && (j < 5 || j >= n_max - 2)) TR(0, 200 + j);
                 if (j == j_draw) {
                     draw(nx);
                     drawn = true;
-                    if (lane == 0) TR(0, 104);
                 }
             }
             ok = __all_sync(0xffffffffu, ok);
@@ -449,15 +427,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         // read from the context slot where they are needed (the slot is not rewritten before this lane has
         // left the next item's last S = Q K^T behind), and only the interior loop keeps its parities in registers.
         volatile uint32_t* const ist = issuer_state;
-        TR_DECL;
-        TR(1, 100);
         ist[0] = ist[1] = ist[2] = ist[3] = 0u;
         bool ok = true;
         for (int k = 0; ok; ++k) {
         const ItemCtx* cs = wait_item(k);
         if (cs == nullptr || cs->live == 0) break;
         const volatile ItemCtx* const vs = cs;
-        TR(1, 1);
         const int n_max = cs->n_max;
         const int n_j[2] = {cs->n_j[0], cs->n_j[1]};
         ok = mbar_wait(smem_u32(&bars.q_full), (uint32_t)k & 1u, abort_flag);
@@ -467,7 +442,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (n_j[0] > 0) issue_qk(I0{}, I0{});
         if (n_j[1] > 0) issue_qk(I1{}, I0{});
         umma_commit(bar_ke[0]);
-        TR(1, 3);
         // q_empty: arrives when every S = Q K^T of the item has completed (the last one is issued in step n_max - 2)
         if (n_max <= 1) umma_commit(bar_qe);
         // ---- interior tiles: both q tiles present and continuing, all 8 pages loaded, not the last tile
@@ -475,25 +449,18 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         auto lean_step = [&](auto S, uint32_t par_v, uint32_t par_k1, uint32_t par_p0, uint32_t par_p1, uint32_t acc0) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
-            TRF(1, 10);
             if (!mbar_wait(bar_vf[st], par_v, abort_flag)) return false;
-            TRF(1, 11);
             if (!mbar_wait(bar_kf[st1], par_k1, abort_flag)) return false;
-            TRF(1, 12);
             if (!mbar_wait(bar_p[0], par_p0, abort_flag)) return false;
-            TRF(1, 13);
             tc_fence_after();
             issue_pv(I0{}, S, 8, acc0);
             issue_qk(I0{}, S1{});
-            TRF(1, 14);
             if (!mbar_wait(bar_p[1], par_p1, abort_flag)) return false;
-            TRF(1, 15);
             tc_fence_after();
             issue_pv(I1{}, S, 8, acc0);
             issue_qk(I1{}, S1{});
             umma_commit(bar_ve[st]);
             umma_commit(bar_ke[st1]);
-            TRF(1, 16);
             return true;
         };
         int j = 0;
@@ -550,9 +517,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
         for (; j < n_max && ok; ++j) {
             ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
-            TR(1, 300 + j);
         }
-        TR(1, 4);
         ist[0] += (uint32_t)(n_max + 1) >> 1;
         ist[1] += (uint32_t)n_max >> 1;
         ist[2] += (uint32_t)n_j[0];
@@ -568,8 +533,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const uint32_t lanes = lane_field(warp);
       const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * D + lanes;
       const float sc = p.scale_log2;
-      TR_DECL;
-      if ((warp & 3) == 0 && lane == 0) TR(2 + t, 100);
       uint32_t sbt = 0u;                       // tiles of this q tile in earlier items: running phase of s_full / p_full / o_done
       bool ok = true;
       for (int k = 0; ok; ++k) {
@@ -585,7 +548,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         for (int j = 0; j < n_jt; ++j) {
             ok = mbar_wait(smem_u32(&bars.s_full[t]), (sbt + (uint32_t)j) & 1u, abort_flag);
             if (!ok) break;
-            if ((warp & 3) == 0 && lane == 0 && (j < 5 || j >= n_jt - 2)) TR(2 + t, 400 + j);
             tc_fence_after();
             float sv[128];
 #pragma unroll
@@ -672,10 +634,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             tc_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(smem_u32(&bars.p_full[t]));
-            if ((warp & 3) == 0 && lane == 0 && (j < 5 || j >= n_jt - 2)) TR(2 + t, 500 + j);
         }
         if (ok && n_jt > 0) ok = mbar_wait(smem_u32(&bars.o_done[t]), (sbt + (uint32_t)(n_jt - 1)) & 1u, abort_flag);
-        if ((warp & 3) == 0 && lane == 0) TR(2 + t, 6);
         if (ok && n_jt > 0) {
             tc_fence_after();
             const float inv = 1.f / l_sum;
@@ -711,7 +671,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             // program order, is what allows the issuer to overwrite it
             tc_fence_before();
         }
-        if ((warp & 3) == 0 && lane == 0) TR(2 + t, 7);
         sbt += (uint32_t)n_jt;
         }
       }
@@ -721,18 +680,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
     tc_fence_before();
     __syncthreads();
     if (abort_s == 1u) {
-        if (threadIdx.x == 0 && p.err) atomicExch(p.err, 1u);
+        if (threadIdx.x == 0 && p.err) atomicOr(p.err, kErrTimeout);
         // let copies and MMAs that may still be in flight settle before tensor memory is handed back
         for (int i = 0; i < 64; ++i) __nanosleep(2000);
         __syncthreads();
     }
     if (warp == 0) tmem_dealloc<512>(tmem);
-#ifdef CF_TRACE
-    if (threadIdx.x == 0 && blockIdx.x == CF_TRACE_CTA) {
-        cf_trace_buf[0][255][0] = 999ull;
-        cf_trace_buf[0][255][1] = (unsigned long long)clock64();
-    }
-#endif
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -813,7 +766,7 @@ __global__ void __launch_bounds__(32) wait_selftest_kernel(uint32_t* err)
     __syncwarp();
     const bool ok = mbar_wait(smem_u32(&bar), 0, &abort_s, 1ll << 23);
     __syncwarp();
-    if (!ok && threadIdx.x == 0 && err) atomicExch(err, 1u);
+    if (!ok && threadIdx.x == 0 && err) atomicOr(err, kErrTimeout);
 }
 
 cudaError_t launch_wait_selftest(uint32_t* err, cudaStream_t stream)
@@ -871,12 +824,6 @@ bool encode_q(CUtensorMap* m, const void* base, int D, int total_rows, int Hq)
 
 }  // namespace
 
-bool prefill_tc_supported(const cf_cache_desc* d)
-{
-    // TMA needs 16-byte aligned strides (checked for every descriptor); rows of 64 or 128 elements
-    return (d->head_dim == 128 || d->head_dim == 64) && d->block_size == 16;
-}
-
 namespace {
 
 template <int D>
@@ -887,19 +834,21 @@ cudaError_t launch_prefill_tc_t(const CUtensorMap& mq, const CUtensorMap& mk, co
     const size_t smem = Geo<D>::SMEM_TOTAL + 1024;
     // The register hand-over inside the kernel (setmaxnreg) is sized for LAUNCH_REGS registers per thread at
     // launch; with any other count a grow request could block forever, so such a build is never launched.
-    static int regs_ok = -1;
-    if (regs_ok < 0) {
+    // (both are set once; host threads racing here compute and store the same values)
+    static std::atomic<int> regs_ok{-1};
+    if (regs_ok.load(std::memory_order_acquire) < 0) {
         cudaFuncAttributes fa;
-        regs_ok = (cudaFuncGetAttributes(&fa, prefill_tc_kernel<D>) == cudaSuccess && fa.numRegs == LAUNCH_REGS) ? 1 : 0;
+        regs_ok.store((cudaFuncGetAttributes(&fa, prefill_tc_kernel<D>) == cudaSuccess && fa.numRegs == LAUNCH_REGS) ? 1 : 0,
+                      std::memory_order_release);
     }
-    if (!regs_ok) return cudaErrorLaunchOutOfResources;
-    static bool configured[64] = {};
+    if (!regs_ok.load(std::memory_order_acquire)) return cudaErrorLaunchOutOfResources;
+    static std::atomic<bool> configured[64];
     int dev = 0;
     cudaGetDevice(&dev);
-    if (dev >= 0 && dev < 64 && !configured[dev]) {
+    if (dev >= 0 && dev < 64 && !configured[dev].load(std::memory_order_acquire)) {
         cudaError_t e = cudaFuncSetAttribute(prefill_tc_kernel<D>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
         if (e != cudaSuccess) return e;
-        configured[dev] = true;
+        configured[dev].store(true, std::memory_order_release);
     }
     // Programmatic dependent launch: barrier set-up and tensor-memory allocation run while the kernel
     // before this one in the stream drains; the kernel waits (griddepcontrol.wait) before its first read.
@@ -933,10 +882,3 @@ cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, in
 }
 
 }  // namespace cf
-
-#ifdef CF_TRACE
-extern "C" int cf_trace_read(void* dst)
-{
-    return (int)cudaMemcpyFromSymbol(dst, cf::cf_trace_buf, sizeof(cf::cf_trace_buf));
-}
-#endif

@@ -101,14 +101,6 @@ __device__ __forceinline__ void tmem_ld16(uint32_t taddr, uint32_t* r)
                    "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
                  : "r"(taddr));
 }
-__device__ __forceinline__ void tmem_st32(uint32_t taddr, const uint32_t* r)
-{
-    asm volatile("tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31,%32};"
-                 ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
-                   "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
-                   "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
-                   "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31]) : "memory");
-}
 __device__ __forceinline__ void tmem_st16(uint32_t taddr, const uint32_t* r)
 {
     asm volatile("tcgen05.st.sync.aligned.32x32b.x16.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16};"
@@ -131,22 +123,6 @@ __device__ __forceinline__ void umma_ts(uint32_t d_tmem, uint32_t a_tmem, uint64
     asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], [%1], %2, %3, p;\n}"
                  ::"r"(d_tmem), "r"(a_tmem), "l"(b_desc), "r"(idesc), "r"(accumulate) : "memory");
 }
-// The same two forms with each shared-memory descriptor given as (low, high) 32-bit halves: the
-// address field sits in the low word, so stepping an operand along K is one 32-bit add.
-__device__ __forceinline__ void umma_ss_lh(uint32_t d_tmem, uint32_t a_lo, uint32_t a_hi, uint32_t b_lo, uint32_t b_hi,
-                                           uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile("{\n.reg .pred p;\n.reg .b64 da, db;\nsetp.ne.b32 p, %6, 0;\nmov.b64 da, {%1, %2};\nmov.b64 db, {%3, %4};\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], da, db, %5, p;\n}"
-                 ::"r"(d_tmem), "r"(a_lo), "r"(a_hi), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void umma_ts_lh(uint32_t d_tmem, uint32_t a_tmem, uint32_t b_lo, uint32_t b_hi, uint32_t idesc,
-                                           uint32_t accumulate)
-{
-    asm volatile("{\n.reg .pred p;\n.reg .b64 db;\nsetp.ne.b32 p, %5, 0;\nmov.b64 db, {%2, %3};\n"
-                 "tcgen05.mma.cta_group::1.kind::f16 [%0], [%1], db, %4, p;\n}"
-                 ::"r"(d_tmem), "r"(a_tmem), "r"(b_lo), "r"(b_hi), "r"(idesc), "r"(accumulate) : "memory");
-}
 // packed pairs of fp32 (one instruction, two lanes of the FMA pipe)
 __device__ __forceinline__ unsigned long long f2_bits(float2 v) { return *reinterpret_cast<unsigned long long*>(&v); }
 __device__ __forceinline__ float2 bits_f2(unsigned long long v) { return *reinterpret_cast<float2*>(&v); }
@@ -162,7 +138,13 @@ __device__ __forceinline__ float2 add2(float2 a, float2 b)
     asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(f2_bits(a)), "l"(f2_bits(b)));
     return bits_f2(d);
 }
-// halves of the 128B-swizzle descriptor (see smem_desc_sw128 below)
+// Shared-memory operand descriptor, 128-byte swizzle: bits 0-13 address>>4, 16-29 leading-dimension
+// byte offset>>4, 32-45 stride-dimension byte offset>>4, 46-47 version (1), 61-63 layout (2 = 128B).
+//   K-major operand ([rows][64 elements] atoms of 8 rows x 128 B): SBO = bytes between 8-row groups,
+//     LBO unused; advance 32 B per K = 16 inside the 64-element row.
+//   MN-major operand ([k][64 elements of M/N] rows of 128 B): LBO = bytes between 64-element groups
+//     along M/N, SBO = bytes between groups of 8 k; advance 16 rows per K = 16.
+// The descriptor is built from its (low, high) 32-bit halves: the address field sits in the low word.
 __device__ __forceinline__ uint32_t desc_lo_sw128(uint32_t saddr, uint32_t lbo_bytes)
 {
     return ((saddr & 0x3FFFFu) >> 4) | (((lbo_bytes >> 4) & 0x3FFFu) << 16);
@@ -177,22 +159,6 @@ __device__ __forceinline__ void umma_commit(uint32_t bar)
     asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
 }
 
-// Shared-memory operand descriptor, 128-byte swizzle: bits 0-13 address>>4, 16-29 leading-dimension
-// byte offset>>4, 32-45 stride-dimension byte offset>>4, 46-47 version (1), 61-63 layout (2 = 128B).
-//   K-major operand ([rows][64 elements] atoms of 8 rows x 128 B): SBO = bytes between 8-row groups,
-//     LBO unused; advance 32 B per K = 16 inside the 64-element row.
-//   MN-major operand ([k][64 elements of M/N] rows of 128 B): LBO = bytes between 64-element groups
-//     along M/N, SBO = bytes between groups of 8 k; advance 16 rows per K = 16.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes)
-{
-    uint64_t d = 0;
-    d |= (uint64_t)((saddr & 0x3FFFFu) >> 4);
-    d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFFu) << 16;
-    d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFFu) << 32;
-    d |= (uint64_t)1 << 46;
-    d |= (uint64_t)2 << 61;
-    return d;
-}
 // Instruction descriptor, kind::f16: D f32 (bit 4), A bf16 (bit 7), B bf16 (bit 10), B MN-major (bit 16),
 // N>>3 at bits 17-22, M>>4 at bits 24-28.
 __host__ __device__ constexpr uint32_t idesc_bf16(uint32_t M, uint32_t N, bool b_mn_major)

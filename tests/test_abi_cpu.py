@@ -94,10 +94,18 @@ def _check_plan(geom, lc, lq, sms=148):
     for s in np.nonzero(lq > 1)[0]:
         mine = pre[pre[:, 0] == s]
         cover = np.zeros((lq[s], geom.num_q_heads), dtype=np.int32)
-        for _, q_row0, row0, n_rows, head, kvh in mine:
-            assert q_row0 == qs[s] + row0 and n_rows >= 1 and kvh == head // G
-            cover[row0:row0 + n_rows, head] += 1
+        tiles_seen = {}
+        for _, q_row0, row0, n_rows, head, kvh, j0, j1 in mine:
+            assert q_row0 == qs[s] + row0 and n_rows >= 1 and kvh == head // G and 0 <= j0 < j1
+            tiles_seen.setdefault((row0, n_rows, head), []).append((j0, j1))
+            if j0 == 0:
+                cover[row0:row0 + n_rows, head] += 1
         assert (cover == 1).all()
+        for (row0, n_rows, head), ranges in tiles_seen.items():
+            # the KV ranges of a q tile tile [0, its number of visible KV tiles) without gap or overlap
+            ranges.sort()
+            assert ranges[0][0] == 0 and ranges[-1][1] == ((lc[s] - lq[s]) + row0 + n_rows + 127) // 128
+            assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
     assert set(int(s) for s in pre[:, 0]) == set(int(s) for s in np.nonzero(lq > 1)[0])
     ext = (lc - lq)[pre[:, 0]] + pre[:, 2] + pre[:, 3]
     if len(ext):
@@ -124,7 +132,7 @@ def test_plan_random_batches():
         lc = lq + rng.integers(0, 5000, size=S)
         _check_plan(syn.GEOM_G4, lc, lq, sms=int(rng.choice([1, 4, 148])))
         _check_plan(syn.Geometry(4, 4, 128, 16, 1 << 16), lc, lq)          # group size 1: row-tile pairs
-        _check_plan(syn.Geometry(8, 2, 64, 16, 1 << 16), lc, lq)           # head_dim 64: mma.sync tiles
+        _check_plan(syn.Geometry(8, 2, 64, 16, 1 << 16), lc, lq)           # head_dim 64
 
 
 def test_calls_without_a_device_fail_with_a_status():
@@ -156,38 +164,48 @@ def test_cost_model_is_sane_on_the_host():
 def test_kv_split_of_the_last_prefill_wave():
     """256 equal items on 148 SMs leave a last wave of 108: the planner cuts those into KV ranges that
     tile each item's extent, never start inside the diagonal band, and fill the machine."""
-    import ctypes
     d = cf.make_desc(32, 8, 128, 16, 65536)
     lc, lq = [24576 + 2048], [2048]
-    st, dec, comb, pre, parts = cf.cf_plan_inspect(d, lc, lq, 4096, 148)
-    counts = np.zeros(6, dtype=np.int32)
-    lcn, lqn = np.array(lc, np.int32), np.array(lq, np.int32)
-    cf.load_library().cf_plan_inspect(ctypes.byref(d), lcn.ctypes.data, lqn.ctypes.data, 1, 4096, 148, None, None, None, 0,
-                                      counts.ctypes.data)
+    st, dec, comb, pre, parts, counts = cf.cf_plan_inspect(d, lc, lq, 4096, 148, want_counts=True)
     n_items = 16 * 16                                   # 16 q tiles x 16 head pairs
     assert counts[5] == n_items % 148                   # the 108 items of the last wave are split
     k = (counts[4] - (n_items - counts[5])) // counts[5]
     assert k >= 2 and counts[4] == (n_items - counts[5]) + counts[5] * k
-    cover = np.zeros((2048, 32), dtype=np.int32)        # listed once per (row, head) all the same
-    for _, q_row0, row0, n_rows, head, kvh in pre:
-        cover[row0:row0 + n_rows, head] += 1
+    cover = np.zeros((2048, 32), dtype=np.int32)        # every (row, head) has exactly one range that starts at tile 0
+    for _, q_row0, row0, n_rows, head, kvh, j0, j1 in pre:
+        if j0 == 0:
+            cover[row0:row0 + n_rows, head] += 1
     assert (cover == 1).all()
     # 128 equal items on 148 SMs: splitting would not pay for its partial traffic
-    cf.load_library().cf_plan_inspect(ctypes.byref(d), np.array([6656, 6656], np.int32).ctypes.data,
-                                      np.array([512, 512], np.int32).ctypes.data, 2, 4096, 148, None, None, None, 0,
-                                      counts.ctypes.data)
+    counts = cf.cf_plan_inspect(d, [6656, 6656], [512, 512], 4096, 148, want_counts=True)[5]
     assert counts[5] == 0 and counts[4] == 128
 
 
 def test_few_items_are_cut_into_kv_ranges():
     """A 512-token chunk over an 8K prefix on one TP4 rank (16 query heads, 2 KV heads) is only 32 tile
     pairs for 148 SMs: the planner cuts them into KV ranges until the machine is about full."""
-    import ctypes
     d = cf.make_desc(16, 2, 128, 16, 65536)
     lc, lq = np.array([8192 + 512], np.int32), np.array([512], np.int32)
-    counts = np.zeros(6, dtype=np.int32)
-    cf.load_library().cf_plan_inspect(ctypes.byref(d), lc.ctypes.data, lq.ctypes.data, 1, 8192, 148, None, None, None, 0,
-                                      counts.ctypes.data)
+    counts = cf.cf_plan_inspect(d, lc, lq, 8192, 148, want_counts=True)[5]
     assert counts[5] > 0 and 96 <= counts[4] <= 148
     _, _, whole = cf.cf_estimate_us(d, lc, lq, 8192, num_sms=148)
     assert whole < 0.6 * (8 + 1.9 * 68)                 # well under the time of one unsplit item
+
+
+def test_forced_kv_split_tiles_every_item():
+    """prefill_force_split = k cuts every item that is long enough into KV ranges; the ranges of every q tile
+    still tile its visible KV tiles (checked inside _check_plan for the default plan; here with the option)."""
+    d = cf.make_desc(32, 8, 128, 16, 65536)
+    lc, lq = [3100 + 700, 50], [700, 1]
+    for k in (2, 3, 8):
+        st, dec, comb, pre, parts, counts = cf.cf_plan_inspect(d, lc, lq, 4096, 148, prefill_force_split=k, want_counts=True)
+        assert counts[5] > 0 and counts[4] > counts[5]
+        by_tile = {}
+        for _, q_row0, row0, n_rows, head, kvh, j0, j1 in pre:
+            by_tile.setdefault((row0, head), []).append((j0, j1))
+        for (row0, head), ranges in by_tile.items():
+            ranges.sort()
+            n_rows = min(128, 700 - row0)
+            assert ranges[0][0] == 0 and ranges[-1][1] == (3100 + row0 + n_rows + 127) // 128
+            assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+            assert len(ranges) <= k

@@ -1,6 +1,7 @@
 """GPU parity at the full sizes of the five workload configurations, in the launch configuration
-the benchmark times.  Decode rows are all checked; prefill rows are checked on a deterministic
-sample (first and last row of every 128-row tile plus every 7th row, thinned to a cap) because
+the benchmark times: every chunk iteration of configs 3 and 4, all 13 sweep points of config 5.
+Decode rows are all checked; prefill rows are checked on a deterministic sample - the first and
+last row of every 128-row q tile, the last row and every 41st row of each chunk, all heads - because
 the fp64 oracle needs ~1 TFLOP per iteration for the long chunks."""
 import pytest
 
@@ -15,17 +16,17 @@ def test_config2_decode_only_full_size():
 
 
 def test_config3_chat_all_iterations():
-    print(run_and_check(syn.config3_chat(), max_prefill_rows=24, check_append=False))
+    print(run_and_check(syn.config3_chat(), tile_rows=True, check_append=False))
 
 
-def test_config4_agentic_first_and_last_iteration():
+def test_config4_agentic_all_iterations():
     sc = syn.config4_agentic()
-    print(run_and_check(sc, max_prefill_rows=12, check_append=False))
+    print(run_and_check(sc, tile_rows=True, check_append=False))
 
 
-@pytest.mark.parametrize("budget,n", [(0, 0), (512, 4), (2048, 3), (8192, 1)])
+@pytest.mark.parametrize("budget,n", syn.CONFIG5_POINTS)
 def test_config5_sweep_points(budget, n):
-    print(run_and_check(syn.config5_sweep_point(budget, n), max_prefill_rows=8, check_append=False))
+    print(run_and_check(syn.config5_sweep_point(budget, n), tile_rows=True, check_append=False))
 
 
 @pytest.mark.parametrize("make", [lambda: syn.config3_chat(iterations=(3,)), lambda: syn.config5_sweep_point(2048, 3)])
@@ -69,4 +70,4 @@ def test_paper_context_limit_128k():
     geom = syn.Geometry(32, 8, 128, 16, 32768)
     limit = 131072 - 512
     sc = syn.scenario_from_lengths("ctx128k", geom, 4242, [limit - 1, 65536 - 1, limit - 300], [[1, 1, 300]])
-    print(run_and_check(sc, max_prefill_rows=16, check_append=False))
+    print(run_and_check(sc, tile_rows=True, check_append=False))

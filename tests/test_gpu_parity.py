@@ -34,18 +34,6 @@ def test_prefill_only_ragged(Hq, Hkv, D):
     run_and_check(small(5, Hq, Hkv, D, prefix, [qlen]))
 
 
-@pytest.mark.parametrize("D", [64, 128])
-def test_mma_sync_prefill_kernel_behind_its_switch(D, monkeypatch):
-    """CF_PREFILL_MMA=1 (read when the context is created) selects the warp-level mma.sync prefill kernel."""
-    monkeypatch.setenv("CF_PREFILL_MMA", "1")
-    ctx = cf.cf_create(0)
-    monkeypatch.delenv("CF_PREFILL_MMA")
-    try:
-        run_and_check(small(5, 8, 2, D, [0, 100, 700, 33], [[129, 64, 200, 1]]), ctx=ctx)
-    finally:
-        cf.cf_destroy(ctx)
-
-
 def test_mixed_shuffled_order_with_empty_sequences():
     prefix = [10, 0, 500, 77, 0, 2000, 31, 640, 5, 1]
     qlen = [1, 90, 1, 0, 1, 1, 130, 1, 0, 64]
@@ -127,49 +115,82 @@ def test_determinism_and_unrelated_calls():
     g.close()
 
 
-@pytest.mark.parametrize("kind", ["decode", "prefill"])
-def test_spike_keys(kind):
-    """A key planted 40+ above the rest must be found wherever it sits: page edges, chunk edges,
-    the prefix/chunk boundary, the diagonal; a key just past the diagonal must have no effect."""
-    Hq, Hkv, D = 8, 2, 128
-    if kind == "decode":
-        Lc, Lq = 20000, 1
-    else:
-        Lc, Lq = 1500, 200
-    P = Lc - Lq
-    sc = small(19, Hq, Hkv, D, [P], [[Lq]], NB=2048)
+def _spike_run(sc, cand, rows_to_check, spike, debug=None):
+    """Plants, at each candidate position in turn, a key whose score towers over the rest and checks
+    that every listed row returns that key's value if it can see the key and is unaffected if not."""
     b = sc.batches[0]
-    g = GpuScenario(sc)
+    geom = sc.geom
+    Hq, Hkv, D = geom.num_q_heads, geom.num_kv_heads, geom.head_dim
+    Lc, Lq = int(b.context_len[0]), int(b.query_len[0])
+    P = Lc - Lq
+    g = GpuScenario(sc, debug=debug)
     g.append(b)
-    d = cf.make_desc(Hq, Hkv, D, 16, 2048)
-    _, dec, _, _, _ = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks)
-    edges = sorted(set(int(x) for x in dec[:, 2]) | set(int(x) for x in dec[:, 3]))
-    cand = {0, 15, 16, 63, 64, 127, 128, P - 1, P, Lc - 2, Lc - 1}
-    for e in edges:
-        cand.update({e - 1, e, e + 1})
-    cand = sorted(j for j in cand if 0 <= j < Lc)
     k0 = g.k.clone()
     big = torch.zeros(D, dtype=torch.bfloat16, device="cuda")
-    big[0] = 96.0
+    big[0] = spike
     q = b.q.copy()
-    q[:, :, 0] = syn.f32_to_bf16_bits(np.float32(8.0))       # every row: score of the planted key = 8*96/sqrt(128) ~ 68
+    q[:, :, 0] = syn.f32_to_bf16_bits(np.float32(8.0))       # every row: score of the planted key = 8 * spike / sqrt(D)
     bq = syn.Batch(b.geom, b.context_len, b.query_len, b.block_table, q, b.k_new, b.v_new)
     v_host = to_host_bits(g.v)
-    for j in cand:
+    for j in sorted(set(int(x) for x in cand if 0 <= x < Lc)):
         g.k.copy_(k0)
         blk, slot = int(b.block_table[0, j // 16]), j % 16
         g.k[blk, :, slot, :] = big
         o, _ = g.attend(bq, want_lse=False)
         o = syn.bf16_bits_to_f64(o)                          # [Lq, Hq, D]
         vj = syn.bf16_bits_to_f64(v_host[blk, :, slot, :])   # [Hkv, D]
-        for i in ([0] if Lq == 1 else [0, 1, Lq // 2, Lq - 2, Lq - 1]):
-            p = P + i
-            want = np.repeat(vj, Hq // Hkv, axis=0)
-            if j <= p:
-                assert np.abs(o[i] - want).max() <= 2e-2, (kind, j, i)
+        want = np.repeat(vj, Hq // Hkv, axis=0)
+        for i in rows_to_check:
+            if j <= P + i:
+                assert np.abs(o[i] - want).max() <= 2e-2, (j, i)
             else:
-                assert np.abs(o[i] - want).max() > 0.5, (kind, j, i)   # invisible key: output is the ordinary average
+                assert np.abs(o[i] - want).max() > 0.5, (j, i)   # invisible key: output is the ordinary average
     g.close()
+
+
+def test_spike_keys_decode():
+    """A key planted ~68 nats above the rest must be found wherever it sits in a split decode sequence: page
+    edges, both sides of every chunk edge of the plan, the last positions."""
+    Hq, Hkv, D = 8, 2, 128
+    Lc = 20000
+    sc = small(19, Hq, Hkv, D, [Lc - 1], [[1]], NB=2048)
+    b = sc.batches[0]
+    d = cf.make_desc(Hq, Hkv, D, 16, 2048)
+    _, dec, _, _, _ = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks)
+    assert len(dec) > 2
+    cand = {0, 15, 16, 63, 64, 127, 128, Lc - 2, Lc - 1}
+    for e in sorted(set(int(x) for x in dec[:, 2]) | set(int(x) for x in dec[:, 3])):
+        cand.update({e - 1, e, e + 1})
+    _spike_run(sc, cand, [0], 96.0)
+
+
+@pytest.mark.parametrize("split", [0, 2, 3])
+@pytest.mark.parametrize("spike", [96.0, 192.0])
+def test_spike_keys_prefill(split, spike):
+    """Chunked prefill, 700 new tokens over a 3100-token prefix (interior tiles of the lean MMA loop, a ragged
+    last q tile): the planted key sits on both sides of every 128-token KV tile boundary, of every KV-range
+    boundary of the (forced) KV split, of the prefix/chunk boundary and of the diagonal, and on the columns of
+    later tiles whose exponentials are evaluated by the polynomial route (14, 15, 30, 31 of every 32).  spike =
+    192 puts the key ~136 nats (196 in log2 units) above the rest: far outside what an exponent field can
+    hold against a stale reference maximum, so the rescale path must catch it in every column."""
+    Hq, Hkv, D = 8, 2, 128
+    Lq, P = 700, 3100
+    Lc = P + Lq
+    sc = small(19, Hq, Hkv, D, [P], [[Lq]], NB=2048)
+    b = sc.batches[0]
+    d = cf.make_desc(Hq, Hkv, D, 16, 2048)
+    _, _, _, pre, _, counts = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks, prefill_force_split=split,
+                                                 want_counts=True)
+    assert (counts[5] > 0) == (split >= 2)
+    cand = {0, 15, 16, 63, 64, P - 1, P, P + 1, Lc - 2, Lc - 1}
+    for t in range(0, Lc + 128, 128):
+        cand.update({t - 1, t, t + 1})
+    for e in sorted(set(int(x) * 128 for x in pre[:, 6]) | set(int(x) * 128 for x in pre[:, 7])):
+        cand.update({e - 1, e, e + 1})
+    for t in (1, 2, 7, 13, P // 128, (Lc - 1) // 128):
+        cand.update({128 * t + c for c in (14, 15, 30, 31, 46, 47, 126, 127)})
+    rows = [0, 1, 127, 128, 300, 511, 512, Lq - 2, Lq - 1]
+    _spike_run(sc, cand, rows, spike, debug={cf.CF_DEBUG_PREFILL_SPLIT: split} if split else None)
 
 
 def test_abi_rejects_bad_arguments_without_launching():
@@ -267,18 +288,16 @@ def test_property_random_batches():
     cf.cf_destroy(ctx)
 
 
-def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge(monkeypatch):
-    """The split-K merge runs inside the decode kernel by default; CF_FUSED_COMBINE=0 (read when the context is
-    created) keeps the separate combine kernel.  Same merge routine, same chunk order: identical bits."""
+def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge():
+    """The split-K merge runs inside the decode kernel by default; the test-only switch CF_DEBUG_SEPARATE_COMBINE
+    keeps the separate combine kernel.  Same merge routine, same chunk order: identical bits."""
     sc = small(47, 32, 8, 128, [9000, 5000, 300, 16000, 2047], [[1, 1, 1, 1, 1]], NB=4096)
     b = sc.batches[0]
     fused = GpuScenario(sc)
     fused.append(b)
     o1, l1 = fused.attend(b)
     assert cf.cf_get_last_launch_count(fused.ctx) == 1
-    monkeypatch.setenv("CF_FUSED_COMBINE", "0")
-    sep = GpuScenario(sc)
-    monkeypatch.delenv("CF_FUSED_COMBINE")
+    sep = GpuScenario(sc, debug={cf.CF_DEBUG_SEPARATE_COMBINE: 1})
     sep.append(b)
     o2, l2 = sep.attend(b)
     assert cf.cf_get_last_launch_count(sep.ctx) == 2
@@ -290,7 +309,7 @@ def test_separate_combine_kernel_gives_the_bits_of_the_fused_merge(monkeypatch):
     sep.close()
 
 
-def test_more_prefill_items_than_sms(monkeypatch):
+def test_more_prefill_items_than_sms():
     """A chunk whose q tiles x head pairs exceed the SM count (11 tiles x 16 pairs + 2 x 16 = 208 items, ragged
     last tiles): every persistent CTA works through several items, in the serial and in the spatial sequence,
     with and without decode sequences beside it (KV split off, so that all sequences run one plan)."""
@@ -298,9 +317,7 @@ def test_more_prefill_items_than_sms(monkeypatch):
         prefix = [700, 40, 5000, 300, 17][:len(qlen[0])]
         sc = small(41, 32, 8, 128, prefix, qlen, NB=2048)
         b = sc.batches[0]
-        monkeypatch.setenv("CF_PREFILL_SPLIT", "1")
-        g = GpuScenario(sc)
-        monkeypatch.delenv("CF_PREFILL_SPLIT")
+        g = GpuScenario(sc, debug={cf.CF_DEBUG_PREFILL_SPLIT: 1})
         g.append(b)
         outs = []
         for mode in (0, 1, 5):
@@ -318,14 +335,12 @@ def test_more_prefill_items_than_sms(monkeypatch):
         g.close()
 
 
-def test_spatial_sequence_is_bit_identical_to_the_serial_sequence(monkeypatch):
+def test_spatial_sequence_is_bit_identical_to_the_serial_sequence():
     """With the planner's KV split switched off the plan does not depend on the launch sequence, and then
     neither does any bit of the result: which CTA runs an item, and when, never matters."""
     sc = small(29, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
     b = sc.batches[0]
-    monkeypatch.setenv("CF_PREFILL_SPLIT", "1")
-    g = GpuScenario(sc)
-    monkeypatch.delenv("CF_PREFILL_SPLIT")
+    g = GpuScenario(sc, debug={cf.CF_DEBUG_PREFILL_SPLIT: 1})
     g.append(b)
     cf.cf_set_overlap(g.ctx, 0)
     serial, lse0 = g.attend(b)
@@ -344,17 +359,15 @@ def test_spatial_sequence_is_bit_identical_to_the_serial_sequence(monkeypatch):
     g.close()
 
 
-def test_spatial_sequence_with_the_resident_wait(monkeypatch):
-    """CF_SPATIAL_WAIT=1 (read when the context is created): decode waits, through a stream memory operation, for
+def test_spatial_sequence_with_the_resident_wait():
+    """CF_DEBUG_SPATIAL_WAIT (test-only switch): decode waits, through a stream memory operation, for
     the front prefill CTAs; same plan, same bits as without the wait, over repeated calls."""
     sc = small(31, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
     b = sc.batches[0]
     plain = GpuScenario(sc)
     plain.append(b)
     o0, l0 = plain.attend(b)
-    monkeypatch.setenv("CF_SPATIAL_WAIT", "1")
-    waited = GpuScenario(sc)
-    monkeypatch.delenv("CF_SPATIAL_WAIT")
+    waited = GpuScenario(sc, debug={cf.CF_DEBUG_SPATIAL_WAIT: 1})
     waited.append(b)
     for n in (1, 1, 5, 1):
         cf.cf_set_overlap(waited.ctx, n)
@@ -501,19 +514,77 @@ def test_sequences_sharing_prefix_pages():
 
 
 @pytest.mark.parametrize("k", [2, 3])
-def test_kv_split_prefill_items_match_the_oracle(k, monkeypatch):
+def test_kv_split_prefill_items_match_the_oracle(k):
     """Every tcgen05 prefill item cut into k KV ranges (fp32 partials + the prefill combine kernel):
     group sizes 1, 4 and 8, ragged chunks, a chunk with no prefix."""
-    monkeypatch.setenv("CF_PREFILL_SPLIT", str(k))           # read when the context is created
     prefix = [2000, 0, 700, 4097, 300]
     qlen = [300, 700, 129, 64, 1]
     for Hq, Hkv in ((4, 4), (32, 8), (16, 2)):
         sc = small(41 + Hq, Hq, Hkv, 128, prefix, [qlen], NB=2048)
         d = cf.make_desc(Hq, Hkv, 128, 16, 2048)
-        import ctypes
-        counts = np.zeros(6, dtype=np.int32)
         b = sc.batches[0]
-        cf.load_library().cf_plan_inspect(ctypes.byref(d), b.context_len.ctypes.data, b.query_len.ctypes.data, b.num_seqs,
-                                          b.max_blocks, 148, None, None, None, 0, counts.ctypes.data)
+        counts = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks, prefill_force_split=k, want_counts=True)[5]
         assert counts[5] > 0                                  # some items really were split
-        run_and_check(sc)
+        run_and_check(sc, debug={cf.CF_DEBUG_PREFILL_SPLIT: k})
+
+
+def test_block_ids_outside_the_pool_are_reported_not_dereferenced():
+    """A block-table entry in use that lies outside the pool: nothing is read or written through it, and
+    cf_get_async_status reports CF_ERR_OUT_OF_RANGE once (decode, prefill and append paths)."""
+    sc = small(51, 8, 2, 128, [100, 700, 300], [[1, 1, 140]], NB=128)
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    k_before, v_before = to_host_bits(g.k), to_host_bits(g.v)
+    for s, col, val in ((0, 2, 128), (1, 40, -7), (2, 5, 1 << 28)):
+        bad = b.block_table.copy()
+        bad[s, col] = val
+        bt = torch.from_numpy(bad).cuda()
+        q = to_dev_bf16(b.q)
+        out = torch.zeros_like(q)
+        cf.cf_mixed_attention(g.ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len, out)
+        torch.cuda.synchronize()
+        assert cf.cf_get_async_status(g.ctx) == cf.CF_ERR_OUT_OF_RANGE
+        assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    # append aimed at a page outside the pool: the row is not written anywhere
+    bad = b.block_table.copy()
+    bad[0, (int(b.context_len[0]) - 1) // 16] = 4096
+    cf.cf_kv_append(g.ctx, g.desc, g.k, g.v, to_dev_bf16(b.k_new), to_dev_bf16(b.v_new), torch.from_numpy(bad).cuda(),
+                    b.max_blocks, b.context_len, b.query_len)
+    torch.cuda.synchronize()
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_ERR_OUT_OF_RANGE
+    assert np.array_equal(to_host_bits(g.k), k_before) and np.array_equal(to_host_bits(g.v), v_before)
+    o_bits, lse = g.attend(b)                                  # the context is still good
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_before, v_before, b.block_table, b.context_len, b.query_len)
+    compare(o_bits, lse, ref_o, ref_lse)
+    g.close()
+
+
+def test_destroy_is_refused_while_a_plan_is_alive():
+    sc = small(53, 8, 2, 64, [100], [[1]], NB=64)
+    b = sc.batches[0]
+    ctx = cf.cf_create(0)
+    d = cf.make_desc(8, 2, 64, 16, 64)
+    plan = cf.cf_plan_create(ctx, d, b.context_len, b.query_len, b.max_blocks)
+    assert cf.load_library().cf_destroy(ctx) == cf.CF_ERR_BUSY
+    cf.cf_plan_destroy(plan)
+    cf.cf_destroy(ctx)
+
+
+def test_set_overlap_one_returns_to_the_default_share():
+    """cf_set_overlap(ctx, n > 1) then cf_set_overlap(ctx, 1): the default share again, i.e. the bits of a fresh
+    context on a batch whose plan depends on the share (KV split balanced over the front grid)."""
+    sc = small(55, 32, 8, 128, [4000, 3000, 800], [[300, 1, 1]], NB=2048)
+    b = sc.batches[0]
+    fresh = GpuScenario(sc)
+    fresh.append(b)
+    o0, l0 = fresh.attend(b)
+    g = GpuScenario(sc)
+    g.append(b)
+    cf.cf_set_overlap(g.ctx, 9)
+    g.attend(b)
+    cf.cf_set_overlap(g.ctx, 1)
+    o1, l1 = g.attend(b)
+    assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+    fresh.close()
+    g.close()

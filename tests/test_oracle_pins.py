@@ -343,3 +343,23 @@ def test_bf16_pipeline_error_is_inside_the_stated_tolerance():
         e64 = np.exp(s64 - s64.max(axis=1, keepdims=True))
         o64 = (e64 / e64.sum(axis=1, keepdims=True)) @ V.astype(np.float64)
         assert np.abs(o - o64).max() < 2e-2 and np.abs(o - o64).mean() < 2e-3
+
+
+def test_empty_sequences_inside_the_batch_match_brute_force():
+    """Sequences with no new tokens (Lq = 0), at the front, in the middle and at the end of the batch, own no
+    packed rows: the rows of the sequences around them must still be found (row -> sequence lookup) and match
+    the dense brute force; asking for an explicit row list gives the same rows."""
+    sc = small_scenario(71, 8, 2, 64, prefix=[40, 3, 0, 77, 19, 5, 60], qlens=[[0, 1, 25, 0, 0, 17, 0]])
+    b = sc.batches[0]
+    assert b.total_q == 43
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    bo, blse = brute_force(b, k, v)
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - blse).max() < 1e-12
+    rows = np.array([0, 1, 25, 26, 42], dtype=np.int64)          # the decode row, first/last rows of both chunks
+    o2, lse2 = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, rows=rows)
+    assert np.array_equal(o2, o[rows]) and np.array_equal(lse2, lse[rows])
+    # the scatter skips them too: slots of the empty sequences keep their sentinel
+    kk, vv = sc.k_pool.copy(), sc.v_pool.copy()
+    oracle.kv_append(kk, vv, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+    blk = int(b.block_table[0, 40 // 16])
+    assert (kk[blk, :, 40 % 16:, :] == syn.BF16_NAN_BITS).all()
