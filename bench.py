@@ -1,22 +1,25 @@
 #!/usr/bin/env python
 """Benchmark of the mixed decode + chunked-prefill paged-attention path on B200.
 
-    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--report]
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--repeats R] [--impl ours|reference] [--no-per-config]
 
-One *step* = one unit of one layer of the chat-like mixed batch: cf_kv_append followed by
-cf_mixed_attention (split-K decode with its merge, chunked prefill) over 48 decode sequences
-(lognormal contexts, median 4096) plus two 512-token prefill chunks that sit on 6144 + 512*t
-cached tokens; steps cycle through the four chunks t = 0..3 of the 2048-token prompts.
-Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank runs
-an independent replica of the batch on its own GPU: the path has no exchange step, so there is no
+One *step* = one unit of one layer of the agentic long-context mixed batch: cf_kv_append followed by
+cf_mixed_attention (split-K decode with its merge, chunked prefill) over 16 decode sequences with
+contexts of 8K..32K plus one 2048-token prefill chunk that sits on 24,576 + 2048*t cached tokens;
+steps cycle through the four chunks t = 0..3 of the 8192-token prompt.
+Prints ONE JSON line (rank 0).  With N > 1 (launched by torch.distributed.run) every rank runs an
+independent replica of the batch on its own GPU: the path has no exchange step, so there is no
 data-path collective; the only collective is the max-over-ranks of the device time.
-`value` is measured in the library's default launch sequence (for this batch: a first grid of
-prefill CTAs beside decode); the `serial` key repeats the steps with one kernel after the other,
-which is also the sequence the per-kernel times under `kernels` / `roofline` are taken in.
+
+The timed region of K steps is repeated R times inside the invocation (synchronised on both sides
+every time); `value` and `ms_per_step` are the median repeat, `repeats` lists every repeat with the
+SM clock sampled while it ran, so that a cold burst and the power-limited steady state can be told
+apart.  `value` is measured in the library's default launch sequence; `serial` repeats the steps with
+one kernel after the other, which is also the sequence the per-kernel times under `kernels` /
+`roofline` are taken in.  `per_config` carries the same measurements for the other workload
+configurations (device times only, fewer repeats).
 
 `--impl reference` times the fp64 CPU oracle (as it stands) on the host cores instead.
-`--report` additionally writes a per-configuration table (all five workload configurations) to
-bench_report.json under $CF_REPORT_DIR (default: ./bench_out).
 """
 from __future__ import annotations
 
@@ -37,13 +40,18 @@ import cf_synth as syn  # noqa: E402
 
 METRIC = "mixed decode+prefill paged-attention query-tokens/s"
 UNIT = "query-tokens/s"
-WORKLOAD = ("configs[2] chat-like mixed batch: 48 decode seqs (lognormal ctx, median 4096, sigma 0.8, clip [128,16384]) "
-            "+ 2 prefills of 2048 new tokens over 6144 cached, 512-token chunks; Hq 32, Hkv 8, D 128, block 16, bf16; "
+WORKLOAD = ("configs[3] agentic long-context mixed batch: 16 decode seqs (ctx uniform in [8192, 32768]) "
+            "+ 1 prefill of 8192 new tokens over 24576 cached, 2048-token chunks; Hq 32, Hkv 8, D 128, block 16, bf16; "
             "one step = kv_append + mixed attention of one chunk iteration (t cycles 0..3)")
 # DRAM traffic per algorithmic byte of the split-K decode kernel, from an ncu capture on the reduced
 # decode case (dram bytes read + written: 560.9 MB for 555.2 MB algorithmic); traffic grows in
 # proportion to the K/V bytes, so a full launch is scaled by its algorithmic bytes.
 DECODE_TRAFFIC_RATIO = 1.010
+# DRAM traffic per algorithmic byte of the tcgen05 prefill kernel, from an ncu capture of a 4096-token chunk
+# over an 8192-token prefix (152.6 MB moved for 117.4 MB algorithmic: K/V come from DRAM ~1.9 times, the other
+# re-reads by the q tiles of a KV head are served by L2).  Prefill is tensor-bound; the figure is scaled by the
+# launch's algorithmic bytes and is approximate, because the re-read share depends on what else competes for L2.
+PREFILL_TRAFFIC_RATIO = 1.30
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
@@ -60,11 +68,12 @@ def load_peaks():
 
 # ------------------------------------------------------------------------------------------ clocks
 class ClockSampler:
-    """Samples SM clock and throttle reasons through NVML (read-only) while a region runs."""
+    """Samples SM clock, power and throttle reasons through NVML (read-only) while a region runs.
+    Samples carry a host timestamp, so a caller can ask for the samples of a sub-interval."""
 
-    def __init__(self, torch_device_index: int, period_s: float = 0.005):
+    def __init__(self, torch_device_index: int, period_s: float = 0.002):
         self.period = period_s
-        self.samples = []
+        self.samples = []            # (perf_counter, sm_mhz, watts)
         self.reasons = set()
         self.max_mhz = None
         self._stop = threading.Event()
@@ -89,7 +98,12 @@ class ClockSampler:
                  "hw_thermal_slowdown": 0x40, "hw_power_brake_slowdown": 0x80}
         while not self._stop.is_set():
             try:
-                self.samples.append(int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM)))
+                mhz = int(nv.nvmlDeviceGetClockInfo(self._h, nv.NVML_CLOCK_SM))
+                try:
+                    watts = nv.nvmlDeviceGetPowerUsage(self._h) / 1000.0
+                except Exception:
+                    watts = None
+                self.samples.append((time.perf_counter(), mhz, watts))
                 mask = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self._h)) if hasattr(nv, "nvmlDeviceGetCurrentClocksEventReasons") \
                     else int(nv.nvmlDeviceGetCurrentClocksThrottleReasons(self._h))
                 for k, bit in names.items():
@@ -110,11 +124,20 @@ class ClockSampler:
         if self._thread is not None:
             self._thread.join(timeout=1.0)
 
-    def summary(self):
-        if not self.samples:
+    def between(self, t0: float, t1: float):
+        """Median SM MHz and peak watts of the samples taken in [t0, t1] (None when there are none)."""
+        sel = [(m, w) for (t, m, w) in self.samples if t0 <= t <= t1]
+        if not sel:
+            return None, None
+        watts = [w for _, w in sel if w is not None]
+        return float(np.median([m for m, _ in sel])), (max(watts) if watts else None)
+
+    def summary(self, t0: float = None, t1: float = None):
+        sel = [m for (t, m, _) in self.samples if (t0 is None or t >= t0) and (t1 is None or t <= t1)]
+        if not sel:
             return {"sm_mhz": None, "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": 0}
-        return {"sm_mhz": float(np.median(self.samples)), "sm_max_mhz": self.max_mhz,
-                "reasons": sorted(self.reasons), "samples": len(self.samples)}
+        return {"sm_mhz": float(np.median(sel)), "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(sel)}
 
 
 # ------------------------------------------------------------------------------------------ device workload
@@ -196,13 +219,32 @@ def time_region(torch, fn, steps: int, stream) -> float:
     return float(e0.elapsed_time(e1))
 
 
+def time_repeats(torch, fn, steps: int, stream, repeats: int, clk: "ClockSampler" = None):
+    """The timed region of `steps` calls, `repeats` times.  Returns a list of
+    {"ms_per_step", "sm_mhz", "watts"} (the clock is the median of the samples taken while the repeat ran)."""
+    out = []
+    for _ in range(repeats):
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        ms = time_region(torch, fn, steps, stream)
+        t1 = time.perf_counter()
+        mhz, watts = clk.between(t0, t1) if clk is not None else (None, None)
+        out.append({"ms_per_step": ms / steps, "sm_mhz": mhz, "watts": watts})
+    return out
+
+
+def median_of(reps):
+    return float(np.median([r["ms_per_step"] for r in reps]))
+
+
 def batch_accounting(sc: syn.Scenario):
     acc = []
     for b in sc.batches:
         acc.append({"tokens": b.total_q,
                     "decode_bytes": syn.decode_algorithmic_bytes(b.geom, b.context_len, b.query_len),
                     "decode_flops": syn.decode_flops(b.geom, b.context_len, b.query_len),
-                    "prefill_flops": syn.prefill_flops(b.geom, b.context_len, b.query_len)})
+                    "prefill_flops": syn.prefill_flops(b.geom, b.context_len, b.query_len),
+                    "prefill_bytes": syn.prefill_algorithmic_bytes(b.geom, b.context_len, b.query_len)})
     return acc
 
 
@@ -211,18 +253,26 @@ NOMINAL_HBM_GBS = 7700.0
 NOMINAL_BF16_TFLOPS = 2250.0
 
 
-def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks):
-    """Per-kernel CUDA-event times (inside the library, on the launching stream) over `steps` steps."""
+def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks, clk: "ClockSampler" = None):
+    """Per-kernel CUDA-event times (inside the library, on the launching stream, serial launch sequence) over
+    `steps` steps.  Fractions: `frac` against the measured burst peak, `frac_of_sustained` against the measured
+    seconds-long figure (what a kernel inside a long power-limited loop can be held to), `frac_of_nominal`."""
     acc = batch_accounting(wl.sc)
     cf.cf_set_timing(wl.ctx, True)
     launches = 0
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
     for i in range(steps):
         launches += wl.step(i, stream)
     ms_dec, ms_comb, ms_pre, n = cf.cf_get_timing_sums(wl.ctx)
+    t1 = time.perf_counter()
     cf.cf_set_timing(wl.ctx, False)
+    mhz, _ = clk.between(t0, t1) if clk is not None else (None, None)
     dec_bytes = sum(acc[i % len(acc)]["decode_bytes"] for i in range(steps))
     pre_flops = sum(acc[i % len(acc)]["prefill_flops"] for i in range(steps))
-    out = {"ms_decode": ms_dec / steps, "ms_combine": ms_comb / steps, "ms_prefill": ms_pre / steps}
+    pre_bytes = sum(acc[i % len(acc)]["prefill_bytes"] for i in range(steps))
+    out = {"ms_decode": ms_dec / steps, "ms_combine": ms_comb / steps, "ms_prefill": ms_pre / steps, "sequence": "serial",
+           "sm_mhz": mhz}
     if ms_dec > 0:
         gbs = dec_bytes / ((ms_dec + ms_comb) * 1e-3) / 1e9
         out["decode"] = {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
@@ -232,9 +282,25 @@ def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks):
     if ms_pre > 0:
         tf = pre_flops / (ms_pre * 1e-3) / 1e12
         out["prefill"] = {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                          "frac": tf / peaks["bf16_tflops"], "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS, "traffic": None,
-                          "flops_per_launch": pre_flops / steps, "ms": ms_pre / steps}
+                          "frac": tf / peaks["bf16_tflops"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
+                          "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS,
+                          "traffic": PREFILL_TRAFFIC_RATIO * pre_bytes / steps, "bytes_per_launch": pre_bytes / steps,
+                          "flops_per_launch": pre_flops / steps, "ms": ms_pre / steps,
+                          "tflops_per_ghz": (tf / (mhz / 1e3)) if mhz else None}
     return out, launches
+
+
+def measure_host_time(torch, cf, wl: DeviceWorkload, steps: int, stream):
+    """Host microseconds the two ABI calls of a step cost the caller's thread, with the stream idle before
+    every step (so nothing waits for a plan slot): validation, planning, plan upload, tensor-map lookup, launches."""
+    cf.cf_get_host_time_sums(wl.ctx)
+    for i in range(steps):
+        torch.cuda.synchronize()
+        wl.step(i, stream)
+    torch.cuda.synchronize()
+    us_append, us_attn, us_plan, n = cf.cf_get_host_time_sums(wl.ctx)
+    n = max(n, 1)
+    return {"append": us_append / n, "attention": us_attn / n, "planner": us_plan / n, "total": (us_append + us_attn) / n}
 
 
 # ------------------------------------------------------------------------------------------ CPU oracle legs
@@ -269,14 +335,27 @@ class OracleWorkload:
         return time.perf_counter() - t0, pairs_s, pairs_t, b.total_q, len(rows)
 
 
-def cpu_baseline(sc: syn.Scenario, prefill_stride: int = 4):
+def _stride_for(ow: "OracleWorkload", it: int, seconds: float):
+    """Calibrates on a thin sample and picks the prefill-row stride whose sample takes about `seconds`."""
+    ow.sample(it, 256)                                  # touch the pages once, untimed
+    dt, ps, pt, _, _ = ow.sample(it, 256)
+    rate = ps / max(dt, 1e-6)                           # visible pairs per second
+    for stride in (1, 2, 4, 8, 16, 32, 64, 128):
+        # pairs of the sample at this stride ~ decode pairs + prefill pairs / stride; bounded by the thin sample's own figure
+        est = ps + (pt - ps) * (256.0 / stride - 1.0) / 255.0
+        if est / rate <= seconds:
+            return stride
+    return 256
+
+
+def cpu_baseline(sc: syn.Scenario, seconds: float = 15.0):
     ow = OracleWorkload(sc)
-    ow.sample(0, 64)                                   # touch the pages once, untimed
-    dt, ps, pt, T, nrows = ow.sample(0, prefill_stride)
+    stride = _stride_for(ow, 0, seconds)
+    dt, ps, pt, T, nrows = ow.sample(0, stride)
     full = dt * pt / ps
     return {"value": T / full, "unit": UNIT, "cores": ow.oracle.num_threads(), "kind": "oracle",
-            "sample": f"iteration 0: all decode rows + every {prefill_stride}th prefill row ({nrows} of {T} rows, "
-                      f"{ps / pt:.3f} of the visible (query,key) pairs) in {dt:.2f} s; whole-step time extrapolated by pair count"}
+            "sample": f"iteration 0: all decode rows + every {stride}th prefill row ({nrows} of {T} rows, "
+                      f"{ps / pt:.4f} of the visible (query,key) pairs) in {dt:.2f} s; whole-step time extrapolated by pair count"}
 
 
 def run_reference(args):
@@ -285,17 +364,9 @@ def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
         return
-    ow = OracleWorkload(syn.config3_chat())
+    ow = OracleWorkload(syn.config4_agentic())
     n_it = len(ow.sc.batches)
-    dt, ps, pt, _, _ = ow.sample(0, 64)                # page-touching pass
-    dt, ps, pt, _, _ = ow.sample(0, 64)
-    budget = 120.0 / max(1, args.steps + args.warmup)
-    stride = 64
-    for cand in (4, 8, 16, 32):
-        est_pairs = ps + (pt - ps) * (64.0 / cand - 1.0) / 63.0 if cand < 64 else ps
-        if dt * est_pairs / ps <= budget:
-            stride = cand
-            break
+    stride = _stride_for(ow, 0, 100.0 / max(1, args.steps + args.warmup))
     times, toks = [], []
     for i in range(args.warmup + args.steps):
         dt, ps, pt, T, nrows = ow.sample(i % n_it, stride)
@@ -327,6 +398,42 @@ def reduce_max(value: float, dist, device) -> float:
     return float(t.item())
 
 
+PER_CONFIG = [("configs[1] decode-only", lambda: syn.config2_decode_only()),
+              ("configs[2] chat-like", lambda: syn.config3_chat()),
+              ("configs[2] chat-like, one TP4 rank's shard (8 q heads, 2 kv heads)", lambda: syn.config3_chat_tp4_shard()),
+              ("configs[4] sweep, budget 0", lambda: syn.config5_sweep_point(0, 0)),
+              ("configs[4] sweep, budget 512 x 4 prompts", lambda: syn.config5_sweep_point(512, 4)),
+              ("configs[4] sweep, budget 2048 x 1 prompt", lambda: syn.config5_sweep_point(2048, 1)),
+              ("configs[4] sweep, budget 8192 x 1 prompt", lambda: syn.config5_sweep_point(8192, 1)),
+              ("configs[4] sweep, budget 8192 x 4 prompts", lambda: syn.config5_sweep_point(8192, 4))]
+
+
+def measure_config(torch, cf, ctx, sc, stream, peaks, clk, steps: int, repeats: int):
+    """Default-sequence and serial-sequence step times (median of `repeats` regions of `steps` steps) and the
+    per-kernel figures of one workload."""
+    wl = DeviceWorkload(sc, torch, cf, ctx)
+    n_it = len(sc.batches)
+    for i in range(max(3, n_it)):
+        wl.step(i, stream)
+    reps = time_repeats(torch, lambda i: wl.step(i, stream), steps, stream, repeats, clk)
+    cf.cf_set_overlap(ctx, 0)
+    for i in range(max(3, n_it)):
+        wl.step(i, stream)
+    reps_serial = time_repeats(torch, lambda i: wl.step(i, stream), steps, stream, max(3, repeats // 2), clk)
+    cf.cf_set_overlap(ctx, 1)
+    kern, _ = measure_kernels(torch, cf, wl, steps, stream, peaks, clk)
+    host = measure_host_time(torch, cf, wl, min(steps, 4 * n_it), stream)
+    toks = sum(wl.tokens(i) for i in range(steps)) / steps
+    ms = median_of(reps)
+    row = {"ms_per_step": ms, "ms_per_step_min": min(r["ms_per_step"] for r in reps), "ms_per_step_serial": median_of(reps_serial),
+           "query_tokens_per_s": toks / (ms * 1e-3), "steps": steps, "repeats": len(reps),
+           "sm_mhz": float(np.median([r["sm_mhz"] for r in reps if r["sm_mhz"]])) if any(r["sm_mhz"] for r in reps) else None,
+           "kernels": kern, "host_us_per_call": host}
+    del wl
+    torch.cuda.empty_cache()
+    return row
+
+
 def run_ours(args):
     import torch
     import paper_2609_27085_b200 as cf
@@ -341,12 +448,13 @@ def run_ours(args):
     if world > 1:
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    device = torch.device("cuda", local)
     peaks = load_peaks()
     ctx = cf.cf_create(local)
-    sc = syn.config3_chat(k=rank % 3)
+    sc = syn.config4_agentic(k=rank % 3)
     wl = DeviceWorkload(sc, torch, cf, ctx)
     stream = torch.cuda.current_stream()
-    steps, warmup = args.steps, max(3, args.warmup)
+    steps, warmup, repeats = args.steps, max(3, args.warmup), max(1, args.repeats)
 
     for i in range(warmup):
         wl.step(i, stream)
@@ -360,127 +468,114 @@ def run_ours(args):
         launches += wl.step(i, stream)
 
     with ClockSampler(local) as clk:
-        ms = time_region(torch, one, steps, stream)
-    if dist is not None:
-        dist.barrier()
-    ms = reduce_max(ms, dist, torch.device("cuda", local))
-    tokens = sum(wl.tokens(i) for i in range(steps))
-    value = world * tokens / (ms * 1e-3)
+        t_first = time.perf_counter()
+        reps = time_repeats(torch, one, steps, stream, repeats, clk)
+        t_last = time.perf_counter()
+        if dist is not None:
+            dist.barrier()
+        launches_per_region = launches // repeats
+        # every repeat is a region of exactly `steps` steps; the slowest rank decides each of them
+        for r in reps:
+            r["ms_per_step"] = reduce_max(r["ms_per_step"], dist, device)
+        ms_step = median_of(reps)
+        tokens_per_step = sum(wl.tokens(i) for i in range(steps)) / steps
+        value = world * tokens_per_step / (ms_step * 1e-3)
+        clocks = clk.summary(t_first, t_last)
 
-    # the same steps as the serial sequence (decode -> combine -> prefill on the caller's stream alone)
-    cf.cf_set_overlap(ctx, 0)
-    for i in range(3):
-        wl.step(i, stream)
-    ms_serial = reduce_max(time_region(torch, lambda i: wl.step(i, stream), steps, stream), dist, torch.device("cuda", local))
-    cf.cf_set_overlap(ctx, 1)
-    # the same steps as replays of captured graphs of the planned calls (plan once per iteration, launch per layer)
-    graphs, plans = wl.capture_graphs()
-    for i in range(3):
-        graphs[i % len(graphs)].replay()
-    ms_graph = reduce_max(time_region(torch, lambda i: graphs[i % len(graphs)].replay(), steps, stream), dist,
-                          torch.device("cuda", local))
-    del graphs
-    for pl in plans:
-        cf.cf_plan_destroy(pl)
-    # per-kernel times on the launching stream, same steps
-    kern, _ = measure_kernels(torch, cf, wl, steps, stream, peaks)
-    # end to end: host buffers in, host result out, every step
-    for i in range(3):
-        wl.step_host(i, stream)
-    cf.cf_host_steps_flush(ctx, stream)
-    torch.cuda.synchronize()
-    if dist is not None:
-        dist.barrier()
+        # the same steps as the serial sequence (decode -> combine -> prefill on the caller's stream alone)
+        side_reps = max(3, repeats // 3)
+        cf.cf_set_overlap(ctx, 0)
+        for i in range(3):
+            wl.step(i, stream)
+        ms_serial = reduce_max(median_of(time_repeats(torch, lambda i: wl.step(i, stream), steps, stream, side_reps, clk)), dist, device)
+        cf.cf_set_overlap(ctx, 1)
+        # the same steps as replays of captured graphs of the planned calls (plan once per iteration, launch per layer)
+        graphs, plans = wl.capture_graphs()
+        for i in range(3):
+            graphs[i % len(graphs)].replay()
+        ms_graph = reduce_max(median_of(time_repeats(torch, lambda i: graphs[i % len(graphs)].replay(), steps, stream, side_reps, clk)),
+                              dist, device)
+        del graphs
+        for pl in plans:
+            cf.cf_plan_destroy(pl)
+        # per-kernel times on the launching stream (serial sequence), same steps
+        kern, _ = measure_kernels(torch, cf, wl, steps, stream, peaks, clk)
+        host = measure_host_time(torch, cf, wl, min(steps, 16), stream)
+        # end to end: host buffers in, host result out, every step
+        for i in range(3):
+            wl.step_host(i, stream)
+        cf.cf_host_steps_flush(ctx, stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
 
-    def host_step(i):
-        wl.step_host(i, stream)
-        if i == steps - 1:
-            cf.cf_host_steps_flush(ctx, stream)          # the last read-backs are inside the timed region
+        def host_step(i):
+            wl.step_host(i, stream)
+            if i == steps - 1:
+                cf.cf_host_steps_flush(ctx, stream)          # the last read-backs are inside the timed region
 
-    ms_e2e = time_region(torch, host_step, steps, stream)
-    ms_e2e = reduce_max(ms_e2e, dist, torch.device("cuda", local))
-    assert cf.cf_get_async_status(ctx) == cf.CF_OK
-    g = sc.geom
-    T = wl.tokens(0)
-    h2d = T * (g.num_q_heads + 2 * g.num_kv_heads) * g.head_dim * 2
-    d2h = T * g.num_q_heads * g.head_dim * 2
+        ms_e2e = reduce_max(median_of(time_repeats(torch, host_step, steps, stream, side_reps, clk)), dist, device)
+        assert cf.cf_get_async_status(ctx) == cf.CF_OK
+        g = sc.geom
+        T = wl.tokens(0)
+        h2d = T * (g.num_q_heads + 2 * g.num_kv_heads) * g.head_dim * 2
+        d2h = T * g.num_q_heads * g.head_dim * 2
+        del wl
+        torch.cuda.empty_cache()
+
+        per_config = None
+        if rank == 0 and world == 1 and not args.no_per_config:
+            per_config = {}
+            pc_repeats = max(3, min(5, repeats))
+            for name, make in PER_CONFIG:
+                scn = make()
+                n_it = len(scn.batches)
+                per_config[name] = measure_config(torch, cf, ctx, scn, stream, peaks, clk, steps=max(8, 4 * n_it), repeats=pc_repeats)
+                del scn
 
     if rank == 0:
         dominant = "prefill" if kern.get("prefill", {}).get("ms", 0) >= kern.get("decode", {}).get("ms", 0) else "decode"
-        roof = {k: kern[dominant][k] for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "frac_of_nominal")}
+        roof = {k: kern[dominant].get(k) for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "frac_of_nominal",
+                                                   "frac_of_sustained", "tflops_per_ghz")}
         roof["kernel"] = "prefill_tc_kernel" if dominant == "prefill" else "decode_splitk_kernel (merge of the partials fused in)"
         roof["peak_source"] = peaks["source"] + (" burst bf16" if dominant == "prefill" else " copy")
+        roof["sequence"] = "serial (per-kernel events need kernels that do not overlap; `value` runs the default sequence)"
+        mhz = [r["sm_mhz"] for r in reps if r["sm_mhz"]]
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
-                "ms_per_step": ms / steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+                "ms_per_step": ms_step, "ms_per_step_min": min(r["ms_per_step"] for r in reps),
+                "ms_per_step_first": reps[0]["ms_per_step"], "repeats": len(reps),
+                "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
                 "dtype": "bf16", "data": "synthetic",
-                "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: ~1.0 GB of paged K/V streamed per step",
+                "config": {"workload": WORKLOAD, "l2": "inputs larger than L2: ~1.3 GB of paged K/V streamed per step",
                            "replicas": world},
                 "roofline": roof,
-                "kernels": {"decode": kern.get("decode"), "prefill": kern.get("prefill"),
-                            "ms_decode": kern["ms_decode"], "ms_combine": kern["ms_combine"], "ms_prefill": kern["ms_prefill"]},
-                "e2e": {"value": world * tokens / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e / steps},
-                "serial": {"value": world * tokens / (ms_serial * 1e-3), "unit": UNIT, "ms_per_step": ms_serial / steps,
+                "kernels": {"decode": kern.get("decode"), "prefill": kern.get("prefill"), "sequence": "serial",
+                            "ms_decode": kern["ms_decode"], "ms_combine": kern["ms_combine"], "ms_prefill": kern["ms_prefill"],
+                            "sm_mhz": kern.get("sm_mhz")},
+                "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
+                        "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
+                "serial": {"value": world * tokens_per_step / (ms_serial * 1e-3), "unit": UNIT, "ms_per_step": ms_serial,
                            "note": "cf_set_overlap(0): decode -> prefill one after the other; `value` is the "
-                                   "library's default sequence (prefill CTAs beside decode, joined per call); the per-kernel "
-                                   "times under `kernels` are taken in the serial sequence"},
-                "planned_graph": {"value": world * tokens / (ms_graph * 1e-3), "unit": UNIT, "ms_per_step": ms_graph / steps,
+                                   "library's default sequence (prefill CTAs beside decode, joined per call)"},
+                "planned_graph": {"value": world * tokens_per_step / (ms_graph * 1e-3), "unit": UNIT, "ms_per_step": ms_graph,
                                   "note": "cf_plan_create once per chunk iteration; cf_kv_append_planned + "
                                           "cf_mixed_attention_planned captured in a CUDA graph and replayed per step"},
-                "gpu_launches": launches, "clocks": clk.summary()}
+                "host_us_per_call": host,
+                "repeat_list": [{"ms_per_step": round(r["ms_per_step"], 5), "sm_mhz": r["sm_mhz"], "watts": r["watts"],
+                                 "ms_x_ghz": (round(r["ms_per_step"] * r["sm_mhz"] / 1e3, 5) if r["sm_mhz"] else None)} for r in reps],
+                "gpu_launches": launches_per_region, "clocks": clocks}
+        if mhz:
+            line["clocks"]["sm_mhz_per_repeat_min"] = min(mhz)
+            line["clocks"]["sm_mhz_per_repeat_max"] = max(mhz)
+        if per_config is not None:
+            line["per_config"] = per_config
         if world == 1:
             line["cpu_baseline"] = cpu_baseline(sc)
         print(json.dumps(line), flush=True)
-        if args.report:
-            write_report(torch, cf, ctx, stream, peaks)
-    del wl
     cf.cf_destroy(ctx)
     if dist is not None:
         dist.barrier()
         dist.destroy_process_group()
-
-
-def write_report(torch, cf, ctx, stream, peaks):
-    """Per-configuration table over the workload configurations (device times only)."""
-    rows = []
-    scenarios = [("cfg2_decode", lambda: syn.config2_decode_only()), ("cfg3_chat", lambda: syn.config3_chat()),
-                 ("cfg3_tp4_shard", lambda: syn.config3_chat_tp4_shard()), ("cfg4_agentic", lambda: syn.config4_agentic())]
-    scenarios += [(f"cfg5_b{b}_n{n}", (lambda b=b, n=n: syn.config5_sweep_point(b, n))) for b, n in
-                  [(0, 0), (512, 4), (2048, 1), (8192, 1), (8192, 4)]]
-    only = [x for x in os.environ.get("CF_REPORT_ONLY", "").split(",") if x]
-    for name, make in scenarios:
-        if only and name not in only:
-            continue
-        sc = make()
-        wl = DeviceWorkload(sc, torch, cf, ctx)
-        n_it = len(sc.batches)
-        for i in range(3 * n_it):
-            wl.step(i, stream)
-        steps = 5 * n_it
-        ms = time_region(torch, lambda i: wl.step(i, stream), steps, stream)
-        cf.cf_set_overlap(ctx, 0)
-        for i in range(n_it):
-            wl.step(i, stream)
-        ms_serial = time_region(torch, lambda i: wl.step(i, stream), steps, stream)
-        cf.cf_set_overlap(ctx, 1)
-        kern, _ = measure_kernels(torch, cf, wl, steps, stream, peaks)
-        toks = sum(wl.tokens(i) for i in range(steps))
-        rows.append({"config": name, "ms_per_step": ms / steps, "ms_per_step_serial": ms_serial / steps,
-                     "query_tokens_per_s": toks / (ms * 1e-3), **kern})
-        del wl
-        torch.cuda.empty_cache()
-    out_dir = os.environ.get("CF_REPORT_DIR", os.path.join(ROOT, "bench_out"))
-    os.makedirs(out_dir, exist_ok=True)
-    with open(os.path.join(out_dir, "bench_report.json"), "w") as f:
-        json.dump({"peaks": peaks, "rows": rows}, f, indent=1)
-    for r in rows:
-        d, p = r.get("decode"), r.get("prefill")
-        print(f"# {r['config']:16s} step {r['ms_per_step'] * 1e3:8.1f} us (serial {r['ms_per_step_serial'] * 1e3:8.1f})  "
-              f"{r['query_tokens_per_s']:12.0f} tok/s | "
-              f"decode {r['ms_decode'] * 1e3:7.1f}+{r['ms_combine'] * 1e3:5.1f} us "
-              f"{(d['achieved'] if d else 0):7.0f} GB/s ({(d['frac'] if d else 0):.2f}) | "
-              f"prefill {r['ms_prefill'] * 1e3:8.1f} us {(p['achieved'] if p else 0):7.1f} TF/s ({(p['frac'] if p else 0):.2f})",
-              file=sys.stderr, flush=True)
 
 
 def small_case(name: str) -> syn.Scenario:
@@ -496,6 +591,9 @@ def small_case(name: str) -> syn.Scenario:
     if name == "prefill_multi":      # 32 q tiles x 16 head pairs = 512 items: every persistent CTA works through 3-4 of them
         geom = syn.Geometry(32, 8, 128, 16, 16384)
         return syn.scenario_from_lengths(name, geom, 45, [8192], [[4096]])
+    if name == "agentic_small":      # the headline's first chunk iteration (2048 new over 24,576 cached) beside 4 decode sequences, in a pool of 1 GB
+        geom = syn.Geometry(32, 8, 128, 16, 8192)
+        return syn.scenario_from_lengths(name, geom, 46, [24576, 20000, 9000, 30000, 12000], [[2048, 1, 1, 1, 1]])
     raise SystemExit(f"unknown case {name}")
 
 
@@ -511,20 +609,24 @@ def run_case(args):
     for i in range(args.warmup):
         wl.step(i, stream)
     kern, launches = measure_kernels(torch, cf, wl, args.steps, stream, peaks)
+    host = measure_host_time(torch, cf, wl, min(args.steps, 8), stream)
     torch.cuda.synchronize()
-    print(json.dumps({"case": args.case, "steps": args.steps, "kernels": kern, "gpu_launches": launches}), flush=True)
+    print(json.dumps({"case": args.case, "steps": args.steps, "kernels": kern, "host_us_per_call": host, "gpu_launches": launches}),
+          flush=True)
     del wl
     cf.cf_destroy(ctx)
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", default=None, help="run a reduced workload (decode_small | prefill_small | prefill_multi) and exit")
+    ap.add_argument("--case", default=None,
+                    help="run a reduced workload (decode_small | prefill_small | prefill_multi | agentic_small) and exit")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
-    ap.add_argument("--report", action="store_true")
+    ap.add_argument("--repeats", type=int, default=15, help="how many times the timed region of --steps steps is repeated")
+    ap.add_argument("--no-per-config", action="store_true", help="skip the per_config block (the other workload configurations)")
     args = ap.parse_args()
     if args.case:
         run_case(args)

@@ -322,6 +322,15 @@ def prefill_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray
     return int(4 * geom.head_dim * geom.num_q_heads * pairs.sum())
 
 
+def prefill_algorithmic_bytes(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
+    """Bytes a prefill pass must move: K and V of every visible token of each chunk's sequence once per KV
+    head, the chunk's q rows in and o rows out."""
+    lq = np.asarray(query_len, dtype=np.int64)
+    lc = np.asarray(context_len, dtype=np.int64)
+    m = lq > 1
+    return int((lc[m] * geom.kv_bytes_per_token()).sum() + (lq[m] * 2 * geom.num_q_heads * geom.head_dim * 2).sum())
+
+
 def decode_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
     m = np.asarray(query_len) == 1
     lc = np.asarray(context_len, dtype=np.int64)[m]

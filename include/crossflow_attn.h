@@ -206,7 +206,13 @@ cf_status cf_selftest_bounded_wait(cf_ctx* ctx, void* cuda_stream);
 cf_status cf_set_timing(cf_ctx* ctx, int enabled);
 cf_status cf_get_timing_sums(cf_ctx* ctx, float* ms_decode, float* ms_combine, float* ms_prefill,
                              int32_t* num_calls);
-/* Number of kernels the last cf_mixed_attention launched (decode, combine, prefill: 0..3). */
+/* Host time (microseconds, wall clock) spent inside cf_kv_append and cf_mixed_attention since the previous
+ * query, summed over the calls, the part of it spent in the planner, and the number of cf_mixed_attention
+ * calls; resets the sums.  What the caller's thread pays per unit: validation, planning, plan upload,
+ * tensor-map lookup and the launches themselves (the GPU work is asynchronous). */
+cf_status cf_get_host_time_sums(cf_ctx* ctx, double* us_append, double* us_attention, double* us_planner,
+                                int32_t* num_steps);
+/* Number of kernels the last cf_mixed_attention launched. */
 cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
 
 /* Decode attention that allocates nothing (the paper has no counterpart; this serves callers that

@@ -42,7 +42,7 @@ CF_DEBUG_SPATIAL_WAIT = 4
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option",
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option", "cf_get_host_time_sums",
            "cf_status_string")
 
 
@@ -92,6 +92,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_get_last_launch_count.argtypes = [vp, i32p]
     lib.cf_plan_inspect.argtypes = [dp, vp, vp, i32, i32, ctypes.POINTER(PlanOptions), vp, vp, vp, i32, vp]
     lib.cf_set_debug_option.argtypes = [vp, ctypes.c_int, ctypes.c_int]
+    dbl = ctypes.POINTER(ctypes.c_double)
+    lib.cf_get_host_time_sums.argtypes = [vp, dbl, dbl, dbl, i32p]
     lib.cf_decode_attention_static.argtypes = [dp, vp, vp, vp, vp, i32, vp, i32, vp, vp, vp]
     lib.cf_selftest_bounded_wait.argtypes = [vp, vp]
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
@@ -230,6 +232,14 @@ def cf_get_timing_sums(ctx) -> Tuple[float, float, float, int]:
     a, b, c, n = ctypes.c_float(), ctypes.c_float(), ctypes.c_float(), ctypes.c_int32()
     _check(load_library().cf_get_timing_sums(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
            "cf_get_timing_sums")
+    return a.value, b.value, c.value, n.value
+
+
+def cf_get_host_time_sums(ctx) -> Tuple[float, float, float, int]:
+    """(us in cf_kv_append, us in cf_mixed_attention, us of that in the planner, attention calls) since the last query."""
+    a, b, c, n = ctypes.c_double(), ctypes.c_double(), ctypes.c_double(), ctypes.c_int32()
+    _check(load_library().cf_get_host_time_sums(ctx, ctypes.byref(a), ctypes.byref(b), ctypes.byref(c), ctypes.byref(n)),
+           "cf_get_host_time_sums")
     return a.value, b.value, c.value, n.value
 
 

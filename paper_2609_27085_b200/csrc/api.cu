@@ -3,6 +3,7 @@
 #include <cuda.h>
 
 #include <atomic>
+#include <chrono>
 #include <cmath>
 #include <cstdio>
 #include <cstdlib>
@@ -38,6 +39,24 @@ struct HostStage {
     cudaEvent_t h2d_done = nullptr, h2d_kv_done = nullptr, compute_done = nullptr, d2h_done = nullptr;
     bool used = false;
 };
+
+// TMA tensor maps of the prefill kernel, kept per (base address, geometry): a serving loop passes the same
+// pools and activation buffer call after call (one set per layer), and encoding three maps costs a few
+// microseconds of host time per launch.
+struct PoolMapEntry {
+    const void* base = nullptr;
+    int D = 0, num_blocks = 0, Hkv = 0;
+    int64_t sb = 0, sh = 0, st = 0;
+    uint64_t stamp = 0;
+    CUtensorMap map;
+};
+struct QMapEntry {
+    const void* base = nullptr;
+    int D = 0, rows = 0, Hq = 0;
+    uint64_t stamp = 0;
+    CUtensorMap map;
+};
+static constexpr int kPoolMaps = 32, kQMaps = 8;
 
 struct PlanSlot {
     uint8_t* host = nullptr;   // pinned
@@ -81,6 +100,13 @@ struct cf_ctx {
     std::vector<cf::TimedCall> timed;
     size_t timed_used = 0;
     int launches = 0;
+    // host time spent inside the entry points (benchmark instrumentation): nanoseconds and call counts
+    int64_t host_ns_append = 0, host_ns_attention = 0, host_ns_planner = 0;
+    int32_t host_calls_append = 0, host_calls_attention = 0;
+    // tensor-map cache (least recently used entry is replaced)
+    cf::PoolMapEntry pool_maps[cf::kPoolMaps];
+    cf::QMapEntry q_maps[cf::kQMaps];
+    uint64_t map_stamp = 0;
 };
 
 // A plan that lives on the device for as long as the caller wants: built once per scheduler iteration
@@ -232,23 +258,69 @@ struct StreamMemOps {
     Fn wait = nullptr, write = nullptr;
     bool ok = false;
 };
-static const StreamMemOps& stream_mem_ops()
+static StreamMemOps lookup_stream_mem_ops()
 {
-    static StreamMemOps ops;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void *w = nullptr, *r = nullptr;
-        cudaDriverEntryPointQueryResult q1, q2;
-        if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &w, cudaEnableDefault, &q1) == cudaSuccess &&
-            cudaGetDriverEntryPoint("cuStreamWriteValue32", &r, cudaEnableDefault, &q2) == cudaSuccess &&
-            q1 == cudaDriverEntryPointSuccess && q2 == cudaDriverEntryPointSuccess && w && r) {
-            ops.wait = reinterpret_cast<StreamMemOps::Fn>(w);
-            ops.write = reinterpret_cast<StreamMemOps::Fn>(r);
-            ops.ok = true;
-        }
+    StreamMemOps ops;
+    void *w = nullptr, *r = nullptr;
+    cudaDriverEntryPointQueryResult q1, q2;
+    if (cudaGetDriverEntryPoint("cuStreamWaitValue32", &w, cudaEnableDefault, &q1) == cudaSuccess &&
+        cudaGetDriverEntryPoint("cuStreamWriteValue32", &r, cudaEnableDefault, &q2) == cudaSuccess &&
+        q1 == cudaDriverEntryPointSuccess && q2 == cudaDriverEntryPointSuccess && w && r) {
+        ops.wait = reinterpret_cast<StreamMemOps::Fn>(w);
+        ops.write = reinterpret_cast<StreamMemOps::Fn>(r);
+        ops.ok = true;
     }
     return ops;
+}
+static const StreamMemOps& stream_mem_ops()
+{
+    static const StreamMemOps ops = lookup_stream_mem_ops();      // initialised once, thread-safe
+    return ops;
+}
+
+static int64_t now_ns()
+{
+    return std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now().time_since_epoch()).count();
+}
+
+static const CUtensorMap* pool_map(cf_ctx* c, const void* base, const cf_cache_desc* d, int64_t sb, int64_t sh, int64_t st)
+{
+    PoolMapEntry* victim = &c->pool_maps[0];
+    for (PoolMapEntry& e : c->pool_maps) {
+        if (e.base == base && e.D == d->head_dim && e.num_blocks == d->num_blocks && e.Hkv == d->num_kv_heads && e.sb == sb &&
+            e.sh == sh && e.st == st) {
+            e.stamp = ++c->map_stamp;
+            return &e.map;
+        }
+        if (e.stamp < victim->stamp) victim = &e;
+    }
+    if (!encode_pool_map(&victim->map, base, d->head_dim, d->num_blocks, d->num_kv_heads, sb, sh, st)) {
+        victim->base = nullptr;
+        return nullptr;
+    }
+    victim->base = base; victim->D = d->head_dim; victim->num_blocks = d->num_blocks; victim->Hkv = d->num_kv_heads;
+    victim->sb = sb; victim->sh = sh; victim->st = st;
+    victim->stamp = ++c->map_stamp;
+    return &victim->map;
+}
+
+static const CUtensorMap* q_map(cf_ctx* c, const void* base, int D, int rows, int Hq)
+{
+    QMapEntry* victim = &c->q_maps[0];
+    for (QMapEntry& e : c->q_maps) {
+        if (e.base == base && e.D == D && e.rows == rows && e.Hq == Hq) {
+            e.stamp = ++c->map_stamp;
+            return &e.map;
+        }
+        if (e.stamp < victim->stamp) victim = &e;
+    }
+    if (!encode_q_map(&victim->map, base, D, rows, Hq)) {
+        victim->base = nullptr;
+        return nullptr;
+    }
+    victim->base = base; victim->D = D; victim->rows = rows; victim->Hq = Hq;
+    victim->stamp = ++c->map_stamp;
+    return &victim->map;
 }
 
 static float scale_log2_of(const cf_cache_desc* d)
@@ -335,6 +407,14 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         tc->ran[2] = n.n_pre_tc > 0;
     }
     const bool has_prefill = n.n_pre_tc > 0;
+    PrefillMaps maps;
+    if (has_prefill) {
+        const CUtensorMap* mq = q_map(c, q, D, n.total_q, Hq);
+        const CUtensorMap* mk = pool_map(c, k_cache, desc, desc->k_stride_block, desc->k_stride_head, desc->k_stride_token);
+        const CUtensorMap* mv = pool_map(c, v_cache, desc, desc->v_stride_block, desc->v_stride_head, desc->v_stride_token);
+        if (!mq || !mk || !mv) return CF_ERR_CUDA;
+        maps.q = *mq; maps.k = *mk; maps.v = *mv;
+    }
     int second_grid = 0;
     const int sms = c->num_sms > 0 ? c->num_sms : 148;
     const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
@@ -369,14 +449,14 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         }
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, front, front + tail, 1, front, resident, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, front, front + tail, 1, front, resident, stream);
         // only after the front grid has been enqueued without an error, so that the count is certain to arrive
         if (e == cudaSuccess && resident &&
             mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, c->side);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
         if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
@@ -386,7 +466,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, desc, n.total_q, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
+        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
@@ -514,6 +594,7 @@ cf_status cf_kv_append(cf_ctx* c, const cf_cache_desc* desc, void* k_cache, void
                        int32_t num_seqs, void* cuda_stream)
 {
     if (!c || !desc) return CF_ERR_INVALID_ARG;
+    const int64_t t_in = now_ns();
     cf_status st = validate_desc(desc);
     if (st != CF_OK) return st;
     Plan pl;
@@ -545,6 +626,8 @@ cf_status cf_kv_append(cf_ctx* c, const cf_cache_desc* desc, void* k_cache, void
     p.query_len = (const int32_t*)(base + L.off_qlen);
     const cudaError_t e = launch_kv_append(p, stream);
     const cf_status fs = finish_slot(slot, stream);
+    c->host_ns_append += now_ns() - t_in;
+    ++c->host_calls_append;
     if (e != cudaSuccess) return CF_ERR_CUDA;
     return fs;
 }
@@ -556,6 +639,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
                              void* out, float* lse, void* cuda_stream)
 {
     if (!c || !desc) return CF_ERR_INVALID_ARG;
+    const int64_t t_in = now_ns();
     cf_status st = validate_desc(desc);
     if (st != CF_OK) return st;
     Plan pl;
@@ -563,6 +647,7 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
+    c->host_ns_planner += now_ns() - t_in;
     c->launches = 0;
     if (pl.total_q == 0) return CF_OK;
     if (!q || !k_cache || !v_cache || !block_table || !out) return CF_ERR_INVALID_ARG;
@@ -589,6 +674,8 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
     const cf_status fs = finish_slot(slot, stream);
+    c->host_ns_attention += now_ns() - t_in;
+    ++c->host_calls_attention;
     return ls != CF_OK ? ls : fs;
 }
 
@@ -914,6 +1001,18 @@ cf_status cf_get_timing_sums(cf_ctx* c, float* ms_decode, float* ms_combine, flo
     if (ms_combine) *ms_combine = (float)t[1];
     if (ms_prefill) *ms_prefill = (float)t[2];
     if (num_calls) *num_calls = (int32_t)n;
+    return CF_OK;
+}
+
+cf_status cf_get_host_time_sums(cf_ctx* c, double* us_append, double* us_attention, double* us_planner, int32_t* num_steps)
+{
+    if (!c) return CF_ERR_INVALID_ARG;
+    if (us_append) *us_append = 1e-3 * (double)c->host_ns_append;
+    if (us_attention) *us_attention = 1e-3 * (double)c->host_ns_attention;
+    if (us_planner) *us_planner = 1e-3 * (double)c->host_ns_planner;
+    if (num_steps) *num_steps = c->host_calls_attention;
+    c->host_ns_append = c->host_ns_attention = c->host_ns_planner = 0;
+    c->host_calls_append = c->host_calls_attention = 0;
     return CF_OK;
 }
 

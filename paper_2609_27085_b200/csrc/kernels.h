@@ -1,5 +1,6 @@
 // Host-callable launchers of the CUDA kernels (one translation unit per kernel family).
 #pragma once
+#include <cuda.h>
 #include <cuda_runtime.h>
 
 #include "device_common.cuh"
@@ -34,7 +35,15 @@ cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaS
 // ticket_base + t; with first_static set, CTA b starts on item b without a draw (then ticket_base = n_ctas of
 // that grid, also for a second grid that shares the counter).  `resident`, when not null, is a device word that
 // every CTA increments as it starts.
-cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
+// The kernel reads q and the two pools through TMA tensor maps; a map depends only on the base address and the
+// geometry, so the caller may build it once and keep it (encode_* return false when the driver refuses).
+struct PrefillMaps {
+    CUtensorMap q, k, v;
+};
+bool encode_q_map(CUtensorMap* m, const void* q, int head_dim, int total_rows, int num_q_heads);
+bool encode_pool_map(CUtensorMap* m, const void* pool, int head_dim, int num_blocks, int num_kv_heads, int64_t stride_block,
+                     int64_t stride_head, int64_t stride_token);
+cudaError_t launch_prefill_tc(const AttnParams& p, const PrefillMaps& maps, int head_dim, int n_items, int n_ctas,
                               int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
 
 // merges the fp32 partials of KV-split prefill items into `out` (one CTA per split item)

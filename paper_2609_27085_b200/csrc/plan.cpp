@@ -121,45 +121,57 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         struct KeyedTc { int64_t extent; PrefillTcItem it; };
         std::vector<KeyedTc> items;
         auto prefix_of = [&](int32_t s) { return context_len[s] - query_len[s]; };
+        // All items of one (sequence, row tile) have the same KV extent, so the longest-first order is found by
+        // sorting those few groups, not the items (a 8192-token chunk with 64 query heads is 2048 items in 64 groups).
+        struct Group { int64_t extent; int32_t s, tile; };
+        std::vector<Group> groups;
+        size_t n_emit = 0;
         for (int32_t s = 0; s < num_seqs; ++s) {
             const int32_t lq = query_len[s];
             if (lq <= 1) continue;
+            const int32_t n_tiles = (lq + TR - 1) / TR;
+            for (int32_t tile = 0; tile < n_tiles; tile += (G >= 2 ? 1 : 2)) {
+                const int32_t last = (G >= 2 || tile + 1 >= n_tiles) ? tile : tile + 1;
+                groups.push_back(Group{(int64_t)prefix_of(s) + last * TR + std::min(TR, lq - last * TR), s, tile});
+                n_emit += (size_t)(G >= 2 ? d->num_kv_heads * (G / 2) : d->num_q_heads);
+            }
+        }
+        std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b) { return a.extent > b.extent; });
+        items.reserve(n_emit);
+        for (const Group& gr : groups) {
+            const int32_t s = gr.s, tile = gr.tile, lq = query_len[s];
             const int32_t prefix = context_len[s] - lq;
             const int32_t n_tiles = (lq + TR - 1) / TR;
-            auto rows_of = [&](int32_t tile) { return std::min(TR, lq - tile * TR); };
+            auto rows_of = [&](int32_t tl) { return std::min(TR, lq - tl * TR); };
+            PrefillTcItem it;
+            it.seq = s; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
+            it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
             if (G >= 2) {
-                for (int32_t tile = 0; tile < n_tiles; ++tile)
-                    for (int32_t kvh = 0; kvh < d->num_kv_heads; ++kvh)
-                        for (int32_t i = 0; i < G; i += 2) {
-                            PrefillTcItem it;
-                            it.seq = s; it.kvh = kvh; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
-                            it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
-                            for (int t = 0; t < 2; ++t) {
-                                it.q_row0[t] = plan->q_start[s] + tile * TR;
-                                it.row0[t] = tile * TR;
-                                it.n_rows[t] = rows_of(tile);
-                                it.head[t] = kvh * G + i + t;
-                            }
-                            items.push_back(KeyedTc{(int64_t)prefix + tile * TR + rows_of(tile), it});
-                        }
-            } else {
-                for (int32_t tile = 0; tile < n_tiles; tile += 2)
-                    for (int32_t h = 0; h < d->num_q_heads; ++h) {
-                        PrefillTcItem it;
-                        it.seq = s; it.kvh = h; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
-                        it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
-                        int32_t last = tile;
-                        for (int t = 0; t < 2; ++t) {
-                            const int32_t tt = tile + t;
-                            const bool present = tt < n_tiles;
-                            it.q_row0[t] = present ? plan->q_start[s] + tt * TR : 0;
-                            it.row0[t] = present ? tt * TR : 0;
-                            it.n_rows[t] = present ? rows_of(tt) : 0;
-                            it.head[t] = h;
-                            if (present) last = tt;
-                        }
-                        items.push_back(KeyedTc{(int64_t)prefix + last * TR + rows_of(last), it});
+                for (int t = 0; t < 2; ++t) {
+                    it.q_row0[t] = plan->q_start[s] + tile * TR;
+                    it.row0[t] = tile * TR;
+                    it.n_rows[t] = rows_of(tile);
+                }
+                for (int32_t kvh = 0; kvh < d->num_kv_heads; ++kvh)
+                    for (int32_t i = 0; i < G; i += 2) {
+                        it.kvh = kvh;
+                        it.head[0] = kvh * G + i;
+                        it.head[1] = kvh * G + i + 1;
+                        items.push_back(KeyedTc{gr.extent, it});
                     }
+            } else {
+                for (int t = 0; t < 2; ++t) {
+                    const int32_t tt = tile + t;
+                    const bool present = tt < n_tiles;
+                    it.q_row0[t] = present ? plan->q_start[s] + tt * TR : 0;
+                    it.row0[t] = present ? tt * TR : 0;
+                    it.n_rows[t] = present ? rows_of(tt) : 0;
+                }
+                for (int32_t h = 0; h < d->num_q_heads; ++h) {
+                    it.kvh = h;
+                    it.head[0] = it.head[1] = h;
+                    items.push_back(KeyedTc{gr.extent, it});
+                }
             }
         }
         // Few items (short chunks, few heads per GPU under tensor parallelism): a CTA's time is set by the
@@ -180,7 +192,6 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 }
             std::stable_sort(singles.begin(), singles.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
         }
-        std::stable_sort(items.begin(), items.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
         // ---- KV split.  Items run one per SM, so a long item or an incomplete last wave leaves SMs idle.
         // An item may be cut into k <= 8 KV ranges that write fp32 partials, merged by a combine pass; k
         // comes from the cost model's constants; a range never starts inside the diagonal band and has at
@@ -262,6 +273,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             }
         }
         const size_t n_items = items.size();
+        plan->prefill_tc.reserve(n_items + 8 * plan->prefill_combine.capacity());
         for (size_t i = 0; i < n_items; ++i) {
             PrefillTcItem it = items[i].it;
             const int32_t k_want = k_of[i];

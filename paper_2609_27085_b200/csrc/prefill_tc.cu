@@ -781,23 +781,25 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
+EncodeTiledFn lookup_encode()
+{
+    void* ptr = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+        return reinterpret_cast<EncodeTiledFn>(ptr);
+    return nullptr;
+}
 EncodeTiledFn get_encode()
 {
-    static EncodeTiledFn fn = nullptr;
-    static bool tried = false;
-    if (!tried) {
-        tried = true;
-        void* ptr = nullptr;
-        cudaDriverEntryPointQueryResult q;
-        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &ptr, cudaEnableDefault, &q) == cudaSuccess &&
-            q == cudaDriverEntryPointSuccess)
-            fn = reinterpret_cast<EncodeTiledFn>(ptr);
-    }
+    static const EncodeTiledFn fn = lookup_encode();      // initialised once, thread-safe
     return fn;
 }
 
+}  // namespace
+
 // pool viewed as (d, token-in-page, head, block); one box = 64 elements x 16 tokens of one head of one page
-bool encode_pool(CUtensorMap* m, const void* base, int D, int num_blocks, int Hkv, int64_t s_block, int64_t s_head, int64_t s_token)
+bool encode_pool_map(CUtensorMap* m, const void* base, int D, int num_blocks, int Hkv, int64_t s_block, int64_t s_head, int64_t s_token)
 {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -810,7 +812,7 @@ bool encode_pool(CUtensorMap* m, const void* base, int D, int num_blocks, int Hk
 }
 
 // q viewed as (d, head, row); one box = 64 elements x 1 head x 128 rows; rows past the end read as zero
-bool encode_q(CUtensorMap* m, const void* base, int D, int total_rows, int Hq)
+bool encode_q_map(CUtensorMap* m, const void* base, int D, int total_rows, int Hq)
 {
     EncodeTiledFn enc = get_encode();
     if (!enc) return false;
@@ -821,8 +823,6 @@ bool encode_q(CUtensorMap* m, const void* base, int D, int total_rows, int Hq)
                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
-
-}  // namespace
 
 namespace {
 
@@ -867,18 +867,13 @@ cudaError_t launch_prefill_tc_t(const CUtensorMap& mq, const CUtensorMap& mk, co
 
 }  // namespace
 
-cudaError_t launch_prefill_tc(const AttnParams& p, const cf_cache_desc* desc, int total_q_rows, int n_items, int n_ctas,
+cudaError_t launch_prefill_tc(const AttnParams& p, const PrefillMaps& maps, int head_dim, int n_items, int n_ctas,
                               int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream)
 {
     if (n_items <= 0 || n_ctas <= 0) return cudaSuccess;
-    const int D = desc->head_dim;
-    CUtensorMap mq, mk, mv;
-    if (!encode_q(&mq, p.q, D, total_q_rows, p.Hq) ||
-        !encode_pool(&mk, p.k_cache, D, desc->num_blocks, p.Hkv, p.ks_block, p.ks_head, p.ks_token) ||
-        !encode_pool(&mv, p.v_cache, D, desc->num_blocks, p.Hkv, p.vs_block, p.vs_head, p.vs_token))
-        return cudaErrorInvalidValue;
-    return D == 128 ? launch_prefill_tc_t<128>(mq, mk, mv, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream)
-                    : launch_prefill_tc_t<64>(mq, mk, mv, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream);
+    return head_dim == 128
+               ? launch_prefill_tc_t<128>(maps.q, maps.k, maps.v, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream)
+               : launch_prefill_tc_t<64>(maps.q, maps.k, maps.v, p, n_items, n_ctas, queue_ctas, first_static, ticket_base, resident, stream);
 }
 
 }  // namespace cf
