@@ -55,7 +55,7 @@ def _load():
         i32, i64, f64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
         lib.cf_oracle_mixed_attention.restype = ctypes.c_int
         lib.cf_oracle_mixed_attention.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i32, vp, vp, i32,
-                                                  i32, i32, i32, i32, f64, vp, i64, vp, vp, vp, i64]
+                                                  i32, i32, i32, i32, f64, vp, i64, vp, vp, vp, i64, i32, vp]
         lib.cf_oracle_kv_append.restype = ctypes.c_int
         lib.cf_oracle_kv_append.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, vp, vp, i32, vp, vp, i32,
                                             i32, i32, i32]
@@ -84,10 +84,13 @@ def _base(pool: np.ndarray) -> ctypes.c_void_p:
 
 def mixed_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, block_table: np.ndarray,
                     context_len: np.ndarray, query_len: np.ndarray, scale: Optional[float] = None,
-                    rows: Optional[np.ndarray] = None, want_weights: int = 0):
+                    rows: Optional[np.ndarray] = None, want_weights: int = 0, window: int = 0,
+                    sinks: Optional[np.ndarray] = None):
     """fp64 paged attention.  q: uint16 [T, Hq, D]; pools: uint16 [NB, Hkv, B, D] (any strides with
     a contiguous last axis).  Returns (out [n, Hq, D], lse [n, Hq]) and, if want_weights > 0, the
-    softmax weights [n, Hq, want_weights]."""
+    softmax weights [n, Hq, want_weights].
+    window > 0: sliding window (the query at position p sees keys (p - window, p]); sinks: per-query-head
+    logits [Hq] that join the softmax denominator only (see the header of cf_oracle.c)."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.uint16)
     T, Hq, D = q.shape
@@ -106,12 +109,15 @@ def mixed_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, block
     out = np.empty((n, Hq, D), dtype=np.float64)
     lse = np.empty((n, Hq), dtype=np.float64)
     w = np.empty((n, Hq, want_weights), dtype=np.float64) if want_weights else None
+    if sinks is not None:
+        sinks = np.ascontiguousarray(sinks, dtype=np.float64)
+        assert sinks.shape == (Hq,)
     ks, vs = _pool_strides(k_pool), _pool_strides(v_pool)
     rc = lib.cf_oracle_mixed_attention(
         _ptr(q), _base(k_pool), _base(v_pool), ks[0], ks[1], ks[2], vs[0], vs[1], vs[2],
         _ptr(bt), bt.shape[1], _ptr(lc), _ptr(lq), S, Hq, Hkv, D, B,
         float(1.0 / math.sqrt(D) if scale is None else scale),
-        _ptr(rows), n, _ptr(out), _ptr(lse), _ptr(w), want_weights)
+        _ptr(rows), n, _ptr(out), _ptr(lse), _ptr(w), want_weights, int(window), _ptr(sinks))
     if rc != 0:
         raise ValueError(f"cf_oracle_mixed_attention rejected its arguments (code {rc})")
     return (out, lse, w) if want_weights else (out, lse)

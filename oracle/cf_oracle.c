@@ -14,7 +14,7 @@
  * Section 5), so the arithmetic is the textbook definition of softmax attention
  * over a paged cache:
  *
- *   for sequence s, new-token row i in [0, Lq[s]), query head h:
+ *   for sequence s, new-token row i in [0, Lq[s]), query head h (full causal attention, no sink):
  *     p = (Lc[s] - Lq[s]) + i                 absolute position of the query token
  *     g = h / (Hq / Hkv)                      KV head serving this query head
  *     k_j, v_j = cache[ block_table[s][j / B] ][ g ][ j % B ]   for j in [0, p]
@@ -24,6 +24,17 @@
  *
  * Everything is evaluated in fp64 from the exact bf16 input values, keys in
  * ascending order, with no blocking, fusion or reordering.
+ *
+ * Variant (model-specific attention; the paper evaluates GPT-OSS-120B, Section 6.1,
+ * without describing its attention, so this is a reading taken from that model's
+ * public description): a sliding window and per-head attention sinks.
+ *   window W > 0 : the query at position p sees keys j in [max(0, p - W + 1), p]
+ *                  (W = 0: every key up to p, as above)
+ *   sink s_h     : a per-query-head logit (natural-log units, not multiplied by
+ *                  scale) that joins the softmax denominator and carries no value:
+ *                    O = sum_j exp(x_j) v_j / (exp(s_h) + sum_j exp(x_j))
+ *                    lse = ln(exp(s_h) + sum_j exp(x_j))
+ *                  (sinks == NULL: no sink)
  *
  * Pins (tests, CPU only): brute-force dense masked attention on gathered
  * contiguous K/V, the library scaled-dot-product routine on an identity block
@@ -78,10 +89,11 @@ int cf_oracle_mixed_attention(
     int32_t num_q_heads, int32_t num_kv_heads, int32_t head_dim, int32_t block_size,
     double scale,
     const int64_t *rows, int64_t n_rows,
-    double *out, double *lse, double *weights, int64_t weights_ld)
+    double *out, double *lse, double *weights, int64_t weights_ld,
+    int32_t window, const double *sinks /* [num_q_heads] or NULL */)
 {
     if (num_q_heads <= 0 || num_kv_heads <= 0 || num_q_heads % num_kv_heads != 0) return -1;
-    if (head_dim <= 0 || block_size <= 0 || num_seqs < 0) return -1;
+    if (head_dim <= 0 || block_size <= 0 || num_seqs < 0 || window < 0) return -1;
     int64_t T = 0;
     for (int32_t s = 0; s < num_seqs; ++s) {
         if (query_len[s] < 0 || query_len[s] > context_len[s]) return -2;
@@ -109,9 +121,13 @@ int cf_oracle_mixed_attention(
         const uint16_t *qrow = q + (r * num_q_heads + h) * (int64_t)head_dim;
         const int32_t *bt = block_table + (int64_t)s * max_blocks_per_seq;
 
+        /* first visible key: 0, or the left edge of the sliding window */
+        const int32_t j_lo = (window > 0 && p - window + 1 > 0) ? p - window + 1 : 0;
+        const double sink = sinks ? sinks[h] : -INFINITY;
+
         double *x = (double *)malloc(sizeof(double) * (size_t)(p + 1));
-        double m = -INFINITY;
-        for (int32_t j = 0; j <= p; ++j) {
+        double m = sink;
+        for (int32_t j = j_lo; j <= p; ++j) {
             const uint16_t *kj = k_cache + (int64_t)bt[j / block_size] * k_stride_block
                                  + (int64_t)g * k_stride_head + (int64_t)(j % block_size) * k_stride_token;
             double dot = 0.0;
@@ -120,13 +136,14 @@ int cf_oracle_mixed_attention(
             if (x[j] > m) m = x[j];
         }
         double l = 0.0;
-        for (int32_t j = 0; j <= p; ++j) {
+        for (int32_t j = j_lo; j <= p; ++j) {
             x[j] = exp(x[j] - m);
             l += x[j];
         }
+        if (sinks) l += exp(sink - m);        /* the sink adds to the denominator only */
         double *o = out + (slot * num_q_heads + h) * (int64_t)head_dim;
         for (int32_t d = 0; d < head_dim; ++d) o[d] = 0.0;
-        for (int32_t j = 0; j <= p; ++j) {
+        for (int32_t j = j_lo; j <= p; ++j) {
             const uint16_t *vj = v_cache + (int64_t)bt[j / block_size] * v_stride_block
                                  + (int64_t)g * v_stride_head + (int64_t)(j % block_size) * v_stride_token;
             for (int32_t d = 0; d < head_dim; ++d) o[d] += x[j] * bf16_to_f64(vj[d]);
@@ -135,7 +152,7 @@ int cf_oracle_mixed_attention(
         if (lse) lse[slot * num_q_heads + h] = m + log(l);
         if (weights) {
             double *wr = weights + (slot * num_q_heads + h) * weights_ld;
-            for (int64_t j = 0; j < weights_ld; ++j) wr[j] = (j <= p) ? x[j] / l : 0.0;
+            for (int64_t j = 0; j < weights_ld; ++j) wr[j] = (j >= j_lo && j <= p) ? x[j] / l : 0.0;
         }
         free(x);
     }

@@ -363,3 +363,132 @@ def test_empty_sequences_inside_the_batch_match_brute_force():
     oracle.kv_append(kk, vv, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
     blk = int(b.block_table[0, 40 // 16])
     assert (kk[blk, :, 40 % 16:, :] == syn.BF16_NAN_BITS).all()
+
+
+# ------------------------------------------------------------------ variant: sliding window + attention sinks
+def brute_force_variant(batch, k_pool, v_pool, window=0, sinks=None, scale=None):
+    """Dense statement of the variant: an explicit [Lq, Lc] boolean band mask (causal edge on the right, the
+    window's edge on the left) and the sink as one extra softmax column that carries a zero value row."""
+    g = batch.geom
+    G = g.num_q_heads // g.num_kv_heads
+    scale = 1.0 / math.sqrt(g.head_dim) if scale is None else scale
+    qs = batch.q_start()
+    out = np.zeros((batch.total_q, g.num_q_heads, g.head_dim))
+    lse = np.zeros((batch.total_q, g.num_q_heads))
+    for s in range(batch.num_seqs):
+        Lq, Lc = int(batch.query_len[s]), int(batch.context_len[s])
+        if Lq == 0:
+            continue
+        K = gather_contiguous(k_pool, batch.block_table[s], Lc)
+        V = gather_contiguous(v_pool, batch.block_table[s], Lc)
+        Q = syn.bf16_bits_to_f64(batch.q[qs[s]:qs[s + 1]])
+        pos = (Lc - Lq + np.arange(Lq))[:, None]
+        keys = np.arange(Lc)[None, :]
+        hidden = keys > pos
+        if window > 0:
+            hidden |= keys <= pos - window
+        for h in range(g.num_q_heads):
+            scores = Q[:, h, :] @ K[h // G].T * scale
+            scores[hidden] = -np.inf
+            vals = V[h // G]
+            if sinks is not None:
+                scores = np.concatenate([scores, np.full((Lq, 1), float(sinks[h]))], axis=1)
+                vals = np.concatenate([vals, np.zeros((1, g.head_dim))], axis=0)
+            logsum = np.logaddexp.reduce(scores, axis=1)
+            out[qs[s]:qs[s + 1], h] = np.exp(scores - logsum[:, None]) @ vals
+            lse[qs[s]:qs[s + 1], h] = logsum
+    return out, lse
+
+
+@pytest.mark.parametrize("window,with_sinks", [(1, False), (7, False), (16, True), (33, True), (0, True), (1000, True)])
+def test_variant_matches_brute_force(window, with_sinks):
+    sc = small_scenario(91, 8, 2, 64, prefix=[0, 5, 37, 16, 99, 0, 31], qlens=[[1, 1, 23, 16, 1, 40, 1]])
+    b = sc.batches[0]
+    sinks = np.random.default_rng(4).normal(0.0, 2.0, size=8) if with_sinks else None
+    (o, lse), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool, window=window, sinks=sinks)
+    bo, blse = brute_force_variant(b, k, v, window=window, sinks=sinks)
+    assert np.abs(o - bo).max() < 1e-12 and np.abs(lse - blse).max() < 1e-12
+
+
+def test_variant_matches_torch_sdpa_with_band_mask_and_sink_column():
+    """Library statement: scaled_dot_product_attention over the gathered keys plus one extra zero key / zero
+    value per KV head, with an additive float mask that is -inf outside the band and the head's sink logit on
+    the extra column (GQA by repeating the KV heads, since the mask is per query head)."""
+    Hq, Hkv, D, B, Lq, P, W = 8, 2, 64, 16, 37, 59, 20
+    Lc = P + Lq
+    nb = (Lc + B - 1) // B
+    geom = syn.Geometry(Hq, Hkv, D, B, nb)
+    rng = np.random.default_rng(78)
+    k_pool, v_pool = syn.empty_pools(geom)
+    ident = np.arange(nb, dtype=np.int32)
+    syn.fill_prefix(rng, geom, k_pool, ident, Lc)
+    syn.fill_prefix(rng, geom, v_pool, ident, Lc)
+    q = syn.normal_bf16(rng, (Lq, Hq, D))
+    sinks = rng.normal(0.0, 1.5, size=Hq)
+    o, lse = oracle.mixed_attention(q, k_pool, v_pool, ident[None, :], [Lc], [Lq], window=W, sinks=sinks)
+
+    G = Hq // Hkv
+    K = torch.from_numpy(gather_contiguous(k_pool, ident, Lc)).repeat_interleave(G, dim=0)      # [Hq, Lc, D]
+    V = torch.from_numpy(gather_contiguous(v_pool, ident, Lc)).repeat_interleave(G, dim=0)
+    K = torch.cat([K, torch.zeros(Hq, 1, D, dtype=torch.float64)], dim=1)[None]
+    V = torch.cat([V, torch.zeros(Hq, 1, D, dtype=torch.float64)], dim=1)[None]
+    Q = torch.from_numpy(syn.bf16_bits_to_f64(q)).permute(1, 0, 2)[None]
+    pos = P + torch.arange(Lq)[:, None]
+    keys = torch.arange(Lc)[None, :]
+    band = (keys <= pos) & (keys > pos - W)
+    bias = torch.full((Hq, Lq, Lc + 1), float("-inf"), dtype=torch.float64)
+    bias[:, :, :Lc][band[None].expand(Hq, -1, -1)] = 0.0
+    bias[:, :, Lc] = torch.from_numpy(sinks)[:, None]
+    ref = torch.nn.functional.scaled_dot_product_attention(Q, K, V, attn_mask=bias[None])
+    assert np.abs(o - ref[0].permute(1, 0, 2).numpy()).max() < 1e-12
+
+
+def test_variant_reduces_to_the_plain_definition():
+    """A window at least as long as the context, and sinks of -inf, give the bits of the plain path."""
+    sc = small_scenario(93, 8, 2, 64, prefix=[10, 77, 0], qlens=[[1, 30, 19]])
+    b = sc.batches[0]
+    (o0, l0), (k, v) = run_oracle(b, sc.k_pool, sc.v_pool)
+    for W in (int(b.context_len.max()), 10 ** 6):
+        o1, l1 = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, window=W)
+        assert np.array_equal(o0, o1) and np.array_equal(l0, l1)
+    o2, l2 = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, sinks=np.full(8, -np.inf))
+    assert np.array_equal(o0, o2) and np.array_equal(l0, l2)
+
+
+def test_variant_closed_forms_with_zero_query():
+    """q = 0: every visible key weighs the same.  Window W -> the mean of the last min(W, p + 1) values and
+    lse = ln min(W, p + 1); with a sink s the n visible keys weigh 1 / (n + e^s) each and lse = ln(n + e^s)."""
+    b, k, v = _single_seq(4, 2, 32, 45, 13)
+    q0 = np.zeros_like(b.q)
+    V = gather_contiguous(v, b.block_table[0], 45)
+    W = 10
+    o, lse = oracle.mixed_attention(q0, k, v, b.block_table, b.context_len, b.query_len, window=W)
+    sinks = np.array([0.0, 1.0, -2.0, 3.5])
+    os_, lses = oracle.mixed_attention(q0, k, v, b.block_table, b.context_len, b.query_len, window=W, sinks=sinks)
+    for i in range(13):
+        p = 45 - 13 + i
+        n = min(W, p + 1)
+        for h in range(4):
+            mean = V[h // 2, p + 1 - n:p + 1].mean(axis=0)
+            assert np.abs(o[i, h] - mean).max() < 1e-13 and abs(lse[i, h] - math.log(n)) < 1e-13
+            assert np.abs(os_[i, h] - mean * n / (n + math.exp(sinks[h]))).max() < 1e-13
+            assert abs(lses[i, h] - math.log(n + math.exp(sinks[h]))) < 1e-13
+
+
+def test_variant_weights_vanish_left_of_the_window():
+    b, k, v = _single_seq(4, 2, 32, 50, 9)
+    sinks = np.array([0.5, -1.0, 2.0, 0.0])
+    o, lse, w = oracle.mixed_attention(b.q, k, v, b.block_table, b.context_len, b.query_len, want_weights=50, window=12,
+                                       sinks=sinks)
+    for i in range(9):
+        p = 50 - 9 + i
+        assert (w[i, :, :p - 11] == 0).all() and (w[i, :, p + 1:] == 0).all() and (w[i, :, p - 11:p + 1] > 0).all()
+    # the key weights plus the sink's share exp(s - lse) sum to one
+    assert np.abs(w.sum(axis=-1) + np.exp(sinks[None, :] - lse) - 1.0).max() < 1e-14
+    # keys left of the window may hold anything (here: Inf) without reaching the result
+    k2, v2 = k.copy(), v.copy()
+    first_page = b.block_table[0, 0]
+    k2[first_page] = 0x7F80
+    v2[first_page] = 0x7F80
+    o2, lse2 = oracle.mixed_attention(b.q, k2, v2, b.block_table, b.context_len, b.query_len, window=12, sinks=sinks)
+    assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
