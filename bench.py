@@ -467,7 +467,7 @@ def run_ours(args):
         nonlocal launches
         launches += wl.step(i, stream)
 
-    with ClockSampler(local) as clk:
+    with ClockSampler(local, period_s=args.clock_period_ms * 1e-3) as clk:
         t_first = time.perf_counter()
         reps = time_repeats(torch, one, steps, stream, repeats, clk)
         t_last = time.perf_counter()
@@ -528,6 +528,8 @@ def run_ours(args):
             per_config = {}
             pc_repeats = max(3, min(5, repeats))
             for name, make in PER_CONFIG:
+                if args.only_config and args.only_config not in name:
+                    continue
                 scn = make()
                 n_it = len(scn.batches)
                 per_config[name] = measure_config(torch, cf, ctx, scn, stream, peaks, clk, steps=max(8, 4 * n_it), repeats=pc_repeats)
@@ -626,6 +628,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
     ap.add_argument("--repeats", type=int, default=15, help="how many times the timed region of --steps steps is repeated")
+    ap.add_argument("--clock-period-ms", type=float, default=10.0, help="sampling period of the SM clock (NVML, read-only)")
+    ap.add_argument("--only-config", default=None, help="with per_config: measure only the configurations whose name contains this")
     ap.add_argument("--no-per-config", action="store_true", help="skip the per_config block (the other workload configurations)")
     args = ap.parse_args()
     if args.case:

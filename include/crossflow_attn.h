@@ -68,6 +68,16 @@ typedef struct {
     int64_t k_stride_block, k_stride_head, k_stride_token;
     int64_t v_stride_block, v_stride_head, v_stride_token;
     float softmax_scale; /* 0 -> 1/sqrt(head_dim) */
+    /* Model-specific attention variant (Section 6.1 evaluates GPT-OSS-120B, whose layers alternate full and
+     * sliding-window attention and carry a learned sink logit per head; the paper itself does not describe it).
+     *   window_size W > 0: the query at position p sees keys j in [max(0, p - W + 1), p]; 0: every key up to p.
+     *     Block-table entries of pages that lie entirely left of every query's window are never read, so an
+     *     engine may have released those pages.
+     *   sink_logits: DEVICE fp32 [num_q_heads] or NULL.  The logit of head h (natural-log units, NOT multiplied
+     *     by softmax_scale) joins the softmax denominator and carries no value:
+     *       out = sum_j exp(x_j) v_j / (exp(sink_h) + sum_j exp(x_j)),  lse = ln(exp(sink_h) + sum_j exp(x_j)). */
+    int32_t window_size;
+    const float* sink_logits;
 } cf_cache_desc;
 
 /* Create a context on `device`.  workspace_bytes = 0: the split-K workspace starts at a default

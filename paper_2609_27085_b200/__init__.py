@@ -52,7 +52,7 @@ class CacheDesc(ctypes.Structure):
                 ("block_size", ctypes.c_int32), ("num_blocks", ctypes.c_int32),
                 ("k_stride_block", ctypes.c_int64), ("k_stride_head", ctypes.c_int64), ("k_stride_token", ctypes.c_int64),
                 ("v_stride_block", ctypes.c_int64), ("v_stride_head", ctypes.c_int64), ("v_stride_token", ctypes.c_int64),
-                ("softmax_scale", ctypes.c_float)]
+                ("softmax_scale", ctypes.c_float), ("window_size", ctypes.c_int32), ("sink_logits", ctypes.c_void_p)]
 
 
 class PlanOptions(ctypes.Structure):
@@ -142,14 +142,16 @@ def _stream(stream) -> Optional[int]:
 
 def make_desc(num_q_heads: int, num_kv_heads: int, head_dim: int, block_size: int, num_blocks: int,
               k_strides: Optional[Tuple[int, int, int]] = None, v_strides: Optional[Tuple[int, int, int]] = None,
-              softmax_scale: float = 0.0) -> CacheDesc:
+              softmax_scale: float = 0.0, window_size: int = 0, sink_logits=None) -> CacheDesc:
     """Descriptor for pools laid out [num_blocks, num_kv_heads, block_size, head_dim] unless
-    (block, head, token) element strides are given."""
+    (block, head, token) element strides are given.  window_size > 0: sliding-window attention;
+    sink_logits: device fp32 tensor [num_q_heads] (or address) of per-head sink logits.  The caller keeps
+    the sink tensor alive for as long as the descriptor is used."""
     default = (num_kv_heads * block_size * head_dim, block_size * head_dim, head_dim)
     ks = k_strides or default
     vs = v_strides or default
     return CacheDesc(num_q_heads, num_kv_heads, head_dim, block_size, num_blocks,
-                     ks[0], ks[1], ks[2], vs[0], vs[1], vs[2], softmax_scale)
+                     ks[0], ks[1], ks[2], vs[0], vs[1], vs[2], softmax_scale, int(window_size), _dev(sink_logits))
 
 
 def cf_create(device: int = 0, workspace_bytes: int = 0) -> ctypes.c_void_p:

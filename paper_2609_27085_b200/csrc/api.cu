@@ -375,6 +375,8 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
     p.scale_log2 = scale_log2_of(desc);
+    p.window = desc->window_size;
+    p.sinks = desc->sink_logits;
     p.q_start = (const int32_t*)(base + L.off_qstart);
     p.context_len = (const int32_t*)(base + L.off_ctx);
     p.query_len = (const int32_t*)(base + L.off_qlen);

@@ -64,7 +64,9 @@ __device__ __forceinline__ void merge_partials(const AttnParams& p, int q_row, i
                 acc.x += v[i].x * f; acc.y += v[i].y * f; acc.z += v[i].z * f; acc.w += v[i].w * f;
             }
     }
-    const float inv = 1.f / L;
+    float shrink = 1.f;
+    if (p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + hq) * kLog2e, M, L);
+    const float inv = shrink / L;
     __nv_bfloat162 lo = __floats2bfloat162_rn(acc.x * inv, acc.y * inv);
     __nv_bfloat162 hi = __floats2bfloat162_rn(acc.z * inv, acc.w * inv);
     uint2 packed;
@@ -139,7 +141,8 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
         for (int r = 0; r < (16 * CPR) / 32; ++r) {
             const int id = r * 32 + lane;
             const int t = id / CPR, c = id % CPR;
-            const bool ok = tok0 + t < it.kv_end;     // slack slots of the last page are zero-filled
+            // slack slots of the last page and tokens left of a sliding window are zero-filled
+            const bool ok = tok0 + t < it.kv_end && tok0 + t >= it.kv_lo;
             const int tt = ok ? t : 0;
             cp_async16_hint(sbase + tile_off<16>(t, c), kp + tt * p.ks_token + c * 8, ok ? 16 : 0, stream_once);
             cp_async16_hint(sbase + PAGE_BYTES + tile_off<16>(t, c), vp + tt * p.vs_token + c * 8, ok ? 16 : 0, stream_once);
@@ -184,7 +187,8 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
         const int tA = tok0 + (lane >> 2);
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
-            const bool ok = (tA + (e >> 1) * 8) < it.kv_end;
+            const int tok = tA + (e >> 1) * 8;
+            const bool ok = tok < it.kv_end && tok >= it.kv_lo;
             s[e] = ok ? (s0[e] + s1[e]) * p.scale_log2 : -INFINITY;
         }
         // per-head (column) max over the 16 tokens of the page: 2 local rows, 8 lane groups
@@ -265,7 +269,9 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
         }
         const int hq = kvh * G + head;
         if (it.part_slot < 0) {
-            const float inv = 1.f / L;
+            float shrink = 1.f;
+            if (p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + hq) * kLog2e, M, L);     // the only chunk: the sink joins here
+            const float inv = shrink / L;
             *reinterpret_cast<__nv_bfloat162*>(p.out + ((int64_t)it.q_row * p.Hq + hq) * D + d) =
                 __floats2bfloat162_rn(o0 * inv, o1 * inv);
             if (p.lse && d == 0) p.lse[(int64_t)it.q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
@@ -461,13 +467,17 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
         if (lc < 1) return CF_ERR_INVALID_ARG;                       // every sequence decodes one token
         if ((int64_t)lc > (int64_t)max_blocks_per_seq * B) return CF_ERR_OUT_OF_RANGE;
     }
-    const int64_t target = decode_target_pages(num_seqs, [&](int32_t s) -> int64_t { return context_len[s]; }, B,
-                                               desc->num_kv_heads, D, cfg, false);
+    const int32_t W = desc->window_size;
+    auto first_page_of = [&](int32_t lc) -> int64_t { return (W > 0 && lc > W) ? (lc - W) / B : 0; };
+    const int64_t target = decode_target_pages(
+        num_seqs, [&](int32_t s) -> int64_t { return (int64_t)context_len[s] - first_page_of(context_len[s]) * B; }, B,
+        desc->num_kv_heads, D, cfg, false);
 
     StaticPlan pl;
     for (int32_t s = 0; s < num_seqs; ++s) {
         const int32_t lc = context_len[s];
-        const int64_t pages = (lc + B - 1) / B;
+        const int64_t page0 = first_page_of(lc);
+        const int64_t pages = (lc + B - 1) / B - page0;
         int64_t n = 1, per = pages;
         decode_split(pages, target, cfg.decode_page_quantum, &n, &per);
         if (pl.n_items + n > kStaticMaxItems) return CF_ERR_WORKSPACE;
@@ -482,9 +492,9 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
             it.seq = s;
             it.q_row = s;
             it.n_chunks = (int32_t)n;
-            it.pad = 0;
-            it.kv_begin = (int32_t)(c * per * B);
-            it.kv_end = (int32_t)(((c + 1) * per * B < lc) ? (c + 1) * per * B : lc);
+            it.kv_lo = (W > 0 && lc > W) ? lc - W : 0;
+            it.kv_begin = (int32_t)((page0 + c * per) * B);
+            it.kv_end = (int32_t)(((page0 + (c + 1) * per) * B < lc) ? (page0 + (c + 1) * per) * B : lc);
             it.part_slot = n > 1 ? first + (int32_t)c : -1;
             it.chunk = (int32_t)c;
         }
@@ -524,6 +534,8 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hq = Hq; p.Hkv = desc->num_kv_heads; p.G = Hq / desc->num_kv_heads;
     p.scale_log2 = (desc->softmax_scale > 0.f ? desc->softmax_scale : 1.0f / sqrtf((float)D)) * 1.4426950408889634f;
+    p.window = desc->window_size;
+    p.sinks = desc->sink_logits;
     p.dec_items = reinterpret_cast<const DecodeItem*>(su.base);
     p.comb_items = reinterpret_cast<const CombineItem*>(su.base + comb_off);
     // Partials need no clearing: every slot the combine kernel reads is fully written by its decode CTA

@@ -21,6 +21,8 @@ struct AttnParams {
     int64_t vs_block, vs_head, vs_token;
     int32_t Hq, Hkv, G;
     float scale_log2;                 // softmax_scale * log2(e)
+    int32_t window;                   // sliding window in tokens (0 = none): row at position p sees keys (p - window, p]
+    const float* sinks;               // [Hq] per-head sink logits (natural-log units) or null
     const int32_t* context_len;       // device copies of the host arrays
     const int32_t* query_len;
     const int32_t* q_start;
@@ -117,5 +119,18 @@ __device__ __forceinline__ uint32_t tile_off(int t, int c)
 }
 
 constexpr float kLn2 = 0.6931471805599453f;
+constexpr float kLog2e = 1.4426950408889634f;
+
+// Joins a sink logit (log2 domain) to a softmax whose running maximum is M and un-normalised sum is L: the sink
+// adds 2^(sink - M') to the sum and carries no value.  Returns the factor by which the un-normalised output
+// must shrink (1 when the maximum does not move); M and L are updated.  M may be -inf only together with L = 0.
+__device__ __forceinline__ float join_sink(float sink2, float& M, float& L)
+{
+    const float Mn = fmaxf(M, sink2);
+    const float f = fast_exp2(M - Mn);
+    L = L * f + fast_exp2(sink2 - Mn);
+    M = Mn;
+    return f;
+}
 
 }  // namespace cf

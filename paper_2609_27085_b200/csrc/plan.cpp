@@ -43,6 +43,7 @@ cf_status validate_desc(const cf_cache_desc* d)
     }
     if (d->k_stride_token < d->head_dim || d->v_stride_token < d->head_dim) return CF_ERR_INVALID_ARG;
     if (!(d->softmax_scale >= 0.0f)) return CF_ERR_INVALID_ARG;   // also rejects NaN
+    if (d->window_size < 0) return CF_ERR_INVALID_ARG;
     return CF_OK;
 }
 
@@ -79,14 +80,20 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         else if (query_len[s] > 1) ++plan->n_prefill_seqs;
     const int32_t quantum = std::max(1, cfg.decode_page_quantum);
     const bool shares_sms = cfg.prefill_sms_mixed > 0 && plan->n_prefill_seqs > 0;   // spatial sequence: decode runs on part of the machine, beside prefill
+    // With a sliding window a decode token at position Lc - 1 sees keys [Lc - W, Lc): the chunks cover the pages
+    // from the one that holds the window's left edge onwards, and nothing left of it is ever touched.
+    const int32_t W = d->window_size;
+    auto first_page_of = [&](int32_t lc) -> int64_t { return (W > 0 && lc > W) ? (lc - W) / B : 0; };
     const int64_t target = decode_target_pages(
-        num_seqs, [&](int32_t s) -> int64_t { return query_len[s] == 1 ? (int64_t)context_len[s] : -1; }, B, d->num_kv_heads,
-        d->head_dim, cfg, shares_sms);
+        num_seqs,
+        [&](int32_t s) -> int64_t { return query_len[s] == 1 ? (int64_t)context_len[s] - first_page_of(context_len[s]) * B : -1; },
+        B, d->num_kv_heads, d->head_dim, cfg, shares_sms);
 
     for (int32_t s = 0; s < num_seqs; ++s) {
         if (query_len[s] != 1) continue;
         const int32_t lc = context_len[s];
-        const int64_t pages = (lc + B - 1) / B;
+        const int64_t page0 = first_page_of(lc);
+        const int64_t pages = (lc + B - 1) / B - page0;
         int64_t n = 1, per = pages;
         decode_split(pages, target, quantum, &n, &per);
         int32_t first = -1;
@@ -99,12 +106,12 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             DecodeItem it;
             it.seq = s;
             it.q_row = plan->q_start[s];
-            it.kv_begin = (int32_t)(c * per * B);
-            it.kv_end = (int32_t)std::min<int64_t>((c + 1) * per * B, lc);
+            it.kv_begin = (int32_t)((page0 + c * per) * B);
+            it.kv_end = (int32_t)std::min<int64_t>((page0 + (c + 1) * per) * B, lc);
             it.part_slot = n > 1 ? first + (int32_t)c : -1;
             it.chunk = (int32_t)c;
             it.n_chunks = (int32_t)n;
-            it.pad = 0;
+            it.kv_lo = (W > 0 && lc > W) ? lc - W : 0;
             plan->decode.push_back(it);
         }
     }
@@ -118,7 +125,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // (group size 1) two consecutive row tiles of one head
         constexpr int32_t TR = 128;
         const int32_t G = d->num_q_heads / d->num_kv_heads;
-        struct KeyedTc { int64_t extent; PrefillTcItem it; };
+        struct KeyedTc { int64_t extent; int32_t tiles; PrefillTcItem it; };   // extent: end of the visible keys; tiles: KV tiles to visit
         std::vector<KeyedTc> items;
         auto prefix_of = [&](int32_t s) { return context_len[s] - query_len[s]; };
         // All items of one (sequence, row tile) have the same KV extent, so the longest-first order is found by
@@ -144,8 +151,13 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             const int32_t n_tiles = (lq + TR - 1) / TR;
             auto rows_of = [&](int32_t tl) { return std::min(TR, lq - tl * TR); };
             PrefillTcItem it;
-            it.seq = s; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad[0] = it.pad[1] = 0;
-            it.j_begin = 0; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
+            it.seq = s; it.prefix = prefix; it.ctx_len = context_len[s]; it.pad = 0;
+            // sliding window: the item's first row (position prefix + tile * TR) sees keys from lo0 on, and no row of
+            // the item sees anything left of that; pages and KV tiles left of lo0 are skipped
+            const int32_t lo0 = (W > 0) ? std::max(0, prefix + tile * TR - W + 1) : 0;
+            it.page_lo = lo0 / B;
+            it.j_begin = lo0 / TR; it.j_end = INT32_MAX; it.part_slot[0] = it.part_slot[1] = -1; it.part_k = 1; it.part_c = 0;
+            const int32_t n_tiles_kv = (int32_t)((gr.extent + TR - 1) / TR) - it.j_begin;
             if (G >= 2) {
                 for (int t = 0; t < 2; ++t) {
                     it.q_row0[t] = plan->q_start[s] + tile * TR;
@@ -157,7 +169,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                         it.kvh = kvh;
                         it.head[0] = kvh * G + i;
                         it.head[1] = kvh * G + i + 1;
-                        items.push_back(KeyedTc{gr.extent, it});
+                        items.push_back(KeyedTc{gr.extent, n_tiles_kv, it});
                     }
             } else {
                 for (int t = 0; t < 2; ++t) {
@@ -170,7 +182,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 for (int32_t h = 0; h < d->num_q_heads; ++h) {
                     it.kvh = h;
                     it.head[0] = it.head[1] = h;
-                    items.push_back(KeyedTc{gr.extent, it});
+                    items.push_back(KeyedTc{gr.extent, n_tiles_kv, it});
                 }
             }
         }
@@ -188,7 +200,11 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     one.q_row0[0] = k.it.q_row0[t]; one.row0[0] = k.it.row0[t]; one.n_rows[0] = k.it.n_rows[t];
                     one.head[0] = k.it.head[t];
                     one.q_row0[1] = 0; one.row0[1] = 0; one.n_rows[1] = 0; one.head[1] = k.it.head[t];
-                    singles.push_back(KeyedTc{(int64_t)prefix_of(k.it.seq) + one.row0[0] + one.n_rows[0], one});
+                    const int64_t ext = (int64_t)prefix_of(k.it.seq) + one.row0[0] + one.n_rows[0];
+                    const int32_t lo1 = (W > 0) ? std::max(0, prefix_of(k.it.seq) + one.row0[0] - W + 1) : 0;
+                    one.page_lo = lo1 / B;
+                    one.j_begin = lo1 / TR;
+                    singles.push_back(KeyedTc{ext, (int32_t)((ext + TR - 1) / TR) - one.j_begin, one});
                 }
             std::stable_sort(singles.begin(), singles.end(), [](const KeyedTc& a, const KeyedTc& b) { return a.extent > b.extent; });
         }
@@ -202,7 +218,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         const size_t n_items = its.size();
         k_of.assign(n_items, 1);
         double predicted = 0.0;
-        auto tiles_of = [&](size_t i) { return (double)((its[i].extent + 127) / 128); };
+        auto tiles_of = [&](size_t i) { return (double)its[i].tiles; };
         // a whole item costs ~8 us + 1.9 us per tile; a KV range pays ~13 us (fp32 partial epilogue);
         // splitting adds the combine launch and the partial write/read
         auto split_extra = [](size_t n_ranges) { return 8.0 + 0.05 * (double)n_ranges; };
@@ -289,7 +305,8 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     n_min = std::min(n_min, (prefix + it.row0[t] + it.n_rows[t] + 127) / 128);
                     safe = std::min(safe, (prefix + it.row0[t]) / 128);
                 }
-            const int32_t k = std::min(k_want, std::max(1, std::min(n_min, safe + 1) / 4));
+            const int32_t j_lo = it.j_begin;          // first tile of the sliding window (0 without one); j_lo <= safe
+            const int32_t k = std::min(k_want, std::max(1, (std::min(n_min, safe + 1) - j_lo) / 4));
             if (k <= 1) {
                 plan->prefill_tc.push_back(it);
                 continue;
@@ -304,8 +321,8 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             plan->prefill_combine.push_back(ci);
             for (int32_t c = 0; c < k; ++c) {
                 PrefillTcItem f = it;
-                f.j_begin = std::min((int32_t)((int64_t)c * n_min / k), safe);
-                f.j_end = c + 1 < k ? std::min((int32_t)((int64_t)(c + 1) * n_min / k), safe) : INT32_MAX;
+                f.j_begin = std::min(j_lo + (int32_t)((int64_t)c * (n_min - j_lo) / k), safe);
+                f.j_end = c + 1 < k ? std::min(j_lo + (int32_t)((int64_t)(c + 1) * (n_min - j_lo) / k), safe) : INT32_MAX;
                 f.part_slot[0] = ci.part_slot[0]; f.part_slot[1] = ci.part_slot[1];
                 f.part_k = k; f.part_c = c;
                 plan->prefill_tc.push_back(f);
@@ -322,7 +339,9 @@ float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len
     const int32_t S = (int32_t)plan.q_start.size() - 1;
     double dec_bytes = 0.0;
     for (int32_t s = 0; s < S; ++s)
-        if (query_len[s] == 1) dec_bytes += (double)context_len[s] * 2.0 * d->num_kv_heads * d->head_dim * 2.0;
+        if (query_len[s] == 1)
+            dec_bytes += (double)(d->window_size > 0 ? std::min(context_len[s], d->window_size) : context_len[s]) * 2.0 *
+                         d->num_kv_heads * d->head_dim * 2.0;
     double work = 0.0;
     for (const PrefillTcItem& it : plan.prefill_tc) {
         int32_t hi = 0;
@@ -347,7 +366,8 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
     double dec_bytes = 0.0;
     for (int32_t s = 0; s < S; ++s)
         if (query_len[s] == 1)
-            dec_bytes += (double)context_len[s] * 2.0 * d->num_kv_heads * d->head_dim * 2.0 + 4.0 * d->num_q_heads * d->head_dim;
+            dec_bytes += (double)(d->window_size > 0 ? std::min(context_len[s], d->window_size) : context_len[s]) * 2.0 *
+                             d->num_kv_heads * d->head_dim * 2.0 + 4.0 * d->num_q_heads * d->head_dim;
     if (!plan.decode.empty()) e.us_decode = (float)(kDecodeFixedUs + dec_bytes / kDecodeBytesPerUs);
     if (!plan.combine.empty()) e.us_combine = (float)kCombineUs;
     if (!plan.prefill_tc.empty()) {

@@ -19,7 +19,8 @@ struct DecodeItem {        // one (decode sequence, KV chunk); the kernel adds t
     int32_t part_slot;     // partial slot to write, or -1: the only chunk, write `out` directly
     int32_t chunk;         // index of this chunk within its sequence
     int32_t n_chunks;      // chunks of the sequence (its partial slots are part_slot - chunk + [0, n_chunks))
-    int32_t pad;
+    int32_t kv_lo;         // first visible token of the sequence (left edge of a sliding window; 0 without one):
+                           // tokens of this chunk below it are masked (only the first chunk can hold any)
 };
 
 struct CombineItem {       // one decode sequence that was split
@@ -42,7 +43,9 @@ struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one
     int32_t part_slot[2];
     int32_t part_k, part_c;
     int32_t prefix, ctx_len;   // of the sequence (copied here so that a role needs one load per item)
-    int32_t pad[2];            // 80 bytes: five 16-byte words
+    int32_t page_lo;           // first page of the sequence any row of the item can see (sliding window; 0 without
+                               // one): pages below it are neither fetched nor multiplied
+    int32_t pad;               // 80 bytes: five 16-byte words
 };
 static_assert(sizeof(PrefillTcItem) == 80, "PrefillTcItem is copied as five 16-byte words");
 

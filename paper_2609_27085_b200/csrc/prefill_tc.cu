@@ -247,20 +247,22 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             const ItemCtx* cs = wait_item(k);
             if (cs == nullptr || cs->live == 0) break;
             const int n_max = cs->n_max, total_pages = cs->total_pages, jb = cs->it.j_begin, kvh = cs->it.kvh;
+            const int page_lo = cs->it.page_lo;          // sliding window: pages below it are not fetched (their table entries may be stale)
             const int32_t* bt = p.block_table + (int64_t)cs->it.seq * p.max_blocks;
-            int32_t pid = lane < min(8, total_pages - 8 * jb) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
+            int32_t pid = (lane < min(8, total_pages - 8 * jb) && 8 * jb + lane >= page_lo) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
             for (int j = 0; j < n_max && ok; ++j) {
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
+                const int p0 = max(0, page_lo - 8 * (jb + j));            // first page of the tile that is fetched
                 const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
                 if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? checked_pid(__ldg(bt + 8 * (jb + j + 1) + lane)) : 0;
                 const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.v_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
-                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), np * 16 * D * 2);
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.v_full[stage]), (np - p0) * 16 * D * 2);
                 __syncwarp();
-                if (lane < HALVES * np)
+                if (lane < HALVES * np && lane >= HALVES * p0)
                     tma_load_4d(smem + SMEM_V + stage * TILE_BYTES + dst_off, &map_v, (lane % HALVES) * 64, 0, kvh, my_pid,
                                 smem_u32(&bars.v_full[stage]));
             }
@@ -329,23 +331,25 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                                         it.q_row0[t], smem_u32(&bars.q_full));
             }
             const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks;
-            const int n_max = cx.n_max, total_pages = cx.total_pages, jb = it.j_begin;
+            const int n_max = cx.n_max, total_pages = cx.total_pages, jb = it.j_begin, page_lo = it.page_lo;
             const int j_draw = min(2, n_max - 1);       // the next ticket is drawn once the first tiles are on their way
             bool drawn = false;
-            // page ids of a tile are fetched while the tile before it is being issued
-            int32_t pid = lane < min(8, total_pages - 8 * jb) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
+            // page ids of a tile are fetched while the tile before it is being issued (never those of pages left of a
+            // sliding window: page_lo lies in the item's first tile)
+            int32_t pid = (lane < min(8, total_pages - 8 * jb) && 8 * jb + lane >= page_lo) ? checked_pid(__ldg(bt + 8 * jb + lane)) : 0;
             for (int j = 0; j < n_max && ok; ++j) {
                 const int stage = j & 1;
                 const uint32_t use = ub[stage] + (uint32_t)(j >> 1);
                 const int np = min(8, total_pages - 8 * (jb + j));
+                const int p0 = max(0, page_lo - 8 * (jb + j));
                 const int32_t my_pid = __shfl_sync(0xffffffffu, pid, lane / HALVES);
                 if (j + 1 < n_max) pid = lane < min(8, total_pages - 8 * (jb + j + 1)) ? checked_pid(__ldg(bt + 8 * (jb + j + 1) + lane)) : 0;
                 const uint32_t dst_off = (lane % HALVES) * HALF_BYTES + (lane / HALVES) * 2048;
                 if (use > 0) ok = __all_sync(0xffffffffu, mbar_wait(smem_u32(&bars.k_empty[stage]), (use - 1) & 1u, abort_flag));
                 if (!ok) break;
-                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), np * 16 * D * 2);
+                if (lane == 0) mbar_arrive_expect_tx(smem_u32(&bars.k_full[stage]), (np - p0) * 16 * D * 2);
                 __syncwarp();
-                if (lane < HALVES * np)
+                if (lane < HALVES * np && lane >= HALVES * p0)
                     tma_load_4d(smem + SMEM_K + stage * TILE_BYTES + dst_off, &map_k, (lane % HALVES) * 64, 0, it.kvh, my_pid,
                                 smem_u32(&bars.k_full[stage]));
                 if (j == j_draw) {
@@ -393,17 +397,19 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             for (int ks = 1; ks < KS; ++ks) umma_ss(dS, qd[t][ks], kd[st][ks], IDESC_QK, 1u);
             umma_commit(bar_s[t]);
         };
-        auto issue_pv = [&](auto T, auto S, int n_steps, uint32_t acc0) {   // O_t (+)= P_t V, one step per loaded page
+        // O_t (+)= P_t V, one K = 16 step per fetched page: pages [ks0, n_steps) of the tile (ks0 > 0 only in the first
+        // tile of a sliding window, n_steps < 8 only in a sequence's last tile)
+        auto issue_pv = [&](auto T, auto S, int ks0, int n_steps, uint32_t acc0) {
             constexpr int t = decltype(T)::value, st = decltype(S)::value;
             const uint32_t dO = tmem + TM_O + t * D, aP = tmem + TM_S + t * 128;
-            umma_ts(dO, aP, vd[st][0], IDESC_PV, acc0);
-            if (n_steps == 8) {
+            if (ks0 == 0 && n_steps == 8) {
+                umma_ts(dO, aP, vd[st][0], IDESC_PV, acc0);
 #pragma unroll
                 for (int ks = 1; ks < 8; ++ks) umma_ts(dO, aP + ks * 8, vd[st][ks], IDESC_PV, 1u);
             } else {
 #pragma unroll
-                for (int ks = 1; ks < 8; ++ks)
-                    if (ks < n_steps) umma_ts(dO, aP + ks * 8, vd[st][ks], IDESC_PV, 1u);
+                for (int ks = 0; ks < 8; ++ks)
+                    if (ks >= ks0 && ks < n_steps) umma_ts(dO, aP + ks * 8, vd[st][ks], IDESC_PV, ks == ks0 ? acc0 : 1u);
             }
             umma_commit(bar_o[t]);
         };
@@ -453,35 +459,23 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (!mbar_wait(bar_kf[st1], par_k1, abort_flag)) return false;
             if (!mbar_wait(bar_p[0], par_p0, abort_flag)) return false;
             tc_fence_after();
-            issue_pv(I0{}, S, 8, acc0);
+            issue_pv(I0{}, S, 0, 8, acc0);
             issue_qk(I0{}, S1{});
             if (!mbar_wait(bar_p[1], par_p1, abort_flag)) return false;
             tc_fence_after();
-            issue_pv(I1{}, S, 8, acc0);
+            issue_pv(I1{}, S, 0, 8, acc0);
             issue_qk(I1{}, S1{});
             umma_commit(bar_ve[st]);
             umma_commit(bar_ke[st1]);
             return true;
         };
-        int j = 0;
-        {
-            // parities of the even tile j of a pair: stage 0 fill ub[0] + j/2 (V now), stage 1 fill ub[1] + j/2
-            // (K of tile j + 1), softmax phases sb[t] + j; the odd tile j + 1 flips all but the stage-0 K
-            // fill of tile j + 2, which is ub[0] + j/2 + 1
-            uint32_t h0 = ist[0] & 1u, h1 = ist[1] & 1u;
-            const uint32_t p0 = ist[2] & 1u, p1 = ist[3] & 1u;
-            for (; ok && j + 1 < n_int; j += 2, h0 ^= 1u, h1 ^= 1u) {
-                ok = lean_step(I0{}, h0, h1, p0, p1, j > 0 ? 1u : 0u);
-                if (ok) ok = lean_step(I1{}, h1, h0 ^ 1u, p0 ^ 1u, p1 ^ 1u, 1u);
-            }
-            if (ok && j > 0 && j >= n_max - 1) umma_commit(bar_qe);     // the pair loop issued the item's last S = Q K^T
-        }
         // ---- general step: PV_0(j) QK_0(j+1) PV_1(j) QK_1(j+1) with every edge case
         auto kv_step = [&](auto S, int j) -> bool {
             constexpr int st = decltype(S)::value, st1 = st ^ 1;
             using S1 = std::integral_constant<int, st1>;
             const int jb = vs->it.j_begin, Lc = vs->it.ctx_len;
             const int np = min(8, vs->total_pages - 8 * (jb + j));
+            const int ks0 = max(0, vs->it.page_lo - 8 * (jb + j));      // sliding window: the tile's first fetched page
             if (!mbar_wait(bar_vf[st], (ist[st] + (uint32_t)(j >> 1)) & 1u, abort_flag)) return false;
             if (j == n_max - 1 && Lc < (8 * (jb + j) + np) * 16) {
                 // slack slots of the sequence's last page came in with the page: zero those V rows so
@@ -503,7 +497,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 if (more && !mbar_wait(bar_kf[st1], (ist[st1] + (uint32_t)((j + 1) >> 1)) & 1u, abort_flag)) return false;
                 if (!mbar_wait(bar_p[t], (ist[2 + t] + (uint32_t)j) & 1u, abort_flag)) return false;
                 tc_fence_after();
-                issue_pv(T, S, np, acc0);
+                issue_pv(T, S, ks0, np, acc0);
                 if (more) issue_qk(T, S1{});
                 return true;
             };
@@ -514,6 +508,26 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             if (j + 1 == n_max - 1) umma_commit(bar_qe);
             return true;
         };
+        int j = 0;
+        // Sliding window: the item's first tile may start with pages that are not fetched; it (and the tile after it,
+        // so that the pair loop below starts on an even tile) take the general step.
+        const bool partial_first = vs->it.page_lo > 8 * vs->it.j_begin;
+        if (partial_first) {
+            for (; j < min(2, n_max) && ok; ++j) ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
+        }
+        const int j_pairs = j;                       // where the pair loop starts: 0 or 2
+        if (ok) {
+            // parities of the even tile j of a pair: stage 0 fill ub[0] + j/2 (V now), stage 1 fill ub[1] + j/2
+            // (K of tile j + 1), softmax phases sb[t] + j; the odd tile j + 1 flips all but the stage-0 K
+            // fill of tile j + 2, which is ub[0] + j/2 + 1
+            uint32_t h0 = (ist[0] + (uint32_t)(j >> 1)) & 1u, h1 = (ist[1] + (uint32_t)(j >> 1)) & 1u;
+            const uint32_t p0 = ist[2] & 1u, p1 = ist[3] & 1u;
+            for (; ok && j + 1 < n_int; j += 2, h0 ^= 1u, h1 ^= 1u) {
+                ok = lean_step(I0{}, h0, h1, p0, p1, j > 0 ? 1u : 0u);
+                if (ok) ok = lean_step(I1{}, h1, h0 ^ 1u, p0 ^ 1u, p1 ^ 1u, 1u);
+            }
+            if (ok && j > j_pairs && j >= n_max - 1) umma_commit(bar_qe);     // the pair loop issued the item's last S = Q K^T
+        }
         static_assert(KV_STAGES == 2, "the stage index is the parity of the tile index");
         for (; j < n_max && ok; ++j) {
             ok = (j & 1) ? kv_step(I1{}, j) : kv_step(I0{}, j);
@@ -544,7 +558,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int it_row0 = cs->it.row0[t], it_n_rows = cs->it.n_rows[t], it_q_row0 = cs->it.q_row0[t], it_head = cs->it.head[t];
         const int it_part_slot = cs->it.part_slot[t], it_part_k = cs->it.part_k, it_part_c = cs->it.part_c;
         const int limit = min(cs->it.prefix + it_row0 + row, kv_hi - 1);   // last visible key of this row
-        float m_used = -INFINITY, l_sum = 0.f;
+        const int first_key = p.window > 0 ? limit - p.window + 1 : -(1 << 30);   // first visible key (sliding window)
+        const uint32_t span = (uint32_t)(limit - first_key);
+        float m_used = -INFINITY, l_sum = 0.f;     // -inf: the row has not met a visible key yet
         for (int j = 0; j < n_jt; ++j) {
             ok = mbar_wait(smem_u32(&bars.s_full[t]), (sbt + (uint32_t)j) & 1u, abort_flag);
             if (!ok) break;
@@ -553,14 +569,17 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 #pragma unroll
             for (int c = 0; c < 4; ++c) tmem_ld32(tS + c * 32, reinterpret_cast<uint32_t*>(&sv[c * 32]));
             tmem_wait_ld();
-            const int col_limit = limit - (jb + j) * KT;     // columns <= col_limit are visible
-            if (__any_sync(0xffffffffu, col_limit < KT - 1)) {
+            const int col_limit = limit - (jb + j) * KT;     // columns [col_first, col_limit] are visible
+            const int col_first = first_key - (jb + j) * KT;
+            if (__any_sync(0xffffffffu, col_limit < KT - 1 || col_first > 0)) {
 #pragma unroll
-                for (int c = 0; c < 128; ++c) sv[c] = (c <= col_limit) ? sv[c] : -INFINITY;
+                for (int c = 0; c < 128; ++c) sv[c] = ((uint32_t)(c - col_first) <= span) ? sv[c] : -INFINITY;
             }
-            if (j == 0) {
-                // first tile: exact row maximum.  It is finite: every row sees a key of the item's first
-                // tile (key 0 for a whole item; the planner never starts a split inside the diagonal band)
+            if (__any_sync(0xffffffffu, m_used == -INFINITY)) {
+                // A row's first tile with a visible key: the exact row maximum becomes its reference.  Without a
+                // sliding window that is the item's first tile for every row (key 0 of a whole item; the planner
+                // never starts a KV range inside the diagonal band); with one, a row of the tile's lower part may
+                // meet its first key one tile later and keeps -inf (all its probabilities are zero) until then.
                 float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
                 for (int c = 4; c < 128; c += 8) {
@@ -571,7 +590,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                         mx4[3] = max3(mx4[3], sv[c + 6], sv[c + 7]);
                     }
                 }
-                m_used = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
+                if (m_used == -INFINITY) m_used = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc;
             }
             // Optimistic pass: exponentials against the current reference maximum, packed two per
             // FMA-pipe instruction.  Whether the reference has to be raised is read off the tile's row
@@ -597,7 +616,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 const float2 a01 = add2(acc2[0], acc2[1]), a23 = add2(acc2[2], acc2[3]);
                 return (a01.x + a01.y) + (a23.x + a23.y);
             };
-            float tile_sum = exp_pass(-m_used);
+            float tile_sum = exp_pass(m_used == -INFINITY ? 0.f : -m_used);
             if (__any_sync(0xffffffffu, !(tile_sum <= 32768.f))) {
                 float mx4[4] = {sv[0], sv[1], sv[2], sv[3]};
 #pragma unroll
@@ -608,7 +627,8 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     mx4[3] = fmaxf(mx4[3], sv[c + 3]);
                 }
                 const float rise = fmaxf(fmaxf(mx4[0], mx4[1]), fmaxf(mx4[2], mx4[3])) * sc - m_used;
-                const float d = fmaxf(rise, 0.f);            // rows that did not rise keep their reference
+                const float d = fmaxf(rise, 0.f);            // rows that did not rise keep their reference (a row without
+                                                             // a visible key so far: -inf - -inf is NaN, which fmaxf drops)
                 const float f = fast_exp2(-d);
                 m_used += d;
                 l_sum *= f;
@@ -627,7 +647,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                     }
                 }
                 tmem_wait_st();
-                tile_sum = exp_pass(-m_used);
+                tile_sum = exp_pass(m_used == -INFINITY ? 0.f : -m_used);
             }
             l_sum += tile_sum;
             tmem_wait_st();
@@ -638,9 +658,12 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         if (ok && n_jt > 0) ok = mbar_wait(smem_u32(&bars.o_done[t]), (sbt + (uint32_t)(n_jt - 1)) & 1u, abort_flag);
         if (ok && n_jt > 0) {
             tc_fence_after();
-            const float inv = 1.f / l_sum;
             const bool live = row < it_n_rows;
             const bool partial = it_part_slot >= 0;
+            // a whole item joins the head's sink logit here; a KV range leaves it to the combine pass
+            float m_fin = m_used, l_fin = l_sum, shrink = 1.f;
+            if (!partial && p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + it_head) * kLog2e, m_fin, l_fin);
+            const float inv = shrink / l_fin;
             __nv_bfloat16* orow = p.out + ((int64_t)(it_q_row0 + row) * p.Hq + it_head) * D;
             // KV-split item: un-normalised fp32 row plus (reference maximum, sum) for the combine pass
             const int64_t pslot = (int64_t)it_part_slot + (int64_t)row * it_part_k + it_part_c;
@@ -666,7 +689,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
                 }
             }
             if (live && partial) *reinterpret_cast<float2*>(p.pre_part_ml + pslot * 2) = make_float2(m_used, l_sum);
-            else if (live && p.lse) p.lse[(int64_t)(it_q_row0 + row) * p.Hq + it_head] = (m_used + log2f(l_sum)) * kLn2;
+            else if (live && p.lse) p.lse[(int64_t)(it_q_row0 + row) * p.Hq + it_head] = (m_fin + log2f(l_fin)) * kLn2;
             // O_t has been read out: the p_full arrival of the next item's first tile, later in this thread's
             // program order, is what allows the issuer to overwrite it
             tc_fence_before();
@@ -727,7 +750,9 @@ __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p
             L += ml[c].y * f;
             acc.x += v[c].x * f; acc.y += v[c].y * f; acc.z += v[c].z * f; acc.w += v[c].w * f;
         }
-    const float inv = 1.f / L;
+    float shrink = 1.f;
+    if (p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + it.head[t]) * kLog2e, M, L);
+    const float inv = shrink / L;
     uint2 w;
     w.x = pack_bf16(acc.x * inv, acc.y * inv);
     w.y = pack_bf16(acc.z * inv, acc.w * inv);

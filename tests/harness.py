@@ -33,9 +33,13 @@ def to_host_bits(t: torch.Tensor) -> np.ndarray:
 class GpuScenario:
     """Device copy of a scenario's pools plus a library context."""
 
-    def __init__(self, sc: syn.Scenario, ctx=None, softmax_scale: float = 0.0, layout: str = "HND", debug=None):
-        """debug: {CF_DEBUG_* option: value} applied to a context created here (test-only planner switches)."""
+    def __init__(self, sc: syn.Scenario, ctx=None, softmax_scale: float = 0.0, layout: str = "HND", debug=None,
+                 window: int = 0, sinks=None):
+        """debug: {CF_DEBUG_* option: value} applied to a context created here (test-only planner switches).
+        window / sinks: the sliding-window and attention-sink variant (sinks: host fp32 array [Hq])."""
         self.geom = g = sc.geom
+        self.sinks_dev = None if sinks is None else torch.from_numpy(np.ascontiguousarray(sinks, dtype=np.float32)).cuda()
+        variant = dict(window_size=window, sink_logits=self.sinks_dev)
         self.layout = layout
         self.own_ctx = ctx is None
         self.ctx = cf.cf_create(0) if ctx is None else ctx
@@ -45,14 +49,14 @@ class GpuScenario:
             self.k = to_dev_bf16(sc.k_pool)
             self.v = to_dev_bf16(sc.v_pool)
             self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks,
-                                     softmax_scale=softmax_scale)
+                                     softmax_scale=softmax_scale, **variant)
         else:  # NHD: [NB, B, Hkv, D] storage
             self.k = to_dev_bf16(np.ascontiguousarray(sc.k_pool.transpose(0, 2, 1, 3)))
             self.v = to_dev_bf16(np.ascontiguousarray(sc.v_pool.transpose(0, 2, 1, 3)))
             H, B, D = g.num_kv_heads, g.block_size, g.head_dim
             st = (B * H * D, D, H * D)
             self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks,
-                                     k_strides=st, v_strides=st, softmax_scale=softmax_scale)
+                                     k_strides=st, v_strides=st, softmax_scale=softmax_scale, **variant)
 
     def pools_host(self):
         k, v = to_host_bits(self.k), to_host_bits(self.v)
@@ -106,11 +110,11 @@ def compare(o_bits: np.ndarray, lse: np.ndarray, ref_o: np.ndarray, ref_lse: np.
 
 
 def run_and_check(sc: syn.Scenario, max_prefill_rows: int = 0, layout: str = "HND", softmax_scale: float = 0.0,
-                  check_append: bool = True, ctx=None, debug=None, tile_rows: bool = False):
+                  check_append: bool = True, ctx=None, debug=None, tile_rows: bool = False, window: int = 0, sinks=None):
     """Every iteration of the scenario: append + attention on both sides, compare.
     Rows compared: all of them, or (max_prefill_rows) a thinned sample per prefill sequence, or (tile_rows) the
     first and last row of every 128-row q tile plus every 41st row of each prefill sequence, all heads."""
-    gpu = GpuScenario(sc, ctx=ctx, softmax_scale=softmax_scale, layout=layout, debug=debug)
+    gpu = GpuScenario(sc, ctx=ctx, softmax_scale=softmax_scale, layout=layout, debug=debug, window=window, sinks=sinks)
     k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
     all_stats = []
     try:
@@ -123,7 +127,8 @@ def run_and_check(sc: syn.Scenario, max_prefill_rows: int = 0, layout: str = "HN
             o_bits, lse = gpu.attend(b)
             rows = syn.tile_edge_rows(b) if tile_rows else (syn.sample_rows(b, max_prefill_rows) if max_prefill_rows else None)
             ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len,
-                                                    scale=(softmax_scale or None), rows=rows)
+                                                    scale=(softmax_scale or None), rows=rows, window=window,
+                                                    sinks=None if sinks is None else np.asarray(sinks, dtype=np.float32).astype(np.float64))
             all_stats.append(compare(o_bits, lse, ref_o, ref_lse, rows=rows, label=b.label))
     finally:
         gpu.close()

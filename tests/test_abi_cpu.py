@@ -209,3 +209,33 @@ def test_forced_kv_split_tiles_every_item():
             assert ranges[0][0] == 0 and ranges[-1][1] == (3100 + row0 + n_rows + 127) // 128
             assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
             assert len(ranges) <= k
+
+
+def test_windowed_plan_skips_what_no_query_can_see():
+    """Sliding window W: decode chunks tile [page of (Lc - W), Lc) and prefill KV ranges tile the tiles from the one
+    that holds the first row's left edge up to the diagonal; nothing left of that is planned."""
+    rng = np.random.default_rng(3)
+    for W in (1, 16, 100, 128, 1000, 4096):
+        d = cf.make_desc(32, 8, 128, 16, 1 << 16, window_size=W)
+        S = 12
+        lq = rng.choice([1, 1, 1, 64, 300, 700], size=S)
+        lc = lq + rng.integers(0, 9000, size=S)
+        for split in (0, 2):
+            st, dec, comb, pre, parts = cf.cf_plan_inspect(d, lc, lq, 1 << 16, 148, prefill_force_split=split)
+            for s in np.nonzero(lq == 1)[0]:
+                mine = dec[dec[:, 0] == s]
+                mine = mine[np.argsort(mine[:, 5])]
+                lo = max(0, lc[s] - W)
+                assert mine[0, 2] == (lo // 16) * 16 and mine[-1, 3] == lc[s]
+                assert (mine[1:, 2] == mine[:-1, 3]).all() and (mine[:, 3] > mine[:, 2]).all()
+            by_tile = {}
+            for s_, q_row0, row0, n_rows, head, kvh, j0, j1 in pre:
+                by_tile.setdefault((s_, row0, n_rows, head), []).append((j0, j1))
+            assert len(by_tile) == sum(((n + 127) // 128) * 32 for n in lq if n > 1)
+            for (s_, row0, n_rows, head), ranges in by_tile.items():
+                ranges.sort()
+                P = lc[s_] - lq[s_]
+                assert ranges[0][0] == max(0, P + row0 - W + 1) // 128
+                assert ranges[-1][1] == (P + row0 + n_rows + 127) // 128
+                assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
+    assert cf.cf_plan_inspect(cf.make_desc(32, 8, 128, 16, 64, window_size=-1), [5], [1], 8, check=False)[0] == cf.CF_ERR_INVALID_ARG

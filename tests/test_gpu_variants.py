@@ -1,0 +1,169 @@
+"""GPU parity of the model-specific attention variant - sliding window and per-head attention sinks -
+against the oracle's statement of it, on the decode kernel, the tcgen05 prefill kernel (whole items and
+KV ranges) and mixed batches."""
+import numpy as np
+import pytest
+import torch
+
+import cf_synth as syn
+import oracle
+import paper_2609_27085_b200 as cf
+from harness import GpuScenario, compare, run_and_check, to_dev_bf16, to_host_bits
+
+pytestmark = pytest.mark.gpu
+
+
+def small(seed, Hq, Hkv, D, prefix, qlens, NB=2048, shuffle=False):
+    return syn.scenario_from_lengths("v", syn.Geometry(Hq, Hkv, D, 16, NB), seed, prefix, qlens, shuffle_seqs=shuffle)
+
+
+def sink_values(Hq, seed=0):
+    return np.random.default_rng(100 + seed).normal(0.0, 2.0, size=Hq).astype(np.float32)
+
+
+@pytest.mark.parametrize("window", [1, 16, 17, 100, 128, 1000, 5000])
+@pytest.mark.parametrize("Hq,Hkv,D,with_sinks", [(32, 8, 128, True), (8, 2, 64, False), (64, 8, 128, True)])
+def test_windowed_decode(window, Hq, Hkv, D, with_sinks):
+    lens = [1, 2, 15, 16, 17, 31, 33, 127, 129, 255, 700, 1025, 2500, 4097, 9000, 20000]
+    sc = small(3, Hq, Hkv, D, [l - 1 for l in lens], [[1] * len(lens)], NB=4096)
+    run_and_check(sc, window=window, sinks=sink_values(Hq) if with_sinks else None)
+
+
+@pytest.mark.parametrize("window", [1, 17, 128, 129, 300, 1024])
+@pytest.mark.parametrize("Hq,Hkv,D,with_sinks", [(32, 8, 128, True), (4, 4, 128, False), (8, 2, 64, True), (16, 2, 128, False)])
+def test_windowed_prefill(window, Hq, Hkv, D, with_sinks):
+    prefix = [0, 0, 5, 16, 63, 64, 100, 1000, 0, 333, 2000]
+    qlen = [2, 64, 65, 17, 1, 128, 129, 200, 300, 31, 700]
+    run_and_check(small(5, Hq, Hkv, D, prefix, [qlen]), window=window, sinks=sink_values(Hq, 1) if with_sinks else None)
+
+
+def test_sinks_without_a_window():
+    prefix = [10, 0, 500, 77, 0, 2000, 31, 640, 5, 1, 9000]
+    qlen = [1, 90, 1, 0, 1, 1, 130, 1, 0, 64, 1]
+    run_and_check(small(7, 32, 8, 128, prefix, [qlen], shuffle=True), sinks=sink_values(32, 2))
+    # a huge sink swallows nearly all of the probability: outputs shrink towards zero, lse follows the sink
+    run_and_check(small(7, 8, 2, 64, prefix, [qlen], shuffle=True), sinks=np.full(8, 30.0, dtype=np.float32))
+    run_and_check(small(7, 8, 2, 64, prefix, [qlen], shuffle=True), sinks=np.full(8, -30.0, dtype=np.float32))
+
+
+@pytest.mark.parametrize("split", [2, 3])
+def test_windowed_prefill_items_cut_into_kv_ranges(split):
+    """A window long enough for the band to hold several KV ranges per item (forced split), with sinks (joined in
+    the combine pass), beside decode sequences."""
+    prefix = [6000, 300, 4097, 50, 8000]
+    qlen = [300, 700, 129, 1, 1]
+    sinks = sink_values(32, 3)
+    for window in (2048, 3000):
+        sc = small(43, 32, 8, 128, prefix, [qlen], NB=2048)
+        b = sc.batches[0]
+        d = cf.make_desc(32, 8, 128, 16, 2048, window_size=window)
+        counts = cf.cf_plan_inspect(d, b.context_len, b.query_len, b.max_blocks, prefill_force_split=split, want_counts=True)[5]
+        assert counts[5] > 0
+        run_and_check(sc, window=window, sinks=sinks, debug={cf.CF_DEBUG_PREFILL_SPLIT: split})
+
+
+def test_pages_left_of_the_window_are_never_touched():
+    """An engine that serves a sliding-window layer releases the pages that no query can see any more.  Here their
+    block-table entries are -1 and their contents NaN: the kernels must neither dereference the entries (the
+    status word would report a block id outside the pool) nor let the contents reach a result."""
+    window = 200
+    prefix = [3000, 5000, 700, 130, 0]
+    qlen = [300, 1, 1, 150, 64]
+    sc = small(45, 32, 8, 128, prefix, [qlen], NB=1024)
+    b = sc.batches[0]
+    g = GpuScenario(sc, window=window, sinks=sink_values(32, 4))
+    g.append(b)
+    k_ref, v_ref = g.pools_host()
+    table = b.block_table.copy()
+    nan = torch.tensor(float("nan"), dtype=torch.bfloat16, device="cuda")
+    for s in range(b.num_seqs):
+        first_visible = int(b.context_len[s]) - int(b.query_len[s]) - window + 1      # left edge of the first row's window
+        for pg in range(max(0, first_visible) // 16):
+            blk = int(table[s, pg])
+            g.k[blk] = nan
+            g.v[blk] = nan
+            k_ref[blk] = syn.BF16_NAN_BITS
+            v_ref[blk] = syn.BF16_NAN_BITS
+            table[s, pg] = -1
+    dead = syn.Batch(b.geom, b.context_len, b.query_len, table, b.q, b.k_new, b.v_new)
+    o_bits, lse = g.attend(dead)
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, table, b.context_len, b.query_len, window=window,
+                                            sinks=sink_values(32, 4).astype(np.float64))
+    assert np.isfinite(ref_o).all()
+    compare(o_bits, lse, ref_o, ref_lse)
+    g.close()
+
+
+def test_window_edges_with_a_spike_key():
+    """A key that towers over the rest, planted on both sides of the window's left edge of several rows: inside
+    the window it must dominate the row, one position further left it must not be seen."""
+    Hq, Hkv, D, window = 8, 2, 128, 300
+    Lq, P = 400, 1500
+    sc = small(47, Hq, Hkv, D, [P, 2000], [[Lq, 1]], NB=1024)
+    b = sc.batches[0]
+    g = GpuScenario(sc, window=window)
+    g.append(b)
+    k0 = g.k.clone()
+    big = torch.zeros(D, dtype=torch.bfloat16, device="cuda")
+    big[0] = 96.0
+    q = b.q.copy()
+    q[:, :, 0] = syn.f32_to_bf16_bits(np.float32(8.0))
+    bq = syn.Batch(b.geom, b.context_len, b.query_len, b.block_table, q, b.k_new, b.v_new)
+    v_host = to_host_bits(g.v)
+    rows = [0, 1, 127, 128, 255, 256, Lq - 1]
+    cand = set()
+    for i in rows:
+        left = P + i - window + 1
+        cand.update({left - 1, left, left + 1, P + i, P + i + 1})
+    for j in sorted(c for c in cand if 0 <= c < P + Lq):
+        g.k.copy_(k0)
+        blk, slot = int(b.block_table[0, j // 16]), j % 16
+        g.k[blk, :, slot, :] = big
+        o, _ = g.attend(bq, want_lse=False)
+        o = syn.bf16_bits_to_f64(o)
+        want = np.repeat(syn.bf16_bits_to_f64(v_host[blk, :, slot, :]), Hq // Hkv, axis=0)
+        for i in rows:
+            visible = P + i - window + 1 <= j <= P + i
+            assert (np.abs(o[i] - want).max() <= 2e-2) == visible, (j, i)
+    # the decode sequence: position 2000, window [1701, 2000]
+    for j, visible in ((1700, False), (1701, True), (2000, True)):
+        g.k.copy_(k0)
+        blk, slot = int(b.block_table[1, j // 16]), j % 16
+        g.k[blk, :, slot, :] = big
+        o, _ = g.attend(bq, want_lse=False)
+        o = syn.bf16_bits_to_f64(o)
+        want = np.repeat(syn.bf16_bits_to_f64(v_host[blk, :, slot, :]), Hq // Hkv, axis=0)
+        assert (np.abs(o[Lq] - want).max() <= 2e-2) == visible, j
+    g.close()
+
+
+def test_windowed_agentic_configuration_at_full_size():
+    """configs[3] (16 decode sequences of 8K..32K, a 2048-token chunk over 24,576 cached tokens) as a sliding-window
+    layer of 128 tokens with sinks - the geometry of the windowed layers of GPT-OSS - and with a 4096-token window:
+    first chunk iteration, decode rows and the edge rows of every q tile against the oracle."""
+    for window in (128, 4096):
+        sc = syn.config4_agentic(iterations=(0,))
+        run_and_check(sc, tile_rows=True, check_append=False, window=window, sinks=sink_values(32, 5))
+
+
+def test_static_entry_point_honours_window_and_sinks():
+    lens = [30000, 17, 4096, 1, 9001, 640]
+    sc = small(49, 32, 8, 128, [l - 1 for l in lens], [[1] * len(lens)], NB=4096)
+    b = sc.batches[0]
+    sinks = sink_values(32, 6)
+    g = GpuScenario(sc, window=1000, sinks=sinks)
+    g.append(b)
+    ctx_o, ctx_lse = g.attend(b)
+    bt = torch.from_numpy(b.block_table).cuda()
+    q = to_dev_bf16(b.q)
+    out = torch.full_like(q, float("nan"))
+    lse = torch.full((b.total_q, 32), float("nan"), dtype=torch.float32, device="cuda")
+    cf.cf_decode_attention_static(g.desc, q, g.k, g.v, bt, b.max_blocks, b.context_len, out, lse)
+    torch.cuda.synchronize()
+    assert np.array_equal(to_host_bits(out), ctx_o) and np.array_equal(lse.cpu().numpy(), ctx_lse)
+    k_ref, v_ref = g.pools_host()
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len, window=1000,
+                                            sinks=sinks.astype(np.float64))
+    compare(ctx_o, ctx_lse, ref_o, ref_lse)
+    g.close()
