@@ -599,8 +599,60 @@ def small_case(name: str) -> syn.Scenario:
     raise SystemExit(f"unknown case {name}")
 
 
+def run_shared_prefix_case(args):
+    """16 decode sequences (Hq 32, Hkv 8, D 128) that share an 8192-token prefix and have 200..900 tokens of their
+    own: the same batch through cf_mixed_attention (every sequence streams the shared pages) and through
+    cf_mixed_attention_shared (the shared pages are streamed once per set of four sequences).  `--variant plain`
+    or `--variant shared` runs only that one (for a profiler capture)."""
+    import torch
+    import paper_2609_27085_b200 as cf
+    torch.cuda.set_device(0)
+    geom = syn.Geometry(32, 8, 128, 16, 16384)
+    rng = np.random.default_rng(7)
+    own = [int(x) for x in rng.integers(200, 900, size=16)]
+    sc, sg, sl = syn.shared_prefix_scenario("shared_prefix", geom, 47, 8192, own, [1] * 16, [0] * 16)
+    b = sc.batches[0]
+    ctx = cf.cf_create(0)
+    wl = DeviceWorkload(sc, torch, cf, ctx)
+    it = wl.its[0]
+    stream = torch.cuda.current_stream()
+    wl.step(0, stream)                                               # append once
+    per_tok = geom.kv_bytes_per_token()
+    bytes_plain = int(sum(int(x) for x in b.context_len) * per_tok)
+    bytes_dedup = int((8192 + sum(int(x) - 8192 for x in b.context_len)) * per_tok)
+    res = {"case": "shared_prefix", "kv_bytes_every_sequence": bytes_plain, "kv_bytes_shared_once": bytes_dedup}
+
+    def plain(i):
+        cf.cf_mixed_attention(ctx, wl.desc, it["q"], wl.k, wl.v, it["bt"], b.max_blocks, b.context_len, b.query_len,
+                              it["out"], None, stream=stream)
+
+    def shared(i):
+        cf.cf_mixed_attention_shared(ctx, wl.desc, it["q"], wl.k, wl.v, it["bt"], b.max_blocks, b.context_len, b.query_len,
+                                     sg, sl, it["out"], None, stream=stream)
+
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")      # larger than L2: every timed call starts cold
+    for name, fn in (("plain", plain), ("shared", shared)):
+        if args.variant not in ("both", name):
+            continue
+        for i in range(args.warmup):
+            fn(i)
+        ts = []
+        for i in range(args.steps):
+            flush.zero_()
+            ts.append(time_region(torch, fn, 1, stream))
+        res[name] = {"ms": float(np.median(ts)), "ms_min": float(min(ts)),
+                     "effective_gbs_of_all_sequences": bytes_plain / (float(np.median(ts)) * 1e-3) / 1e9,
+                     "plan_counts": [int(x) for x in cf.cf_get_last_plan_counts(ctx)]}
+    assert cf.cf_get_async_status(ctx) == cf.CF_OK
+    print(json.dumps(res), flush=True)
+    del wl
+    cf.cf_destroy(ctx)
+
+
 def run_case(args):
     """Runs one reduced workload for `warmup + steps` steps and prints its per-kernel times."""
+    if args.case == "shared_prefix":
+        return run_shared_prefix_case(args)
     import torch
     import paper_2609_27085_b200 as cf
     torch.cuda.set_device(0)
@@ -622,7 +674,8 @@ def run_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None,
-                    help="run a reduced workload (decode_small | prefill_small | prefill_multi | agentic_small) and exit")
+                    help="run a reduced workload (decode_small | prefill_small | prefill_multi | agentic_small | shared_prefix) and exit")
+    ap.add_argument("--variant", default="both", choices=["both", "plain", "shared"], help="shared_prefix case: which entry point")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=5)

@@ -373,3 +373,50 @@ def sample_rows(batch: Batch, max_prefill_rows_per_seq: int = 0) -> np.ndarray:
                 idx = idx[pick]
         rows.append(qs[s] + idx)
     return np.concatenate(rows).astype(np.int64) if rows else np.zeros(0, dtype=np.int64)
+
+
+def shared_prefix_scenario(name: str, geom: Geometry, seed: int, shared_tokens: int, own_prefix: Sequence[int],
+                           query_len: Sequence[int], group: Optional[Sequence[int]] = None):
+    """Sequences whose block tables alias the same pages for a common prefix (radix-cache reuse: turns of one
+    agent session, sub-agents forked from one context).  Sequence s with group[s] >= 0 starts with the
+    `shared_tokens` tokens of its group's prefix (a multiple of the block size, the same physical pages for every
+    member), followed by own_prefix[s] cached tokens of its own and query_len[s] new ones; group[s] < 0: no
+    shared part.  Returns (scenario with one batch, share_group int32 [S], shared_len int32 [S])."""
+    B = geom.block_size
+    assert shared_tokens % B == 0
+    S = len(own_prefix)
+    group = np.zeros(S, dtype=np.int32) if group is None else np.asarray(group, dtype=np.int32)
+    rng = np.random.default_rng(seed)
+    k_pool, v_pool = empty_pools(geom)
+    perm = rng.permutation(geom.num_blocks).astype(np.int32)
+    at = 0
+    n_shared_pages = shared_tokens // B
+    group_pages = {}
+    for gid in sorted(set(int(x) for x in group if x >= 0)):
+        pages = perm[at:at + n_shared_pages]
+        at += n_shared_pages
+        fill_prefix(rng, geom, k_pool, pages, shared_tokens)
+        fill_prefix(rng, geom, v_pool, pages, shared_tokens)
+        group_pages[gid] = pages
+    lens = []
+    rows = []
+    for s in range(S):
+        sh = shared_tokens if group[s] >= 0 else 0
+        total = sh + int(own_prefix[s]) + int(query_len[s])
+        n_own_pages = (total + B - 1) // B - sh // B
+        own = perm[at:at + n_own_pages]
+        at += n_own_pages
+        assert at <= geom.num_blocks, "pool too small"
+        row = np.concatenate([group_pages[int(group[s])], own]) if group[s] >= 0 else own
+        fill_prefix(rng, geom, k_pool, own, int(own_prefix[s]))
+        fill_prefix(rng, geom, v_pool, own, int(own_prefix[s]))
+        rows.append(row)
+        lens.append(total)
+    width = max(len(r) for r in rows)
+    table = np.full((S, width), -1, dtype=np.int32)
+    for s, r in enumerate(rows):
+        table[s, :len(r)] = r
+    b = make_batch(rng, geom, lens, query_len, table, label=name)
+    sc = Scenario(name, geom, k_pool, v_pool, [b])
+    shared_len = np.where(group >= 0, shared_tokens, 0).astype(np.int32)
+    return sc, group.astype(np.int32), shared_len

@@ -117,6 +117,23 @@ cf_status cf_mixed_attention(cf_ctx* ctx, const cf_cache_desc* desc, const void*
                              const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
                              void* out, float* lse, void* cuda_stream);
 
+/* The same with a description of shared prefixes (Section 4.4: a radix-cache lookup tells how much of a prompt
+ * is already resident; Section 2.1: agent turns and sub-agents share long prefixes).  Sequences with the same
+ * share_group[s] >= 0 promise that their block-table rows are identical for the first shared_len[s] tokens (the
+ * same physical pages); share_group[s] < 0: shares nothing.  The result is what cf_mixed_attention gives for the
+ * same arguments - aliased block tables define it - but the decode sequences of a group (two or more, full
+ * attention, at least 256 common tokens) read the common pages once per KV chunk for a whole set of members
+ * instead of once each; each member's own suffix is read as usual and merged with it.  Prefill chunks and
+ * sliding-window layers are served as by cf_mixed_attention.  share_group, shared_len: HOST int32 [num_seqs],
+ * both or neither (neither: exactly cf_mixed_attention).  If the promise does not hold the affected rows are
+ * meaningless, but nothing is read outside the pages the tables name. */
+cf_status cf_mixed_attention_shared(cf_ctx* ctx, const cf_cache_desc* desc, const void* q,
+                                    const void* k_cache, const void* v_cache,
+                                    const int32_t* block_table, int32_t max_blocks_per_seq,
+                                    const int32_t* context_len, const int32_t* query_len,
+                                    const int32_t* share_group, const int32_t* shared_len, int32_t num_seqs,
+                                    void* out, float* lse, void* cuda_stream);
+
 /* Plan once, launch many times.  The lengths of a scheduler iteration are the same for every layer
  * of the model (Section 5: one mixed batch per iteration), so the host planning and the plan upload can
  * be done once: cf_plan_create validates, plans and uploads (it allocates the plan's own device buffers
@@ -169,7 +186,8 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  *     caller's stream alone.
  *   cf_set_overlap(ctx, n), n > 0 (the initial state is n = 1): n persistent prefill CTAs, one per SM (n = 1:
  *     the library's default share of the SMs), are enqueued first, on the caller's stream; a context-owned
- *     side stream, forked from the caller's, runs decode on the SMs left over, and behind it a second prefill
+ *     side stream, forked from the caller's, runs decode on the SMs left over as soon as those CTAs hold their
+ *     SMs (it waits for their count with a stream memory operation), and behind it a second prefill
  *     grid that draws from the same work queue, so the SMs decode frees join the prefill.  The side stream is
  *     joined back into the caller's stream inside the call, so the caller still sees one stream.
  * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n (the share that n = 1 stands for).
@@ -191,14 +209,15 @@ cf_status cf_validate_block_table(cf_ctx* ctx, const cf_cache_desc* desc, const 
  *   CF_DEBUG_SEPARATE_COMBINE       1: merge split-K decode partials in the separate combine kernel
  *   CF_DEBUG_DECODE_WAVES           target number of decode CTA waves
  *   CF_DEBUG_DECODE_MIN_CHUNK_PAGES shortest decode chunk, in pages
- *   CF_DEBUG_SPATIAL_WAIT           1: in the spatial sequence decode waits, through a stream memory operation,
- *                                   until the first prefill grid's CTAs hold their SMs */
+ *   CF_DEBUG_SPATIAL_NO_WAIT        1: in the spatial sequence decode does not wait (through a stream memory
+ *                                   operation) until the first prefill grid's CTAs hold their SMs, but relies on
+ *                                   the order of the launches */
 typedef enum {
     CF_DEBUG_PREFILL_SPLIT = 0,
     CF_DEBUG_SEPARATE_COMBINE = 1,
     CF_DEBUG_DECODE_WAVES = 2,
     CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3,
-    CF_DEBUG_SPATIAL_WAIT = 4
+    CF_DEBUG_SPATIAL_NO_WAIT = 4
 } cf_debug_option;
 cf_status cf_set_debug_option(cf_ctx* ctx, cf_debug_option option, int value);
 
@@ -222,6 +241,10 @@ cf_status cf_get_timing_sums(cf_ctx* ctx, float* ms_decode, float* ms_combine, f
  * tensor-map lookup and the launches themselves (the GPU work is asynchronous). */
 cf_status cf_get_host_time_sums(cf_ctx* ctx, double* us_append, double* us_attention, double* us_planner,
                                 int32_t* num_steps);
+/* Item counts of the plan the last cf_mixed_attention(_shared) built, for tests and reports: counts[8] =
+ * {decode items, split decode sequences, prefill CTAs, decode partial slots, KV-split prefill items,
+ *  shared-prefix items, members of shared-prefix sets, 0}. */
+cf_status cf_get_last_plan_counts(cf_ctx* ctx, int32_t* counts);
 /* Number of kernels the last cf_mixed_attention launched. */
 cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
 

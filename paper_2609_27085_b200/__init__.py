@@ -37,12 +37,12 @@ CF_DEBUG_PREFILL_SPLIT = 0
 CF_DEBUG_SEPARATE_COMBINE = 1
 CF_DEBUG_DECODE_WAVES = 2
 CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3
-CF_DEBUG_SPATIAL_WAIT = 4
+CF_DEBUG_SPATIAL_NO_WAIT = 4
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option", "cf_get_host_time_sums",
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option", "cf_get_host_time_sums", "cf_mixed_attention_shared", "cf_get_last_plan_counts",
            "cf_status_string")
 
 
@@ -84,6 +84,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_destroy.argtypes = [vp]
     lib.cf_kv_append.argtypes = [vp, dp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp]
     lib.cf_mixed_attention.argtypes = [vp, dp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp, vp]
+    lib.cf_mixed_attention_shared.argtypes = [vp, dp, vp, vp, vp, vp, i32, vp, vp, vp, vp, i32, vp, vp, vp]
+    lib.cf_get_last_plan_counts.argtypes = [vp, vp]
     lib.cf_mixed_step_host.argtypes = [vp, dp, vp, vp, vp, vp, vp, vp, i32, vp, vp, i32, vp, vp]
     lib.cf_host_steps_flush.argtypes = [vp, vp]
     lib.cf_get_async_status.argtypes = [vp]
@@ -185,6 +187,29 @@ def cf_mixed_attention(ctx, desc: CacheDesc, q, k_cache, v_cache, block_table, m
     if check:
         _check(st, "cf_mixed_attention")
     return st
+
+
+def cf_mixed_attention_shared(ctx, desc: CacheDesc, q, k_cache, v_cache, block_table, max_blocks_per_seq: int,
+                              context_len, query_len, share_group, shared_len, out, lse=None, stream=None,
+                              check: bool = True) -> int:
+    """cf_mixed_attention with shared prefixes described: share_group[s] >= 0 names the group whose members have
+    the same pages for their first shared_len[s] tokens (host int32 arrays)."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    sg, sl = _host_i32(share_group), _host_i32(shared_len)
+    st = load_library().cf_mixed_attention_shared(ctx, ctypes.byref(desc), _dev(q), _dev(k_cache), _dev(v_cache),
+                                                  _dev(block_table), int(max_blocks_per_seq), lc.ctypes.data, lq.ctypes.data,
+                                                  sg.ctypes.data, sl.ctypes.data, int(lc.shape[0]), _dev(out), _dev(lse),
+                                                  _stream(stream))
+    if check:
+        _check(st, "cf_mixed_attention_shared")
+    return st
+
+
+def cf_get_last_plan_counts(ctx) -> np.ndarray:
+    """Item counts of the last plan built by cf_mixed_attention(_shared): see the header."""
+    counts = np.zeros(8, dtype=np.int32)
+    _check(load_library().cf_get_last_plan_counts(ctx, counts.ctypes.data), "cf_get_last_plan_counts")
+    return counts
 
 
 def cf_mixed_step_host(ctx, desc: CacheDesc, q_host, k_new_host, v_new_host, k_cache, v_cache, block_table,

@@ -86,7 +86,7 @@ struct cf_ctx {
     cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
     cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
     bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
-    bool spatial_wait = false; // CF_DEBUG_SPATIAL_WAIT: decode waits (stream memory operation) for the front prefill CTAs to be resident
+    bool spatial_wait = true;  // decode waits (stream memory operation) for the front prefill CTAs to be resident; CF_DEBUG_SPATIAL_NO_WAIT: launch order only
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths)
     int spatial_sms_default = 0;   // CF_SPATIAL_SMS at cf_create: what cf_set_overlap(ctx, 1) goes back to
     cudaStream_t side = nullptr;
@@ -107,6 +107,7 @@ struct cf_ctx {
     cf::PoolMapEntry pool_maps[cf::kPoolMaps];
     cf::QMapEntry q_maps[cf::kQMaps];
     uint64_t map_stamp = 0;
+    int32_t last_counts[8] = {0, 0, 0, 0, 0, 0, 0, 0};   // item counts of the plan the last cf_mixed_attention built
 };
 
 // A plan that lives on the device for as long as the caller wants: built once per scheduler iteration
@@ -119,7 +120,7 @@ struct cf_plan {
     uint8_t* dev = nullptr;
     float* part = nullptr;         // this plan's own split-K partials
     int n_part_slots = 0, n_pre_slots = 0;
-    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
+    size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_sh = 0, off_shm = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     float pre_over_dec = 0.f;
 };
@@ -190,7 +191,7 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_pre_tc, off_pre_comb, off_queue, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_sh, off_shm, off_pre_tc, off_pre_comb, off_queue, total;
 };
 
 static PlanLayout layout_of(int32_t S, const Plan& pl)
@@ -202,6 +203,8 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_qlen = at;   at = align_up(at + sizeof(int32_t) * (size_t)S, 16);
     L.off_dec = at;    at = align_up(at + sizeof(DecodeItem) * pl.decode.size(), 16);
     L.off_comb = at;   at = align_up(at + sizeof(CombineItem) * pl.combine.size(), 16);
+    L.off_sh = at;     at = align_up(at + sizeof(SharedDecodeItem) * pl.shared_decode.size(), 16);
+    L.off_shm = at;    at = align_up(at + sizeof(ShareMember) * pl.share_members.size(), 16);
     L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
     L.off_pre_comb = at; at = align_up(at + sizeof(PrefillCombineItem) * pl.prefill_combine.size(), 16);
     L.off_queue = at;  at += 16;   // ticket counter + exit counter of the persistent prefill CTAs; uploaded as zeros
@@ -226,6 +229,10 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
     }
     if (!pl.decode.empty()) std::memcpy(s.host + L->off_dec, pl.decode.data(), sizeof(DecodeItem) * pl.decode.size());
     if (!pl.combine.empty()) std::memcpy(s.host + L->off_comb, pl.combine.data(), sizeof(CombineItem) * pl.combine.size());
+    if (!pl.shared_decode.empty())
+        std::memcpy(s.host + L->off_sh, pl.shared_decode.data(), sizeof(SharedDecodeItem) * pl.shared_decode.size());
+    if (!pl.share_members.empty())
+        std::memcpy(s.host + L->off_shm, pl.share_members.data(), sizeof(ShareMember) * pl.share_members.size());
     if (!pl.prefill_tc.empty())
         std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
     if (!pl.prefill_combine.empty())
@@ -334,7 +341,7 @@ static float scale_log2_of(const cf_cache_desc* d)
 namespace cf {
 
 struct PlanCounts {
-    int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    int n_dec = 0, n_comb = 0, n_shared = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
     int n_part_slots = 0;
 };
@@ -382,6 +389,8 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.query_len = (const int32_t*)(base + L.off_qlen);
     p.dec_items = (const DecodeItem*)(base + L.off_dec);
     p.comb_items = (const CombineItem*)(base + L.off_comb);
+    p.sh_items = (const SharedDecodeItem*)(base + L.off_sh);
+    p.sh_members = (const ShareMember*)(base + L.off_shm);
     p.pre_tc_items = (const PrefillTcItem*)(base + L.off_pre_tc);
     p.part_o = (float*)((uint8_t*)ws + W.dec_o);
     p.part_ml = (float*)((uint8_t*)ws + W.dec_ml);
@@ -436,12 +445,12 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tail > sms) tail = sms;
         second_grid = tail > 0;
         // Decode must not start before the front CTAs hold their SMs (its grid would otherwise fill the
-        // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end).  The
-        // front grid is therefore enqueued first and on the stream that needs no cross-stream event, which in
-        // every measurement so far is enough.  CF_SPATIAL_WAIT=1 adds a guarantee: the front CTAs count
-        // themselves in and the side stream waits for that count with a stream memory operation before decode
-        // (3-9 us per step; never while the stream is being captured: in a graph the two branches start
-        // together and the memory-operation nodes cost more than they return).
+        // machine first and the prefill CTAs, which need an SM to themselves, would wait for its end: the call
+        // then takes longer than the serial sequence).  Enqueueing the front grid first, on the stream that needs
+        // no cross-stream event, wins that race only some of the time, so the order is enforced: the front CTAs
+        // count themselves in and the side stream waits for that count with a stream memory operation before
+        // decode (a few microseconds per call; not while the stream is being captured: in a graph the two branches
+        // start together, front grid first, and memory-operation nodes cost more than they return).
         uint32_t* resident = nullptr;
         const StreamMemOps& mo = stream_mem_ops();
         cudaStreamCaptureStatus cap = cudaStreamCaptureStatusNone;
@@ -456,6 +465,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess && resident &&
             mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
+        if (e == cudaSuccess) e = launch_decode_shared(p, D, n.n_shared, c->side);
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, c->side);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
         if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
@@ -464,6 +474,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
     } else {
         if (tc) cudaEventRecord(tc->ev[0], stream);
+        if (e == cudaSuccess) e = launch_decode_shared(p, D, n.n_shared, stream);
         if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
@@ -472,7 +483,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_shared > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 
@@ -640,14 +651,26 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
                              const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
                              void* out, float* lse, void* cuda_stream)
 {
+    return cf_mixed_attention_shared(c, desc, q, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
+                                     nullptr, nullptr, num_seqs, out, lse, cuda_stream);
+}
+
+cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const void* q,
+                                    const void* k_cache, const void* v_cache,
+                                    const int32_t* block_table, int32_t max_blocks_per_seq,
+                                    const int32_t* context_len, const int32_t* query_len,
+                                    const int32_t* share_group, const int32_t* shared_len, int32_t num_seqs,
+                                    void* out, float* lse, void* cuda_stream)
+{
     if (!c || !desc) return CF_ERR_INVALID_ARG;
+    if ((share_group == nullptr) != (shared_len == nullptr)) return CF_ERR_INVALID_ARG;
     const int64_t t_in = now_ns();
     cf_status st = validate_desc(desc);
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
-    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
+    st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl, share_group, shared_len);
     if (st != CF_OK) return st;
     c->host_ns_planner += now_ns() - t_in;
     c->launches = 0;
@@ -669,9 +692,12 @@ cf_status cf_mixed_attention(cf_ctx* c, const cf_cache_desc* desc, const void* q
     if (st != CF_OK) return st;
 
     PlanCounts n;
-    n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size();
+    n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_shared = (int)pl.shared_decode.size();
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
     n.n_part_slots = pl.n_part_slots;
+    c->last_counts[0] = n.n_dec; c->last_counts[1] = n.n_comb; c->last_counts[2] = n.n_pre_tc; c->last_counts[3] = n.n_part_slots;
+    c->last_counts[4] = n.n_pre_comb; c->last_counts[5] = n.n_shared; c->last_counts[6] = (int32_t)pl.share_members.size();
+    c->last_counts[7] = 0;
     n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
@@ -703,7 +729,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->max_blocks = max_blocks_per_seq;
     const PlanLayout L = layout_of(num_seqs, pl);
     P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
-    P->off_comb = L.off_comb; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
+    P->off_comb = L.off_comb; P->off_sh = L.off_sh; P->off_shm = L.off_shm; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
     P->total = L.total;
     P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size();
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
@@ -789,7 +815,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     if (!guard.ok) return CF_ERR_CUDA;
     PlanLayout L;
     L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
-    L.off_comb = P->off_comb; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
+    L.off_comb = P->off_comb; L.off_sh = P->off_sh; L.off_shm = P->off_shm; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
     L.total = P->total;
     PlanCounts n;
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
@@ -961,7 +987,7 @@ cf_status cf_set_debug_option(cf_ctx* c, cf_debug_option option, int value)
         case CF_DEBUG_DECODE_MIN_CHUNK_PAGES:
             c->cfg.decode_min_chunk_pages = value > 0 ? value : defaults.decode_min_chunk_pages;
             return CF_OK;
-        case CF_DEBUG_SPATIAL_WAIT: c->spatial_wait = value > 0; return CF_OK;
+        case CF_DEBUG_SPATIAL_NO_WAIT: c->spatial_wait = value <= 0; return CF_OK;
     }
     return CF_ERR_INVALID_ARG;
 }
@@ -1015,6 +1041,13 @@ cf_status cf_get_host_time_sums(cf_ctx* c, double* us_append, double* us_attenti
     if (num_steps) *num_steps = c->host_calls_attention;
     c->host_ns_append = c->host_ns_attention = c->host_ns_planner = 0;
     c->host_calls_append = c->host_calls_attention = 0;
+    return CF_OK;
+}
+
+cf_status cf_get_last_plan_counts(cf_ctx* c, int32_t* counts)
+{
+    if (!c || !counts) return CF_ERR_INVALID_ARG;
+    for (int i = 0; i < 8; ++i) counts[i] = c->last_counts[i];
     return CF_OK;
 }
 

@@ -305,6 +305,223 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
 }
 
 // ---------------------------------------------------------------------------------------------
+// Shared-prefix decode: one CTA serves one (share group, shared KV chunk, KV head) for a SET of member sequences.
+// The chunk lies inside the prefix that all members have in common (same physical pages), so its K/V is streamed
+// once and the members' query heads ride along as MMA columns: NCG column groups of 8, column c of the set =
+// head c % G of member c / G.  Loop structure, ring and fragment layouts are those of decode_splitk_kernel; there
+// is no masking at all (whole pages, every token visible to every member).  Every (member, head) gets an fp32
+// partial in the member's slot for this chunk; the member's own chunks and the merge follow in the next kernel.
+// Pages are fetched with the default L2 policy: other member sets of the group read them again.
+template <int D, int NWARPS, int NSTAGE, int NCG>
+__global__ void __launch_bounds__(NWARPS * 32, 2) decode_shared_kernel(const AttnParams p)
+{
+    constexpr int CPR = D / 8;
+    constexpr int PAGE_BYTES = 16 * D * 2;
+    constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+    constexpr int WARP_BYTES = NSTAGE * STAGE_BYTES;
+    constexpr int KSTEPS = D / 16;
+    constexpr int DP = D + 4;
+    constexpr int NCOL = NCG * 8;
+    extern __shared__ __align__(1024) uint8_t smem[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const SharedDecodeItem it = p.sh_items[item_id];
+    const ShareMember* members = p.sh_members + it.member_first;
+    const int G = p.G;
+
+    // ---- Q^T fragments of every column group (B operands)
+    uint32_t qf[NCG][KSTEPS][2];
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) {
+        const int col = cg * 8 + (lane >> 2);
+        const int m = col / G, head = col % G;
+        const bool live = m < it.n_members;
+        const int q_row = live ? __ldg(&members[m].q_row) : 0;
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)q_row * p.Hq + (int64_t)kvh * G + head) * D);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            qf[cg][ks][0] = live ? __ldg(qrow + ks * 8 + (lane & 3)) : 0u;
+            qf[cg][ks][1] = live ? __ldg(qrow + ks * 8 + 4 + (lane & 3)) : 0u;
+        }
+    }
+
+    const int first_page = it.kv_begin >> 4;
+    const int n_pages = (it.kv_end - it.kv_begin) >> 4;
+    const int my_n = n_pages > warp ? (n_pages - warp + NWARPS - 1) / NWARPS : 0;
+    const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks + first_page + warp;
+    const uint32_t wbase = smem_u32(smem) + warp * WARP_BYTES;
+    const __nv_bfloat16* kbase = p.k_cache + (int64_t)kvh * p.ks_head;
+    const __nv_bfloat16* vbase = p.v_cache + (int64_t)kvh * p.vs_head;
+
+    auto checked = [&](int32_t id) -> int32_t {
+        if ((uint32_t)id < (uint32_t)p.num_blocks) return id;
+        if (p.err) atomicOr(p.err, kErrBlockId);
+        return 0;
+    };
+    int cache_base = 0;
+    int32_t pid_cache = (lane < my_n) ? checked(__ldg(bt + lane * NWARPS)) : 0;
+
+    auto issue = [&](int i) {
+        if (i - cache_base == 32) {
+            cache_base = i;
+            pid_cache = (i + lane < my_n) ? checked(__ldg(bt + (i + lane) * NWARPS)) : 0;
+        }
+        const int32_t pid = __shfl_sync(0xffffffffu, pid_cache, i - cache_base);
+        const uint32_t sbase = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const __nv_bfloat16* kp = kbase + (int64_t)pid * p.ks_block;
+        const __nv_bfloat16* vp = vbase + (int64_t)pid * p.vs_block;
+#pragma unroll
+        for (int r = 0; r < (16 * CPR) / 32; ++r) {
+            const int id = r * 32 + lane;
+            const int t = id / CPR, c = id % CPR;
+            cp_async16(sbase + tile_off<16>(t, c), kp + t * p.ks_token + c * 8, 16);
+            cp_async16(sbase + PAGE_BYTES + tile_off<16>(t, c), vp + t * p.vs_token + c * 8, 16);
+        }
+    };
+
+    float o[NCG][KSTEPS][4];
+    float m_run[NCG][2], l_run[NCG][2];
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) {
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt) o[cg][mt][0] = o[cg][mt][1] = o[cg][mt][2] = o[cg][mt][3] = 0.f;
+        m_run[cg][0] = m_run[cg][1] = -INFINITY;
+        l_run[cg][0] = l_run[cg][1] = 0.f;
+    }
+
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (s < my_n) issue(s);
+        cp_async_commit();
+    }
+
+    for (int i = 0; i < my_n; ++i) {
+        cp_async_wait<NSTAGE - 2>();
+        __syncwarp();
+        if (i + NSTAGE - 1 < my_n) issue(i + NSTAGE - 1);
+        cp_async_commit();
+
+        const uint32_t sK = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const uint32_t sV = sK + PAGE_BYTES;
+
+        // S^T = K Q^T: one K fragment feeds every column group
+        float sacc[NCG][4];
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) sacc[cg][0] = sacc[cg][1] = sacc[cg][2] = sacc[cg][3] = 0.f;
+        {
+            const int t = (lane & 7) + ((lane >> 3) & 1) * 8;
+#pragma unroll
+            for (int ks = 0; ks < KSTEPS; ++ks) {
+                uint32_t a[4];
+                ldmatrix_x4(a, sK + tile_off<16>(t, 2 * ks + (lane >> 4)));
+#pragma unroll
+                for (int cg = 0; cg < NCG; ++cg) mma_bf16_16816(sacc[cg], a, qf[cg][ks][0], qf[cg][ks][1]);
+            }
+        }
+        uint32_t pb[NCG][2];
+#pragma unroll
+        for (int cg = 0; cg < NCG; ++cg) {
+            float s[4];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) s[e] = sacc[cg][e] * p.scale_log2;
+            float alpha[2];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                float mx = fmaxf(s[j], s[2 + j]);
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+                mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+                const float mnew = fmaxf(m_run[cg][j], mx);
+                alpha[j] = fast_exp2(m_run[cg][j] - mnew);
+                m_run[cg][j] = mnew;
+                s[j] = fast_exp2(s[j] - mnew);
+                s[2 + j] = fast_exp2(s[2 + j] - mnew);
+                l_run[cg][j] = l_run[cg][j] * alpha[j] + s[j] + s[2 + j];
+            }
+#pragma unroll
+            for (int mt = 0; mt < KSTEPS; ++mt) {
+                o[cg][mt][0] *= alpha[0]; o[cg][mt][1] *= alpha[1];
+                o[cg][mt][2] *= alpha[0]; o[cg][mt][3] *= alpha[1];
+            }
+            pb[cg][0] = movmatrix_trans(pack_bf16(s[0], s[1]));
+            pb[cg][1] = movmatrix_trans(pack_bf16(s[2], s[3]));
+        }
+        {
+            const int t = (lane & 7) + (lane >> 4) * 8;
+#pragma unroll
+            for (int mt = 0; mt < KSTEPS; ++mt) {
+                uint32_t a[4];
+                ldmatrix_x4_trans(a, sV + tile_off<16>(t, 2 * mt + ((lane >> 3) & 1)));
+#pragma unroll
+                for (int cg = 0; cg < NCG; ++cg) mma_bf16_16816(o[cg][mt], a, pb[cg][0], pb[cg][1]);
+            }
+        }
+    }
+    cp_async_wait<0>();
+
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg)
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            l_run[cg][j] += __shfl_xor_sync(0xffffffffu, l_run[cg][j], 4);
+            l_run[cg][j] += __shfl_xor_sync(0xffffffffu, l_run[cg][j], 8);
+            l_run[cg][j] += __shfl_xor_sync(0xffffffffu, l_run[cg][j], 16);
+        }
+    __syncthreads();                                  // every warp is done with its ring
+    float* mo = reinterpret_cast<float*>(smem);       // [NWARPS][NCOL][DP]
+    float* mm = mo + NWARPS * NCOL * DP;              // [NWARPS][NCOL]
+    float* ml = mm + NWARPS * NCOL;                   // [NWARPS][NCOL]
+#pragma unroll
+    for (int cg = 0; cg < NCG; ++cg) {
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt)
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const int d = mt * 16 + (lane >> 2) + (e >> 1) * 8;
+                const int col = cg * 8 + 2 * (lane & 3) + (e & 1);
+                mo[(warp * NCOL + col) * DP + d] = o[cg][mt][e];
+            }
+        if (lane < 4) {
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+                mm[warp * NCOL + cg * 8 + 2 * lane + j] = m_run[cg][j];
+                ml[warp * NCOL + cg * 8 + 2 * lane + j] = l_run[cg][j];
+            }
+        }
+    }
+    __syncthreads();
+
+    const int n_cols = it.n_members * G;
+    for (int idx = threadIdx.x; idx < n_cols * (D / 2); idx += NWARPS * 32) {
+        const int col = idx / (D / 2), d = (idx % (D / 2)) * 2;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) M = fmaxf(M, mm[w * NCOL + col]);
+        float L = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) {
+            const float f = fast_exp2(mm[w * NCOL + col] - M);   // idle warps: 2^(-inf) = 0
+            L += ml[w * NCOL + col] * f;
+            o0 += mo[(w * NCOL + col) * DP + d] * f;
+            o1 += mo[(w * NCOL + col) * DP + d + 1] * f;
+        }
+        const int m = col / G, hq = kvh * G + col % G;
+        const int64_t pr = (int64_t)(__ldg(&members[m].part_first) + it.chunk) * p.Hq + hq;
+        *reinterpret_cast<float2*>(p.part_o + pr * D + d) = make_float2(o0, o1);
+        if (d == 0) *reinterpret_cast<float2*>(p.part_ml + pr * 2) = make_float2(M, L);
+    }
+    // Fused merge: this chunk counts as done for every member (the member's own chunks, which run in the next
+    // kernel, draw the remaining tickets, so the last ticket is never drawn here).
+    if (p.dec_counters != nullptr) {
+        __threadfence();
+        __syncthreads();
+        if ((int)threadIdx.x < it.n_members)
+            atomicAdd(p.dec_counters + (int64_t)__ldg(&members[threadIdx.x].part_first) * p.Hkv + kvh, 1u);
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
 // Combine: merges the partials of a split sequence in fixed chunk order (deterministic).
 //   M = max_c m_c ; O = sum_c 2^(m_c - M) o_c / sum_c 2^(m_c - M) l_c ; lse = (M + log2 sum) ln 2
 // (evaluated as a running merge over groups of eight chunks)
@@ -352,6 +569,32 @@ cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaSt
 {
     if (n_items <= 0) return cudaSuccess;
     return head_dim == 128 ? launch_decode_t<128>(p, n_items, stream) : launch_decode_t<64>(p, n_items, stream);
+}
+
+template <int D>
+static cudaError_t launch_decode_shared_t(const AttnParams& p, int n_items, cudaStream_t stream)
+{
+    constexpr int NCG = kSharedColumns / 8;
+    auto kern = decode_shared_kernel<D, kDecWarps, kDecStages, NCG>;
+    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * D * 2;
+    const size_t merge = (size_t)kDecWarps * kSharedColumns * (D + 4) * 4 + (size_t)kDecWarps * kSharedColumns * 4 * 2;
+    const size_t smem = ring > merge ? ring : merge;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev].load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev].store(true, std::memory_order_release);
+    }
+    kern<<<n_items * p.Hkv, kDecWarps * 32, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
+cudaError_t launch_decode_shared(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    return head_dim == 128 ? launch_decode_shared_t<128>(p, n_items, stream) : launch_decode_shared_t<64>(p, n_items, stream);
 }
 
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)

@@ -28,6 +28,8 @@ struct AttnParams {
     const int32_t* q_start;
     const DecodeItem* dec_items;
     const CombineItem* comb_items;
+    const SharedDecodeItem* sh_items; // shared-prefix chunks and their member sets (null when the batch has none)
+    const ShareMember* sh_members;
     const PrefillTcItem* pre_tc_items;
     float* part_o;                    // [slot, Hq, D] fp32 un-normalised partial outputs
     float* part_ml;                   // [slot, Hq, 2] running max (log2 domain) and sum

@@ -5,6 +5,7 @@
 #include <cmath>
 #include <functional>
 #include <queue>
+#include <utility>
 #include <cstdint>
 
 namespace cf {
@@ -67,7 +68,8 @@ cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, c
 }
 
 cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
-                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan)
+                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan,
+                     const int32_t* share_group, const int32_t* shared_len)
 {
     *plan = Plan();
     cf_status st = validate_lengths(d, context_len, query_len, num_seqs, max_blocks_per_seq, plan);
@@ -84,23 +86,84 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     // from the one that holds the window's left edge onwards, and nothing left of it is ever touched.
     const int32_t W = d->window_size;
     auto first_page_of = [&](int32_t lc) -> int64_t { return (W > 0 && lc > W) ? (lc - W) / B : 0; };
+
+    // Shared prefixes: decode sequences of a group (at least two, full attention) whose common prefix is at least
+    // kMinSharedPages pages long leave those pages to shared items; their own chunks start behind them.
+    // shared_pages[s] = pages of sequence s that a shared item covers (0: none).
+    const int32_t G = d->num_q_heads / d->num_kv_heads;
+    std::vector<int32_t> shared_pages;
+    struct GroupInfo { int32_t group; int32_t pages; std::vector<int32_t> members; };
+    std::vector<GroupInfo> groups_sh;
+    int64_t extra_pages = 0;
+    if (share_group != nullptr && shared_len != nullptr && W == 0) {
+        std::vector<std::pair<int32_t, int32_t>> keyed;          // (group, sequence) of the decode sequences that share
+        for (int32_t s = 0; s < num_seqs; ++s)
+            if (query_len[s] == 1 && share_group[s] >= 0 && shared_len[s] > 0) keyed.emplace_back(share_group[s], s);
+        std::sort(keyed.begin(), keyed.end());
+        for (size_t i = 0; i < keyed.size();) {
+            size_t j = i;
+            int32_t pages = INT32_MAX;
+            while (j < keyed.size() && keyed[j].first == keyed[i].first) {
+                const int32_t s = keyed[j].second;
+                // a sequence's new token is never part of the shared prefix
+                pages = std::min(pages, std::min(shared_len[s], context_len[s] - 1) / B);
+                ++j;
+            }
+            if (j - i >= 2 && pages >= kMinSharedPages) {
+                GroupInfo gi;
+                gi.group = keyed[i].first;
+                gi.pages = pages;
+                for (size_t m = i; m < j; ++m) gi.members.push_back(keyed[m].second);
+                const int64_t sets = ((int64_t)gi.members.size() * G + kSharedColumns - 1) / kSharedColumns;
+                extra_pages += sets * pages;
+                groups_sh.push_back(std::move(gi));
+            }
+            i = j;
+        }
+        if (!groups_sh.empty()) {
+            shared_pages.assign((size_t)num_seqs, 0);
+            for (const GroupInfo& gi : groups_sh)
+                for (int32_t s : gi.members) shared_pages[(size_t)s] = gi.pages;
+        }
+    }
+    auto own_first_page = [&](int32_t s) -> int64_t {
+        return shared_pages.empty() ? first_page_of(context_len[s]) : (int64_t)shared_pages[(size_t)s];
+    };
     const int64_t target = decode_target_pages(
         num_seqs,
-        [&](int32_t s) -> int64_t { return query_len[s] == 1 ? (int64_t)context_len[s] - first_page_of(context_len[s]) * B : -1; },
-        B, d->num_kv_heads, d->head_dim, cfg, shares_sms);
+        [&](int32_t s) -> int64_t { return query_len[s] == 1 ? (int64_t)context_len[s] - own_first_page(s) * B : -1; },
+        B, d->num_kv_heads, d->head_dim, cfg, shares_sms, extra_pages);
 
+    // chunks of the shared part of every group, the same for all of its members
+    std::vector<int32_t> n_shared_chunks;      // per sequence
+    std::vector<int64_t> shared_per;           // per group: pages per shared chunk
+    if (!groups_sh.empty()) {
+        n_shared_chunks.assign((size_t)num_seqs, 0);
+        for (const GroupInfo& gi : groups_sh) {
+            int64_t n = 1, per = gi.pages;
+            decode_split(gi.pages, target, quantum, &n, &per);
+            shared_per.push_back(per);
+            for (int32_t s : gi.members) n_shared_chunks[(size_t)s] = (int32_t)n;
+        }
+    }
+
+    std::vector<int32_t> part_first_of;        // per sequence: its first partial slot (-1: writes out directly)
+    if (!groups_sh.empty()) part_first_of.assign((size_t)num_seqs, -1);
     for (int32_t s = 0; s < num_seqs; ++s) {
         if (query_len[s] != 1) continue;
         const int32_t lc = context_len[s];
-        const int64_t page0 = first_page_of(lc);
+        const int64_t page0 = own_first_page(s);
         const int64_t pages = (lc + B - 1) / B - page0;
+        const int32_t n_sh = n_shared_chunks.empty() ? 0 : n_shared_chunks[(size_t)s];
         int64_t n = 1, per = pages;
         decode_split(pages, target, quantum, &n, &per);
+        const int32_t n_all = (int32_t)n + n_sh;
         int32_t first = -1;
-        if (n > 1) {
+        if (n_all > 1) {
             first = plan->n_part_slots;
-            plan->combine.push_back(CombineItem{plan->q_start[s], first, (int32_t)n});
-            plan->n_part_slots += (int32_t)n;
+            plan->combine.push_back(CombineItem{plan->q_start[s], first, n_all});
+            plan->n_part_slots += n_all;
+            if (!part_first_of.empty()) part_first_of[(size_t)s] = first;
         }
         for (int64_t c = 0; c < n; ++c) {
             DecodeItem it;
@@ -108,11 +171,37 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             it.q_row = plan->q_start[s];
             it.kv_begin = (int32_t)((page0 + c * per) * B);
             it.kv_end = (int32_t)std::min<int64_t>((page0 + (c + 1) * per) * B, lc);
-            it.part_slot = n > 1 ? first + (int32_t)c : -1;
-            it.chunk = (int32_t)c;
-            it.n_chunks = (int32_t)n;
+            it.part_slot = n_all > 1 ? first + n_sh + (int32_t)c : -1;
+            it.chunk = n_sh + (int32_t)c;
+            it.n_chunks = n_all;
             it.kv_lo = (W > 0 && lc > W) ? lc - W : 0;
             plan->decode.push_back(it);
+        }
+    }
+    // shared items: per group, member sets of kSharedColumns / G sequences, one item per (set, shared chunk)
+    for (size_t gi_idx = 0; gi_idx < groups_sh.size(); ++gi_idx) {
+        const GroupInfo& gi = groups_sh[gi_idx];
+        const int64_t per = shared_per[gi_idx];
+        const int32_t n_sh = n_shared_chunks[(size_t)gi.members[0]];
+        const int32_t per_set = std::max(1, kSharedColumns / G);
+        for (size_t m0 = 0; m0 < gi.members.size(); m0 += (size_t)per_set) {
+            const int32_t n_mem = (int32_t)std::min<size_t>((size_t)per_set, gi.members.size() - m0);
+            const int32_t member_first = (int32_t)plan->share_members.size();
+            for (int32_t m = 0; m < n_mem; ++m) {
+                const int32_t s = gi.members[m0 + (size_t)m];
+                plan->share_members.push_back(ShareMember{plan->q_start[s], part_first_of[(size_t)s]});
+            }
+            for (int32_t c = 0; c < n_sh; ++c) {
+                SharedDecodeItem it;
+                it.seq = gi.members[m0];
+                it.kv_begin = (int32_t)(c * per * B);
+                it.kv_end = (int32_t)std::min<int64_t>((c + 1) * per, gi.pages) * B;
+                it.chunk = c;
+                it.member_first = member_first;
+                it.n_members = n_mem;
+                it.pad[0] = it.pad[1] = 0;
+                plan->shared_decode.push_back(it);
+            }
         }
     }
     std::stable_sort(plan->decode.begin(), plan->decode.end(), [](const DecodeItem& a, const DecodeItem& b) {
@@ -124,7 +213,6 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // pairs of 128-row tiles that share a KV head: two heads of a group over the same rows, or
         // (group size 1) two consecutive row tiles of one head
         constexpr int32_t TR = 128;
-        const int32_t G = d->num_q_heads / d->num_kv_heads;
         struct KeyedTc { int64_t extent; int32_t tiles; PrefillTcItem it; };   // extent: end of the visible keys; tiles: KV tiles to visit
         std::vector<KeyedTc> items;
         auto prefix_of = [&](int32_t s) { return context_len[s] - query_len[s]; };

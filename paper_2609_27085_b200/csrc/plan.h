@@ -23,6 +23,27 @@ struct DecodeItem {        // one (decode sequence, KV chunk); the kernel adds t
                            // tokens of this chunk below it are masked (only the first chunk can hold any)
 };
 
+// Shared prefix (radix-cache reuse, Section 4.4: a lookup tells how much of a prompt is already resident; agent
+// turns share long prefixes): decode sequences of one share group point at the same physical pages for the first
+// `shared_len` tokens.  Those pages are streamed once per KV chunk for a whole set of members, whose query heads
+// ride along as extra MMA columns; every member gets a partial per shared chunk, merged with the partials of
+// its own suffix by the usual split-K merge.
+struct SharedDecodeItem {  // one (share group, shared KV chunk, member set); the kernel adds the KV-head index
+    int32_t seq;           // the member whose block-table row is read for the shared pages
+    int32_t kv_begin;      // whole pages of the shared prefix: [kv_begin, kv_end)
+    int32_t kv_end;
+    int32_t chunk;         // index of this chunk in every member's chunk list (shared chunks come first)
+    int32_t member_first;  // first entry of this set in the member list
+    int32_t n_members;     // members in the set (<= kSharedColumns / G)
+    int32_t pad[2];
+};
+struct ShareMember {       // one member of a set
+    int32_t q_row;         // packed row of its query token
+    int32_t part_first;    // first partial slot of the sequence (its chunk c writes slot part_first + c)
+};
+constexpr int32_t kSharedColumns = 16;      // query-head columns a shared-prefix CTA carries (two 8-wide MMA operands)
+constexpr int32_t kMinSharedPages = 16;     // shorter shared prefixes are not worth a separate pass
+
 struct CombineItem {       // one decode sequence that was split
     int32_t q_row;
     int32_t part_first;    // its chunks occupy slots [part_first, part_first + n_chunks)
@@ -72,6 +93,8 @@ struct Plan {
     std::vector<int32_t> q_start;     // [S+1] exclusive prefix sum of query_len
     std::vector<DecodeItem> decode;   // longest chunk first
     std::vector<CombineItem> combine;
+    std::vector<SharedDecodeItem> shared_decode;   // shared-prefix chunks (empty unless the caller described sharing)
+    std::vector<ShareMember> share_members;
     std::vector<PrefillTcItem> prefill_tc;   // longest KV extent first (tcgen05 kernel); KV-split items appear part_k times
     std::vector<PrefillCombineItem> prefill_combine;   // one per KV-split item
     int32_t n_pre_slots = 0;          // fp32 partial rows of KV-split prefill items (compact, D floats each)
@@ -94,7 +117,7 @@ cf_status validate_lengths(const cf_cache_desc* d, const int32_t* context_len, c
 //   decode_split: near-equal chunks of at most `target` pages, each a multiple of the page quantum.
 template <class LcOf>
 inline int64_t decode_target_pages(int32_t num_seqs, LcOf lc_of, int32_t B, int32_t Hkv, int32_t D, const PlanConfig& cfg,
-                                   bool shares_sms)
+                                   bool shares_sms, int64_t extra_pages = 0)
 {
     const int64_t wave = (int64_t)(cfg.num_sms > 1 ? cfg.num_sms : 1) * (cfg.decode_ctas_per_sm > 1 ? cfg.decode_ctas_per_sm : 1);
     const int64_t slots = wave * (cfg.decode_waves > 1 ? cfg.decode_waves : 1);
@@ -105,8 +128,9 @@ inline int64_t decode_target_pages(int32_t num_seqs, LcOf lc_of, int32_t B, int3
         const int64_t lc = lc_of(s);
         if (lc >= 0) total_pages += (lc + B - 1) / B;
     }
+    total_pages += extra_pages;                         // pages streamed by shared-prefix items
     int64_t target = (total_pages * Hkv + slots - 1) / slots;
-    if (target < min_pages && total_pages > 0 && !shares_sms) {
+    if (target < min_pages && total_pages > 0 && !shares_sms && extra_pages == 0) {
         // A small batch: chunks of the minimum length would not fill `decode_waves` waves, and how many waves
         // of (num_sms x ctas_per_sm) CTAs they do fall into decides the time (a last wave that is a quarter
         // full costs a whole CTA time).  Try chunk lengths from the minimum to four times it and keep the
@@ -152,8 +176,11 @@ inline void decode_split(int64_t pages, int64_t target, int32_t quantum, int64_t
 }
 
 // Full plan (calls validate_lengths).
+// share_group / shared_len (both or neither; HOST [num_seqs]): share_group[s] >= 0 names the group of sequence s,
+// whose members have identical block-table entries for the first shared_len[s] tokens; < 0: shares nothing.
 cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len,
-                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan);
+                     int32_t num_seqs, int32_t max_blocks_per_seq, const PlanConfig& cfg, Plan* plan,
+                     const int32_t* share_group = nullptr, const int32_t* shared_len = nullptr);
 
 // Predicted device time of one cf_mixed_attention call, in microseconds, from a model fitted to this
 // library's measured kernel times on B200 (decode: fixed cost + bytes at the sustained split-K rate;

@@ -190,7 +190,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
 
     if (threadIdx.x == 0) {
         abort_s = (p.err != nullptr && (*reinterpret_cast<volatile uint32_t*>(p.err) & kErrTimeout) != 0u) ? 2u : 0u;   // an earlier CTA gave up
-        // spatial launch sequence with CF_SPATIAL_WAIT=1: the stream that carries the decode kernel waits (a
+        // spatial launch sequence: the stream that carries the decode kernel waits (a
         // stream memory operation, not a kernel) until every CTA of this grid holds its SM
         if (resident != nullptr) atomicAdd(resident, 1u);
         mbar_init(smem_u32(&bars.q_full), 1);

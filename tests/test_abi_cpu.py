@@ -239,3 +239,14 @@ def test_windowed_plan_skips_what_no_query_can_see():
                 assert ranges[-1][1] == (P + row0 + n_rows + 127) // 128
                 assert all(a[1] == b[0] for a, b in zip(ranges, ranges[1:]))
     assert cf.cf_plan_inspect(cf.make_desc(32, 8, 128, 16, 64, window_size=-1), [5], [1], 8, check=False)[0] == cf.CF_ERR_INVALID_ARG
+
+
+def test_shared_prefix_argument_check_needs_no_device():
+    """share_group and shared_len come together or not at all (checked before anything else is touched)."""
+    lib = cf.load_library()
+    d = cf.make_desc(32, 8, 128, 16, 64)
+    arr = np.zeros(2, dtype=np.int32)
+    fake_ctx = ctypes.c_void_p(1)                      # never dereferenced: the pairing check comes first
+    st = lib.cf_mixed_attention_shared(fake_ctx, ctypes.byref(d), None, None, None, None, 4, arr.ctypes.data, arr.ctypes.data,
+                                       arr.ctypes.data, None, 2, None, None, None)
+    assert st == cf.CF_ERR_INVALID_ARG

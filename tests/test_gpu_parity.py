@@ -359,15 +359,16 @@ def test_spatial_sequence_is_bit_identical_to_the_serial_sequence():
     g.close()
 
 
-def test_spatial_sequence_with_the_resident_wait():
-    """CF_DEBUG_SPATIAL_WAIT (test-only switch): decode waits, through a stream memory operation, for
-    the front prefill CTAs; same plan, same bits as without the wait, over repeated calls."""
+def test_spatial_sequence_without_the_resident_wait():
+    """By default decode waits, through a stream memory operation, until the front prefill CTAs hold their SMs;
+    CF_DEBUG_SPATIAL_NO_WAIT (test-only switch) leaves the order to the launches.  Same plan, same bits either
+    way, over repeated calls."""
     sc = small(31, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]], NB=2048)
     b = sc.batches[0]
     plain = GpuScenario(sc)
     plain.append(b)
     o0, l0 = plain.attend(b)
-    waited = GpuScenario(sc, debug={cf.CF_DEBUG_SPATIAL_WAIT: 1})
+    waited = GpuScenario(sc, debug={cf.CF_DEBUG_SPATIAL_NO_WAIT: 1})      # (the variable keeps its name: this is the one without the wait)
     waited.append(b)
     for n in (1, 1, 5, 1):
         cf.cf_set_overlap(waited.ctx, n)

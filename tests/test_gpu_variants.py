@@ -167,3 +167,143 @@ def test_static_entry_point_honours_window_and_sinks():
                                             sinks=sinks.astype(np.float64))
     compare(ctx_o, ctx_lse, ref_o, ref_lse)
     g.close()
+
+
+# ------------------------------------------------------------------ tensor-parallel head sharding (Section 6.1: one TP4 worker per server)
+def _run_shard(ctx, sc, b, g_full, r, ranks, debug_single_partition):
+    """Rank r's share of the heads through the ABI: strided views of the SAME pools (the descriptor keeps the
+    pool's block stride and says Hkv / ranks heads; the base pointer is moved to the shard's first KV head)."""
+    geom = sc.geom
+    Hq, Hkv, D, B = geom.num_q_heads, geom.num_kv_heads, geom.head_dim, geom.block_size
+    hq, hkv = Hq // ranks, Hkv // ranks
+    st = (Hkv * B * D, B * D, D)
+    desc = cf.make_desc(hq, hkv, D, B, geom.num_blocks, k_strides=st, v_strides=st)
+    k_ptr = g_full.k.data_ptr() + r * hkv * B * D * 2
+    v_ptr = g_full.v.data_ptr() + r * hkv * B * D * 2
+    q = to_dev_bf16(np.ascontiguousarray(b.q[:, r * hq:(r + 1) * hq, :]))
+    bt = torch.from_numpy(b.block_table).cuda()
+    out = torch.full((b.total_q, hq, D), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((b.total_q, hq), float("nan"), dtype=torch.float32, device="cuda")
+    cf.cf_mixed_attention(ctx, desc, q, k_ptr, v_ptr, bt, b.max_blocks, b.context_len, b.query_len, out, lse)
+    torch.cuda.synchronize()
+    assert cf.cf_get_async_status(ctx) == cf.CF_OK
+    return to_host_bits(out), lse.cpu().numpy()
+
+
+@pytest.mark.parametrize("same_partition", [True, False])
+def test_four_head_shards_reproduce_the_unsharded_result(same_partition):
+    """The chat-like configuration split four ways by KV-head group, each shard run on its own through the ABI
+    on strided views of the same pools, concatenated along the head axis.  With the planner held to one
+    partition (one KV chunk per decode sequence, no KV split of prefill items) a head's arithmetic does not
+    depend on which other heads ride in the call: the concatenation equals the unsharded call bit for bit.  With
+    the planner left to itself the shards are cut differently (fewer heads per call) and agree to rounding;
+    both ways the shards match the oracle."""
+    sc = syn.config3_chat(iterations=(0,))
+    b = sc.batches[0]
+    debug = {cf.CF_DEBUG_PREFILL_SPLIT: 1, cf.CF_DEBUG_DECODE_MIN_CHUNK_PAGES: 1 << 20} if same_partition else None
+    g = GpuScenario(sc, debug=debug)
+    g.append(b)
+    full_o, full_lse = g.attend(b)
+    shards = [_run_shard(g.ctx, sc, b, g, r, 4, same_partition) for r in range(4)]
+    cat_o = np.concatenate([o for o, _ in shards], axis=1)
+    cat_lse = np.concatenate([l for _, l in shards], axis=1)
+    if same_partition:
+        assert np.array_equal(cat_o, full_o) and np.array_equal(cat_lse, full_lse)
+    else:
+        diff = np.abs(syn.bf16_bits_to_f64(cat_o) - syn.bf16_bits_to_f64(full_o))
+        assert diff.max() <= 2e-2 and diff.mean() <= 2e-3
+    k_ref, v_ref = g.pools_host()
+    rows = syn.tile_edge_rows(b)
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len, rows=rows)
+    compare(cat_o, cat_lse, ref_o, ref_lse, rows=rows, label="concatenated shards vs oracle")
+    g.close()
+
+
+# ------------------------------------------------------------------ shared prefixes read once
+def _run_shared(sc, share_group, shared_len, expect_shared_items=True):
+    b = sc.batches[0]
+    g = GpuScenario(sc)
+    g.append(b)
+    plain_o, plain_lse = g.attend(b)                      # aliased block tables alone already define the result
+    geom = sc.geom
+    bt = torch.from_numpy(b.block_table).cuda()
+    q = to_dev_bf16(b.q)
+    out = torch.full((b.total_q, geom.num_q_heads, geom.head_dim), float("nan"), dtype=torch.bfloat16, device="cuda")
+    lse = torch.full((b.total_q, geom.num_q_heads), float("nan"), dtype=torch.float32, device="cuda")
+    for _ in range(2):                                    # twice: the ticket counters must be back at zero
+        out.fill_(float("nan"))
+        cf.cf_mixed_attention_shared(g.ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len,
+                                     share_group, shared_len, out, lse)
+        torch.cuda.synchronize()
+        assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+        counts = cf.cf_get_last_plan_counts(g.ctx)
+        assert (counts[5] > 0) == expect_shared_items, counts
+        k_ref, v_ref = g.pools_host()
+        ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
+        o_bits, lse_h = to_host_bits(out), lse.cpu().numpy()
+        compare(o_bits, lse_h, ref_o, ref_lse, label="shared-prefix path vs oracle")
+    diff = np.abs(syn.bf16_bits_to_f64(o_bits) - syn.bf16_bits_to_f64(plain_o))
+    assert diff.max() <= 2e-2 and diff.mean() <= 2e-3
+    g.close()
+    return counts
+
+
+@pytest.mark.parametrize("n_sharers", [2, 4, 8, 16])
+@pytest.mark.parametrize("Hq,Hkv,D", [(4, 4, 128), (32, 8, 128), (64, 8, 128), (8, 2, 64)])
+def test_shared_prefix_is_read_once_for_all_sharers(n_sharers, Hq, Hkv, D):
+    """2 to 16 decode sequences that share a 2048-token prefix (group sizes 1, 4 and 8, both head dims), each with
+    a suffix of its own, beside sequences that share nothing and a prefill chunk of the same group."""
+    geom = syn.Geometry(Hq, Hkv, D, 16, 4096)
+    rng = np.random.default_rng(n_sharers)
+    own = [int(x) for x in rng.integers(0, 700, size=n_sharers)] + [900, 3000, 40]
+    qlen = [1] * n_sharers + [1, 1, 150]
+    group = [0] * n_sharers + [-1, -1, 0]
+    sc, sg, sl = syn.shared_prefix_scenario("shared", geom, 61 + n_sharers, 2048, own, qlen, group)
+    counts = _run_shared(sc, sg, sl)
+    per_set = max(1, 16 // (Hq // Hkv))
+    assert counts[6] == n_sharers and counts[5] % ((n_sharers + per_set - 1) // per_set) == 0
+
+
+def test_two_share_groups_and_a_short_prefix():
+    """Two groups with prefixes of their own; a group whose common prefix is shorter than the threshold, a group
+    with a single decode member and a member whose shared_len exceeds its context are served the ordinary way."""
+    geom = syn.Geometry(32, 8, 128, 16, 4096)
+    own = [10, 500, 33, 0, 1200, 77, 5, 300]
+    qlen = [1, 1, 1, 1, 1, 1, 1, 1]
+    sc, sg, sl = syn.shared_prefix_scenario("two-groups", geom, 71, 4096, own, qlen, [0, 0, 0, 1, 1, 1, 1, -1])
+    counts = _run_shared(sc, sg, sl)
+    assert counts[6] == 7
+    sc, sg, sl = syn.shared_prefix_scenario("short", geom, 72, 128, own[:4], qlen[:4], [0, 0, 0, 0])
+    _run_shared(sc, sg, sl, expect_shared_items=False)
+    sc, sg, sl = syn.shared_prefix_scenario("lonely", geom, 73, 2048, own[:3], [1, 40, 1], [0, 0, -1])
+    _run_shared(sc, sg, sl, expect_shared_items=False)
+    # shared_len claims more than a member has: clamped to the member's context minus its new token
+    sc, sg, sl = syn.shared_prefix_scenario("clamped", geom, 74, 1024, [0, 0, 0], [1, 1, 1], [0, 0, 0])
+    sl[:] = 1 << 20
+    counts = _run_shared(sc, sg, sl)
+    assert counts[6] == 3
+
+
+def test_shared_prefix_with_many_chunks_and_the_separate_combine_kernel():
+    """A 40K-token shared prefix (many shared chunks per member) with short and long suffixes, merged by the fused
+    merge and by the separate combine kernel: identical bits."""
+    geom = syn.Geometry(32, 8, 128, 16, 8192)
+    sc, sg, sl = syn.shared_prefix_scenario("long-shared", geom, 75, 40000 // 16 * 16, [0, 15, 3000, 9000, 17, 600], [1] * 6, [0] * 6)
+    b = sc.batches[0]
+    outs = []
+    for debug in (None, {cf.CF_DEBUG_SEPARATE_COMBINE: 1}):
+        g = GpuScenario(sc, debug=debug)
+        g.append(b)
+        bt = torch.from_numpy(b.block_table).cuda()
+        q = to_dev_bf16(b.q)
+        out = torch.full_like(q, float("nan"))
+        lse = torch.full((b.total_q, 32), float("nan"), dtype=torch.float32, device="cuda")
+        cf.cf_mixed_attention_shared(g.ctx, g.desc, q, g.k, g.v, bt, b.max_blocks, b.context_len, b.query_len, sg, sl, out, lse)
+        torch.cuda.synchronize()
+        assert cf.cf_get_last_plan_counts(g.ctx)[5] > 1
+        outs.append((to_host_bits(out), lse.cpu().numpy()))
+        k_ref, v_ref = g.pools_host()
+        g.close()
+    assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
+    compare(outs[0][0], outs[0][1], ref_o, ref_lse)
