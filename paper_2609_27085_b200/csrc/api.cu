@@ -465,8 +465,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess && resident &&
             mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_decode_shared(p, D, n.n_shared, c->side);
-        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, c->side);
+        if (e == cudaSuccess) e = launch_decode_with_shared(p, D, n.n_shared, n.n_dec, c->side);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
         if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
         if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
@@ -474,8 +473,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
     } else {
         if (tc) cudaEventRecord(tc->ev[0], stream);
-        if (e == cudaSuccess) e = launch_decode_shared(p, D, n.n_shared, stream);
-        if (e == cudaSuccess) e = launch_decode(p, D, n.n_dec, stream);
+        if (e == cudaSuccess) e = launch_decode_with_shared(p, D, n.n_shared, n.n_dec, stream);
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
@@ -483,7 +481,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
-    c->launches = (int)(n.n_dec > 0) + (int)(n.n_shared > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
+    c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
     return e == cudaSuccess ? CF_OK : CF_ERR_CUDA;
 }
 

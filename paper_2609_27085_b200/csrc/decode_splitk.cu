@@ -77,7 +77,7 @@ __device__ __forceinline__ void merge_partials(const AttnParams& p, int q_row, i
 }
 
 template <int D, int NWARPS, int NSTAGE>
-__global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const AttnParams p)
+__device__ __forceinline__ void decode_cta(const AttnParams& p, const int cta)
 {
     constexpr int CPR = D / 8;                  // 16-byte chunks per token row
     constexpr int PAGE_BYTES = 16 * D * 2;      // one (page, head) of K or of V
@@ -88,7 +88,7 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
     extern __shared__ __align__(1024) uint8_t smem[];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const int item_id = cta / p.Hkv, kvh = cta % p.Hkv;
     const DecodeItem it = p.dec_items[item_id];
     const int G = p.G;
     // lets the combine kernel (launched with programmatic stream serialisation) become resident while
@@ -313,7 +313,7 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const Att
 // partial in the member's slot for this chunk; the member's own chunks and the merge follow in the next kernel.
 // Pages are fetched with the default L2 policy: other member sets of the group read them again.
 template <int D, int NWARPS, int NSTAGE, int NCG>
-__global__ void __launch_bounds__(NWARPS * 32, 2) decode_shared_kernel(const AttnParams p)
+__device__ __forceinline__ void decode_shared_cta(const AttnParams& p, const int cta)
 {
     constexpr int CPR = D / 8;
     constexpr int PAGE_BYTES = 16 * D * 2;
@@ -325,8 +325,9 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_shared_kernel(const Att
     extern __shared__ __align__(1024) uint8_t smem[];
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const int item_id = cta / p.Hkv, kvh = cta % p.Hkv;
     const SharedDecodeItem it = p.sh_items[item_id];
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
     const ShareMember* members = p.sh_members + it.member_first;
     const int G = p.G;
 
@@ -511,14 +512,50 @@ __global__ void __launch_bounds__(NWARPS * 32, 2) decode_shared_kernel(const Att
         *reinterpret_cast<float2*>(p.part_o + pr * D + d) = make_float2(o0, o1);
         if (d == 0) *reinterpret_cast<float2*>(p.part_ml + pr * 2) = make_float2(M, L);
     }
-    // Fused merge: this chunk counts as done for every member (the member's own chunks, which run in the next
-    // kernel, draw the remaining tickets, so the last ticket is never drawn here).
+    // Fused merge: this chunk counts as done for every member of the set.  The members' own chunks run in the
+    // same grid; whichever CTA draws a member's last ticket - this one or one of those - merges that member's
+    // partials for this KV head (all of them were published, fence + ticket, before the last ticket was drawn).
     if (p.dec_counters != nullptr) {
+        __shared__ uint32_t last_mask_s;
+        if (threadIdx.x == 0) last_mask_s = 0u;
         __threadfence();
         __syncthreads();
-        if ((int)threadIdx.x < it.n_members)
-            atomicAdd(p.dec_counters + (int64_t)__ldg(&members[threadIdx.x].part_first) * p.Hkv + kvh, 1u);
+        if ((int)threadIdx.x < it.n_members) {
+            uint32_t* counter = p.dec_counters + (int64_t)__ldg(&members[threadIdx.x].part_first) * p.Hkv + kvh;
+            if (atomicAdd(counter, 1u) == (uint32_t)(__ldg(&members[threadIdx.x].n_chunks) - 1)) atomicOr(&last_mask_s, 1u << threadIdx.x);
+        }
+        __syncthreads();
+        const uint32_t last_mask = last_mask_s;
+        if (last_mask != 0u) {
+            __threadfence();
+            for (int m = 0; m < it.n_members; ++m) {
+                if (!((last_mask >> m) & 1u)) continue;
+                const int q_row = __ldg(&members[m].q_row), part_first = __ldg(&members[m].part_first);
+                const int n_chunks = __ldg(&members[m].n_chunks);
+                for (int idx = threadIdx.x; idx < G * (D / 4); idx += NWARPS * 32) {
+                    const int head = idx / (D / 4), d = (idx % (D / 4)) * 4;
+                    merge_partials<D>(p, q_row, part_first, n_chunks, kvh * G + head, d, d == 0);
+                }
+                if (threadIdx.x == 0) p.dec_counters[(int64_t)part_first * p.Hkv + kvh] = 0u;
+            }
+        }
     }
+}
+
+template <int D, int NWARPS, int NSTAGE>
+__global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_kernel(const AttnParams p)
+{
+    decode_cta<D, NWARPS, NSTAGE>(p, (int)blockIdx.x);
+}
+
+// One grid for a batch with shared prefixes: the first n_shared_ctas CTAs serve the shared chunks (longer items
+// first), the rest the sequences' own chunks.  Both kinds need half an SM's shared memory, so the larger register
+// footprint of the shared role costs no occupancy; batches without sharing launch decode_splitk_kernel.
+template <int D, int NWARPS, int NSTAGE, int NCG>
+__global__ void __launch_bounds__(NWARPS * 32, 2) decode_with_shared_kernel(const AttnParams p, const int n_shared_ctas)
+{
+    if ((int)blockIdx.x < n_shared_ctas) decode_shared_cta<D, NWARPS, NSTAGE, NCG>(p, (int)blockIdx.x);
+    else decode_cta<D, NWARPS, NSTAGE>(p, (int)blockIdx.x - n_shared_ctas);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -572,10 +609,10 @@ cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaSt
 }
 
 template <int D>
-static cudaError_t launch_decode_shared_t(const AttnParams& p, int n_items, cudaStream_t stream)
+static cudaError_t launch_decode_shared_t(const AttnParams& p, int n_shared_items, int n_items, cudaStream_t stream)
 {
     constexpr int NCG = kSharedColumns / 8;
-    auto kern = decode_shared_kernel<D, kDecWarps, kDecStages, NCG>;
+    auto kern = decode_with_shared_kernel<D, kDecWarps, kDecStages, NCG>;
     const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * D * 2;
     const size_t merge = (size_t)kDecWarps * kSharedColumns * (D + 4) * 4 + (size_t)kDecWarps * kSharedColumns * 4 * 2;
     const size_t smem = ring > merge ? ring : merge;
@@ -587,14 +624,16 @@ static cudaError_t launch_decode_shared_t(const AttnParams& p, int n_items, cuda
         if (e != cudaSuccess) return e;
         configured[dev].store(true, std::memory_order_release);
     }
-    kern<<<n_items * p.Hkv, kDecWarps * 32, smem, stream>>>(p);
+    kern<<<(n_shared_items + n_items) * p.Hkv, kDecWarps * 32, smem, stream>>>(p, n_shared_items * p.Hkv);
     return cudaGetLastError();
 }
 
-cudaError_t launch_decode_shared(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
+cudaError_t launch_decode_with_shared(const AttnParams& p, int head_dim, int n_shared_items, int n_items, cudaStream_t stream)
 {
-    if (n_items <= 0) return cudaSuccess;
-    return head_dim == 128 ? launch_decode_shared_t<128>(p, n_items, stream) : launch_decode_shared_t<64>(p, n_items, stream);
+    if (n_shared_items + n_items <= 0) return cudaSuccess;
+    if (n_shared_items <= 0) return launch_decode(p, head_dim, n_items, stream);
+    return head_dim == 128 ? launch_decode_shared_t<128>(p, n_shared_items, n_items, stream)
+                           : launch_decode_shared_t<64>(p, n_shared_items, n_items, stream);
 }
 
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)

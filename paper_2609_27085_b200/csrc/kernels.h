@@ -29,9 +29,11 @@ cudaError_t launch_validate_table(const int32_t* block_table, int32_t max_blocks
                                   int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
-// shared-prefix chunks: one CTA per (shared item, KV head) streams the chunk once for all members of the set and
-// writes one partial per member and head; launched before launch_decode, whose merge then finds those partials
-cudaError_t launch_decode_shared(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
+// a batch with shared prefixes: one grid whose first CTAs serve the shared-prefix chunks (one CTA per shared item
+// and KV head streams the chunk once for all members of its set and writes one partial per member and head) and
+// whose other CTAs serve the sequences' own chunks; n_shared_items = 0 is launch_decode
+cudaError_t launch_decode_with_shared(const AttnParams& p, int head_dim, int n_shared_items, int n_items, cudaStream_t stream);
+
 // tcgen05 / tensor-memory chunked prefill (head_dim 64 or 128): `n_ctas` persistent CTAs draw the `n_items`
 // PrefillTcItems from the ticket counter p.pre_queue, which `queue_ctas` CTAs share in total (several
 // launches may draw from one counter; the last CTA to leave resets it).  Ticket t stands for item

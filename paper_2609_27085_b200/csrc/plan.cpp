@@ -147,8 +147,11 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         }
     }
 
-    std::vector<int32_t> part_first_of;        // per sequence: its first partial slot (-1: writes out directly)
-    if (!groups_sh.empty()) part_first_of.assign((size_t)num_seqs, -1);
+    std::vector<int32_t> part_first_of, n_chunks_of;   // per sequence: its first partial slot (-1: writes out directly), its chunks
+    if (!groups_sh.empty()) {
+        part_first_of.assign((size_t)num_seqs, -1);
+        n_chunks_of.assign((size_t)num_seqs, 0);
+    }
     for (int32_t s = 0; s < num_seqs; ++s) {
         if (query_len[s] != 1) continue;
         const int32_t lc = context_len[s];
@@ -163,7 +166,10 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             first = plan->n_part_slots;
             plan->combine.push_back(CombineItem{plan->q_start[s], first, n_all});
             plan->n_part_slots += n_all;
-            if (!part_first_of.empty()) part_first_of[(size_t)s] = first;
+            if (!part_first_of.empty()) {
+                part_first_of[(size_t)s] = first;
+                n_chunks_of[(size_t)s] = n_all;
+            }
         }
         for (int64_t c = 0; c < n; ++c) {
             DecodeItem it;
@@ -189,7 +195,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             const int32_t member_first = (int32_t)plan->share_members.size();
             for (int32_t m = 0; m < n_mem; ++m) {
                 const int32_t s = gi.members[m0 + (size_t)m];
-                plan->share_members.push_back(ShareMember{plan->q_start[s], part_first_of[(size_t)s]});
+                plan->share_members.push_back(ShareMember{plan->q_start[s], part_first_of[(size_t)s], n_chunks_of[(size_t)s], 0});
             }
             for (int32_t c = 0; c < n_sh; ++c) {
                 SharedDecodeItem it;

@@ -40,6 +40,8 @@ struct SharedDecodeItem {  // one (share group, shared KV chunk, member set); th
 struct ShareMember {       // one member of a set
     int32_t q_row;         // packed row of its query token
     int32_t part_first;    // first partial slot of the sequence (its chunk c writes slot part_first + c)
+    int32_t n_chunks;      // chunks of the sequence, shared ones and its own
+    int32_t pad;
 };
 constexpr int32_t kSharedColumns = 16;      // query-head columns a shared-prefix CTA carries (two 8-wide MMA operands)
 constexpr int32_t kMinSharedPages = 16;     // shorter shared prefixes are not worth a separate pass
