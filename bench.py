@@ -658,6 +658,8 @@ def run_case(args):
     torch.cuda.set_device(0)
     peaks = load_peaks()
     ctx = cf.cf_create(0)
+    if args.pairs:
+        cf.cf_set_debug_option(ctx, cf.CF_DEBUG_PREFILL_PAIRS, 1)
     wl = DeviceWorkload(small_case(args.case), torch, cf, ctx)
     stream = torch.cuda.current_stream()
     for i in range(args.warmup):
@@ -665,7 +667,7 @@ def run_case(args):
     kern, launches = measure_kernels(torch, cf, wl, args.steps, stream, peaks)
     host = measure_host_time(torch, cf, wl, min(args.steps, 8), stream)
     torch.cuda.synchronize()
-    print(json.dumps({"case": args.case, "steps": args.steps, "kernels": kern, "host_us_per_call": host, "gpu_launches": launches}),
+    print(json.dumps({"case": args.case, "pairs": bool(args.pairs), "steps": args.steps, "kernels": kern, "host_us_per_call": host, "gpu_launches": launches}),
           flush=True)
     del wl
     cf.cf_destroy(ctx)
@@ -675,6 +677,7 @@ def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None,
                     help="run a reduced workload (decode_small | prefill_small | prefill_multi | agentic_small | shared_prefix) and exit")
+    ap.add_argument("--pairs", action="store_true", help="reduced workloads: chunked prefill on the two-CTA (cta_group::2) kernel")
     ap.add_argument("--variant", default="both", choices=["both", "plain", "shared"], help="shared_prefix case: which entry point")
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)

@@ -211,13 +211,18 @@ cf_status cf_validate_block_table(cf_ctx* ctx, const cf_cache_desc* desc, const 
  *   CF_DEBUG_DECODE_MIN_CHUNK_PAGES shortest decode chunk, in pages
  *   CF_DEBUG_SPATIAL_NO_WAIT        1: in the spatial sequence decode does not wait (through a stream memory
  *                                   operation) until the first prefill grid's CTAs hold their SMs, but relies on
- *                                   the order of the launches */
+ *                                   the order of the launches
+ *   CF_DEBUG_PREFILL_PAIRS          1: chunked prefill on pairs of SMs (tcgen05.mma.cta_group::2: two CTAs work on four
+ *                                   heads of a group and share every K/V tile) where head_dim is 128 and the group
+ *                                   size 4 or 8; correct and tested, but measured ~20 % slower than the default
+ *                                   one-CTA-per-item kernel */
 typedef enum {
     CF_DEBUG_PREFILL_SPLIT = 0,
     CF_DEBUG_SEPARATE_COMBINE = 1,
     CF_DEBUG_DECODE_WAVES = 2,
     CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3,
-    CF_DEBUG_SPATIAL_NO_WAIT = 4
+    CF_DEBUG_SPATIAL_NO_WAIT = 4,
+    CF_DEBUG_PREFILL_PAIRS = 5
 } cf_debug_option;
 cf_status cf_set_debug_option(cf_ctx* ctx, cf_debug_option option, int value);
 
@@ -243,7 +248,7 @@ cf_status cf_get_host_time_sums(cf_ctx* ctx, double* us_append, double* us_atten
                                 int32_t* num_steps);
 /* Item counts of the plan the last cf_mixed_attention(_shared) built, for tests and reports: counts[8] =
  * {decode items, split decode sequences, prefill CTAs, decode partial slots, KV-split prefill items,
- *  shared-prefix items, members of shared-prefix sets, 0}. */
+ *  shared-prefix items, members of shared-prefix sets, 1 if the prefill items are pair items (two CTAs each)}. */
 cf_status cf_get_last_plan_counts(cf_ctx* ctx, int32_t* counts);
 /* Number of kernels the last cf_mixed_attention launched. */
 cf_status cf_get_last_launch_count(cf_ctx* ctx, int32_t* num_launches);
@@ -290,7 +295,8 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
  * cf_mixed_attention would build and copies out up to `cap` items of each kind.
  *   opts          : planner settings, or NULL for the defaults of a 148-SM device.  Zero fields mean
  *                   "default"; prefill_sms_mixed > 0 plans a mixed batch for the spatial sequence with
- *                   that many SMs in the first prefill grid; prefill_force_split as CF_DEBUG_PREFILL_SPLIT.
+ *                   that many SMs in the first prefill grid; prefill_force_split as CF_DEBUG_PREFILL_SPLIT;
+ *                   prefill_pairs as CF_DEBUG_PREFILL_PAIRS.
  *   decode_items  : int32 [cap, 6] = {seq, q_row, kv_begin, kv_end, partial_slot (-1 = writes out directly), chunk_index}
  *   combine_items : int32 [cap, 3] = {q_row, first_partial_slot, num_chunks}
  *   prefill_items : int32 [cap, 8] = {seq, q_row_of_tile, first_row_in_chunk, num_rows, query_head, kv_head,
@@ -298,10 +304,12 @@ cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, 
  *                   order; KV tiles are 128 tokens, end_kv_tile is clamped to the tile's own extent; an item
  *                   that is not KV-split has one entry covering all of its tiles
  *   counts        : int32 [6]      = {n_decode_items, n_combine_items, n_prefill_entries, n_partial_slots,
- *                                     n_prefill_ctas (KV ranges of split items counted), n_kv_split_prefill_items}
+ *                                     n_prefill_work_items (KV ranges of split items counted; an item occupies one
+ *                                     SM, or a pair of SMs where pairs are used and then carries four heads),
+ *                                     n_prefill_combine_items (one per KV-split item and CTA of a pair)}
  * Any output pointer may be NULL. */
 typedef struct {
-    int32_t num_sms, prefill_sms_mixed, prefill_force_split, decode_waves, decode_min_chunk_pages;
+    int32_t num_sms, prefill_sms_mixed, prefill_force_split, decode_waves, decode_min_chunk_pages, prefill_pairs;
 } cf_plan_options;
 cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
                           int32_t num_seqs, int32_t max_blocks_per_seq, const cf_plan_options* opts,

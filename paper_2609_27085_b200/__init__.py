@@ -38,6 +38,7 @@ CF_DEBUG_SEPARATE_COMBINE = 1
 CF_DEBUG_DECODE_WAVES = 2
 CF_DEBUG_DECODE_MIN_CHUNK_PAGES = 3
 CF_DEBUG_SPATIAL_NO_WAIT = 4
+CF_DEBUG_PREFILL_PAIRS = 5
 
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
@@ -58,7 +59,7 @@ class CacheDesc(ctypes.Structure):
 class PlanOptions(ctypes.Structure):
     """Mirror of ``cf_plan_options`` (zero = default)."""
     _fields_ = [("num_sms", ctypes.c_int32), ("prefill_sms_mixed", ctypes.c_int32), ("prefill_force_split", ctypes.c_int32),
-                ("decode_waves", ctypes.c_int32), ("decode_min_chunk_pages", ctypes.c_int32)]
+                ("decode_waves", ctypes.c_int32), ("decode_min_chunk_pages", ctypes.c_int32), ("prefill_pairs", ctypes.c_int32)]
 
 
 class CfError(RuntimeError):
@@ -278,7 +279,7 @@ def cf_get_last_launch_count(ctx) -> int:
 
 def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148,
                     cap: int = 1 << 16, check: bool = True, prefill_sms_mixed: int = 0, prefill_force_split: int = 0,
-                    decode_waves: int = 0, decode_min_chunk_pages: int = 0, want_counts: bool = False):
+                    decode_waves: int = 0, decode_min_chunk_pages: int = 0, want_counts: bool = False, prefill_pairs: int = 0):
     """Returns (status, decode_items [n,6], combine_items [n,3], prefill_items [n,8], n_partial_slots)
     and, with want_counts, the six counters as a last element."""
     lc, lq = _host_i32(context_len), _host_i32(query_len)
@@ -287,7 +288,7 @@ def cf_plan_inspect(desc: CacheDesc, context_len, query_len, max_blocks_per_seq:
     pre = np.zeros((cap, 8), dtype=np.int32)
     counts = np.zeros(6, dtype=np.int32)
     opts = PlanOptions(int(num_sms), int(prefill_sms_mixed), int(prefill_force_split), int(decode_waves),
-                       int(decode_min_chunk_pages))
+                       int(decode_min_chunk_pages), int(prefill_pairs))
     st = load_library().cf_plan_inspect(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]),
                                         int(max_blocks_per_seq), ctypes.byref(opts), dec.ctypes.data, comb.ctypes.data,
                                         pre.ctypes.data, cap, counts.ctypes.data)

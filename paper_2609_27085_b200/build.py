@@ -15,7 +15,7 @@ import sys
 HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libcrossflow_attn.so")
-SOURCES = ["api.cu", "plan.cpp", "kv_append.cu", "decode_splitk.cu", "prefill_tc.cu"]
+SOURCES = ["api.cu", "plan.cpp", "kv_append.cu", "decode_splitk.cu", "prefill_tc.cu", "prefill_tc2.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-O3", "-lineinfo", "-std=c++17",
               "-Xcompiler", "-fPIC", "--expt-relaxed-constexpr"]
 

@@ -80,6 +80,8 @@ struct cf_ctx {
     bool workspace_fixed = false;
     uint32_t* err_dev = nullptr;      // [0] device-side findings (bit 0: a wait expired, bit 1: block id outside the pool); [1] scratch counter of cf_validate_block_table
     bool fused_combine = true; // split-K merge inside the decode kernel (CF_DEBUG_SEPARATE_COMBINE: the separate combine kernel)
+    bool use_pairs = false;    // CF_DEBUG_PREFILL_PAIRS: chunked prefill on pairs of SMs where the geometry allows it (measured slower
+                               // than one CTA per item, see prefill_tc2.cu; kept as a tested alternative)
     std::atomic<int> live_plans{0};
     // concurrent execution of the prefill kernel beside decode + combine (side stream, fork/join events)
     bool overlap = true;
@@ -122,6 +124,7 @@ struct cf_plan {
     int n_part_slots = 0, n_pre_slots = 0;
     size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_sh = 0, off_shm = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    bool pair = false;
     float pre_over_dec = 0.f;
 };
 
@@ -342,6 +345,7 @@ namespace cf {
 
 struct PlanCounts {
     int n_dec = 0, n_comb = 0, n_shared = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    bool pair = false;          // the prefill items are pair items (two CTAs each)
     float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
     int n_part_slots = 0;
 };
@@ -427,8 +431,15 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         maps.q = *mq; maps.k = *mk; maps.v = *mv;
     }
     int second_grid = 0;
-    const int sms = c->num_sms > 0 ? c->num_sms : 148;
-    const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs of the serial sequence
+    // Slots that take a prefill item: SMs, or pairs of SMs for pair items.  Grid sizes, the shared work queue and
+    // the front / tail split below are counted in slots.
+    const int per_slot = n.pair ? 2 : 1;
+    const int sms = (c->num_sms > 0 ? c->num_sms : 148) / per_slot;
+    const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs (pairs) of the serial sequence
+    auto launch_prefill = [&](int n_slots, int queue_slots, int first_static, int ticket_base, uint32_t* resident, cudaStream_t st) {
+        return n.pair ? launch_prefill_tc2(p, maps, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st)
+                      : launch_prefill_tc(p, maps, D, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st);
+    };
     if (c->overlap && !c->in_host_step && !tc && has_prefill && (n.n_dec > 0)) {
         // Spatial partition.  `front` persistent prefill CTAs (one per SM: a CTA takes an SM's whole shared
         // memory) go first, on the caller's stream; decode runs on the SMs left over, on a context-owned side
@@ -438,7 +449,8 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         // Default share: three fifths of the SMs.  When the prefill work dwarfs the decode kernel, sharing the
         // machine no longer pays (the tensor-bound kernel already runs at the power limit): prefill takes
         // every SM first and decode fills in as its CTAs retire.
-        int front = c->spatial_sms > 0 ? c->spatial_sms : (n.pre_over_dec > 3.9f ? sms : (sms * 3) / 5);
+        int front = c->spatial_sms > 0 ? c->spatial_sms / per_slot : (n.pre_over_dec > 3.9f ? sms : (sms * 3) / 5);
+        if (front < 1) front = 1;
         if (front > sms) front = sms;
         if (front > n.n_pre_tc) front = n.n_pre_tc;
         int tail = n.n_pre_tc - front;
@@ -460,14 +472,14 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         }
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, front, front + tail, 1, front, resident, stream);
+        if (e == cudaSuccess) e = launch_prefill(front, front + tail, 1, front, resident, stream);
         // only after the front grid has been enqueued without an error, so that the count is certain to arrive
         if (e == cudaSuccess && resident &&
-            mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)front, CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
+            mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)(front * per_slot), CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_decode_with_shared(p, D, n.n_shared, n.n_dec, c->side);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, tail, front + tail, 0, front, nullptr, c->side);
+        if (e == cudaSuccess) e = launch_prefill(tail, front + tail, 0, front, nullptr, c->side);
         if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
@@ -477,7 +489,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
-        if (e == cudaSuccess) e = launch_prefill_tc(p, maps, D, n.n_pre_tc, pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
+        if (e == cudaSuccess) e = launch_prefill(pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
         if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
@@ -668,6 +680,7 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     Plan pl;
     PlanConfig cfg = c->cfg;
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
+    cfg.prefill_pair = c->use_pairs && prefill_pair_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl, share_group, shared_len);
     if (st != CF_OK) return st;
     c->host_ns_planner += now_ns() - t_in;
@@ -693,9 +706,10 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     n.n_dec = (int)pl.decode.size(); n.n_comb = (int)pl.combine.size(); n.n_shared = (int)pl.shared_decode.size();
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
     n.n_part_slots = pl.n_part_slots;
+    n.pair = pl.pair;
     c->last_counts[0] = n.n_dec; c->last_counts[1] = n.n_comb; c->last_counts[2] = n.n_pre_tc; c->last_counts[3] = n.n_part_slots;
     c->last_counts[4] = n.n_pre_comb; c->last_counts[5] = n.n_shared; c->last_counts[6] = (int32_t)pl.share_members.size();
-    c->last_counts[7] = 0;
+    c->last_counts[7] = pl.pair ? 1 : 0;
     n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
@@ -715,6 +729,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     Plan pl;
     PlanConfig cfg = c->cfg;
     cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
+    cfg.prefill_pair = c->use_pairs && prefill_pair_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
     DeviceGuard guard(c->device);
@@ -733,6 +748,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
     P->pre_over_dec = prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms);
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
+    P->pair = pl.pair;
     const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
     // the ticket counters are zeroed on the caller's stream, like the plan copy: every launch that uses the plan
@@ -820,6 +836,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     n.total_q = P->total_q;
     n.pre_over_dec = P->pre_over_dec;
     n.n_part_slots = P->n_part_slots;
+    n.pair = P->pair;
     const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim);
     return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, W, q, k_cache,
                             v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);
@@ -986,6 +1003,7 @@ cf_status cf_set_debug_option(cf_ctx* c, cf_debug_option option, int value)
             c->cfg.decode_min_chunk_pages = value > 0 ? value : defaults.decode_min_chunk_pages;
             return CF_OK;
         case CF_DEBUG_SPATIAL_NO_WAIT: c->spatial_wait = value <= 0; return CF_OK;
+        case CF_DEBUG_PREFILL_PAIRS: c->use_pairs = value > 0; return CF_OK;
     }
     return CF_ERR_INVALID_ARG;
 }
@@ -1089,6 +1107,7 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
         if (opts->decode_waves > 0) cfg.decode_waves = opts->decode_waves;
         if (opts->decode_min_chunk_pages > 0) cfg.decode_min_chunk_pages = opts->decode_min_chunk_pages;
     }
+    cfg.prefill_pair = prefill_pair_supported(desc) && opts && opts->prefill_pairs > 0;
     Plan pl;
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -1116,6 +1135,14 @@ cf_status cf_plan_inspect(const cf_cache_desc* desc, const int32_t* context_len,
                 o[7] = it.j_end < tiles ? it.j_end : tiles;
             }
             ++n_pre;
+            if (pl.pair) {                               // the second CTA of the pair: the same q tile for head + 2
+                if (prefill_items && n_pre < (size_t)cap) {
+                    int32_t* o = prefill_items + 8 * n_pre;
+                    for (int i = 0; i < 8; ++i) o[i] = o[i - 8];
+                    o[4] += 2;
+                }
+                ++n_pre;
+            }
         }
     if (counts) {
         counts[0] = (int32_t)pl.decode.size();

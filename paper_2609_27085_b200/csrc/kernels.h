@@ -51,6 +51,13 @@ bool encode_pool_map(CUtensorMap* m, const void* pool, int head_dim, int num_blo
 cudaError_t launch_prefill_tc(const AttnParams& p, const PrefillMaps& maps, int head_dim, int n_items, int n_ctas,
                               int queue_ctas, int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
 
+// The same work on pairs of SMs (tcgen05.mma.cta_group::2; head_dim 128, group size a multiple of 4): an item is four
+// q tiles (four heads of a group over the same rows), CTA r of a pair taking heads head[t] + 2 r and partial slots
+// part_slot[t] + r * pad; n_pairs persistent pairs (2 n_pairs CTAs), queue_pairs pairs drawing from the counter.
+bool prefill_pair_supported(const cf_cache_desc* desc);
+cudaError_t launch_prefill_tc2(const AttnParams& p, const PrefillMaps& maps, int n_items, int n_pairs, int queue_pairs,
+                               int first_static, int ticket_base, uint32_t* resident, cudaStream_t stream);
+
 // merges the fp32 partials of KV-split prefill items into `out` (one CTA per split item)
 cudaError_t launch_prefill_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 // one CTA whose bounded wait must expire: sets *err and returns normally (status-path self-test)

@@ -219,6 +219,10 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // pairs of 128-row tiles that share a KV head: two heads of a group over the same rows, or
         // (group size 1) two consecutive row tiles of one head
         constexpr int32_t TR = 128;
+        // pair items: four heads of a group per item, run by two CTAs on two SMs
+        const bool pair = cfg.prefill_pair && d->head_dim == 128 && G % 4 == 0;
+        const int32_t heads_per_item = pair ? 4 : 2;
+        plan->pair = pair;
         struct KeyedTc { int64_t extent; int32_t tiles; PrefillTcItem it; };   // extent: end of the visible keys; tiles: KV tiles to visit
         std::vector<KeyedTc> items;
         auto prefix_of = [&](int32_t s) { return context_len[s] - query_len[s]; };
@@ -234,7 +238,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
             for (int32_t tile = 0; tile < n_tiles; tile += (G >= 2 ? 1 : 2)) {
                 const int32_t last = (G >= 2 || tile + 1 >= n_tiles) ? tile : tile + 1;
                 groups.push_back(Group{(int64_t)prefix_of(s) + last * TR + std::min(TR, lq - last * TR), s, tile});
-                n_emit += (size_t)(G >= 2 ? d->num_kv_heads * (G / 2) : d->num_q_heads);
+                n_emit += (size_t)(G >= 2 ? d->num_kv_heads * (G / heads_per_item) : d->num_q_heads);
             }
         }
         std::stable_sort(groups.begin(), groups.end(), [](const Group& a, const Group& b) { return a.extent > b.extent; });
@@ -259,7 +263,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                     it.n_rows[t] = rows_of(tile);
                 }
                 for (int32_t kvh = 0; kvh < d->num_kv_heads; ++kvh)
-                    for (int32_t i = 0; i < G; i += 2) {
+                    for (int32_t i = 0; i < G; i += heads_per_item) {
                         it.kvh = kvh;
                         it.head[0] = kvh * G + i;
                         it.head[1] = kvh * G + i + 1;
@@ -285,7 +289,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // alternative while pairs would leave SMs idle (sharing K/V tiles matters only when the machine is
         // full).  Whether pairs or singles are used is decided below, together with the KV split.
         std::vector<KeyedTc> singles;
-        if (items.size() * 2 <= (size_t)std::max(1, cfg.num_sms)) {
+        if (!pair && items.size() * 2 <= (size_t)std::max(1, cfg.num_sms)) {
             singles.reserve(items.size() * 2);
             for (const KeyedTc& k : items)
                 for (int t = 0; t < 2; ++t) {
@@ -306,7 +310,8 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
         // An item may be cut into k <= 8 KV ranges that write fp32 partials, merged by a combine pass; k
         // comes from the cost model's constants; a range never starts inside the diagonal band and has at
         // least 4 tiles.
-        const size_t M = (size_t)std::max(1, (cfg.prefill_sms_mixed > 0 && !plan->decode.empty()) ? cfg.prefill_sms_mixed : cfg.num_sms);
+        const size_t M = (size_t)std::max(1, ((cfg.prefill_sms_mixed > 0 && !plan->decode.empty()) ? cfg.prefill_sms_mixed : cfg.num_sms) /
+                                                 (pair ? 2 : 1));      // slots that take an item: SMs, or pairs of SMs
         // decides the KV ranges per item for one candidate item list; returns the predicted time (us)
         auto decide = [&](const std::vector<KeyedTc>& its, const double tile_us, std::vector<int32_t>& k_of) -> double {
         const size_t n_items = its.size();
@@ -413,6 +418,17 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
                 plan->n_pre_slots += it.n_rows[t] * k;
             }
             plan->prefill_combine.push_back(ci);
+            if (pair) {
+                // the second CTA's two q tiles (heads + 2) get slots of their own, a fixed distance behind the first CTA's
+                PrefillCombineItem cj = ci;
+                it.pad = plan->n_pre_slots - ci.part_slot[0];
+                for (int t = 0; t < 2; ++t) {
+                    cj.head[t] = it.head[t] + 2;
+                    cj.part_slot[t] = it.n_rows[t] > 0 ? plan->n_pre_slots : -1;
+                    plan->n_pre_slots += it.n_rows[t] * k;
+                }
+                plan->prefill_combine.push_back(cj);
+            }
             for (int32_t c = 0; c < k; ++c) {
                 PrefillTcItem f = it;
                 f.j_begin = std::min(j_lo + (int32_t)((int64_t)c * (n_min - j_lo) / k), safe);
@@ -443,7 +459,7 @@ float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len
             if (it.n_rows[t] > 0) hi = std::max(hi, it.prefix + it.row0[t] + it.n_rows[t]);
         work += 8.0 + 1.9 * (double)std::max(0, std::min((hi + 127) / 128, it.j_end) - it.j_begin);
     }
-    return (float)((work / (double)std::max(1, num_sms)) / (17.0 + dec_bytes / 7.1e6));
+    return (float)((work / (double)std::max(1, plan.pair ? num_sms / 2 : num_sms)) / (17.0 + dec_bytes / 7.1e6));
 }
 
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
@@ -477,7 +493,7 @@ Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const i
             const double cost = kTcItemFixedUs + kTcTileUs * tiles;
             jobs.push_back(cost);
         }
-        e.us_prefill = (float)(kLaunchUs + list_schedule(jobs, (size_t)std::max(1, num_sms)));
+        e.us_prefill = (float)(kLaunchUs + list_schedule(jobs, (size_t)std::max(1, plan.pair ? num_sms / 2 : num_sms)));
         if (!plan.prefill_combine.empty()) e.us_prefill += (float)(6.0 + 0.05 * (double)plan.prefill_tc.size());
     }
     return e;

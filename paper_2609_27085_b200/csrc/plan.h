@@ -68,7 +68,8 @@ struct PrefillTcItem {     // tcgen05 kernel: two 128-row q tiles that share one
     int32_t prefix, ctx_len;   // of the sequence (copied here so that a role needs one load per item)
     int32_t page_lo;           // first page of the sequence any row of the item can see (sliding window; 0 without
                                // one): pages below it are neither fetched nor multiplied
-    int32_t pad;               // 80 bytes: five 16-byte words
+    int32_t pad;               // pair items (two CTAs, four q tiles): offset of the second CTA's partial slots from
+                               // part_slot[]; 0 otherwise.  80 bytes: five 16-byte words
 };
 static_assert(sizeof(PrefillTcItem) == 80, "PrefillTcItem is copied as five 16-byte words");
 
@@ -89,6 +90,8 @@ struct PlanConfig {
     int32_t prefill_sms_mixed = 0;    // > 0: SMs the prefill items are balanced over when the batch also holds decode
                                       // work (spatial launch sequence: the first prefill grid's share); 0: num_sms
     int32_t prefill_force_split = 0;  // >= 2: split every tcgen05 item that many ways (tests); 0: cost model decides
+    bool prefill_pair = false;        // plan for the two-CTA kernel where the geometry allows it (head_dim 128, group
+                                      // size a multiple of 4): an item carries four heads, the machine has num_sms / 2 slots
 };
 
 struct Plan {
@@ -104,6 +107,7 @@ struct Plan {
     int32_t total_q = 0;
     int32_t n_decode_seqs = 0;
     int32_t n_prefill_seqs = 0;
+    bool pair = false;                // prefill_tc items are pair items (four q tiles, two CTAs)
 };
 
 // Validates geometry (supported head_dim / block_size / group / strides).

@@ -179,6 +179,18 @@ def test_kv_split_of_the_last_prefill_wave():
     # 128 equal items on 148 SMs: splitting would not pay for its partial traffic
     counts = cf.cf_plan_inspect(d, [6656, 6656], [512, 512], 4096, 148, want_counts=True)[5]
     assert counts[5] == 0 and counts[4] == 128
+    # on pairs of SMs: 128 four-head items on 74 pairs leave a last wave of 54, cut into KV ranges; two combine
+    # items (one per CTA of the pair) per split item; every (row, head) still has exactly one range from tile 0
+    st, dec, comb, pre, parts, counts = cf.cf_plan_inspect(d, lc, lq, 4096, 148, want_counts=True, prefill_pairs=1)
+    assert counts[5] == 2 * (128 % 74)
+    k = (counts[4] - (128 - 54)) // 54
+    assert k >= 2 and counts[4] == (128 - 54) + 54 * k
+    cover = np.zeros((2048, 32), dtype=np.int32)
+    for _, q_row0, row0, n_rows, head, kvh, j0, j1 in pre:
+        assert kvh == head // 4
+        if j0 == 0:
+            cover[row0:row0 + n_rows, head] += 1
+    assert (cover == 1).all()
 
 
 def test_few_items_are_cut_into_kv_ranges():
@@ -188,6 +200,8 @@ def test_few_items_are_cut_into_kv_ranges():
     lc, lq = np.array([8192 + 512], np.int32), np.array([512], np.int32)
     counts = cf.cf_plan_inspect(d, lc, lq, 8192, 148, want_counts=True)[5]
     assert counts[5] > 0 and 96 <= counts[4] <= 148
+    counts = cf.cf_plan_inspect(d, lc, lq, 8192, 148, want_counts=True, prefill_pairs=1)[5]          # pairs: 8 four-head items for 74 pairs
+    assert counts[5] > 0 and 48 <= counts[4] <= 74
     _, _, whole = cf.cf_estimate_us(d, lc, lq, 8192, num_sms=148)
     assert whole < 0.6 * (8 + 1.9 * 68)                 # well under the time of one unsplit item
 
@@ -199,7 +213,7 @@ def test_forced_kv_split_tiles_every_item():
     lc, lq = [3100 + 700, 50], [700, 1]
     for k in (2, 3, 8):
         st, dec, comb, pre, parts, counts = cf.cf_plan_inspect(d, lc, lq, 4096, 148, prefill_force_split=k, want_counts=True)
-        assert counts[5] > 0 and counts[4] > counts[5]
+        assert counts[5] > 0 and counts[4] >= counts[5]       # (pairs of SMs: two combine items per split item)
         by_tile = {}
         for _, q_row0, row0, n_rows, head, kvh, j0, j1 in pre:
             by_tile.setdefault((row0, head), []).append((j0, j1))

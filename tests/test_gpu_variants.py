@@ -307,3 +307,53 @@ def test_shared_prefix_with_many_chunks_and_the_separate_combine_kernel():
     assert np.array_equal(outs[0][0], outs[1][0]) and np.array_equal(outs[0][1], outs[1][1])
     ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len)
     compare(outs[0][0], outs[0][1], ref_o, ref_lse)
+
+
+# ------------------------------------------------------------------ chunked prefill on pairs of SMs (opt-in kernel)
+PAIRS = {cf.CF_DEBUG_PREFILL_PAIRS: 1}
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(4, 1), (32, 8), (16, 2), (64, 8)])
+def test_pair_kernel_ragged_prefill(Hq, Hkv):
+    """The two-CTA prefill kernel (four heads of a group per work item, K/V tiles split between two SMs) on ragged
+    chunks: group sizes 4 and 8, chunks shorter than a tile, without a prefix, ending in the middle of a page."""
+    prefix = [0, 0, 5, 16, 63, 64, 100, 1000, 0, 333, 2000]
+    qlen = [2, 64, 65, 17, 1, 128, 129, 200, 300, 31, 700]
+    sc = small(5, Hq, Hkv, 128, prefix, [qlen])
+    g = GpuScenario(sc, debug=PAIRS)
+    g.append(sc.batches[0])
+    g.attend(sc.batches[0])
+    assert cf.cf_get_last_plan_counts(g.ctx)[7] == 1          # the plan really was a pair plan
+    g.close()
+    run_and_check(sc, debug=PAIRS)
+
+
+def test_pair_kernel_mixed_batches_kv_split_window_and_sinks():
+    mixed = small(8, 32, 8, 128, [3000, 700, 9000, 50, 0], [[1, 300, 1, 1, 130]])
+    run_and_check(mixed, debug=PAIRS)
+    for split in (2, 3):
+        run_and_check(small(7, 32, 8, 128, [2000, 0, 700, 4097, 300], [[300, 700, 129, 64, 1]]),
+                      debug={**PAIRS, cf.CF_DEBUG_PREFILL_SPLIT: split})
+    run_and_check(small(9, 32, 8, 128, [3000, 700, 100], [[300, 700, 64]]), window=300, sinks=sink_values(32, 7), debug=PAIRS)
+    # more items than pairs of SMs (11 x 8 + 2 x 8 = 104 four-head items for 74 pairs), in the serial and the spatial sequence
+    many = small(41, 32, 8, 128, [700, 40, 5000, 300, 17], [[1300, 130, 1, 1, 1]])
+    b = many.batches[0]
+    g = GpuScenario(many, debug={**PAIRS, cf.CF_DEBUG_PREFILL_SPLIT: 1})
+    g.append(b)
+    outs = []
+    for mode in (0, 1, 10):
+        cf.cf_set_overlap(g.ctx, mode)
+        outs.append(g.attend(b))
+    for o, l in outs[1:]:
+        assert np.array_equal(o, outs[0][0]) and np.array_equal(l, outs[0][1])
+    k_ref, v_ref = g.pools_host()
+    rows = syn.tile_edge_rows(b)
+    ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len, rows=rows)
+    compare(outs[0][0], outs[0][1], ref_o, ref_lse, rows=rows)
+    assert cf.cf_get_async_status(g.ctx) == cf.CF_OK
+    g.close()
+
+
+def test_pair_kernel_chat_configuration_at_full_size():
+    sc = syn.config3_chat(iterations=(0, 3))
+    run_and_check(sc, tile_rows=True, check_append=False, debug=PAIRS)
