@@ -55,7 +55,12 @@ def _load():
         i32, i64, f64, vp = ctypes.c_int32, ctypes.c_int64, ctypes.c_double, ctypes.c_void_p
         lib.cf_oracle_mixed_attention.restype = ctypes.c_int
         lib.cf_oracle_mixed_attention.argtypes = [vp, vp, vp, i64, i64, i64, i64, i64, i64, vp, i32, vp, vp, i32,
-                                                  i32, i32, i32, i32, f64, vp, i64, vp, vp, vp, i64, i32, vp]
+                                                  i32, i32, i32, i32, f64, vp, i64, vp, vp, vp, i64, i32, vp, i32, vp, vp]
+        lib.cf_oracle_kv_append_fp8.restype = ctypes.c_int
+        lib.cf_oracle_kv_append_fp8.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, vp, vp, i32, vp, vp, i32,
+                                                i32, i32, i32, vp, vp]
+        lib.cf_oracle_e4m3_decode.argtypes = [vp, i64, vp]
+        lib.cf_oracle_e4m3_encode.argtypes = [vp, i64, vp]
         lib.cf_oracle_kv_append.restype = ctypes.c_int
         lib.cf_oracle_kv_append.argtypes = [vp, vp, i64, i64, i64, i64, i64, i64, vp, vp, vp, i32, vp, vp, i32,
                                             i32, i32, i32]
@@ -73,9 +78,10 @@ def _ptr(a: Optional[np.ndarray]):
 
 
 def _pool_strides(pool: np.ndarray) -> Tuple[int, int, int]:
-    """Element strides (block, head, token) of a [NB, Hkv, B, D] uint16 pool view."""
-    assert pool.dtype == np.uint16 and pool.ndim == 4 and pool.strides[3] == 2
-    return pool.strides[0] // 2, pool.strides[1] // 2, pool.strides[2] // 2
+    """Element strides (block, head, token) of a [NB, Hkv, B, D] pool view (uint16: bf16 bits; uint8: e4m3 codes)."""
+    es = pool.dtype.itemsize
+    assert pool.dtype in (np.uint16, np.uint8) and pool.ndim == 4 and pool.strides[3] == es
+    return pool.strides[0] // es, pool.strides[1] // es, pool.strides[2] // es
 
 
 def _base(pool: np.ndarray) -> ctypes.c_void_p:
@@ -85,12 +91,14 @@ def _base(pool: np.ndarray) -> ctypes.c_void_p:
 def mixed_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, block_table: np.ndarray,
                     context_len: np.ndarray, query_len: np.ndarray, scale: Optional[float] = None,
                     rows: Optional[np.ndarray] = None, want_weights: int = 0, window: int = 0,
-                    sinks: Optional[np.ndarray] = None):
+                    sinks: Optional[np.ndarray] = None, k_scale: Optional[np.ndarray] = None,
+                    v_scale: Optional[np.ndarray] = None):
     """fp64 paged attention.  q: uint16 [T, Hq, D]; pools: uint16 [NB, Hkv, B, D] (any strides with
     a contiguous last axis).  Returns (out [n, Hq, D], lse [n, Hq]) and, if want_weights > 0, the
     softmax weights [n, Hq, want_weights].
     window > 0: sliding window (the query at position p sees keys (p - window, p]); sinks: per-query-head
-    logits [Hq] that join the softmax denominator only (see the header of cf_oracle.c)."""
+    logits [Hq] that join the softmax denominator only (see the header of cf_oracle.c).
+    uint8 pools hold e4m3 codes and need k_scale / v_scale (per KV head, [Hkv])."""
     lib = _load()
     q = np.ascontiguousarray(q, dtype=np.uint16)
     T, Hq, D = q.shape
@@ -112,21 +120,62 @@ def mixed_attention(q: np.ndarray, k_pool: np.ndarray, v_pool: np.ndarray, block
     if sinks is not None:
         sinks = np.ascontiguousarray(sinks, dtype=np.float64)
         assert sinks.shape == (Hq,)
+    fp8 = k_pool.dtype == np.uint8
+    assert v_pool.dtype == k_pool.dtype
+    if fp8:
+        k_scale = np.ascontiguousarray(k_scale, dtype=np.float64)
+        v_scale = np.ascontiguousarray(v_scale, dtype=np.float64)
+        assert k_scale.shape == (Hkv,) and v_scale.shape == (Hkv,)
     ks, vs = _pool_strides(k_pool), _pool_strides(v_pool)
     rc = lib.cf_oracle_mixed_attention(
         _ptr(q), _base(k_pool), _base(v_pool), ks[0], ks[1], ks[2], vs[0], vs[1], vs[2],
         _ptr(bt), bt.shape[1], _ptr(lc), _ptr(lq), S, Hq, Hkv, D, B,
         float(1.0 / math.sqrt(D) if scale is None else scale),
-        _ptr(rows), n, _ptr(out), _ptr(lse), _ptr(w), want_weights, int(window), _ptr(sinks))
+        _ptr(rows), n, _ptr(out), _ptr(lse), _ptr(w), want_weights, int(window), _ptr(sinks),
+        int(fp8), _ptr(k_scale) if fp8 else None, _ptr(v_scale) if fp8 else None)
     if rc != 0:
         raise ValueError(f"cf_oracle_mixed_attention rejected its arguments (code {rc})")
     return (out, lse, w) if want_weights else (out, lse)
 
 
+def e4m3_decode(codes: np.ndarray) -> np.ndarray:
+    codes = np.ascontiguousarray(codes, dtype=np.uint8)
+    out = np.empty(codes.shape, dtype=np.float64)
+    _load().cf_oracle_e4m3_decode(_ptr(codes), codes.size, _ptr(out))
+    return out
+
+
+def e4m3_encode(x: np.ndarray) -> np.ndarray:
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    out = np.empty(x.shape, dtype=np.uint8)
+    _load().cf_oracle_e4m3_encode(_ptr(x), x.size, _ptr(out))
+    return out
+
+
 def kv_append(k_pool: np.ndarray, v_pool: np.ndarray, k_new: np.ndarray, v_new: np.ndarray,
-              block_table: np.ndarray, context_len: np.ndarray, query_len: np.ndarray) -> None:
-    """In-place scatter of the new rows (uint16 [T, Hkv, D]) into the pools."""
+              block_table: np.ndarray, context_len: np.ndarray, query_len: np.ndarray,
+              k_scale: Optional[np.ndarray] = None, v_scale: Optional[np.ndarray] = None) -> None:
+    """In-place scatter of the new rows (uint16 [T, Hkv, D]) into the pools; uint8 pools are fp8 caches and the
+    rows are quantised with the per-head scales (see the header of cf_oracle.c)."""
     lib = _load()
+    if k_pool.dtype == np.uint8:
+        k_new = np.ascontiguousarray(k_new, dtype=np.uint16)
+        v_new = np.ascontiguousarray(v_new, dtype=np.uint16)
+        NB, Hkv, B, D = k_pool.shape
+        bt = np.ascontiguousarray(block_table, dtype=np.int32)
+        lc = np.ascontiguousarray(context_len, dtype=np.int32)
+        lq = np.ascontiguousarray(query_len, dtype=np.int32)
+        ksc = np.ascontiguousarray(k_scale, dtype=np.float32)
+        vsc = np.ascontiguousarray(v_scale, dtype=np.float32)
+        assert ksc.shape == (Hkv,) and vsc.shape == (Hkv,) and v_pool.dtype == np.uint8
+        assert k_new.shape == (int(lq.sum()), Hkv, D) and v_new.shape == k_new.shape
+        ks, vs = _pool_strides(k_pool), _pool_strides(v_pool)
+        rc = lib.cf_oracle_kv_append_fp8(_base(k_pool), _base(v_pool), ks[0], ks[1], ks[2], vs[0], vs[1], vs[2],
+                                         _ptr(k_new), _ptr(v_new), _ptr(bt), bt.shape[1], _ptr(lc), _ptr(lq),
+                                         lc.shape[0], Hkv, D, B, _ptr(ksc), _ptr(vsc))
+        if rc != 0:
+            raise ValueError(f"cf_oracle_kv_append_fp8 rejected its arguments (code {rc})")
+        return
     k_new = np.ascontiguousarray(k_new, dtype=np.uint16)
     v_new = np.ascontiguousarray(v_new, dtype=np.uint16)
     NB, Hkv, B, D = k_pool.shape

@@ -492,3 +492,101 @@ def test_variant_weights_vanish_left_of_the_window():
     v2[first_page] = 0x7F80
     o2, lse2 = oracle.mixed_attention(b.q, k2, v2, b.block_table, b.context_len, b.query_len, window=12, sinks=sinks)
     assert np.array_equal(o, o2) and np.array_equal(lse, lse2)
+
+
+# ------------------------------------------------------------------ variant: fp8 (e4m3) KV cache
+def test_e4m3_decode_matches_the_library_type_for_every_code():
+    codes = np.arange(256, dtype=np.uint8)
+    mine = oracle.e4m3_decode(codes)
+    lib = torch.from_numpy(codes.copy()).view(torch.float8_e4m3fn).to(torch.float64).numpy()
+    nan = np.isnan(lib)
+    assert list(np.nonzero(nan)[0]) == [0x7F, 0xFF] and np.isnan(mine[nan]).all()
+    assert np.array_equal(mine[~nan], lib[~nan])
+    assert mine[0x7E] == 448.0 and mine[0x01] == 2.0 ** -9 and mine[0x08] == 2.0 ** -6       # the format's corner values
+
+
+def test_e4m3_encode_rounds_to_nearest_even_and_saturates():
+    rng = np.random.default_rng(5)
+    x = np.concatenate([rng.normal(0, 1, 20000), rng.normal(0, 100, 20000), rng.uniform(-0.02, 0.02, 20000),
+                        # every representable value and every midpoint between neighbours (the ties)
+                        oracle.e4m3_decode(np.arange(0x7F, dtype=np.uint8)),
+                        (oracle.e4m3_decode(np.arange(0x7E, dtype=np.uint8)) + oracle.e4m3_decode(np.arange(1, 0x7F, dtype=np.uint8))) / 2,
+                        [0.0, -0.0, 447.9, 448.0, 463.9]]).astype(np.float32)
+    x = np.concatenate([x, -x])
+    mine = oracle.e4m3_encode(x)
+    lib = torch.from_numpy(x).to(torch.float8_e4m3fn).view(torch.uint8).numpy()        # the library's cast: nearest even inside the range
+    assert np.array_equal(mine, lib)
+    # nearest: no other code is closer (brute force over the whole grid)
+    grid = oracle.e4m3_decode(np.arange(0x7F, dtype=np.uint8))
+    sample = np.abs(x[:2000]).astype(np.float64)
+    best = np.abs(sample[:, None] - grid[None, :]).min(axis=1)
+    assert np.allclose(np.abs(oracle.e4m3_decode(mine[:2000] & 0x7F) - sample), best, rtol=0, atol=0)
+    # beyond the largest finite value the library's cast gives NaN; this one saturates
+    big = np.array([464.0, 500.0, 1e9, -480.0, np.inf, -np.inf], dtype=np.float32)
+    assert list(oracle.e4m3_encode(big)) == [0x7E, 0x7E, 0x7E, 0xFE, 0x7E, 0xFE]
+    assert oracle.e4m3_encode(np.array([np.nan], dtype=np.float32))[0] == 0x7F
+
+
+def _fp8_case(seed=21):
+    sc = small_scenario(seed, 8, 2, 64, prefix=[40, 3, 0, 77], qlens=[[1, 25, 17, 1]])
+    b = sc.batches[0]
+    k8 = np.zeros(sc.k_pool.shape, dtype=np.uint8)
+    v8 = np.zeros(sc.v_pool.shape, dtype=np.uint8)
+    return sc, b, k8, v8
+
+
+def test_fp8_append_matches_a_python_loop():
+    sc, b, k8, v8 = _fp8_case()
+    k_scale, v_scale = np.array([0.5, 0.013], dtype=np.float32), np.array([2.0, 0.3], dtype=np.float32)
+    k8[...] = 0xAA
+    v8[...] = 0x55
+    oracle.kv_append(k8, v8, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len, k_scale, v_scale)
+    want_k, want_v = np.full_like(k8, 0xAA), np.full_like(v8, 0x55)
+    kn, vn = syn.bf16_bits_to_f32(b.k_new), syn.bf16_bits_to_f32(b.v_new)
+    row = 0
+    for s in range(b.num_seqs):
+        P = int(b.context_len[s] - b.query_len[s])
+        for i in range(int(b.query_len[s])):
+            blk, slot = b.block_table[s, (P + i) // 16], (P + i) % 16
+            for g in range(2):
+                want_k[blk, g, slot] = oracle.e4m3_encode((kn[row, g] / k_scale[g]).astype(np.float32))
+                want_v[blk, g, slot] = oracle.e4m3_encode((vn[row, g] / v_scale[g]).astype(np.float32))
+            row += 1
+    assert np.array_equal(k8, want_k) and np.array_equal(v8, want_v)
+
+
+def test_fp8_cache_reduces_to_the_bf16_path_when_the_values_fit():
+    """With power-of-two scales every dequantised value e4m3(code) * scale is exactly a bf16 number: the fp8 read
+    path must give the bits of the (already pinned) bf16 path on a pool that holds those values."""
+    sc, b, k8, v8 = _fp8_case()
+    rng = np.random.default_rng(3)
+    codes = rng.integers(0, 256, size=k8.shape, dtype=np.uint8)
+    codes[(codes & 0x7F) == 0x7F] = 0x10                       # no NaN codes
+    k8[...] = codes
+    v8[...] = rng.permutation(codes.reshape(-1)).reshape(codes.shape)
+    k_scale, v_scale = np.array([0.25, 4.0]), np.array([1.0, 0.125])
+    o8, lse8 = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len, k_scale=k_scale, v_scale=v_scale,
+                                      window=20, sinks=np.linspace(-1, 1, 8))
+    kb = syn.f32_to_bf16_bits((oracle.e4m3_decode(k8) * k_scale[None, :, None, None]).astype(np.float32))
+    vb = syn.f32_to_bf16_bits((oracle.e4m3_decode(v8) * v_scale[None, :, None, None]).astype(np.float32))
+    assert np.array_equal(syn.bf16_bits_to_f64(kb), oracle.e4m3_decode(k8) * k_scale[None, :, None, None])   # exact in bf16
+    ob, lseb = oracle.mixed_attention(b.q, kb, vb, b.block_table, b.context_len, b.query_len, window=20, sinks=np.linspace(-1, 1, 8))
+    assert np.array_equal(o8, ob) and np.array_equal(lse8, lseb)
+
+
+def test_fp8_scales_are_per_kv_head():
+    """Doubling one KV head's k_scale is the same as doubling the softmax scale for its query heads only; doubling
+    v_scale doubles those heads' outputs."""
+    sc, b, k8, v8 = _fp8_case()
+    rng = np.random.default_rng(9)
+    k8[...] = rng.integers(0x20, 0x50, size=k8.shape, dtype=np.uint8)
+    v8[...] = rng.integers(0x20, 0x50, size=v8.shape, dtype=np.uint8)
+    base = dict(k_scale=np.array([1.0, 1.0]), v_scale=np.array([1.0, 1.0]))
+    o0, _ = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len, **base)
+    o1, _ = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len, k_scale=np.array([1.0, 1.0]),
+                                   v_scale=np.array([1.0, 2.0]))
+    assert np.array_equal(o1[:, :4], o0[:, :4]) and np.array_equal(o1[:, 4:], 2.0 * o0[:, 4:])
+    o2, _ = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len, k_scale=np.array([2.0, 1.0]),
+                                   v_scale=np.array([1.0, 1.0]))
+    o3, _ = oracle.mixed_attention(b.q, k8, v8, b.block_table, b.context_len, b.query_len, scale=2.0 / 8.0, **base)
+    assert np.array_equal(o2[:, 4:], o0[:, 4:]) and np.abs(o2[:, :4] - o3[:, :4]).max() < 1e-13
