@@ -78,7 +78,20 @@ typedef struct {
      *       out = sum_j exp(x_j) v_j / (exp(sink_h) + sum_j exp(x_j)),  lse = ln(exp(sink_h) + sum_j exp(x_j)). */
     int32_t window_size;
     const float* sink_logits;
+    /* Precision of the cache (the paper does not state the KV precision of its runs, Section 6.1).
+     *   kv_dtype = CF_KV_BF16 (0): the pools hold bf16.
+     *   kv_dtype = CF_KV_FP8_E4M3 (1): the pools hold e4m3 codes (one byte per element; strides in elements are then
+     *     strides in bytes and must be multiples of 16; head_dim must be 128) with one fp32 scale per KV head:
+     *     a cached value reads as e4m3(code) * k_scale[g] (v_scale[g]).  cf_kv_append stores
+     *     e4m3_rne_sat((float)x / scale[g]) (IEEE fp32 division, nearest-even, saturating at +-448).  Halves the bytes
+     *     decode has to stream.  k_scale, v_scale: DEVICE fp32 [num_kv_heads].  Attention reads the codes exactly
+     *     (e4m3 -> fp16 / bf16 is exact) and applies the scales in fp32; prefill chunks first expand the pages they
+     *     need into a bf16 staging area inside the workspace.  Not available through cf_decode_attention_static. */
+    int32_t kv_dtype;
+    const float* k_scale;
+    const float* v_scale;
 } cf_cache_desc;
+enum { CF_KV_BF16 = 0, CF_KV_FP8_E4M3 = 1 };
 
 /* Create a context on `device`.  workspace_bytes = 0: the split-K workspace starts at a default
  * size and grows when a batch needs more (growth allocates and synchronises the device);

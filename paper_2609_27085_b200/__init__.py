@@ -32,6 +32,9 @@ CF_ERR_TIMEOUT = 6
 CF_ERR_ARCH = 7
 CF_ERR_BUSY = 8
 
+CF_KV_BF16 = 0
+CF_KV_FP8_E4M3 = 1
+
 # cf_debug_option (test-only switches)
 CF_DEBUG_PREFILL_SPLIT = 0
 CF_DEBUG_SEPARATE_COMBINE = 1
@@ -53,7 +56,8 @@ class CacheDesc(ctypes.Structure):
                 ("block_size", ctypes.c_int32), ("num_blocks", ctypes.c_int32),
                 ("k_stride_block", ctypes.c_int64), ("k_stride_head", ctypes.c_int64), ("k_stride_token", ctypes.c_int64),
                 ("v_stride_block", ctypes.c_int64), ("v_stride_head", ctypes.c_int64), ("v_stride_token", ctypes.c_int64),
-                ("softmax_scale", ctypes.c_float), ("window_size", ctypes.c_int32), ("sink_logits", ctypes.c_void_p)]
+                ("softmax_scale", ctypes.c_float), ("window_size", ctypes.c_int32), ("sink_logits", ctypes.c_void_p),
+                ("kv_dtype", ctypes.c_int32), ("k_scale", ctypes.c_void_p), ("v_scale", ctypes.c_void_p)]
 
 
 class PlanOptions(ctypes.Structure):
@@ -145,16 +149,19 @@ def _stream(stream) -> Optional[int]:
 
 def make_desc(num_q_heads: int, num_kv_heads: int, head_dim: int, block_size: int, num_blocks: int,
               k_strides: Optional[Tuple[int, int, int]] = None, v_strides: Optional[Tuple[int, int, int]] = None,
-              softmax_scale: float = 0.0, window_size: int = 0, sink_logits=None) -> CacheDesc:
+              softmax_scale: float = 0.0, window_size: int = 0, sink_logits=None, kv_dtype: int = 0, k_scale=None,
+              v_scale=None) -> CacheDesc:
     """Descriptor for pools laid out [num_blocks, num_kv_heads, block_size, head_dim] unless
     (block, head, token) element strides are given.  window_size > 0: sliding-window attention;
     sink_logits: device fp32 tensor [num_q_heads] (or address) of per-head sink logits.  The caller keeps
-    the sink tensor alive for as long as the descriptor is used."""
+    the sink tensor alive for as long as the descriptor is used.  kv_dtype = CF_KV_FP8_E4M3: the pools hold e4m3
+    codes (one byte per element) and k_scale / v_scale are device fp32 tensors [num_kv_heads]."""
     default = (num_kv_heads * block_size * head_dim, block_size * head_dim, head_dim)
     ks = k_strides or default
     vs = v_strides or default
     return CacheDesc(num_q_heads, num_kv_heads, head_dim, block_size, num_blocks,
-                     ks[0], ks[1], ks[2], vs[0], vs[1], vs[2], softmax_scale, int(window_size), _dev(sink_logits))
+                     ks[0], ks[1], ks[2], vs[0], vs[1], vs[2], softmax_scale, int(window_size), _dev(sink_logits),
+                     int(kv_dtype), _dev(k_scale), _dev(v_scale))
 
 
 def cf_create(device: int = 0, workspace_bytes: int = 0) -> ctypes.c_void_p:

@@ -122,6 +122,8 @@ struct cf_plan {
     uint8_t* dev = nullptr;
     float* part = nullptr;         // this plan's own split-K partials
     int n_part_slots = 0, n_pre_slots = 0;
+    size_t off_stage = 0;
+    int n_stage_seqs = 0, n_stage_pages = 0, max_stage_pages = 0;
     size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_sh = 0, off_shm = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     bool pair = false;
@@ -194,10 +196,10 @@ static cf_status ensure_workspace(cf_ctx* c, size_t need)
 
 // Layout of one uploaded plan: [q_start S+1][context_len S][query_len S][decode][combine][prefill]
 struct PlanLayout {
-    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_sh, off_shm, off_pre_tc, off_pre_comb, off_queue, total;
+    size_t off_qstart, off_ctx, off_qlen, off_dec, off_comb, off_sh, off_shm, off_pre_tc, off_pre_comb, off_stage, off_queue, total;
 };
 
-static PlanLayout layout_of(int32_t S, const Plan& pl)
+static PlanLayout layout_of(int32_t S, const Plan& pl, size_t n_stage_seqs = 0)
 {
     PlanLayout L;
     size_t at = 0;
@@ -210,6 +212,7 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
     L.off_shm = at;    at = align_up(at + sizeof(ShareMember) * pl.share_members.size(), 16);
     L.off_pre_tc = at; at = align_up(at + sizeof(PrefillTcItem) * pl.prefill_tc.size(), 16);
     L.off_pre_comb = at; at = align_up(at + sizeof(PrefillCombineItem) * pl.prefill_combine.size(), 16);
+    L.off_stage = at;  at = align_up(at + sizeof(StageSeq) * n_stage_seqs, 16);
     L.off_queue = at;  at += 16;   // ticket counter + exit counter of the persistent prefill CTAs; uploaded as zeros
     L.total = at;
     return L;
@@ -217,9 +220,10 @@ static PlanLayout layout_of(int32_t S, const Plan& pl)
 
 // Copies the plan into the next pinned slot and enqueues its upload.  Returns the device base.
 static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, const int32_t* query_len,
-                             const Plan& pl, cudaStream_t stream, PlanLayout* L, uint8_t** dev_base, PlanSlot** slot_out)
+                             const Plan& pl, cudaStream_t stream, PlanLayout* L, uint8_t** dev_base, PlanSlot** slot_out,
+                             const std::vector<StageSeq>* stage = nullptr)
 {
-    *L = layout_of(S, pl);
+    *L = layout_of(S, pl, stage ? stage->size() : 0);
     cf_status st = ensure_plan_capacity(c, L->total);
     if (st != CF_OK) return st;
     PlanSlot& s = c->slots[c->next_slot];
@@ -240,6 +244,7 @@ static cf_status upload_plan(cf_ctx* c, int32_t S, const int32_t* context_len, c
         std::memcpy(s.host + L->off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
     if (!pl.prefill_combine.empty())
         std::memcpy(s.host + L->off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
+    if (stage && !stage->empty()) std::memcpy(s.host + L->off_stage, stage->data(), sizeof(StageSeq) * stage->size());
     std::memset(s.host + L->off_queue, 0, 16);
     // The copy does not go on the caller's stream: there it would start only when that stream's earlier
     // kernels are done (a few microseconds of copy-engine latency between kernels, every call) and, queued in
@@ -345,6 +350,7 @@ namespace cf {
 
 struct PlanCounts {
     int n_dec = 0, n_comb = 0, n_shared = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
+    int n_stage_seqs = 0, n_stage_pages = 0, max_stage_pages = 0, num_seqs = 0;   // fp8 cache: pages to expand for the prefill chunks
     bool pair = false;          // the prefill items are pair items (two CTAs each)
     float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
     int n_part_slots = 0;
@@ -352,18 +358,48 @@ struct PlanCounts {
 
 // Split-K workspace: the ticket counters, decode partials [slot, Hq, D] + [slot, Hq, 2], then the compact
 // partial rows of KV-split prefill items [row slot, D] + [row slot, 2].
+// For an fp8 cache the workspace also holds the bf16 staging pools of the prefill chunks' pages (K and V,
+// [stage page, Hkv, 16, D]) and the staging block table [S, max_blocks].
 struct WsLayout {
-    size_t dec_o = 0, dec_ml = 0, pre_o = 0, pre_ml = 0, total = 0;
+    size_t dec_o = 0, dec_ml = 0, pre_o = 0, pre_ml = 0, stage_k = 0, stage_v = 0, stage_bt = 0, total = 0;
 };
-static WsLayout ws_layout(int n_part_slots, int n_pre_slots, int Hq, int D)
+static WsLayout ws_layout(int n_part_slots, int n_pre_slots, int Hq, int D, int n_stage_pages = 0, int Hkv = 0, int64_t table_entries = 0)
 {
     WsLayout w;
     w.dec_o = kCounterBytes;
     w.dec_ml = w.dec_o + align_up((size_t)n_part_slots * Hq * D * sizeof(float), 256);
     w.pre_o = w.dec_ml + align_up((size_t)n_part_slots * Hq * 2 * sizeof(float), 256);
     w.pre_ml = w.pre_o + align_up((size_t)n_pre_slots * D * sizeof(float), 256);
-    w.total = w.pre_ml + align_up((size_t)n_pre_slots * 2 * sizeof(float), 256);
+    w.stage_k = w.pre_ml + align_up((size_t)n_pre_slots * 2 * sizeof(float), 256);
+    const size_t pool = n_stage_pages > 0 ? align_up((size_t)n_stage_pages * Hkv * 16 * D * 2, 1024) : 0;
+    w.stage_v = w.stage_k + pool;
+    w.stage_bt = w.stage_v + pool;
+    w.total = w.stage_bt + (n_stage_pages > 0 ? align_up((size_t)table_entries * sizeof(int32_t), 256) : 0);
     return w;
+}
+
+// fp8 cache: which pages of which prefill sequences have to be expanded to bf16 for the prefill kernel (from the first
+// page any row of the chunk can see - 0 without a sliding window - to the last page of the context)
+static void stage_list(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, int32_t S,
+                       std::vector<StageSeq>* seqs, int* n_pages, int* max_pages)
+{
+    seqs->clear();
+    *n_pages = 0;
+    *max_pages = 0;
+    if (d->kv_dtype != CF_KV_FP8_E4M3) return;
+    for (int32_t s = 0; s < S; ++s) {
+        if (query_len[s] <= 1) continue;
+        const int32_t prefix = context_len[s] - query_len[s];
+        const int32_t lo = d->window_size > 0 ? std::max(0, prefix - d->window_size + 1) : 0;
+        StageSeq q;
+        q.seq = s;
+        q.page0 = lo / 16;
+        q.n_pages = (context_len[s] + 15) / 16 - q.page0;
+        q.stage_base = *n_pages;
+        *n_pages += q.n_pages;
+        *max_pages = std::max(*max_pages, q.n_pages);
+        seqs->push_back(q);
+    }
 }
 
 // Enqueues decode -> combine -> prefill for a plan that already sits in device memory at `base`.
@@ -388,6 +424,9 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     p.scale_log2 = scale_log2_of(desc);
     p.window = desc->window_size;
     p.sinks = desc->sink_logits;
+    const bool fp8 = desc->kv_dtype == CF_KV_FP8_E4M3;
+    p.k_scale = fp8 ? desc->k_scale : nullptr;
+    p.v_scale = fp8 ? desc->v_scale : nullptr;
     p.q_start = (const int32_t*)(base + L.off_qstart);
     p.context_len = (const int32_t*)(base + L.off_ctx);
     p.query_len = (const int32_t*)(base + L.off_qlen);
@@ -422,14 +461,41 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         tc->ran[2] = n.n_pre_tc > 0;
     }
     const bool has_prefill = n.n_pre_tc > 0;
+    // the prefill kernels' view of the cache: the caller's pools, or (fp8 cache) the bf16 staging pools in the workspace
+    AttnParams pp = p;
+    cf_cache_desc pdesc = *desc;
+    if (fp8 && has_prefill) {
+        pp.k_cache = (const __nv_bfloat16*)((uint8_t*)ws + W.stage_k);
+        pp.v_cache = (const __nv_bfloat16*)((uint8_t*)ws + W.stage_v);
+        pp.block_table = (const int32_t*)((uint8_t*)ws + W.stage_bt);
+        pp.num_blocks = n.n_stage_pages;
+        pdesc.num_blocks = n.n_stage_pages;
+        pdesc.k_stride_block = pdesc.v_stride_block = (int64_t)desc->num_kv_heads * 16 * D;
+        pdesc.k_stride_head = pdesc.v_stride_head = 16 * D;
+        pdesc.k_stride_token = pdesc.v_stride_token = D;
+        pp.ks_block = pp.vs_block = pdesc.k_stride_block;
+        pp.ks_head = pp.vs_head = pdesc.k_stride_head;
+        pp.ks_token = pp.vs_token = pdesc.k_stride_token;
+    }
     PrefillMaps maps;
     if (has_prefill) {
         const CUtensorMap* mq = q_map(c, q, D, n.total_q, Hq);
-        const CUtensorMap* mk = pool_map(c, k_cache, desc, desc->k_stride_block, desc->k_stride_head, desc->k_stride_token);
-        const CUtensorMap* mv = pool_map(c, v_cache, desc, desc->v_stride_block, desc->v_stride_head, desc->v_stride_token);
+        const CUtensorMap* mk = pool_map(c, pp.k_cache, &pdesc, pdesc.k_stride_block, pdesc.k_stride_head, pdesc.k_stride_token);
+        const CUtensorMap* mv = pool_map(c, pp.v_cache, &pdesc, pdesc.v_stride_block, pdesc.v_stride_head, pdesc.v_stride_token);
         if (!mq || !mk || !mv) return CF_ERR_CUDA;
         maps.q = *mq; maps.k = *mk; maps.v = *mv;
     }
+    // fp8 cache: the pages of the prefill chunks are expanded first, on the caller's stream (the prefill kernel behind
+    // it waits for the grid before it in the stream to complete before its first read)
+    auto stage_pages = [&](cudaStream_t st) -> cudaError_t {
+        if (!(fp8 && has_prefill)) return cudaSuccess;
+        return launch_kv_dequant_gather(p, (const StageSeq*)(base + L.off_stage), n.n_stage_seqs, n.max_stage_pages,
+                                        (__nv_bfloat16*)((uint8_t*)ws + W.stage_k), (__nv_bfloat16*)((uint8_t*)ws + W.stage_v),
+                                        (int32_t*)((uint8_t*)ws + W.stage_bt), st);
+    };
+    auto decode_launch = [&](cudaStream_t st) -> cudaError_t {
+        return fp8 ? launch_decode_fp8(p, n.n_dec, st) : launch_decode_with_shared(p, D, n.n_shared, n.n_dec, st);
+    };
     int second_grid = 0;
     // Slots that take a prefill item: SMs, or pairs of SMs for pair items.  Grid sizes, the shared work queue and
     // the front / tail split below are counted in slots.
@@ -437,8 +503,8 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
     const int sms = (c->num_sms > 0 ? c->num_sms : 148) / per_slot;
     const int pre_ctas = n.n_pre_tc < sms ? n.n_pre_tc : sms;      // persistent CTAs (pairs) of the serial sequence
     auto launch_prefill = [&](int n_slots, int queue_slots, int first_static, int ticket_base, uint32_t* resident, cudaStream_t st) {
-        return n.pair ? launch_prefill_tc2(p, maps, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st)
-                      : launch_prefill_tc(p, maps, D, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st);
+        return n.pair ? launch_prefill_tc2(pp, maps, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st)
+                      : launch_prefill_tc(pp, maps, D, n.n_pre_tc, n_slots, queue_slots, first_static, ticket_base, resident, st);
     };
     if (c->overlap && !c->in_host_step && !tc && has_prefill && (n.n_dec > 0)) {
         // Spatial partition.  `front` persistent prefill CTAs (one per SM: a CTA takes an SM's whole shared
@@ -470,6 +536,7 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
             resident = p.pre_queue + 2;
             if (mo.write(stream, (CUdeviceptr)(uintptr_t)resident, 0u, 0u) != CUDA_SUCCESS) e = cudaErrorUnknown;
         }
+        if (e == cudaSuccess) e = stage_pages(stream);      // before the fork: the second prefill grid on the side stream reads the staging area too
         if (cudaEventRecord(c->ev_fork, stream) != cudaSuccess || cudaStreamWaitEvent(c->side, c->ev_fork, 0) != cudaSuccess)
             e = cudaErrorUnknown;
         if (e == cudaSuccess) e = launch_prefill(front, front + tail, 1, front, resident, stream);
@@ -477,20 +544,21 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         if (e == cudaSuccess && resident &&
             mo.wait(c->side, (CUdeviceptr)(uintptr_t)resident, (cuuint32_t)(front * per_slot), CU_STREAM_WAIT_VALUE_GEQ) != CUDA_SUCCESS)
             e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_decode_with_shared(p, D, n.n_shared, n.n_dec, c->side);
+        if (e == cudaSuccess) e = decode_launch(c->side);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, c->side);
         if (e == cudaSuccess) e = launch_prefill(tail, front + tail, 0, front, nullptr, c->side);
         if (cudaEventRecord(c->ev_join, c->side) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
         if (cudaStreamWaitEvent(stream, c->ev_join, 0) != cudaSuccess && e == cudaSuccess) e = cudaErrorUnknown;
-        if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
+        if (e == cudaSuccess) e = launch_prefill_combine(pp, D, n.n_pre_comb, stream);
     } else {
         if (tc) cudaEventRecord(tc->ev[0], stream);
-        if (e == cudaSuccess) e = launch_decode_with_shared(p, D, n.n_shared, n.n_dec, stream);
+        if (e == cudaSuccess) e = decode_launch(stream);
         if (tc) cudaEventRecord(tc->ev[1], stream);
         if (e == cudaSuccess) e = launch_combine(p, D, fused_combine ? 0 : n.n_comb, stream);
         if (tc) cudaEventRecord(tc->ev[2], stream);
+        if (e == cudaSuccess) e = stage_pages(stream);
         if (e == cudaSuccess) e = launch_prefill(pre_ctas, pre_ctas, 1, pre_ctas, nullptr, stream);
-        if (e == cudaSuccess) e = launch_prefill_combine(p, D, n.n_pre_comb, stream);
+        if (e == cudaSuccess) e = launch_prefill_combine(pp, D, n.n_pre_comb, stream);
         if (tc) cudaEventRecord(tc->ev[3], stream);
     }
     c->launches = (int)(n.n_dec > 0) + (int)(n.n_comb > 0 && !fused_combine) + (int)(n.n_pre_tc > 0) + (int)(n.n_pre_comb > 0) + second_grid;
@@ -644,6 +712,8 @@ cf_status cf_kv_append(cf_ctx* c, const cf_cache_desc* desc, void* k_cache, void
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = num_seqs; p.total_rows = pl.total_q;
     p.num_blocks = desc->num_blocks; p.err = c->err_dev;
+    p.k_scale = desc->kv_dtype == CF_KV_FP8_E4M3 ? desc->k_scale : nullptr;
+    p.v_scale = desc->kv_dtype == CF_KV_FP8_E4M3 ? desc->v_scale : nullptr;
     p.q_start = (const int32_t*)(base + L.off_qstart);
     p.context_len = (const int32_t*)(base + L.off_ctx);
     p.query_len = (const int32_t*)(base + L.off_qlen);
@@ -692,14 +762,18 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     cudaStream_t stream = (cudaStream_t)cuda_stream;
 
     const int Hq = desc->num_q_heads, D = desc->head_dim;
-    const WsLayout W = ws_layout(pl.n_part_slots, pl.n_pre_slots, Hq, D);
+    std::vector<StageSeq> stage;
+    int n_stage_pages = 0, max_stage_pages = 0;
+    if (!pl.prefill_tc.empty()) stage_list(desc, context_len, query_len, num_seqs, &stage, &n_stage_pages, &max_stage_pages);
+    const WsLayout W = ws_layout(pl.n_part_slots, pl.n_pre_slots, Hq, D, n_stage_pages, desc->num_kv_heads,
+                                 (int64_t)num_seqs * max_blocks_per_seq);
     st = ensure_workspace(c, W.total);
     if (st != CF_OK) return st;
 
     PlanLayout L;
     uint8_t* base = nullptr;
     PlanSlot* slot = nullptr;
-    st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot);
+    st = upload_plan(c, num_seqs, context_len, query_len, pl, stream, &L, &base, &slot, &stage);
     if (st != CF_OK) return st;
 
     PlanCounts n;
@@ -707,6 +781,7 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     n.n_pre_tc = (int)pl.prefill_tc.size(); n.n_pre_comb = (int)pl.prefill_combine.size(); n.total_q = pl.total_q;
     n.n_part_slots = pl.n_part_slots;
     n.pair = pl.pair;
+    n.n_stage_seqs = (int)stage.size(); n.n_stage_pages = n_stage_pages; n.max_stage_pages = max_stage_pages; n.num_seqs = num_seqs;
     c->last_counts[0] = n.n_dec; c->last_counts[1] = n.n_comb; c->last_counts[2] = n.n_pre_tc; c->last_counts[3] = n.n_part_slots;
     c->last_counts[4] = n.n_pre_comb; c->last_counts[5] = n.n_shared; c->last_counts[6] = (int32_t)pl.share_members.size();
     c->last_counts[7] = pl.pair ? 1 : 0;
@@ -740,7 +815,12 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->desc = *desc;
     P->num_seqs = num_seqs;
     P->max_blocks = max_blocks_per_seq;
-    const PlanLayout L = layout_of(num_seqs, pl);
+    std::vector<StageSeq> stage;
+    int n_stage_pages = 0, max_stage_pages = 0;
+    if (!pl.prefill_tc.empty()) stage_list(desc, context_len, query_len, num_seqs, &stage, &n_stage_pages, &max_stage_pages);
+    const PlanLayout L = layout_of(num_seqs, pl, stage.size());
+    P->off_stage = L.off_stage;
+    P->n_stage_seqs = (int)stage.size(); P->n_stage_pages = n_stage_pages; P->max_stage_pages = max_stage_pages;
     P->off_qstart = L.off_qstart; P->off_ctx = L.off_ctx; P->off_qlen = L.off_qlen; P->off_dec = L.off_dec;
     P->off_comb = L.off_comb; P->off_sh = L.off_sh; P->off_shm = L.off_shm; P->off_pre_tc = L.off_pre_tc; P->off_pre_comb = L.off_pre_comb; P->off_queue = L.off_queue;
     P->total = L.total;
@@ -749,7 +829,8 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->pre_over_dec = prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms);
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
     P->pair = pl.pair;
-    const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim).total;
+    const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim, n_stage_pages,
+                                        desc->num_kv_heads, (int64_t)num_seqs * max_blocks_per_seq).total;
     bool ok = cudaMallocHost((void**)&P->host, L.total) == cudaSuccess && cudaMalloc((void**)&P->dev, L.total) == cudaSuccess;
     // the ticket counters are zeroed on the caller's stream, like the plan copy: every launch that uses the plan
     // is ordered behind this call on that stream (or by the caller)
@@ -767,6 +848,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
         if (P->n_pre_tc) std::memcpy(P->host + L.off_pre_tc, pl.prefill_tc.data(), sizeof(PrefillTcItem) * pl.prefill_tc.size());
         if (P->n_pre_comb)
             std::memcpy(P->host + L.off_pre_comb, pl.prefill_combine.data(), sizeof(PrefillCombineItem) * pl.prefill_combine.size());
+        if (!stage.empty()) std::memcpy(P->host + L.off_stage, stage.data(), sizeof(StageSeq) * stage.size());
         std::memset(P->host + L.off_queue, 0, 16);
         ok = cudaMemcpyAsync(P->dev, P->host, L.total, cudaMemcpyHostToDevice, (cudaStream_t)cuda_stream) == cudaSuccess;
     }
@@ -812,6 +894,8 @@ cf_status cf_kv_append_planned(cf_plan* P, void* k_cache, void* v_cache, const v
     p.vs_block = desc->v_stride_block; p.vs_head = desc->v_stride_head; p.vs_token = desc->v_stride_token;
     p.Hkv = desc->num_kv_heads; p.D = desc->head_dim; p.num_seqs = P->num_seqs; p.total_rows = P->total_q;
     p.num_blocks = desc->num_blocks; p.err = P->ctx->err_dev;
+    p.k_scale = desc->kv_dtype == CF_KV_FP8_E4M3 ? desc->k_scale : nullptr;
+    p.v_scale = desc->kv_dtype == CF_KV_FP8_E4M3 ? desc->v_scale : nullptr;
     p.q_start = (const int32_t*)(P->dev + P->off_qstart);
     p.context_len = (const int32_t*)(P->dev + P->off_ctx);
     p.query_len = (const int32_t*)(P->dev + P->off_qlen);
@@ -829,7 +913,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     if (!guard.ok) return CF_ERR_CUDA;
     PlanLayout L;
     L.off_qstart = P->off_qstart; L.off_ctx = P->off_ctx; L.off_qlen = P->off_qlen; L.off_dec = P->off_dec;
-    L.off_comb = P->off_comb; L.off_sh = P->off_sh; L.off_shm = P->off_shm; L.off_pre_tc = P->off_pre_tc; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
+    L.off_comb = P->off_comb; L.off_sh = P->off_sh; L.off_shm = P->off_shm; L.off_pre_tc = P->off_pre_tc; L.off_stage = P->off_stage; L.off_pre_comb = P->off_pre_comb; L.off_queue = P->off_queue;
     L.total = P->total;
     PlanCounts n;
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
@@ -837,7 +921,9 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     n.pre_over_dec = P->pre_over_dec;
     n.n_part_slots = P->n_part_slots;
     n.pair = P->pair;
-    const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim);
+    n.n_stage_seqs = P->n_stage_seqs; n.n_stage_pages = P->n_stage_pages; n.max_stage_pages = P->max_stage_pages; n.num_seqs = P->num_seqs;
+    const WsLayout W = ws_layout(P->n_part_slots, P->n_pre_slots, P->desc.num_q_heads, P->desc.head_dim, P->n_stage_pages,
+                                 P->desc.num_kv_heads, (int64_t)P->num_seqs * P->max_blocks);
     return launch_attention(P->ctx, &P->desc, n, L, P->dev, P->part, W, q, k_cache,
                             v_cache, block_table, P->max_blocks, out, lse, (cudaStream_t)cuda_stream, false);
 }

@@ -15,6 +15,8 @@
 //
 // Output: a sequence with a single chunk writes bf16 `out` (and lse) directly; otherwise the CTA
 // writes an fp32 partial (o, m, l) that the combine kernel merges in fixed chunk order.
+#include <cuda_fp16.h>
+
 #include <algorithm>
 #include <atomic>
 #include <mutex>
@@ -286,6 +288,282 @@ __device__ __forceinline__ void decode_cta(const AttnParams& p, const int cta)
     // Every CTA publishes its partial (fence), then takes a ticket; the one that draws the last ticket sees
     // all of them (fence again, L2 loads).  The merge walks the chunks in index order, so the result does
     // not depend on which CTA performs it; that CTA also puts the counter back to zero for the next launch.
+    if (it.part_slot >= 0 && p.dec_counters != nullptr) {
+        __shared__ int last_s;
+        __threadfence();
+        __syncthreads();
+        uint32_t* counter = p.dec_counters + (int64_t)(it.part_slot - it.chunk) * p.Hkv + kvh;
+        if (threadIdx.x == 0) last_s = (atomicAdd(counter, 1u) == (uint32_t)(it.n_chunks - 1)) ? 1 : 0;
+        __syncthreads();
+        if (last_s) {
+            __threadfence();
+            for (int idx = threadIdx.x; idx < G * (D / 4); idx += NWARPS * 32) {
+                const int head = idx / (D / 4), d = (idx % (D / 4)) * 4;
+                merge_partials<D>(p, it.q_row, it.part_slot - it.chunk, it.n_chunks, kvh * G + head, d, d == 0);
+            }
+            if (threadIdx.x == 0) *counter = 0u;
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Split-K decode over an fp8 (e4m3) cache, head_dim 128: the same work items, online softmax, partials and merge as
+// decode_splitk_kernel; a (page, head) of K or V is 2 KB instead of 4 KB, so the bytes to stream halve.
+// The codes are turned into fp16 on the way into the MMA fragments (e4m3 -> fp16 is exact) and the MMAs run in
+// fp16 with fp32 accumulation (Q is converted bf16 -> fp16 once, the probabilities are rounded to fp16); the per-head
+// scales multiply the scores (k_scale) and the output (v_scale) in fp32.
+// ldmatrix moves 16-bit elements and cannot gather bytes, so the fragments are loaded with plain 8- and 16-byte
+// shared-memory loads, which wants each thread's elements contiguous.  Both contractions allow that, because a
+// sum does not care about the order of its terms and an output row may be produced by any thread:
+//   S^T = K Q^T: the 16 k-slots of MMA step ks are mapped to head-dim elements so that thread (g, c) - g = lane / 4,
+//     c = lane % 4 - reads, per row, the 8 contiguous bytes d = 32 (ks / 2) + 8 c + 4 (ks % 2) + {0..3} for two steps;
+//     the Q fragments use the same map.
+//   O^T = V^T P^T: output row i of MMA mt is head-dim element d = 16 (i % 8) + 2 mt + (i / 8), so thread (g, c) owns
+//     d in [16 g, 16 g + 16) and reads one 16-byte chunk per token for all 8 MMAs; byte pairs of two tokens are
+//     brought together with one byte-permute.
+__device__ __forceinline__ uint32_t e4m3x2_to_f16x2(uint32_t two_codes)
+{
+    uint32_t d;
+    asm("{\n.reg .b16 lo;\ncvt.u16.u32 lo, %1;\ncvt.rn.f16x2.e4m3x2 %0, lo;\n}" : "=r"(d) : "r"(two_codes));
+    return d;
+}
+__device__ __forceinline__ void mma_f16_16816(float (&c)[4], const uint32_t (&a)[4], uint32_t b0, uint32_t b1)
+{
+    asm volatile("mma.sync.aligned.m16n8k16.row.col.f32.f16.f16.f32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};\n"
+                 : "+f"(c[0]), "+f"(c[1]), "+f"(c[2]), "+f"(c[3])
+                 : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
+}
+__device__ __forceinline__ uint32_t pack_f16(float lo, float hi)
+{
+    __half2 v = __floats2half2_rn(lo, hi);
+    return *reinterpret_cast<uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t bf16x2_to_f16x2(uint32_t v)
+{
+    const float2 f = __bfloat1622float2(*reinterpret_cast<__nv_bfloat162*>(&v));
+    return pack_f16(f.x, f.y);
+}
+
+template <int NWARPS, int NSTAGE>
+__global__ void __launch_bounds__(NWARPS * 32, 2) decode_splitk_fp8_kernel(const AttnParams p)
+{
+    constexpr int D = 128;
+    constexpr int PAGE_BYTES = 16 * D;          // one (page, head) of K or of V: 16 tokens x 128 one-byte codes
+    constexpr int STAGE_BYTES = 2 * PAGE_BYTES;
+    constexpr int WARP_BYTES = NSTAGE * STAGE_BYTES;
+    constexpr int KSTEPS = D / 16;
+    constexpr int DP = D + 4;
+    extern __shared__ __align__(1024) uint8_t smem[];
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int g = lane >> 2, c = lane & 3;
+    const int item_id = blockIdx.x / p.Hkv, kvh = blockIdx.x % p.Hkv;
+    const DecodeItem it = p.dec_items[item_id];
+    const int G = p.G;
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    const float score_scale = p.scale_log2 * __ldg(p.k_scale + kvh);
+    const float out_scale = __ldg(p.v_scale + kvh);
+
+    // ---- Q^T fragments (fp16), k-slots permuted like the K bytes: step ks, slots {2c, 2c+1 | 2c+8, 2c+9} <-> d0 + {0, 1 | 2, 3}
+    uint32_t qf[KSTEPS][2];
+    {
+        const uint32_t* qrow = reinterpret_cast<const uint32_t*>(p.q + ((int64_t)it.q_row * p.Hq + (int64_t)kvh * G + g) * D);
+#pragma unroll
+        for (int ks = 0; ks < KSTEPS; ++ks) {
+            const int d0 = 32 * (ks >> 1) + 8 * c + 4 * (ks & 1);
+            qf[ks][0] = g < G ? bf16x2_to_f16x2(__ldg(qrow + (d0 >> 1))) : 0u;
+            qf[ks][1] = g < G ? bf16x2_to_f16x2(__ldg(qrow + (d0 >> 1) + 1)) : 0u;
+        }
+    }
+
+    const int first_page = it.kv_begin >> 4;
+    const int n_pages = (it.kv_end - it.kv_begin + 15) >> 4;
+    const int my_n = n_pages > warp ? (n_pages - warp + NWARPS - 1) / NWARPS : 0;
+    const int32_t* bt = p.block_table + (int64_t)it.seq * p.max_blocks + first_page + warp;
+    const uint32_t wbase = smem_u32(smem) + warp * WARP_BYTES;
+    const uint8_t* kbase = reinterpret_cast<const uint8_t*>(p.k_cache) + (int64_t)kvh * p.ks_head;
+    const uint8_t* vbase = reinterpret_cast<const uint8_t*>(p.v_cache) + (int64_t)kvh * p.vs_head;
+
+    auto checked = [&](int32_t id) -> int32_t {
+        if ((uint32_t)id < (uint32_t)p.num_blocks) return id;
+        if (p.err) atomicOr(p.err, kErrBlockId);
+        return 0;
+    };
+    int cache_base = 0;
+    int32_t pid_cache = (lane < my_n) ? checked(__ldg(bt + lane * NWARPS)) : 0;
+    const uint64_t stream_once = l2_policy_evict_first();
+
+    // a page in shared memory: [16 tokens][128 bytes], the eight 16-byte chunks of a row XOR-swizzled by the row index
+    auto issue = [&](int i) {
+        if (i - cache_base == 32) {
+            cache_base = i;
+            pid_cache = (i + lane < my_n) ? checked(__ldg(bt + (i + lane) * NWARPS)) : 0;
+        }
+        const int32_t pid = __shfl_sync(0xffffffffu, pid_cache, i - cache_base);
+        const int tok0 = it.kv_begin + (i * NWARPS + warp) * 16;
+        const uint32_t sbase = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const uint8_t* kp = kbase + (int64_t)pid * p.ks_block;
+        const uint8_t* vp = vbase + (int64_t)pid * p.vs_block;
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+            const int id = r * 32 + lane;
+            const int t = id >> 3, ch = id & 7;
+            const bool ok = tok0 + t < it.kv_end && tok0 + t >= it.kv_lo;     // slack slots and tokens left of a window: zero-filled
+            const int tt = ok ? t : 0;
+            const uint32_t off = (uint32_t)(t * 128 + ((ch ^ (t & 7)) << 4));
+            cp_async16_hint(sbase + off, kp + tt * p.ks_token + ch * 16, ok ? 16 : 0, stream_once);
+            cp_async16_hint(sbase + PAGE_BYTES + off, vp + tt * p.vs_token + ch * 16, ok ? 16 : 0, stream_once);
+        }
+    };
+
+    float o[KSTEPS][4];
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt) o[mt][0] = o[mt][1] = o[mt][2] = o[mt][3] = 0.f;
+    float m_run[2] = {-INFINITY, -INFINITY};
+    float l_run[2] = {0.f, 0.f};
+
+#pragma unroll
+    for (int s = 0; s < NSTAGE - 1; ++s) {
+        if (s < my_n) issue(s);
+        cp_async_commit();
+    }
+
+    for (int i = 0; i < my_n; ++i) {
+        cp_async_wait<NSTAGE - 2>();
+        __syncwarp();
+        if (i + NSTAGE - 1 < my_n) issue(i + NSTAGE - 1);
+        cp_async_commit();
+
+        const uint32_t sK = wbase + (i % NSTAGE) * STAGE_BYTES;
+        const uint32_t sV = sK + PAGE_BYTES;
+        const int tok0 = it.kv_begin + (i * NWARPS + warp) * 16;
+
+        // S^T = K Q^T
+        float s0[4] = {0.f, 0.f, 0.f, 0.f}, s1[4] = {0.f, 0.f, 0.f, 0.f};
+#pragma unroll
+        for (int m = 0; m < 4; ++m) {
+            uint32_t lo[2], hi[2];                    // rows g and g + 8: bytes d = 32 m + 8 c + {0..7}
+#pragma unroll
+            for (int rh = 0; rh < 2; ++rh) {
+                const int row = g + 8 * rh;
+                const uint32_t addr = sK + row * 128 + (((2 * m + (c >> 1)) ^ (row & 7)) << 4) + 8 * (c & 1);
+                asm volatile("ld.shared.v2.u32 {%0, %1}, [%2];" : "=r"(lo[rh]), "=r"(hi[rh]) : "r"(addr));
+            }
+            {
+                const uint32_t a[4] = {e4m3x2_to_f16x2(lo[0]), e4m3x2_to_f16x2(lo[1]), e4m3x2_to_f16x2(lo[0] >> 16), e4m3x2_to_f16x2(lo[1] >> 16)};
+                mma_f16_16816(s0, a, qf[2 * m][0], qf[2 * m][1]);
+            }
+            {
+                const uint32_t a[4] = {e4m3x2_to_f16x2(hi[0]), e4m3x2_to_f16x2(hi[1]), e4m3x2_to_f16x2(hi[0] >> 16), e4m3x2_to_f16x2(hi[1] >> 16)};
+                mma_f16_16816(s1, a, qf[2 * m + 1][0], qf[2 * m + 1][1]);
+            }
+        }
+        float s[4];
+        const int tA = tok0 + g;
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int tok = tA + (e >> 1) * 8;
+            const bool ok = tok < it.kv_end && tok >= it.kv_lo;
+            s[e] = ok ? (s0[e] + s1[e]) * score_scale : -INFINITY;
+        }
+        float alpha[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            float mx = fmaxf(s[j], s[2 + j]);
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 4));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 8));
+            mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, 16));
+            const float mnew = fmaxf(m_run[j], mx);
+            alpha[j] = fast_exp2(m_run[j] - mnew);
+            m_run[j] = mnew;
+            s[j] = fast_exp2(s[j] - mnew);
+            s[2 + j] = fast_exp2(s[2 + j] - mnew);
+            l_run[j] = l_run[j] * alpha[j] + s[j] + s[2 + j];
+        }
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt) {
+            o[mt][0] *= alpha[0]; o[mt][1] *= alpha[1];
+            o[mt][2] *= alpha[0]; o[mt][3] *= alpha[1];
+        }
+        const uint32_t pb0 = movmatrix_trans(pack_f16(s[0], s[1]));
+        const uint32_t pb1 = movmatrix_trans(pack_f16(s[2], s[3]));
+        // O^T += V^T P^T: this thread's 16 head-dim elements of its four tokens (2c, 2c+1, 2c+8, 2c+9)
+        uint32_t vw[4][4];
+#pragma unroll
+        for (int q4 = 0; q4 < 4; ++q4) {
+            const int tk = 2 * c + (q4 & 1) + 8 * (q4 >> 1);
+            const uint32_t addr = sV + tk * 128 + ((g ^ (tk & 7)) << 4);
+            asm volatile("ld.shared.v4.u32 {%0, %1, %2, %3}, [%4];" : "=r"(vw[q4][0]), "=r"(vw[q4][1]), "=r"(vw[q4][2]), "=r"(vw[q4][3]) : "r"(addr));
+        }
+#pragma unroll
+        for (int mt = 0; mt < KSTEPS; ++mt) {
+            // bytes 2 mt (row d) and 2 mt + 1 (row d + 1) of both tokens of a pair -> {tokA[b], tokB[b], tokA[b+1], tokB[b+1]}
+            const int w = mt >> 1;
+            const uint32_t sel = (mt & 1) ? 0x7362u : 0x5140u;
+            const uint32_t pa = __byte_perm(vw[0][w], vw[1][w], sel), pc = __byte_perm(vw[2][w], vw[3][w], sel);
+            const uint32_t a[4] = {e4m3x2_to_f16x2(pa), e4m3x2_to_f16x2(pa >> 16), e4m3x2_to_f16x2(pc), e4m3x2_to_f16x2(pc >> 16)};
+            mma_f16_16816(o[mt], a, pb0, pb1);
+        }
+    }
+    cp_async_wait<0>();
+
+#pragma unroll
+    for (int j = 0; j < 2; ++j) {
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 4);
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 8);
+        l_run[j] += __shfl_xor_sync(0xffffffffu, l_run[j], 16);
+    }
+    __syncthreads();
+    float* mo = reinterpret_cast<float*>(smem);       // [NWARPS][8][DP]
+    float* mm = mo + NWARPS * 8 * DP;
+    float* ml = mm + NWARPS * 8;
+#pragma unroll
+    for (int mt = 0; mt < KSTEPS; ++mt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+            const int d = 16 * g + 2 * mt + (e >> 1);       // the output rows of MMA mt in this thread (see the head of the kernel)
+            const int head = 2 * c + (e & 1);
+            mo[(warp * 8 + head) * DP + d] = o[mt][e];
+        }
+    if (lane < 4) {
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            mm[warp * 8 + 2 * lane + j] = m_run[j];
+            ml[warp * 8 + 2 * lane + j] = l_run[j];
+        }
+    }
+    __syncthreads();
+
+    for (int idx = threadIdx.x; idx < G * (D / 2); idx += NWARPS * 32) {
+        const int head = idx / (D / 2), d = (idx % (D / 2)) * 2;
+        float M = -INFINITY;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) M = fmaxf(M, mm[w * 8 + head]);
+        float L = 0.f, o0 = 0.f, o1 = 0.f;
+#pragma unroll
+        for (int w = 0; w < NWARPS; ++w) {
+            const float f = fast_exp2(mm[w * 8 + head] - M);
+            L += ml[w * 8 + head] * f;
+            o0 += mo[(w * 8 + head) * DP + d] * f;
+            o1 += mo[(w * 8 + head) * DP + d + 1] * f;
+        }
+        o0 *= out_scale;                                   // the value scale, once, in fp32
+        o1 *= out_scale;
+        const int hq = kvh * G + head;
+        if (it.part_slot < 0) {
+            float shrink = 1.f;
+            if (p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + hq) * kLog2e, M, L);
+            const float inv = shrink / L;
+            *reinterpret_cast<__nv_bfloat162*>(p.out + ((int64_t)it.q_row * p.Hq + hq) * D + d) =
+                __floats2bfloat162_rn(o0 * inv, o1 * inv);
+            if (p.lse && d == 0) p.lse[(int64_t)it.q_row * p.Hq + hq] = (M + log2f(L)) * kLn2;
+        } else {
+            const int64_t pr = (int64_t)it.part_slot * p.Hq + hq;
+            *reinterpret_cast<float2*>(p.part_o + pr * D + d) = make_float2(o0, o1);
+            if (d == 0) *reinterpret_cast<float2*>(p.part_ml + pr * 2) = make_float2(M, L);
+        }
+    }
+
     if (it.part_slot >= 0 && p.dec_counters != nullptr) {
         __shared__ int last_s;
         __threadfence();
@@ -602,6 +880,25 @@ static cudaError_t launch_decode_t(const AttnParams& p, int n_items, cudaStream_
     return cudaGetLastError();
 }
 
+cudaError_t launch_decode_fp8(const AttnParams& p, int n_items, cudaStream_t stream)
+{
+    if (n_items <= 0) return cudaSuccess;
+    auto kern = decode_splitk_fp8_kernel<kDecWarps, kDecStages>;
+    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * 128;
+    const size_t merge = (size_t)kDecWarps * 8 * (128 + 4) * 4 + (size_t)kDecWarps * 8 * 4 * 2;
+    const size_t smem = ring > merge ? ring : merge;
+    static std::atomic<bool> configured[64];
+    int dev = 0;
+    cudaGetDevice(&dev);
+    if (dev >= 0 && dev < 64 && !configured[dev].load(std::memory_order_acquire)) {
+        cudaError_t e = cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+        if (e != cudaSuccess) return e;
+        configured[dev].store(true, std::memory_order_release);
+    }
+    kern<<<n_items * p.Hkv, kDecWarps * 32, smem, stream>>>(p);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream)
 {
     if (n_items <= 0) return cudaSuccess;
@@ -711,6 +1008,7 @@ extern "C" cf_status cf_decode_attention_static(const cf_cache_desc* desc, const
     if (num_seqs == 0) return CF_OK;
     if (!q || !k_cache || !v_cache || !block_table || !context_len || !out) return CF_ERR_INVALID_ARG;
     if (num_seqs > kStaticMaxSeqs) return CF_ERR_WORKSPACE;
+    if (desc->kv_dtype != CF_KV_BF16) return CF_ERR_UNSUPPORTED;      // the fp8 cache is served by the context-based calls
     cudaStream_t stream = (cudaStream_t)cuda_stream;
     // The plan is copied from this function's stack frame: a captured copy node would read a dead frame on
     // every replay, so the call is refused while the stream is being captured.

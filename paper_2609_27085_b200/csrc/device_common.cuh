@@ -23,6 +23,8 @@ struct AttnParams {
     float scale_log2;                 // softmax_scale * log2(e)
     int32_t window;                   // sliding window in tokens (0 = none): row at position p sees keys (p - window, p]
     const float* sinks;               // [Hq] per-head sink logits (natural-log units) or null
+    const float* k_scale;             // fp8 cache: [Hkv] dequantisation scales (null: bf16 cache, or scale 1)
+    const float* v_scale;
     const int32_t* context_len;       // device copies of the host arrays
     const int32_t* query_len;
     const int32_t* q_start;

@@ -18,6 +18,8 @@ struct AppendParams {
     int64_t vs_block, vs_head, vs_token;
     int32_t Hkv, D, num_seqs, total_rows;
     int32_t num_blocks;               // pool size: a block id outside [0, num_blocks) is reported, its row not written
+    const float* k_scale;             // fp8 cache (non-null): rows are stored as e4m3_rne_sat(x / scale[head])
+    const float* v_scale;
     uint32_t* err;                    // device error word (may be null)
     const int32_t* context_len;
     const int32_t* query_len;
@@ -29,6 +31,18 @@ cudaError_t launch_validate_table(const int32_t* block_table, int32_t max_blocks
                                   int32_t num_seqs, int32_t num_blocks, uint32_t* bad_count, cudaStream_t stream);
 cudaError_t launch_decode(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
 cudaError_t launch_combine(const AttnParams& p, int head_dim, int n_items, cudaStream_t stream);
+// split-K decode over an fp8 (e4m3) cache, head_dim 128: same items, partials and merge as launch_decode
+cudaError_t launch_decode_fp8(const AttnParams& p, int n_items, cudaStream_t stream);
+// fp8 cache: expands the pages that prefill chunks need into bf16 staging pools [n_stage_pages, Hkv, 16, 128] (the codes
+// exactly, without the scales) and fills the staging block table; one entry per prefill sequence
+struct StageSeq {
+    int32_t seq;         // sequence (row of the block tables)
+    int32_t page0;       // first page of the sequence that is expanded
+    int32_t n_pages;
+    int32_t stage_base;  // staging page of page0
+};
+cudaError_t launch_kv_dequant_gather(const AttnParams& p, const StageSeq* seqs_dev, int n_seqs, int max_pages,
+                                     __nv_bfloat16* stage_k, __nv_bfloat16* stage_v, int32_t* stage_table, cudaStream_t stream);
 // a batch with shared prefixes: one grid whose first CTAs serve the shared-prefix chunks (one CTA per shared item
 // and KV head streams the chunk once for all members of its set and writes one partial per member and head) and
 // whose other CTAs serve the sequences' own chunks; n_shared_items = 0 is launch_decode

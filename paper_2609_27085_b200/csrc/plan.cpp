@@ -45,6 +45,13 @@ cf_status validate_desc(const cf_cache_desc* d)
     if (d->k_stride_token < d->head_dim || d->v_stride_token < d->head_dim) return CF_ERR_INVALID_ARG;
     if (!(d->softmax_scale >= 0.0f)) return CF_ERR_INVALID_ARG;   // also rejects NaN
     if (d->window_size < 0) return CF_ERR_INVALID_ARG;
+    if (d->kv_dtype != CF_KV_BF16 && d->kv_dtype != CF_KV_FP8_E4M3) return CF_ERR_INVALID_ARG;
+    if (d->kv_dtype == CF_KV_FP8_E4M3) {
+        if (d->head_dim != 128) return CF_ERR_UNSUPPORTED;
+        if (!d->k_scale || !d->v_scale) return CF_ERR_INVALID_ARG;
+        for (int i = 0; i < 6; ++i)
+            if (st[i] % 16 != 0) return CF_ERR_UNSUPPORTED;          // 16-byte copies of one-byte elements
+    }
     return CF_OK;
 }
 
@@ -95,7 +102,7 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     struct GroupInfo { int32_t group; int32_t pages; std::vector<int32_t> members; };
     std::vector<GroupInfo> groups_sh;
     int64_t extra_pages = 0;
-    if (share_group != nullptr && shared_len != nullptr && W == 0) {
+    if (share_group != nullptr && shared_len != nullptr && W == 0 && d->kv_dtype == CF_KV_BF16) {
         std::vector<std::pair<int32_t, int32_t>> keyed;          // (group, sequence) of the decode sequences that share
         for (int32_t s = 0; s < num_seqs; ++s)
             if (query_len[s] == 1 && share_group[s] >= 0 && shared_len[s] > 0) keyed.emplace_back(share_group[s], s);

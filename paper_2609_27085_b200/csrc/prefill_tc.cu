@@ -460,7 +460,6 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
       const int row = (warp & 3) * 32 + lane;
       const uint32_t lanes = lane_field(warp);
       const uint32_t tS = tmem + TM_S + t * 128 + lanes, tO = tmem + TM_O + t * D + lanes;
-      const float sc = p.scale_log2;
       uint32_t sbt = 0u;                       // tiles of this q tile in earlier items: running phase of s_full / p_full / o_done
       bool ok = true;
       for (int k = 0; ok; ++k) {
@@ -471,6 +470,9 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
         const int jb = cs->it.j_begin, n_jt = cs->n_j[t], kv_hi = cs->kv_hi_t[t];
         const int it_row0 = cs->it.row0[t], it_n_rows = cs->it.n_rows[t], it_q_row0 = cs->it.q_row0[t], it_head = cs->it.head[t];
         const int it_part_slot = cs->it.part_slot[t], it_part_k = cs->it.part_k, it_part_c = cs->it.part_c;
+        // fp8 cache: the staged K/V hold the codes; their per-head scales join the softmax scale and the output here
+        const float sc = p.k_scale != nullptr ? p.scale_log2 * __ldg(p.k_scale + cs->it.kvh) : p.scale_log2;
+        const float v_scale = p.v_scale != nullptr ? __ldg(p.v_scale + cs->it.kvh) : 1.f;
         const int limit = min(cs->it.prefix + it_row0 + row, kv_hi - 1);   // last visible key of this row
         const int first_key = p.window > 0 ? limit - p.window + 1 : -(1 << 30);   // first visible key (sliding window)
         const uint32_t span = (uint32_t)(limit - first_key);
@@ -577,7 +579,7 @@ prefill_tc_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_consta
             // a whole item joins the head's sink logit here; a KV range leaves it to the combine pass
             float m_fin = m_used, l_fin = l_sum, shrink = 1.f;
             if (!partial && p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + it_head) * kLog2e, m_fin, l_fin);
-            const float inv = shrink / l_fin;
+            const float inv = shrink * v_scale / l_fin;
             __nv_bfloat16* orow = p.out + ((int64_t)(it_q_row0 + row) * p.Hq + it_head) * D;
             // KV-split item: un-normalised fp32 row plus (reference maximum, sum) for the combine pass
             const int64_t pslot = (int64_t)it_part_slot + (int64_t)row * it_part_k + it_part_c;
@@ -666,6 +668,7 @@ __global__ void __launch_bounds__(256) prefill_combine_kernel(const AttnParams p
         }
     float shrink = 1.f;
     if (p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + it.head[t]) * kLog2e, M, L);
+    if (p.v_scale != nullptr) shrink *= __ldg(p.v_scale + it.head[t] / p.G);      // fp8 cache: the value scale of the head's KV head
     const float inv = shrink / L;
     uint2 w;
     w.x = pack_bf16(acc.x * inv, acc.y * inv);

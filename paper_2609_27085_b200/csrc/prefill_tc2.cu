@@ -471,7 +471,6 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
       const int row = (warp & 3) * 32 + lane;
       const uint32_t lanes = lane_field(warp);
       const uint32_t tS = tmem + PT_S + t * 128 + lanes, tO = tmem + PT_O + t * D + lanes;
-      const float sc = p.scale_log2;
       uint32_t sbt = 0u;
       bool ok = true;
       for (int k = 0; ok; ++k) {
@@ -483,6 +482,9 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
         const int it_head = cs->it.head[t] + 2 * (int)rank;                                         // this CTA's heads of the group
         const int it_part_slot = cs->it.part_slot[t] < 0 ? -1 : cs->it.part_slot[t] + (int)rank * cs->it.pad;
         const int it_part_k = cs->it.part_k, it_part_c = cs->it.part_c;
+        // fp8 cache: the staged K/V hold the codes; their per-head scales join the softmax scale and the output here
+        const float sc = p.k_scale != nullptr ? p.scale_log2 * __ldg(p.k_scale + cs->it.kvh) : p.scale_log2;
+        const float v_scale = p.v_scale != nullptr ? __ldg(p.v_scale + cs->it.kvh) : 1.f;
         const int limit = min(cs->it.prefix + it_row0 + row, kv_hi - 1);
         const int first_key = p.window > 0 ? limit - p.window + 1 : -(1 << 30);
         const uint32_t span = (uint32_t)(limit - first_key);
@@ -579,7 +581,7 @@ prefill_tc2_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_const
             const bool partial = it_part_slot >= 0;
             float m_fin = m_used, l_fin = l_sum, shrink = 1.f;
             if (!partial && p.sinks != nullptr) shrink = join_sink(__ldg(p.sinks + it_head) * kLog2e, m_fin, l_fin);
-            const float inv = shrink / l_fin;
+            const float inv = shrink * v_scale / l_fin;
             __nv_bfloat16* orow = p.out + ((int64_t)(it_q_row0 + row) * p.Hq + it_head) * D;
             const int64_t pslot = (int64_t)it_part_slot + (int64_t)row * it_part_k + it_part_c;
             float* prow = p.pre_part_o + pslot * D;

@@ -34,10 +34,13 @@ class GpuScenario:
     """Device copy of a scenario's pools plus a library context."""
 
     def __init__(self, sc: syn.Scenario, ctx=None, softmax_scale: float = 0.0, layout: str = "HND", debug=None,
-                 window: int = 0, sinks=None):
+                 window: int = 0, sinks=None, fp8=None):
         """debug: {CF_DEBUG_* option: value} applied to a context created here (test-only planner switches).
-        window / sinks: the sliding-window and attention-sink variant (sinks: host fp32 array [Hq])."""
+        window / sinks: the sliding-window and attention-sink variant (sinks: host fp32 array [Hq]).
+        fp8: (k_scale, v_scale) host fp32 arrays [Hkv]: the cache is an e4m3 cache; the scenario's bf16 prefix is
+        quantised on the host by the oracle's encoder (NaN sentinels stay NaN codes)."""
         self.geom = g = sc.geom
+        self.fp8 = fp8
         self.sinks_dev = None if sinks is None else torch.from_numpy(np.ascontiguousarray(sinks, dtype=np.float32)).cuda()
         variant = dict(window_size=window, sink_logits=self.sinks_dev)
         self.layout = layout
@@ -45,7 +48,17 @@ class GpuScenario:
         self.ctx = cf.cf_create(0) if ctx is None else ctx
         for opt, val in (debug or {}).items():
             cf.cf_set_debug_option(self.ctx, opt, val)
-        if layout == "HND":
+        if fp8 is not None:
+            assert layout == "HND"
+            self.k_scale = np.ascontiguousarray(fp8[0], dtype=np.float32)
+            self.v_scale = np.ascontiguousarray(fp8[1], dtype=np.float32)
+            self.k_scale_dev, self.v_scale_dev = torch.from_numpy(self.k_scale).cuda(), torch.from_numpy(self.v_scale).cuda()
+            self.k = torch.from_numpy(quantise_pool(sc.k_pool, self.k_scale)).cuda()
+            self.v = torch.from_numpy(quantise_pool(sc.v_pool, self.v_scale)).cuda()
+            self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks,
+                                     softmax_scale=softmax_scale, kv_dtype=cf.CF_KV_FP8_E4M3, k_scale=self.k_scale_dev,
+                                     v_scale=self.v_scale_dev, **variant)
+        elif layout == "HND":
             self.k = to_dev_bf16(sc.k_pool)
             self.v = to_dev_bf16(sc.v_pool)
             self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks,
@@ -59,6 +72,8 @@ class GpuScenario:
                                      k_strides=st, v_strides=st, softmax_scale=softmax_scale, **variant)
 
     def pools_host(self):
+        if self.fp8 is not None:
+            return self.k.cpu().numpy(), self.v.cpu().numpy()
         k, v = to_host_bits(self.k), to_host_bits(self.v)
         if self.layout != "HND":
             k, v = k.transpose(0, 2, 1, 3), v.transpose(0, 2, 1, 3)
@@ -90,6 +105,12 @@ class GpuScenario:
             self.ctx = None
 
 
+def quantise_pool(pool_bits: np.ndarray, scale: np.ndarray) -> np.ndarray:
+    """bf16 pool [NB, Hkv, B, D] -> e4m3 codes of value / scale[head] (the oracle's encoder; fp32 division)."""
+    vals = syn.bf16_bits_to_f32(pool_bits) / np.asarray(scale, dtype=np.float32)[None, :, None, None]
+    return oracle.e4m3_encode(vals.astype(np.float32))
+
+
 def compare(o_bits: np.ndarray, lse: np.ndarray, ref_o: np.ndarray, ref_lse: np.ndarray, rows=None, label=""):
     """Element-by-element comparison against the oracle (on `rows` if given)."""
     o = syn.bf16_bits_to_f64(o_bits if rows is None else o_bits[rows])
@@ -110,17 +131,23 @@ def compare(o_bits: np.ndarray, lse: np.ndarray, ref_o: np.ndarray, ref_lse: np.
 
 
 def run_and_check(sc: syn.Scenario, max_prefill_rows: int = 0, layout: str = "HND", softmax_scale: float = 0.0,
-                  check_append: bool = True, ctx=None, debug=None, tile_rows: bool = False, window: int = 0, sinks=None):
+                  check_append: bool = True, ctx=None, debug=None, tile_rows: bool = False, window: int = 0, sinks=None,
+                  fp8=None):
     """Every iteration of the scenario: append + attention on both sides, compare.
     Rows compared: all of them, or (max_prefill_rows) a thinned sample per prefill sequence, or (tile_rows) the
     first and last row of every 128-row q tile plus every 41st row of each prefill sequence, all heads."""
-    gpu = GpuScenario(sc, ctx=ctx, softmax_scale=softmax_scale, layout=layout, debug=debug, window=window, sinks=sinks)
-    k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    gpu = GpuScenario(sc, ctx=ctx, softmax_scale=softmax_scale, layout=layout, debug=debug, window=window, sinks=sinks, fp8=fp8)
+    scales = {}
+    if fp8 is None:
+        k_ref, v_ref = sc.k_pool.copy(), sc.v_pool.copy()
+    else:
+        k_ref, v_ref = quantise_pool(sc.k_pool, gpu.k_scale), quantise_pool(sc.v_pool, gpu.v_scale)
+        scales = dict(k_scale=gpu.k_scale, v_scale=gpu.v_scale)
     all_stats = []
     try:
         for b in sc.batches:
             gpu.append(b)
-            oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len)
+            oracle.kv_append(k_ref, v_ref, b.k_new, b.v_new, b.block_table, b.context_len, b.query_len, **scales)
             if check_append:
                 kg, vg = gpu.pools_host()
                 assert np.array_equal(kg, k_ref) and np.array_equal(vg, v_ref), f"{b.label}: kv_append not bit-exact"
@@ -128,7 +155,8 @@ def run_and_check(sc: syn.Scenario, max_prefill_rows: int = 0, layout: str = "HN
             rows = syn.tile_edge_rows(b) if tile_rows else (syn.sample_rows(b, max_prefill_rows) if max_prefill_rows else None)
             ref_o, ref_lse = oracle.mixed_attention(b.q, k_ref, v_ref, b.block_table, b.context_len, b.query_len,
                                                     scale=(softmax_scale or None), rows=rows, window=window,
-                                                    sinks=None if sinks is None else np.asarray(sinks, dtype=np.float32).astype(np.float64))
+                                                    sinks=None if sinks is None else np.asarray(sinks, dtype=np.float32).astype(np.float64),
+                                                    **scales)
             all_stats.append(compare(o_bits, lse, ref_o, ref_lse, rows=rows, label=b.label))
     finally:
         gpu.close()

@@ -357,3 +357,61 @@ def test_pair_kernel_mixed_batches_kv_split_window_and_sinks():
 def test_pair_kernel_chat_configuration_at_full_size():
     sc = syn.config3_chat(iterations=(0, 3))
     run_and_check(sc, tile_rows=True, check_append=False, debug=PAIRS)
+
+
+# ------------------------------------------------------------------ fp8 (e4m3) KV cache
+def scales(Hkv, seed=0, pow2=False):
+    rng = np.random.default_rng(200 + seed)
+    if pow2:
+        return (2.0 ** rng.integers(-6, -2, size=Hkv)).astype(np.float32), (2.0 ** rng.integers(-6, -2, size=Hkv)).astype(np.float32)
+    return rng.uniform(0.01, 0.05, size=Hkv).astype(np.float32), rng.uniform(0.01, 0.05, size=Hkv).astype(np.float32)
+
+
+@pytest.mark.parametrize("Hq,Hkv", [(32, 8), (8, 8), (16, 2), (64, 8)])
+def test_fp8_cache_decode(Hq, Hkv):
+    """Decode over an e4m3 cache: the append stores the oracle's codes bit for bit (whole-pool compare), attention
+    matches the oracle's reading of the same codes; ragged lengths, split and unsplit sequences."""
+    lens = [1, 2, 15, 16, 17, 31, 33, 127, 129, 255, 700, 1025, 2500, 4097, 9000, 20000]
+    sc = small(3, Hq, Hkv, 128, [l - 1 for l in lens], [[1] * len(lens)], NB=4096)
+    run_and_check(sc, fp8=scales(Hkv, 1))
+
+
+def test_fp8_cache_mixed_batches_and_chunked_prefill():
+    """Prefill chunks over an e4m3 cache (their pages are expanded into the bf16 staging area first), beside decode
+    sequences, over several iterations; with KV-split items, with a sliding window and sinks."""
+    prefix = [300, 40, 999, 0, 5000]
+    qlens = [[100, 1, 1, 64, 1], [37, 1, 1, 64, 1], [200, 1, 1, 1, 300]]
+    run_and_check(small(9, 32, 8, 128, prefix, qlens), fp8=scales(8, 2))
+    run_and_check(small(9, 32, 8, 128, prefix, qlens), fp8=scales(8, 3, pow2=True), window=150, sinks=sink_values(32, 8))
+    run_and_check(small(7, 32, 8, 128, [2000, 0, 700, 4097, 300], [[300, 700, 129, 64, 1]]), fp8=scales(8, 4),
+                  debug={cf.CF_DEBUG_PREFILL_SPLIT: 3})
+    run_and_check(small(7, 4, 4, 128, [2000, 0, 700], [[300, 700, 1]]), fp8=scales(4, 5))
+
+
+def test_fp8_cache_values_at_the_edges_of_the_format():
+    """New K/V values far outside the format's range saturate at +-448 * scale and tiny ones fall on the subnormal
+    grid - on both sides alike, because the rounding decision is taken in fp32 by both."""
+    sc = small(11, 8, 2, 128, [100, 40], [[60, 1]])
+    b = sc.batches[0]
+    rng = np.random.default_rng(1)
+    kn = syn.bf16_bits_to_f32(b.k_new) * rng.choice([1e-4, 1.0, 300.0], size=b.k_new.shape).astype(np.float32)
+    vn = syn.bf16_bits_to_f32(b.v_new) * rng.choice([1e-4, 1.0, 40.0], size=b.v_new.shape).astype(np.float32)
+    b.k_new[...] = syn.f32_to_bf16_bits(kn)
+    b.v_new[...] = syn.f32_to_bf16_bits(vn)
+    # (v_scale small enough that the saturated values, +-448 * v_scale, keep the outputs of order one: the
+    # comparison's absolute tolerance is meant for such outputs)
+    stats = run_and_check(sc, fp8=(np.array([0.5, 0.02], np.float32), np.array([0.004, 0.003], np.float32)))
+    print(stats)
+
+
+def test_fp8_cache_at_full_size_and_what_is_refused():
+    sc = syn.config3_chat(iterations=(0,))
+    run_and_check(sc, tile_rows=True, check_append=False, fp8=scales(8, 6))
+    # head_dim 64 and the allocation-free entry point do not take an fp8 cache
+    ks = torch.ones(2, device="cuda")
+    d64 = cf.make_desc(8, 2, 64, 16, 64, kv_dtype=cf.CF_KV_FP8_E4M3, k_scale=ks, v_scale=ks)
+    assert cf.cf_plan_inspect(d64, [5], [1], 8, check=False)[0] == cf.CF_ERR_UNSUPPORTED
+    d128 = cf.make_desc(8, 2, 128, 16, 64, kv_dtype=cf.CF_KV_FP8_E4M3, k_scale=ks, v_scale=ks)
+    assert cf.cf_decode_attention_static(d128, 1, 1, 1, 1, 8, [5], 1, check=False) == cf.CF_ERR_UNSUPPORTED
+    no_scale = cf.make_desc(8, 2, 128, 16, 64, kv_dtype=cf.CF_KV_FP8_E4M3)
+    assert cf.cf_plan_inspect(no_scale, [5], [1], 8, check=False)[0] == cf.CF_ERR_INVALID_ARG
