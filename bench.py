@@ -144,15 +144,27 @@ class ClockSampler:
 class DeviceWorkload:
     """A scenario resident on the GPU: pools, block table, per-iteration inputs."""
 
-    def __init__(self, sc: syn.Scenario, torch, cf, ctx):
+    def __init__(self, sc: syn.Scenario, torch, cf, ctx, window: int = 0, sinks: bool = False, fp8: bool = False):
+        """window / sinks: the sliding-window + attention-sink variant; fp8: the pools are converted to an e4m3
+        cache (per-head scale 1/32: N(0,1) values use the format's upper half without saturating)."""
         self.sc, self.torch, self.cf, self.ctx = sc, torch, cf, ctx
+        self.window, self.kv_elem_bytes = window, (1 if fp8 else 2)
         g = sc.geom
-        self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks)
 
         def dev(bits):
             return torch.from_numpy(np.ascontiguousarray(bits).view(np.int16)).cuda().view(torch.bfloat16)
 
-        self.k, self.v = dev(sc.k_pool), dev(sc.v_pool)
+        self.sinks = torch.linspace(-2.0, 2.0, g.num_q_heads, device="cuda") if sinks else None
+        variant = dict(window_size=window, sink_logits=self.sinks)
+        if fp8:
+            self.k_scale = torch.full((g.num_kv_heads,), 1.0 / 32.0, device="cuda")
+            self.v_scale = torch.full((g.num_kv_heads,), 1.0 / 32.0, device="cuda")
+            self.k = (dev(sc.k_pool).float() * 32.0).to(torch.float8_e4m3fn)        # input preparation only
+            self.v = (dev(sc.v_pool).float() * 32.0).to(torch.float8_e4m3fn)
+            variant.update(kv_dtype=cf.CF_KV_FP8_E4M3, k_scale=self.k_scale, v_scale=self.v_scale)
+        else:
+            self.k, self.v = dev(sc.k_pool), dev(sc.v_pool)
+        self.desc = cf.make_desc(g.num_q_heads, g.num_kv_heads, g.head_dim, g.block_size, g.num_blocks, **variant)
         self.its = []
         for b in sc.batches:
             it = {"b": b, "bt": torch.from_numpy(b.block_table).cuda(), "q": dev(b.q), "kn": dev(b.k_new), "vn": dev(b.v_new),
@@ -237,14 +249,14 @@ def median_of(reps):
     return float(np.median([r["ms_per_step"] for r in reps]))
 
 
-def batch_accounting(sc: syn.Scenario):
+def batch_accounting(sc: syn.Scenario, window: int = 0, kv_elem_bytes: int = 2):
     acc = []
     for b in sc.batches:
         acc.append({"tokens": b.total_q,
-                    "decode_bytes": syn.decode_algorithmic_bytes(b.geom, b.context_len, b.query_len),
-                    "decode_flops": syn.decode_flops(b.geom, b.context_len, b.query_len),
-                    "prefill_flops": syn.prefill_flops(b.geom, b.context_len, b.query_len),
-                    "prefill_bytes": syn.prefill_algorithmic_bytes(b.geom, b.context_len, b.query_len)})
+                    "decode_bytes": syn.decode_algorithmic_bytes(b.geom, b.context_len, b.query_len, window, kv_elem_bytes),
+                    "decode_flops": syn.decode_flops(b.geom, b.context_len, b.query_len, window),
+                    "prefill_flops": syn.prefill_flops(b.geom, b.context_len, b.query_len, window),
+                    "prefill_bytes": syn.prefill_algorithmic_bytes(b.geom, b.context_len, b.query_len, window, kv_elem_bytes)})
     return acc
 
 
@@ -257,7 +269,7 @@ def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks, cl
     """Per-kernel CUDA-event times (inside the library, on the launching stream, serial launch sequence) over
     `steps` steps.  Fractions: `frac` against the measured burst peak, `frac_of_sustained` against the measured
     seconds-long figure (what a kernel inside a long power-limited loop can be held to), `frac_of_nominal`."""
-    acc = batch_accounting(wl.sc)
+    acc = batch_accounting(wl.sc, wl.window, wl.kv_elem_bytes)
     cf.cf_set_timing(wl.ctx, True)
     launches = 0
     torch.cuda.synchronize()
@@ -398,20 +410,26 @@ def reduce_max(value: float, dist, device) -> float:
     return float(t.item())
 
 
-PER_CONFIG = [("configs[1] decode-only", lambda: syn.config2_decode_only()),
-              ("configs[2] chat-like", lambda: syn.config3_chat()),
-              ("configs[2] chat-like, one TP4 rank's shard (8 q heads, 2 kv heads)", lambda: syn.config3_chat_tp4_shard()),
-              ("configs[4] sweep, budget 0", lambda: syn.config5_sweep_point(0, 0)),
-              ("configs[4] sweep, budget 512 x 4 prompts", lambda: syn.config5_sweep_point(512, 4)),
-              ("configs[4] sweep, budget 2048 x 1 prompt", lambda: syn.config5_sweep_point(2048, 1)),
-              ("configs[4] sweep, budget 8192 x 1 prompt", lambda: syn.config5_sweep_point(8192, 1)),
-              ("configs[4] sweep, budget 8192 x 4 prompts", lambda: syn.config5_sweep_point(8192, 4))]
+# (name, scenario, variant of the layer): the other workload configurations, and two configurations again as a
+# sliding-window layer with sinks and on an fp8 cache (rooflines against the bytes / FLOPs those variants need)
+PER_CONFIG = [("configs[1] decode-only", lambda: syn.config2_decode_only(), {}),
+              ("configs[2] chat-like", lambda: syn.config3_chat(), {}),
+              ("configs[2] chat-like, one TP4 rank's shard (8 q heads, 2 kv heads)", lambda: syn.config3_chat_tp4_shard(), {}),
+              ("configs[4] sweep, budget 0", lambda: syn.config5_sweep_point(0, 0), {}),
+              ("configs[4] sweep, budget 512 x 4 prompts", lambda: syn.config5_sweep_point(512, 4), {}),
+              ("configs[4] sweep, budget 2048 x 1 prompt", lambda: syn.config5_sweep_point(2048, 1), {}),
+              ("configs[4] sweep, budget 8192 x 1 prompt", lambda: syn.config5_sweep_point(8192, 1), {}),
+              ("configs[4] sweep, budget 8192 x 4 prompts", lambda: syn.config5_sweep_point(8192, 4), {}),
+              ("configs[3] agentic as a sliding-window layer (window 4096) with sinks", lambda: syn.config4_agentic(),
+               {"window": 4096, "sinks": True}),
+              ("configs[1] decode-only on an fp8 (e4m3) cache", lambda: syn.config2_decode_only(), {"fp8": True}),
+              ("configs[4] sweep, budget 0, on an fp8 (e4m3) cache", lambda: syn.config5_sweep_point(0, 0), {"fp8": True})]
 
 
-def measure_config(torch, cf, ctx, sc, stream, peaks, clk, steps: int, repeats: int):
+def measure_config(torch, cf, ctx, sc, stream, peaks, clk, steps: int, repeats: int, variant=None):
     """Default-sequence and serial-sequence step times (median of `repeats` regions of `steps` steps) and the
     per-kernel figures of one workload."""
-    wl = DeviceWorkload(sc, torch, cf, ctx)
+    wl = DeviceWorkload(sc, torch, cf, ctx, **(variant or {}))
     n_it = len(sc.batches)
     for i in range(max(3, n_it)):
         wl.step(i, stream)
@@ -527,12 +545,13 @@ def run_ours(args):
         if rank == 0 and world == 1 and not args.no_per_config:
             per_config = {}
             pc_repeats = max(3, min(5, repeats))
-            for name, make in PER_CONFIG:
+            for name, make, variant in PER_CONFIG:
                 if args.only_config and args.only_config not in name:
                     continue
                 scn = make()
                 n_it = len(scn.batches)
-                per_config[name] = measure_config(torch, cf, ctx, scn, stream, peaks, clk, steps=max(8, 4 * n_it), repeats=pc_repeats)
+                per_config[name] = measure_config(torch, cf, ctx, scn, stream, peaks, clk, steps=max(8, 4 * n_it),
+                                                  repeats=pc_repeats, variant=variant)
                 del scn
 
     if rank == 0:

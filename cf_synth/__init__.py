@@ -302,39 +302,53 @@ def config5_sweep_point(budget: int, n_prompts: int, k: int = 0) -> Scenario:
 
 
 # --------------------------------------------------------------------------- accounting (sizes only)
-def decode_algorithmic_bytes(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
-    """Bytes a decode pass must move: K and V of every visible token once per KV head, the q row
-    in and the o row out, and the block-table entries."""
+def decode_algorithmic_bytes(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray, window: int = 0,
+                            kv_elem_bytes: int = 2) -> int:
+    """Bytes a decode pass must move: K and V of every visible token once per KV head (the last `window` tokens
+    with a sliding window; one byte per element for an fp8 cache), the q row in and the o row out, and the
+    block-table entries."""
     m = np.asarray(query_len) == 1
     lc = np.asarray(context_len, dtype=np.int64)[m]
-    per_tok = geom.kv_bytes_per_token()
-    return int((lc * per_tok).sum() + m.sum() * 2 * geom.num_q_heads * geom.head_dim * 2
-               + 4 * ((lc + geom.block_size - 1) // geom.block_size).sum())
+    vis = np.minimum(lc, window) if window > 0 else lc
+    per_tok = 2 * geom.num_kv_heads * geom.head_dim * kv_elem_bytes
+    return int((vis * per_tok).sum() + m.sum() * 2 * geom.num_q_heads * geom.head_dim * 2
+               + 4 * ((vis + geom.block_size - 1) // geom.block_size).sum())
 
 
-def prefill_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
+def _visible_pairs(lc: np.ndarray, lq: np.ndarray, window: int) -> int:
+    """Number of (query row, visible key) pairs of the chunks: row i of a chunk sees min(P + i + 1, window) keys."""
+    total = 0
+    for c, q in zip(lc, lq):
+        rows = np.arange(int(c - q) + 1, int(c) + 1, dtype=np.int64)
+        total += int((np.minimum(rows, window) if window > 0 else rows).sum())
+    return total
+
+
+def prefill_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray, window: int = 0) -> int:
     """4*D*Hq * (number of visible (query, key) pairs) over the sequences with Lq > 1."""
     lq = np.asarray(query_len, dtype=np.int64)
     lc = np.asarray(context_len, dtype=np.int64)
     m = lq > 1
-    lq, p = lq[m], (lc - lq)[m]
-    pairs = lq * p + lq * (lq + 1) // 2
-    return int(4 * geom.head_dim * geom.num_q_heads * pairs.sum())
+    return int(4 * geom.head_dim * geom.num_q_heads * _visible_pairs(lc[m], lq[m], window))
 
 
-def prefill_algorithmic_bytes(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
-    """Bytes a prefill pass must move: K and V of every visible token of each chunk's sequence once per KV
-    head, the chunk's q rows in and o rows out."""
+def prefill_algorithmic_bytes(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray, window: int = 0,
+                              kv_elem_bytes: int = 2) -> int:
+    """Bytes a prefill pass must move: K and V of every token some row of the chunk can see, once per KV head, the
+    chunk's q rows in and o rows out."""
     lq = np.asarray(query_len, dtype=np.int64)
     lc = np.asarray(context_len, dtype=np.int64)
     m = lq > 1
-    return int((lc[m] * geom.kv_bytes_per_token()).sum() + (lq[m] * 2 * geom.num_q_heads * geom.head_dim * 2).sum())
+    vis = lc[m] if window <= 0 else np.minimum(lc[m], lq[m] + window - 1)
+    per_tok = 2 * geom.num_kv_heads * geom.head_dim * kv_elem_bytes
+    return int((vis * per_tok).sum() + (lq[m] * 2 * geom.num_q_heads * geom.head_dim * 2).sum())
 
 
-def decode_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray) -> int:
+def decode_flops(geom: Geometry, context_len: np.ndarray, query_len: np.ndarray, window: int = 0) -> int:
     m = np.asarray(query_len) == 1
     lc = np.asarray(context_len, dtype=np.int64)[m]
-    return int(4 * geom.head_dim * geom.num_q_heads * lc.sum())
+    vis = np.minimum(lc, window) if window > 0 else lc
+    return int(4 * geom.head_dim * geom.num_q_heads * vis.sum())
 
 
 def tile_edge_rows(batch: Batch, tile: int = 128, stride: int = 41) -> np.ndarray:
