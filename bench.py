@@ -606,6 +606,10 @@ def small_case(name: str) -> syn.Scenario:
         geom = syn.Geometry(32, 8, 128, 16, 16384)
         lens = syn.uniform_int(np.random.default_rng(42), 32, 2048, 6144)
         return syn.scenario_from_lengths(name, geom, 43, lens - 1, [[1] * 32])
+    if name == "decode_small_fp8":   # the same lengths on an fp8 (e4m3) cache (run_case converts the pools)
+        geom = syn.Geometry(32, 8, 128, 16, 16384)
+        lens = syn.uniform_int(np.random.default_rng(42), 32, 2048, 6144)
+        return syn.scenario_from_lengths(name, geom, 43, lens - 1, [[1] * 32])
     if name == "prefill_small":
         geom = syn.Geometry(32, 8, 128, 16, 4096)
         return syn.scenario_from_lengths(name, geom, 44, [3072], [[1024]])
@@ -679,7 +683,7 @@ def run_case(args):
     ctx = cf.cf_create(0)
     if args.pairs:
         cf.cf_set_debug_option(ctx, cf.CF_DEBUG_PREFILL_PAIRS, 1)
-    wl = DeviceWorkload(small_case(args.case), torch, cf, ctx)
+    wl = DeviceWorkload(small_case(args.case), torch, cf, ctx, fp8=args.case.endswith("_fp8"))
     stream = torch.cuda.current_stream()
     for i in range(args.warmup):
         wl.step(i, stream)
@@ -695,7 +699,7 @@ def run_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", default=None,
-                    help="run a reduced workload (decode_small | prefill_small | prefill_multi | agentic_small | shared_prefix) and exit")
+                    help="run a reduced workload (decode_small | decode_small_fp8 | prefill_small | prefill_multi | agentic_small | shared_prefix) and exit")
     ap.add_argument("--pairs", action="store_true", help="reduced workloads: chunked prefill on the two-CTA (cta_group::2) kernel")
     ap.add_argument("--variant", default="both", choices=["both", "plain", "shared"], help="shared_prefix case: which entry point")
     ap.add_argument("--gpus", type=int, default=1)
