@@ -4,7 +4,7 @@
 
 nvcc cross-compiles without a GPU.  The library links the static CUDA runtime, so it can be
 loaded (and its symbols listed) on a machine with no driver; any CUDA call there fails with a
-status code instead.
+status code instead.  Extra nvcc flags (a -D for a development build) are taken from CF_NVCC_EXTRA.
 """
 from __future__ import annotations
 
@@ -43,7 +43,7 @@ def build(force: bool = False, verbose: bool = False) -> str:
     for src in SOURCES:
         obj = os.path.join(objdir, os.path.splitext(src)[0] + ".o")
         objs.append(obj)
-        cmd = [_nvcc(), *NVCC_FLAGS, "-c", os.path.join(CSRC, src), "-o", obj]
+        cmd = [_nvcc(), *NVCC_FLAGS, *os.environ.get("CF_NVCC_EXTRA", "").split(), "-c", os.path.join(CSRC, src), "-o", obj]
         if verbose:
             cmd.insert(1, "-Xptxas")
             cmd.insert(2, "-v")
