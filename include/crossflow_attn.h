@@ -198,7 +198,7 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  *   cf_set_overlap(ctx, 0): serial sequence, decode -> (combine) -> prefill -> (prefill combine) on the
  *     caller's stream alone.
  *   cf_set_overlap(ctx, n), n > 0 (the initial state is n = 1): n persistent prefill CTAs, one per SM (n = 1:
- *     the library's default share of the SMs), are enqueued first, on the caller's stream; a context-owned
+ *     the library's default share of the SMs, cf_spatial_share), are enqueued first, on the caller's stream; a context-owned
  *     side stream, forked from the caller's, runs decode on the SMs left over as soon as those CTAs hold their
  *     SMs (it waits for their count with a stream memory operation), and behind it a second prefill
  *     grid that draws from the same work queue, so the SMs decode frees join the prefill.  The side stream is
@@ -206,6 +206,15 @@ cf_status cf_get_async_status(cf_ctx* ctx);
  * Environment at cf_create: CF_OVERLAP=0 (serial), CF_SPATIAL_SMS=n (the share that n = 1 stands for).
  * cf_set_timing and cf_mixed_step_host use the serial sequence. */
 cf_status cf_set_overlap(cf_ctx* ctx, int n);
+
+/* The library's default share (host only, no GPU needed): how many of num_sms SMs (0 = 148) the first prefill grid
+ * of the spatial sequence takes for these lengths; 0 when the batch has no decode or no prefill part.  Decode is
+ * left the SMs it needs to be done by the time the prefill is - it saturates HBM from about 65 SMs (about 100 with
+ * eight query heads per KV head) and needs that many times (its own time / the call's time) - and the share is kept
+ * within [3/5, 7/8] of the SMs.  A scheduler that lends a decode node's capacity (Section 4.2) can read off it how
+ * much of the node a chunk will occupy beside the running decode batch. */
+int32_t cf_spatial_share(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t num_sms);
 
 /* Debug aid (synchronous): checks every block-table entry that cf_kv_append / cf_mixed_attention would
  * dereference for these lengths (entries [0, ceil(context_len/B)) of each row) against [0, num_blocks).

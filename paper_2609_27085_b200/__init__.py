@@ -46,7 +46,7 @@ CF_DEBUG_PREFILL_PAIRS = 5
 EXPORTS = ("cf_create", "cf_destroy", "cf_kv_append", "cf_mixed_attention", "cf_mixed_step_host", "cf_host_steps_flush",
            "cf_get_async_status", "cf_set_timing", "cf_get_timing_sums", "cf_get_last_launch_count", "cf_plan_inspect",
            "cf_decode_attention_static", "cf_selftest_bounded_wait", "cf_set_overlap", "cf_plan_create", "cf_plan_destroy",
-           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option", "cf_get_host_time_sums", "cf_mixed_attention_shared", "cf_get_last_plan_counts",
+           "cf_kv_append_planned", "cf_mixed_attention_planned", "cf_estimate_us", "cf_validate_block_table", "cf_set_debug_option", "cf_get_host_time_sums", "cf_mixed_attention_shared", "cf_get_last_plan_counts", "cf_spatial_share",
            "cf_status_string")
 
 
@@ -106,6 +106,8 @@ def load_library() -> ctypes.CDLL:
     lib.cf_set_overlap.argtypes = [vp, ctypes.c_int]
     lib.cf_validate_block_table.argtypes = [vp, dp, vp, i32, vp, vp, i32, vp, i32p]
     lib.cf_estimate_us.argtypes = [dp, vp, vp, i32, i32, i32, fp, fp, fp]
+    lib.cf_spatial_share.argtypes = [dp, vp, vp, i32, i32]
+    lib.cf_spatial_share.restype = ctypes.c_int32
     lib.cf_plan_create.argtypes = [vp, dp, vp, vp, i32, i32, vp, ctypes.POINTER(vp)]
     lib.cf_plan_destroy.argtypes = [vp]
     lib.cf_kv_append_planned.argtypes = [vp, vp, vp, vp, vp, vp, vp]
@@ -342,6 +344,12 @@ def cf_kv_append_planned(plan, k_cache, v_cache, k_new, v_new, block_table, stre
 def cf_mixed_attention_planned(plan, q, k_cache, v_cache, block_table, out, lse=None, stream=None) -> None:
     _check(load_library().cf_mixed_attention_planned(plan, _dev(q), _dev(k_cache), _dev(v_cache), _dev(block_table),
                                                      _dev(out), _dev(lse), _stream(stream)), "cf_mixed_attention_planned")
+
+
+def cf_spatial_share(desc: CacheDesc, context_len, query_len, num_sms: int = 148) -> int:
+    """SMs the first prefill grid of the spatial sequence takes for these lengths (0: no mixed batch)."""
+    lc, lq = _host_i32(context_len), _host_i32(query_len)
+    return int(load_library().cf_spatial_share(ctypes.byref(desc), lc.ctypes.data, lq.ctypes.data, int(lc.shape[0]), int(num_sms)))
 
 
 def cf_estimate_us(desc: CacheDesc, context_len, query_len, max_blocks_per_seq: int, num_sms: int = 148) -> Tuple[float, float, float]:

@@ -87,7 +87,7 @@ struct cf_ctx {
     bool overlap = true;
     cudaStream_t upload_stream = nullptr;      // plan uploads of cf_kv_append / cf_mixed_attention
     cudaStream_t plan_copy_stream = nullptr;   // set while cf_mixed_step_host runs
-    bool in_host_step = false; // cf_mixed_step_host keeps the serial sequence (its steps are bound by the host copies)
+    bool in_host_step = false; // inside a cf_mixed_step_host call that keeps the serial sequence (a step bound by the host copies)
     bool spatial_wait = true;  // decode waits (stream memory operation) for the front prefill CTAs to be resident; CF_DEBUG_SPATIAL_NO_WAIT: launch order only
     int spatial_sms = 0;       // SMs given to the first prefill grid in that mode (0 = three fifths)
     int spatial_sms_default = 0;   // CF_SPATIAL_SMS at cf_create: what cf_set_overlap(ctx, 1) goes back to
@@ -127,7 +127,7 @@ struct cf_plan {
     size_t off_qstart = 0, off_ctx = 0, off_qlen = 0, off_dec = 0, off_comb = 0, off_sh = 0, off_shm = 0, off_pre_tc = 0, off_pre_comb = 0, off_queue = 0, total = 0;
     int n_dec = 0, n_comb = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     bool pair = false;
-    float pre_over_dec = 0.f;
+    int front_sms = 0;          // spatial sequence: SMs of the first prefill grid (spatial_front_sms or cf_set_overlap)
 };
 
 namespace cf {
@@ -352,7 +352,7 @@ struct PlanCounts {
     int n_dec = 0, n_comb = 0, n_shared = 0, n_pre_tc = 0, n_pre_comb = 0, total_q = 0;
     int n_stage_seqs = 0, n_stage_pages = 0, max_stage_pages = 0, num_seqs = 0;   // fp8 cache: pages to expand for the prefill chunks
     bool pair = false;          // the prefill items are pair items (two CTAs each)
-    float pre_over_dec = 0.f;   // prefill_to_decode_ratio of the plan
+    int front_sms = 0;          // spatial sequence: SMs of the first prefill grid, as the plan was balanced for
     int n_part_slots = 0;
 };
 
@@ -512,10 +512,9 @@ static cf_status launch_attention(cf_ctx* c, const cf_cache_desc* desc, const Pl
         // stream forked from the caller's; a second prefill grid behind decode on that stream draws from the
         // same ticket counter, so the SMs that decode frees join the prefill as soon as decode is done; the
         // side stream is joined back before the prefill combine.
-        // Default share: three fifths of the SMs.  When the prefill work dwarfs the decode kernel, sharing the
-        // machine no longer pays (the tensor-bound kernel already runs at the power limit): prefill takes
-        // every SM first and decode fills in as its CTAs retire.
-        int front = c->spatial_sms > 0 ? c->spatial_sms / per_slot : (n.pre_over_dec > 3.9f ? sms : (sms * 3) / 5);
+        // The front grid's share comes from spatial_front_sms (or cf_set_overlap): decode keeps the SMs it needs to be
+        // done by the time the prefill is.
+        int front = (c->spatial_sms > 0 ? c->spatial_sms : n.front_sms > 0 ? n.front_sms : (c->num_sms * 3) / 5) / per_slot;
         if (front < 1) front = 1;
         if (front > sms) front = sms;
         if (front > n.n_pre_tc) front = n.n_pre_tc;
@@ -749,7 +748,9 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
-    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step && !c->timing) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
+    const int front_sms = !(c->overlap && !c->in_host_step) ? 0 : c->spatial_sms > 0 ? c->spatial_sms
+                              : spatial_front_sms(desc, context_len, query_len, num_seqs, c->num_sms);
+    cfg.prefill_sms_mixed = c->timing ? 0 : front_sms;
     cfg.prefill_pair = c->use_pairs && prefill_pair_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl, share_group, shared_len);
     if (st != CF_OK) return st;
@@ -785,7 +786,7 @@ cf_status cf_mixed_attention_shared(cf_ctx* c, const cf_cache_desc* desc, const 
     c->last_counts[0] = n.n_dec; c->last_counts[1] = n.n_comb; c->last_counts[2] = n.n_pre_tc; c->last_counts[3] = n.n_part_slots;
     c->last_counts[4] = n.n_pre_comb; c->last_counts[5] = n.n_shared; c->last_counts[6] = (int32_t)pl.share_members.size();
     c->last_counts[7] = pl.pair ? 1 : 0;
-    n.pre_over_dec = (c->overlap && !c->in_host_step) ? prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms) : 0.f;
+    n.front_sms = front_sms;
     const cf_status ls = launch_attention(c, desc, n, L, base, c->workspace, W,
                                           q, k_cache, v_cache, block_table, max_blocks_per_seq, out, lse, stream, true);
     const cf_status fs = finish_slot(slot, stream);
@@ -803,7 +804,9 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     if (st != CF_OK) return st;
     Plan pl;
     PlanConfig cfg = c->cfg;
-    cfg.prefill_sms_mixed = (c->overlap && !c->in_host_step) ? (c->spatial_sms > 0 ? c->spatial_sms : (c->num_sms * 3) / 5) : 0;
+    const int front_sms = !(c->overlap && !c->in_host_step) ? 0 : c->spatial_sms > 0 ? c->spatial_sms
+                              : spatial_front_sms(desc, context_len, query_len, num_seqs, c->num_sms);
+    cfg.prefill_sms_mixed = front_sms;
     cfg.prefill_pair = c->use_pairs && prefill_pair_supported(desc);
     st = build_plan(desc, context_len, query_len, num_seqs, max_blocks_per_seq, cfg, &pl);
     if (st != CF_OK) return st;
@@ -826,7 +829,7 @@ cf_status cf_plan_create(cf_ctx* c, const cf_cache_desc* desc, const int32_t* co
     P->total = L.total;
     P->n_dec = (int)pl.decode.size(); P->n_comb = (int)pl.combine.size();
     P->n_pre_tc = (int)pl.prefill_tc.size(); P->n_pre_comb = (int)pl.prefill_combine.size(); P->total_q = pl.total_q;
-    P->pre_over_dec = prefill_to_decode_ratio(desc, context_len, query_len, pl, c->num_sms);
+    P->front_sms = front_sms;
     P->n_part_slots = pl.n_part_slots; P->n_pre_slots = pl.n_pre_slots;
     P->pair = pl.pair;
     const size_t part_bytes = ws_layout(pl.n_part_slots, pl.n_pre_slots, desc->num_q_heads, desc->head_dim, n_stage_pages,
@@ -918,7 +921,7 @@ cf_status cf_mixed_attention_planned(cf_plan* P, const void* q, const void* k_ca
     PlanCounts n;
     n.n_dec = P->n_dec; n.n_comb = P->n_comb; n.n_pre_tc = P->n_pre_tc; n.n_pre_comb = P->n_pre_comb;
     n.total_q = P->total_q;
-    n.pre_over_dec = P->pre_over_dec;
+    n.front_sms = P->front_sms;
     n.n_part_slots = P->n_part_slots;
     n.pair = P->pair;
     n.n_stage_seqs = P->n_stage_seqs; n.n_stage_pages = P->n_stage_pages; n.max_stage_pages = P->max_stage_pages; n.num_seqs = P->num_seqs;
@@ -988,13 +991,15 @@ cf_status cf_mixed_step_host(cf_ctx* c, const cf_cache_desc* desc,
         c->plan_copy_stream = nullptr;
         return st;
     }
-    // The step is bound by the copies over PCIe, not by the kernels; measured on the chat-like workload the
-    // spatial sequence made it slower (0.40 ms against 0.355 ms).
+    // A step whose decode part weighs as much as its prefill part is bound by the copies over PCIe, not by the
+    // kernels: measured on the chat-like workload the spatial sequence made it slower (0.40 ms against 0.355 ms),
+    // so such steps keep the serial sequence.  A prefill-heavy step (the spatial share above its floor) is bound by
+    // the kernels and runs the sequence cf_mixed_attention would run.
     if (cudaStreamWaitEvent(stream, hs.h2d_done, 0) != cudaSuccess) {
         c->plan_copy_stream = nullptr;
         return CF_ERR_CUDA;
     }
-    c->in_host_step = true;
+    c->in_host_step = spatial_front_sms(desc, context_len, query_len, num_seqs, c->num_sms) <= (c->num_sms * 3) / 5;
     st = cf_mixed_attention(c, desc, dq, k_cache, v_cache, block_table, max_blocks_per_seq, context_len, query_len,
                             num_seqs, dout, nullptr, cuda_stream);
     c->in_host_step = false;
@@ -1158,6 +1163,13 @@ cf_status cf_get_last_launch_count(cf_ctx* c, int32_t* num_launches)
     if (!c || !num_launches) return CF_ERR_INVALID_ARG;
     *num_launches = c->launches;
     return CF_OK;
+}
+
+int32_t cf_spatial_share(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,
+                         int32_t num_seqs, int32_t num_sms)
+{
+    if (validate_desc(desc) != CF_OK || num_seqs < 0 || (num_seqs > 0 && (!context_len || !query_len))) return 0;
+    return spatial_front_sms(desc, context_len, query_len, num_seqs, num_sms > 0 ? num_sms : 148);
 }
 
 cf_status cf_estimate_us(const cf_cache_desc* desc, const int32_t* context_len, const int32_t* query_len,

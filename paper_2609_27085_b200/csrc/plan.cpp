@@ -449,24 +449,32 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
     return CF_OK;
 }
 
-float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
-                              int32_t num_sms)
+int32_t spatial_front_sms(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                          int32_t num_sms)
 {
-    if (plan.decode.empty() || plan.prefill_tc.empty()) return 0.f;
-    const int32_t S = (int32_t)plan.q_start.size() - 1;
-    double dec_bytes = 0.0;
-    for (int32_t s = 0; s < S; ++s)
-        if (query_len[s] == 1)
-            dec_bytes += (double)(d->window_size > 0 ? std::min(context_len[s], d->window_size) : context_len[s]) * 2.0 *
-                         d->num_kv_heads * d->head_dim * 2.0;
-    double work = 0.0;
-    for (const PrefillTcItem& it : plan.prefill_tc) {
-        int32_t hi = 0;
-        for (int t = 0; t < 2; ++t)
-            if (it.n_rows[t] > 0) hi = std::max(hi, it.prefix + it.row0[t] + it.n_rows[t]);
-        work += 8.0 + 1.9 * (double)std::max(0, std::min((hi + 127) / 128, it.j_end) - it.j_begin);
+    const int32_t G = d->num_q_heads / d->num_kv_heads, W = d->window_size;
+    const double items_per_tile = G >= 2 ? (double)d->num_kv_heads * (double)(G / 2) : 0.5 * (double)d->num_q_heads;
+    double dec_bytes = 0.0, work = 0.0;      // bytes the decode kernel streams; SM-microseconds of the prefill items
+    for (int32_t s = 0; s < num_seqs; ++s) {
+        const int32_t lq = query_len[s], lc = context_len[s];
+        if (lq == 1) {
+            dec_bytes += (double)(W > 0 ? std::min(lc, W) : lc) * 2.0 * d->num_kv_heads * d->head_dim * 2.0;
+        } else if (lq > 1) {
+            const int32_t prefix = lc - lq;
+            for (int32_t row = 0; row < lq; row += 128) {
+                const int32_t hi = prefix + std::min(lq, row + 128);
+                const int32_t lo = W > 0 ? std::max(0, prefix + row - W + 1) / 128 : 0;
+                work += items_per_tile * (8.0 + 1.9 * (double)((hi + 127) / 128 - lo));
+            }
+        }
     }
-    return (float)((work / (double)std::max(1, plan.pair ? num_sms / 2 : num_sms)) / (17.0 + dec_bytes / 7.1e6));
+    if (dec_bytes == 0.0 || work == 0.0) return 0;
+    const double sms = (double)std::max(1, num_sms);
+    const double t_dec = 17.0 + dec_bytes / 7.1e6, k_sat = G > 4 ? 100.0 : 65.0;
+    const double t_call = work / sms + t_dec * k_sat / sms;              // both parts packed without idle SMs
+    const double k_dec = 1.15 * k_sat * t_dec / t_call;
+    const double front = std::min(std::max(sms - k_dec, 0.6 * sms), 0.875 * sms);
+    return std::max(1, (int32_t)front);
 }
 
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,

@@ -195,10 +195,16 @@ cf_status build_plan(const cf_cache_desc* d, const int32_t* context_len, const i
 struct Estimate {
     float us_decode = 0.f, us_combine = 0.f, us_prefill = 0.f;
 };
-// Time the tcgen05 prefill items would take spread evenly over num_sms SMs, divided by the time of the
-// decode kernel (same constants as estimate_us; no scheduling, O(items)).  0 when either part is absent.
-float prefill_to_decode_ratio(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
-                              int32_t num_sms);
+// Spatial launch sequence: how many SMs the first prefill grid takes when a batch holds decode and prefill work
+// (0 when either part is absent).  Computed from the lengths alone, before the plan exists, because the planner
+// balances the prefill items over this many SMs.  Decode gets what it needs to be done when the prefill is, and no
+// more: it saturates HBM from k_sat SMs (about 65 with up to four heads per KV head, about 100 with eight, where the
+// MMAs per byte double), so over a call of length T it needs k_sat * t_decode / T of them, taken with a margin of 1.15;
+// the share of the prefill grid is clamped to [3/5, 7/8] of the SMs.  t_decode and the prefill work come from the
+// constants of estimate_us.  Fitted against sweeps of the share on the bench configurations (within a few per
+// cent of the best share on each).
+int32_t spatial_front_sms(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, int32_t num_seqs,
+                          int32_t num_sms);
 Estimate estimate_us(const cf_cache_desc* d, const int32_t* context_len, const int32_t* query_len, const Plan& plan,
                      int32_t num_sms);
 

@@ -161,6 +161,26 @@ def test_cost_model_is_sane_on_the_host():
     assert cf.cf_estimate_us(d, [7], [0], 4096) == (0.0, 0.0, 0.0)
 
 
+def test_spatial_share_follows_what_decode_needs():
+    """The first prefill grid's share of the SMs: none without a mixed batch; 3/5 of the machine when decode needs
+    most of the call's time; more, up to 7/8, as the prefill grows against a fixed decode batch; less for a group
+    size of 8 (decode needs more SMs to saturate HBM) than for 4 on the same lengths."""
+    g4, g8 = cf.make_desc(32, 8, 128, 16, 65536), cf.make_desc(64, 8, 128, 16, 65536)
+    dec = [4096] * 48
+    assert cf.cf_spatial_share(g4, dec, [1] * 48) == 0
+    assert cf.cf_spatial_share(g4, [6656], [512]) == 0
+    assert cf.cf_spatial_share(g4, [], []) == 0
+    chat = cf.cf_spatial_share(g4, [6656, 6656] + dec, [512, 512] + [1] * 48)
+    assert chat == 148 * 3 // 5
+    shares = [cf.cf_spatial_share(g4, [p + 2048] + [20000] * 16, [2048] + [1] * 16) for p in (0, 4096, 12288, 24576, 65536)]
+    assert shares == sorted(shares) and shares[0] == 88 and shares[-1] == 129
+    assert all(88 <= s <= 129 for s in shares)
+    mid4 = cf.cf_spatial_share(g4, [8192 + 8192] + [2048] * 256, [8192] + [1] * 256)
+    mid8 = cf.cf_spatial_share(g8, [8192 + 8192] + [2048] * 256, [8192] + [1] * 256)
+    assert 88 <= mid8 <= mid4 <= 129
+    assert cf.cf_spatial_share(g4, [26624] + [20000] * 16, [2048] + [1] * 16, num_sms=74) <= 74 * 7 // 8
+
+
 def test_kv_split_of_the_last_prefill_wave():
     """256 equal items on 148 SMs leave a last wave of 108: the planner cuts those into KV ranges that
     tile each item's extent, never start inside the diagonal band, and fill the machine."""
