@@ -20,7 +20,13 @@ constexpr int NTHREADS = 384;
 // first warpgroup shrinks to REGS_ROLE and the two softmax warpgroups grow to REGS_SOFTMAX.  A grow
 // request blocks until the CTA's pool holds enough released registers, so the released amount MUST
 // cover the growth or the kernel never returns; the launcher also checks the compiled register count.
-constexpr int LAUNCH_REGS = 168, REGS_ROLE = 136, REGS_SOFTMAX = 184;
+#ifndef CF_REGS_ROLE
+#define CF_REGS_ROLE 136
+#endif
+#ifndef CF_REGS_SOFTMAX
+#define CF_REGS_SOFTMAX 184
+#endif
+constexpr int LAUNCH_REGS = 168, REGS_ROLE = CF_REGS_ROLE, REGS_SOFTMAX = CF_REGS_SOFTMAX;
 static_assert(4 * (LAUNCH_REGS - REGS_ROLE) >= 8 * (REGS_SOFTMAX - LAUNCH_REGS), "setmaxnreg.inc would block forever");
 __device__ __forceinline__ uint32_t lane_field(int warp) { return (uint32_t)((warp & 3) * 32) << 16; }
 template <int N> __device__ __forceinline__ void reg_dec() { asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(N)); }
@@ -50,10 +56,11 @@ __device__ __forceinline__ float2 exp2_poly2(float2 x)
 }
 // Of the 16 pairs of a 32-column chunk, the pairs whose bit is set here take the polynomial route.
 // The exp2 unit (16 results per clock per SM) is shared by both softmax warpgroups and is the busiest
-// unit next to the tensor pipe; measured on the reduced prefill case: 1/8 of the pairs +3 %, 1/4 -1 %,
-// 1/2 -10 % (the extra FMA-pipe instructions lengthen the in-order instruction stream of each warp).
+// unit next to the tensor pipe; measured on the multi-item prefill case against no polynomial at all: 1/16 of
+// the pairs +1.7 % (any position in the chunk), 1/8 -0.7 %, 3/16 0 %, 1/4 -8 % (the extra FMA-pipe instructions
+// lengthen the in-order instruction stream of each warp).
 #ifndef CF_POLY_MASK
-#define CF_POLY_MASK 0x8080u
+#define CF_POLY_MASK 0x0080u
 #endif
 #ifndef CF_POLY_MASK_D64
 #define CF_POLY_MASK_D64 0x8080u
