@@ -48,12 +48,11 @@ WORKLOAD = ("configs[3] agentic long-context mixed batch: 16 decode seqs (ctx un
 # proportion to the K/V bytes, so a full launch is scaled by its algorithmic bytes.
 DECODE_TRAFFIC_RATIO = 1.010
 # DRAM traffic per algorithmic byte of the tcgen05 prefill kernel, from an ncu capture of the headline's own prefill
-# launch in the serial sequence (first chunk iteration: 2048 new tokens over 24,576 cached; 470.5 MB moved for
-# 142.6 MB algorithmic: the 109 MB of K/V no longer stay in L2 and come from DRAM ~3.5 times, and the fp32 partial
-# rows of the KV-split items add 55 MB).  A 4096-token chunk over 8192 cached tokens measures 1.28.  Prefill is
-# tensor-bound; the figure is scaled by the launch's algorithmic bytes and is approximate for the later chunk
-# iterations.
-PREFILL_TRAFFIC_RATIO = 3.30
+# launch in the serial sequence (first chunk iteration: 2048 new tokens over 24,576 cached; 162.5 MB moved for
+# 142.6 MB algorithmic: K/V once, q, out and the fp32 partial rows of the KV-split items).  A 4096-token chunk over
+# 8192 cached tokens measures 1.28.  Prefill is tensor-bound; the figure is scaled by the launch's algorithmic bytes
+# and is approximate for the later chunk iterations.
+PREFILL_TRAFFIC_RATIO = 1.14
 FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
 
 
