@@ -415,3 +415,42 @@ def test_fp8_cache_at_full_size_and_what_is_refused():
     assert cf.cf_decode_attention_static(d128, 1, 1, 1, 1, 8, [5], 1, check=False) == cf.CF_ERR_UNSUPPORTED
     no_scale = cf.make_desc(8, 2, 128, 16, 64, kv_dtype=cf.CF_KV_FP8_E4M3)
     assert cf.cf_plan_inspect(no_scale, [5], [1], 8, check=False)[0] == cf.CF_ERR_INVALID_ARG
+
+
+def test_property_random_batches_of_every_variant():
+    """Seeded random geometries, lengths and launch sequences, each with a random variant of the layer: a sliding
+    window, sinks, an fp8 cache (head_dim 128), or several at once.  Every row against the oracle."""
+    rng = np.random.default_rng(4242)
+    ctx = cf.cf_create(0)
+    try:
+        for trial in range(36):
+            fp8 = rng.random() < 0.3
+            Hkv = int(rng.choice([1, 2, 4, 8]))
+            G = int(rng.choice([1, 2, 4, 8]))
+            D = 128 if fp8 else int(rng.choice([64, 128]))
+            S = int(rng.integers(1, 9))
+            kind = int(rng.integers(0, 3))
+            if kind == 0:      # many small chunks and decode sequences
+                qlen = [int(x) for x in rng.choice([0, 1, 1, 1, 2, 31, 128, 129, 300, 513], size=S)]
+                prefix = [int(x) for x in rng.integers(0, 1500, size=S)]
+            elif kind == 1:    # long decode sequences (many KV chunks) beside one chunk
+                qlen = [1] * S
+                qlen[0] = int(rng.integers(2, 700))
+                prefix = [int(x) for x in rng.integers(0, 12000, size=S)]
+            else:              # one large chunk (sometimes more work items than SMs)
+                qlen = [int(rng.integers(300, 1500))] + [1] * (S - 1)
+                prefix = [int(rng.integers(0, 3000))] + [int(x) for x in rng.integers(0, 6000, size=S - 1)]
+            if sum(qlen) == 0:
+                qlen[0] = 1
+            window = int(rng.choice([0, 0, 1, 16, 100, 128, 1000, 4096]))
+            sinks = (rng.standard_normal(Hkv * G) * 2).astype(np.float32) if rng.random() < 0.5 else None
+            need = sum((p + q + 15) // 16 for p, q in zip(prefix, qlen)) + 8
+            sc = syn.scenario_from_lengths("rv", syn.Geometry(Hkv * G, Hkv, D, 16, max(256, int(need * 1.1))), 5100 + trial,
+                                           prefix, [qlen], shuffle_seqs=True)
+            cf.cf_set_overlap(ctx, int(rng.choice([0, 1, 1, 7, 40, 129])))
+            scales = ((0.004 + 0.004 * rng.random(Hkv)).astype(np.float32),
+                      (0.003 + 0.003 * rng.random(Hkv)).astype(np.float32)) if fp8 else None
+            run_and_check(sc, ctx=ctx, window=window, sinks=sinks, fp8=scales, max_prefill_rows=(24 if sum(qlen) > 400 else 0))
+    finally:
+        cf.cf_set_overlap(ctx, 1)
+        cf.cf_destroy(ctx)
