@@ -495,6 +495,15 @@ def run_ours(args):
         launches += wl.step(i, stream)
 
     with ClockSampler(local, period_s=args.clock_period_ms * 1e-3) as clk:
+        # per-kernel times before the long timed region, while the GPU is not yet held at its power cap: what the
+        # kernels do at the idle clock (the figures after the region, below, are the sustained ones)
+        kern_start, _ = measure_kernels(torch, cf, wl, min(steps, 8), stream, peaks, clk)
+        for i in range(2):
+            wl.step(i, stream)
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+        launches = 0
         t_first = time.perf_counter()
         reps = time_repeats(torch, one, steps, stream, repeats, clk)
         t_last = time.perf_counter()
@@ -583,6 +592,10 @@ def run_ours(args):
                 "kernels": {"decode": kern.get("decode"), "prefill": kern.get("prefill"), "sequence": "serial",
                             "ms_decode": kern["ms_decode"], "ms_combine": kern["ms_combine"], "ms_prefill": kern["ms_prefill"],
                             "sm_mhz": kern.get("sm_mhz")},
+                "kernels_at_start": {"decode": kern_start.get("decode"), "prefill": kern_start.get("prefill"), "sequence": "serial",
+                                     "sm_mhz": kern_start.get("sm_mhz"),
+                                     "note": "the same per-kernel measurement taken before the timed repeats (few steps, "
+                                             "GPU not yet at its power cap)"},
                 "e2e": {"value": world * tokens_per_step / (ms_e2e * 1e-3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                         "d2h_bytes_per_step": d2h, "ms_per_step": ms_e2e},
                 "serial": {"value": world * tokens_per_step / (ms_serial * 1e-3), "unit": UNIT, "ms_per_step": ms_serial,
