@@ -853,6 +853,10 @@ __global__ void __launch_bounds__(D / 4) combine_kernel(const AttnParams p)
 // ---------------------------------------------------------------------------------------------
 static constexpr int kDecWarps = 4;
 static constexpr int kDecStages = 3;
+#ifndef CF_FP8_STAGES
+#define CF_FP8_STAGES 4
+#endif
+static constexpr int kDecStagesFp8 = CF_FP8_STAGES;   // pages of an fp8 cache are half the size: the ring can be deeper in the same shared memory
 
 template <int D>
 static size_t decode_smem_bytes()
@@ -883,8 +887,8 @@ static cudaError_t launch_decode_t(const AttnParams& p, int n_items, cudaStream_
 cudaError_t launch_decode_fp8(const AttnParams& p, int n_items, cudaStream_t stream)
 {
     if (n_items <= 0) return cudaSuccess;
-    auto kern = decode_splitk_fp8_kernel<kDecWarps, kDecStages>;
-    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * 128;
+    auto kern = decode_splitk_fp8_kernel<kDecWarps, kDecStagesFp8>;
+    const size_t ring = (size_t)kDecWarps * kDecStagesFp8 * 2 * 16 * 128;
     const size_t merge = (size_t)kDecWarps * 8 * (128 + 4) * 4 + (size_t)kDecWarps * 8 * 4 * 2;
     const size_t smem = ring > merge ? ring : merge;
     static std::atomic<bool> configured[64];
