@@ -858,10 +858,16 @@ static constexpr int kDecStages = 3;
 #endif
 static constexpr int kDecStagesFp8 = CF_FP8_STAGES;   // pages of an fp8 cache are half the size: the ring can be deeper in the same shared memory
 
+#ifndef CF_D64_STAGES
+#define CF_D64_STAGES 4
+#endif
+// head_dim 64: a (page, head) is 2 KB, so four stages per warp fit in 64 KB per CTA and three CTAs on an SM (+3.5 %)
+template <int D> constexpr int dec_stages() { return D == 64 ? CF_D64_STAGES : kDecStages; }
+
 template <int D>
 static size_t decode_smem_bytes()
 {
-    const size_t ring = (size_t)kDecWarps * kDecStages * 2 * 16 * D * 2;
+    const size_t ring = (size_t)kDecWarps * dec_stages<D>() * 2 * 16 * D * 2;
     const size_t merge = (size_t)kDecWarps * 8 * (D + 4) * 4 + (size_t)kDecWarps * 8 * 4 * 2;
     return ring > merge ? ring : merge;
 }
@@ -869,7 +875,7 @@ static size_t decode_smem_bytes()
 template <int D>
 static cudaError_t launch_decode_t(const AttnParams& p, int n_items, cudaStream_t stream)
 {
-    auto kern = decode_splitk_kernel<D, kDecWarps, kDecStages>;
+    auto kern = decode_splitk_kernel<D, kDecWarps, dec_stages<D>()>;
     const size_t smem = decode_smem_bytes<D>();
     // set once per device; two host threads racing here both set the same value
     static std::atomic<bool> configured[64];
