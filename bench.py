@@ -296,19 +296,27 @@ def measure_kernels(torch, cf, wl: DeviceWorkload, steps: int, stream, peaks, cl
                          "bytes_per_launch": dec_bytes / steps, "ms": (ms_dec + ms_comb) / steps}
     if ms_pre > 0:
         tf = pre_flops / (ms_pre * 1e-3) / 1e12
-        # Denominator: the measured cuBLAS burst figure for a kernel timed at the idle clock, the measured sustained
-        # figure (a seconds-long cuBLAS loop under the 1000 W cap) when this kernel, too, was timed inside a long
-        # power-capped run - the SM clock sampled while it ran sits well below the maximum.  Both fractions are given.
-        capped = mhz is not None and mhz < 0.9 * peaks.get("sm_max_mhz", 1965.0)
-        peak = peaks["bf16_tflops_sustained"] if capped else peaks["bf16_tflops"]
-        out["prefill"] = {"bound": "tensor", "achieved": tf, "peak": peak, "unit": "TFLOP/s", "frac": tf / peak,
-                          "peak_kind": "sustained (power-capped run)" if capped else "burst",
+        out["prefill"] = {"bound": "tensor", "achieved": tf, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                          "frac": tf / peaks["bf16_tflops"], "peak_kind": "burst",
                           "frac_of_burst": tf / peaks["bf16_tflops"], "frac_of_sustained": tf / peaks["bf16_tflops_sustained"],
                           "frac_of_nominal": tf / NOMINAL_BF16_TFLOPS,
                           "traffic": PREFILL_TRAFFIC_RATIO * pre_bytes / steps, "bytes_per_launch": pre_bytes / steps,
                           "flops_per_launch": pre_flops / steps, "ms": ms_pre / steps,
                           "tflops_per_ghz": (tf / (mhz / 1e3)) if mhz else None}
     return out, launches
+
+
+def apply_peak_rule(kern, region_mhz, peaks):
+    """Denominator of the prefill kernel's roofline: the measured cuBLAS burst figure for a kernel timed at the idle
+    clock, the measured sustained figure (a seconds-long cuBLAS loop under the 1000 W cap) when this kernel, too, was
+    timed inside a long power-capped run - the median SM clock of the timed region that preceded the per-kernel
+    measurement sits more than 10 % below the maximum.  Both fractions stay in the record."""
+    pre = kern.get("prefill")
+    if not pre or region_mhz is None or region_mhz >= 0.9 * peaks.get("sm_max_mhz", 1965.0):
+        return
+    pre["peak"] = peaks["bf16_tflops_sustained"]
+    pre["frac"] = pre["achieved"] / pre["peak"]
+    pre["peak_kind"] = "sustained (power-capped run: SM clock %.0f MHz over the timed region)" % region_mhz
 
 
 def measure_host_time(torch, cf, wl: DeviceWorkload, steps: int, stream):
@@ -452,6 +460,8 @@ def measure_config(torch, cf, ctx, sc, stream, peaks, clk, steps: int, repeats: 
     host = measure_host_time(torch, cf, wl, min(steps, 4 * n_it), stream)
     toks = sum(wl.tokens(i) for i in range(steps)) / steps
     ms = median_of(reps)
+    region = [r["sm_mhz"] for r in reps if r["sm_mhz"]]
+    apply_peak_rule(kern, float(np.median(region)) if region else None, peaks)
     row = {"ms_per_step": ms, "ms_per_step_min": min(r["ms_per_step"] for r in reps), "ms_per_step_serial": median_of(reps_serial),
            "query_tokens_per_s": toks / (ms * 1e-3), "steps": steps, "repeats": len(reps),
            "sm_mhz": float(np.median([r["sm_mhz"] for r in reps if r["sm_mhz"]])) if any(r["sm_mhz"] for r in reps) else None,
@@ -573,12 +583,12 @@ def run_ours(args):
                 del scn
 
     if rank == 0:
+        apply_peak_rule(kern, clocks.get("sm_mhz"), peaks)
         dominant = "prefill" if kern.get("prefill", {}).get("ms", 0) >= kern.get("decode", {}).get("ms", 0) else "decode"
         roof = {k: kern[dominant].get(k) for k in ("bound", "achieved", "peak", "unit", "frac", "traffic", "frac_of_nominal",
                                                    "frac_of_burst", "frac_of_sustained", "tflops_per_ghz")}
         roof["kernel"] = "prefill_tc_kernel" if dominant == "prefill" else "decode_splitk_kernel (merge of the partials fused in)"
-        roof["peak_source"] = peaks["source"] + ((" bf16, " + kern["prefill"]["peak_kind"] + (", SM clock %.0f MHz while timed" % kern["sm_mhz"] if kern.get("sm_mhz") else ""))
-                                                 if dominant == "prefill" else " copy")
+        roof["peak_source"] = peaks["source"] + ((" bf16, " + kern["prefill"]["peak_kind"]) if dominant == "prefill" else " copy")
         roof["sequence"] = "serial (per-kernel events need kernels that do not overlap; `value` runs the default sequence)"
         mhz = [r["sm_mhz"] for r in reps if r["sm_mhz"]]
         line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": steps, "warmup": warmup,
